@@ -1,0 +1,6 @@
+"""Seeded synthetic inputs shared by the CPU checker and the GPU harness.
+
+Input generation only; nothing of the TSVD forward is computed here.
+"""
+from .configs import CONFIGS, Case, CaseSpec, make_case, make_weights, make_x, scaled  # noqa: F401
+from . import rng  # noqa: F401
