@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the TSVD linear map y = U(diag(S)(V x)) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config cfg2]
+
+One step = one full forward (V-stage, S scale, U-stage) over one batch of B synthetic
+tokens.  Prints ONE JSON line: tokens/s with inputs resident in HBM (`value`), the same
+through the host-buffer entry point with copies inside the timed region (`e2e`), the
+roofline figures of the dominant kernel, and the CPU checker timed on the host cores.
+With N > 1 (torchrun) every rank runs its own replica on its own tokens (weak scaling,
+no data-path collective); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+METRIC = "tsvd_linear_tokens_per_s"
+UNIT = "tokens/s"
+L2_FLUSH_BYTES = 256 << 20
+# measured on this machine's B200s (copy bandwidth, cuBLAS bf16 burst / sustained); used when
+# MEASURED_PEAKS.json is not next to this file
+PEAKS_COPY = {"hbm_gbs": 6524.9, "bf16_tflops": 1681.0, "bf16_tflops_sustained": 1398.7}
+INT8_OVER_BF16 = 2.0  # nominal dense tensor ratio (4.5 / 2.25 PFLOP/s)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in PEAKS_COPY}, "MEASURED_PEAKS.json"
+    except Exception:
+        return dict(PEAKS_COPY), "copy of MEASURED_PEAKS.json values recorded in bench.py"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason sampler running during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1])); mx.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                    "sw_power_cap"), parts[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        finally:
+            try:
+                os.unlink(self.path)
+            except OSError:
+                pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def cpu_baseline(spec, U, S, V, x_np, target_s=8.0, y_gpu=None):
+    """Time the CPU checker, as it stands, on a bounded sample of the workload's tokens."""
+    import oracle
+    from tests import _util
+    cores = oracle.threads()
+    n0 = min(spec.B, max(cores, 8))
+    xs = _util.oracle_x(x_np[:n0], spec.x_dtype)
+    oracle.forward(U, S, V, xs[:1])                      # warm-up (page in, thread pool)
+    t0 = time.perf_counter(); oracle.forward(U, S, V, xs); t1 = time.perf_counter()
+    per_tok = (t1 - t0) / n0
+    n = int(min(spec.B, max(n0, target_s / max(per_tok, 1e-9))))
+    n = max(cores, n - n % cores) if n >= cores else n
+    xs = _util.oracle_x(x_np[:n], spec.x_dtype)
+    t0 = time.perf_counter(); ref = oracle.forward(U, S, V, xs); t1 = time.perf_counter()
+    out = {"value": n / (t1 - t0), "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"first {n} of {spec.B} tokens of {spec.name}, one call, {t1 - t0:.2f} s wall"}
+    parity = None
+    if y_gpu is not None:
+        err = np.abs(y_gpu[:n] - ref.y)
+        if spec.x_dtype == "bf16":
+            tol = 1e-2 * np.abs(ref.y) + 1e-3
+            parity = {"tokens": n, "violations": int((err > tol).sum()), "worst_err_over_tol": float((err / tol).max())}
+        else:
+            parity = {"tokens": n, "max_err_over_max_ref": float(err.max() / np.abs(ref.y).max())}
+    return out, parity
+
+
+def run_reference(args, spec):
+    """--impl reference: the CPU checker on the host cores, same workload and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from tests import _util
+    U, V, S = gen.make_weights(spec)
+    cores = oracle.threads()
+    # size the per-step sample so that warmup+steps stay within about two minutes
+    x_probe = gen.make_x(spec, 0, min(spec.B, cores))
+    xp = _util.oracle_x(x_probe, spec.x_dtype)
+    oracle.forward(U, S, V, xp[:1])
+    t0 = time.perf_counter(); oracle.forward(U, S, V, xp); per_tok = (time.perf_counter() - t0) / len(xp)
+    budget = 100.0 / max(1, args.steps + args.warmup)
+    n = int(min(spec.B, max(cores, budget / max(per_tok, 1e-9))))
+    n = max(1, n - n % cores) if n >= cores else n
+    x = _util.oracle_x(gen.make_x(spec, 0, n), spec.x_dtype)
+    for _ in range(args.warmup):
+        oracle.forward(U, S, V, x)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.forward(U, S, V, x)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = n / dt
+    sample = f"{n} of {spec.B} tokens of {spec.name} per step"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(spec, "host cores; no GPU"),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(spec, l2_note):
+    return {"workload": spec.name, "M": spec.M, "N": spec.N, "K": spec.K, "B": spec.B,
+            "density": spec.density, "x_dtype": spec.x_dtype, "s_dist": spec.s_dist, "seed": spec.seed,
+            "l2": l2_note}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg2", choices=sorted(gen.CONFIGS))
+    ap.add_argument("--path", default="auto", choices=["auto", "simple", "decode", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    spec = gen.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        run_reference(args, spec)
+        return
+
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear, binding, build as lib_build
+    from paper_2308_07641_b200 import TSVD_FLAG_PATH_DECODE, TSVD_FLAG_PATH_SIMPLE, TSVD_FLAG_PATH_TENSOR
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the TSVD library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        lib_build.build()
+    if dist:
+        dist.barrier()
+
+    flags = {"auto": 0, "simple": TSVD_FLAG_PATH_SIMPLE, "decode": TSVD_FLAG_PATH_DECODE,
+             "tensor": TSVD_FLAG_PATH_TENSOR}[args.path]
+    U, V, S = gen.make_weights(spec)
+    x_np = gen.make_x(gen.scaled(spec, seed=spec.seed + 1000 * rank) if rank else spec)
+    layer = TSVDLinear(U, S, V)
+    info = layer.info
+    from tests._util import torch_x
+    x = torch_x(x_np, spec.x_dtype)
+    y = layer.forward(x, flags=flags)
+    torch.cuda.synchronize()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        layer.forward(x, out=y, flags=flags)
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    binding.tsvd_profile_enable(layer.handle, True)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = binding.tsvd_launch_count()
+    barrier()
+    for a, b in ev:
+        flush.zero_()                 # evict inputs, outputs and weights from L2 between steps
+        a.record()
+        layer.forward(x, out=y, flags=flags)
+        b.record()
+    barrier()
+    launches = binding.tsvd_launch_count() - launches0
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = float(sum(step_ms))
+    stage_ms, stage_n = binding.tsvd_profile_read(layer.handle)
+    binding.tsvd_profile_enable(layer.handle, False)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * spec.B / (ms_per_step * 1e-3)
+
+    # end to end: host buffers, copies inside the timed region
+    x_host = torch.from_numpy(x_np.view(np.int16) if spec.x_dtype == "bf16" else x_np).pin_memory()
+    y_bf16 = y.dtype == torch.bfloat16
+    y_host = torch.empty((spec.B, spec.M), dtype=torch.int16 if y_bf16 else torch.float32).pin_memory()
+    dt_code = binding.DTYPES[spec.x_dtype]
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        binding.tsvd_forward_host(layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        binding.tsvd_forward_host(layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if dist:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * spec.B / e2e_s, "unit": UNIT,
+           "h2d_bytes_per_step": int(x_host.numel() * x_host.element_size()),
+           "d2h_bytes_per_step": int(y_host.numel() * y_host.element_size()), "steps": e2e_steps}
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    # roofline of the dominant kernel
+    peaks, peaks_src = load_peaks()
+    dom = int(np.argmax(stage_ms))
+    dom_ms = stage_ms[dom] / max(1, stage_n[dom])
+    rows, contr = ((spec.K, spec.N) if dom == 1 else (spec.M, spec.K))
+    # executed dense operations of that launch: 2 * rows * contraction * columns
+    dense_flop = 2.0 * rows * contr * spec.B
+    achieved_tf = dense_flop / (dom_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved_tf,
+                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"],
+                "traffic": None, "peak_source": f"bf16 burst, {peaks_src} (of measured)",
+                "ms_per_launch": dom_ms, "flop_per_launch": dense_flop,
+                "stage_ms_per_step": {n: m / args.steps for n, m in zip(binding.STAGE_NAMES, stage_ms)}}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": {"f32": "f32", "bf16": "f32", "i8": "int32"}[spec.x_dtype], "data": "synthetic",
+            "config": workload_config(spec, "flushed between steps (256 MiB memset)"),
+            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks,
+            "packed_bytes": info["packed_bytes"],
+            "algorithmic_adds_per_token": info["density_u"] * spec.M * spec.K + info["density_v"] * spec.K * spec.N,
+            "path": args.path}
+    if world == 1 and not args.no_cpu_baseline:
+        y_gpu = y.float().double().cpu().numpy()
+        cb, parity = cpu_baseline(spec, U, S, V, x_np, y_gpu=y_gpu)
+        line["cpu_baseline"] = cb
+        line["parity_on_cpu_sample"] = parity
+    print(json.dumps(line), flush=True)
+    layer.close()
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

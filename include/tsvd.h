@@ -1,0 +1,143 @@
+/*
+ * libtsvd -- the Ternary-SVD parameterised linear map on one NVIDIA B200 (sm_100a).
+ *
+ *     y = U ( diag(S) ( V x ) )
+ *
+ * U [M,K] and V [K,N] hold only -1, 0, +1; S is a real vector of length K; x is a
+ * batch of B activation columns.  This is the inference-time form of the paper's
+ * TSVD layer (Section "Truncated SVD in Network Compression", Eq. 1-2 and the
+ * display that follows them; Section "Ternary SVD"), whose cost the paper counts
+ * as r*K*(M+N) additions and K multiplications per column (supplement, Table S1).
+ *
+ * Plain C ABI: pointers and sizes only.  Every call returns a status; nothing is
+ * thrown across the boundary; arguments are validated on the host before any
+ * kernel is launched.  There is no CPU implementation behind these calls: without
+ * a CUDA device they return TSVD_E_CUDA.
+ */
+#ifndef TSVD_H
+#define TSVD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tsvd_handle_s* tsvd_handle_t; /* opaque; owns device memory on one GPU */
+
+/* storage type of the activations x */
+typedef enum { TSVD_F32 = 0, TSVD_BF16 = 1, TSVD_I8 = 2 } tsvd_dtype_t;
+
+typedef enum {
+    TSVD_OK = 0,
+    TSVD_E_NULL = 1,    /* a required pointer is NULL                              */
+    TSVD_E_SHAPE = 2,   /* a size is < 1, a leading dimension is too small, ...    */
+    TSVD_E_VALUE = 3,   /* an entry of U or V is outside {-1,0,+1}                  */
+    TSVD_E_DTYPE = 4,   /* unknown dtype or unsupported flag combination           */
+    TSVD_E_ALIGN = 5,   /* a pointer or leading dimension breaks the stated rule   */
+    TSVD_E_CUDA = 6,    /* a CUDA runtime call failed (or there is no device)      */
+    TSVD_E_TIMEOUT = 7, /* a bounded device-side wait gave up                      */
+    TSVD_E_NOMEM = 8    /* host or device allocation failed                        */
+} tsvd_status_t;
+
+/* flags of tsvd_forward_ex */
+#define TSVD_FLAG_OUT_F32 0x1u      /* write y as fp32 even for bf16 activations            */
+#define TSVD_FLAG_PATH_SIMPLE 0x10u /* force the CUDA-core reference kernels               */
+#define TSVD_FLAG_PATH_DECODE 0x20u /* force the small-batch streaming kernels             */
+#define TSVD_FLAG_PATH_TENSOR 0x40u /* force the tcgen05 tensor-core kernels               */
+
+/*
+ * tsvd_pack -- store U and V in the 2-bit sign/nonzero form (the paper: "we only
+ * need 2 bits to store each element of a ternary matrix", Section "Connection with
+ * BNN and What Next"; the split U = U+ - U-, V = V+ - V- of the same section) and
+ * copy S.
+ *
+ *   U  host, int8 [M,K] row-major        V  host, int8 [K,N] row-major
+ *   S  host, float [K] (any finite values: negative, zero, unsorted are all fine)
+ *   flags  must be 0
+ *   out    receives the handle; device memory lives on the current CUDA device
+ *
+ * The inputs are copied; the caller keeps ownership of U, S, V.  Any M,K,N >= 1:
+ * ragged sizes are padded with zero entries, which contribute nothing.
+ * Synchronous.  Errors: E_NULL, E_SHAPE, E_VALUE (nothing is kept), E_NOMEM, E_CUDA.
+ */
+tsvd_status_t tsvd_pack(const int8_t* U, const float* S, const int8_t* V, int M, int K, int N,
+                        unsigned flags, tsvd_handle_t* out);
+
+/*
+ * tsvd_forward -- y = U(diag(S)(V x)) for B columns (display after Eq. 2):
+ * V-stage additions, K multiplications by S, U-stage additions (Table S1).
+ *
+ *   x  device; column b is the N contiguous values at x + b*N (token-major)
+ *   y  device; column b is the M contiguous values at y + b*M
+ *      y is fp32 for TSVD_F32 and TSVD_I8 activations, bf16 (round-to-nearest-even
+ *      from the fp32 result) for TSVD_BF16
+ *   stream  a cudaStream_t (NULL = default stream); the call is asynchronous
+ *
+ * x and y stay owned by the caller and must be 16-byte aligned.  The handle's
+ * scratch memory is shared by all calls on it: calls on one handle must be
+ * ordered on one stream (or otherwise serialised).  Scratch grows on the first call
+ * with a larger B (that call synchronises the device once).
+ * Errors: E_NULL, E_SHAPE (B < 1), E_DTYPE, E_ALIGN, E_NOMEM, E_CUDA.
+ */
+tsvd_status_t tsvd_forward(tsvd_handle_t h, const void* x, void* y, int B, tsvd_dtype_t dtype,
+                           void* stream);
+
+/*
+ * tsvd_forward_ex -- tsvd_forward with leading dimensions, flags and the V-stage
+ * result exposed (Table S1, row "V(.)").
+ *
+ *   ldx >= N, ldy >= M   in elements; column b at x + b*ldx, y + b*ldy
+ *   z_out  optional device buffer [B][K] receiving V x BEFORE the S scale:
+ *          int32 (exact) for TSVD_I8, fp32 otherwise
+ */
+tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx, void* y, int ldy, int B,
+                              tsvd_dtype_t dtype, unsigned flags, void* z_out, void* stream);
+
+/*
+ * tsvd_forward_host -- the same map with HOST buffers: copies x to the device,
+ * runs tsvd_forward_ex, copies y (and z_out) back, and waits.  x, y, z_out are
+ * host pointers (pinned memory makes the copies faster); layout as tsvd_forward.
+ */
+tsvd_status_t tsvd_forward_host(tsvd_handle_t h, const void* x, void* y, int B,
+                                tsvd_dtype_t dtype, unsigned flags, void* z_out);
+
+/* Device-side error word of the last forward on this handle (read after the
+ * stream has been synchronised): TSVD_OK, or TSVD_E_TIMEOUT if a bounded wait
+ * inside a kernel gave up.  Resets the word. */
+tsvd_status_t tsvd_last_status(tsvd_handle_t h);
+
+/* Shapes, packed size in bytes (U and V codes plus S: the bytes a forward must
+ * stream) and the measured nonzero rates r of U and V (the r of Table S1). */
+tsvd_status_t tsvd_info(tsvd_handle_t h, int* M, int* K, int* N, size_t* packed_bytes,
+                        double* density_u, double* density_v);
+
+/* Inverse of tsvd_pack, for tests: writes the stored U [M,K], V [K,N] (int8) and
+ * S [K] back to HOST buffers (any of them may be NULL). */
+tsvd_status_t tsvd_unpack(tsvd_handle_t h, int8_t* U, float* S, int8_t* V);
+
+/*
+ * Per-stage device timing (measurement support; the paper reports operation counts
+ * per stage in Table S1 and no timings).  While enabled, every forward on the handle
+ * records CUDA events on its own stream around each kernel it launches.
+ * tsvd_profile_read waits for those events, then returns, per stage, the summed
+ * device time in milliseconds and the number of launches since the last read (both
+ * arrays have TSVD_N_STAGES entries), and resets the sums.
+ *   stage 0: activations -> integer digits     stage 1: V-stage (+ S scale)
+ *   stage 2: S*(V x)     -> integer digits     stage 3: U-stage
+ */
+#define TSVD_N_STAGES 4
+tsvd_status_t tsvd_profile_enable(tsvd_handle_t h, int on);
+tsvd_status_t tsvd_profile_read(tsvd_handle_t h, float* ms_sum, unsigned* launches);
+
+/* Number of kernels this library has launched in this process (all handles). */
+unsigned long long tsvd_launch_count(void);
+
+void tsvd_destroy(tsvd_handle_t h);
+const char* tsvd_strerror(tsvd_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSVD_H */

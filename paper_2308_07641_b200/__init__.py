@@ -1,0 +1,59 @@
+"""Ternary-SVD linear map y = U(diag(S)(V x)) on one B200, behind the C ABI of include/tsvd.h.
+
+`binding` mirrors the C entry points one to one; `TSVDLinear` is a small
+convenience over them for torch tensors (it owns a handle and passes data
+pointers and the current stream; it computes nothing itself).
+"""
+from __future__ import annotations
+
+from . import binding
+from .binding import (DTYPES, TSVD_BF16, TSVD_F32, TSVD_I8, TSVD_FLAG_OUT_F32,  # noqa: F401
+                      TSVD_FLAG_PATH_DECODE, TSVD_FLAG_PATH_SIMPLE, TSVD_FLAG_PATH_TENSOR,
+                      TSVDError)
+
+
+class TSVDLinear:
+    """A packed TSVD layer living on the current CUDA device."""
+
+    def __init__(self, U, S, V):
+        self.handle = binding.tsvd_pack(U, S, V)
+        self.info = binding.tsvd_info(self.handle)
+
+    @staticmethod
+    def _dtype_of(x) -> int:
+        import torch
+        if x.dtype == torch.float32:
+            return TSVD_F32
+        if x.dtype == torch.bfloat16:
+            return TSVD_BF16
+        if x.dtype == torch.int8:
+            return TSVD_I8
+        raise TSVDError(binding.TSVD_E_DTYPE, "TSVDLinear.forward")
+
+    def forward(self, x, out=None, flags: int = 0, z_out=None):
+        """x: CUDA tensor [B,N] (float32, bfloat16 or int8), row stride >= N. Returns y [B,M]."""
+        import torch
+        if not x.is_cuda or x.dim() != 2 or x.stride(1) != 1:
+            raise TSVDError(binding.TSVD_E_SHAPE, "TSVDLinear.forward")
+        B = x.shape[0]
+        dt = self._dtype_of(x)
+        out_dtype = torch.bfloat16 if (dt == TSVD_BF16 and not flags & TSVD_FLAG_OUT_F32) else torch.float32
+        if out is None:
+            out = torch.empty((B, self.info["M"]), dtype=out_dtype, device=x.device)
+        stream = torch.cuda.current_stream(x.device).cuda_stream
+        binding.tsvd_forward_ex(self.handle, x.data_ptr(), x.stride(0), out.data_ptr(), out.stride(0),
+                                B, dt, flags, z_out.data_ptr() if z_out is not None else 0, stream)
+        return out
+
+    __call__ = forward
+
+    def close(self):
+        if getattr(self, "handle", None):
+            binding.tsvd_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,172 @@
+"""ctypes binding of libtsvd: the same names as include/tsvd.h, argument marshalling only.
+
+Every step of the map runs in the CUDA library.  There is no Python or CPU
+implementation behind these calls: if libtsvd.so is missing the import of the
+symbols fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtsvd.so")
+
+TSVD_F32, TSVD_BF16, TSVD_I8 = 0, 1, 2
+TSVD_OK = 0
+(TSVD_E_NULL, TSVD_E_SHAPE, TSVD_E_VALUE, TSVD_E_DTYPE, TSVD_E_ALIGN, TSVD_E_CUDA,
+ TSVD_E_TIMEOUT, TSVD_E_NOMEM) = range(1, 9)
+TSVD_FLAG_OUT_F32 = 0x1
+TSVD_FLAG_PATH_SIMPLE = 0x10
+TSVD_FLAG_PATH_DECODE = 0x20
+TSVD_FLAG_PATH_TENSOR = 0x40
+
+DTYPES = {"f32": TSVD_F32, "bf16": TSVD_BF16, "i8": TSVD_I8}
+
+# every symbol include/tsvd.h declares
+EXPORTS = ("tsvd_pack", "tsvd_forward", "tsvd_forward_ex", "tsvd_forward_host", "tsvd_last_status",
+           "tsvd_info", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read", "tsvd_launch_count", "tsvd_destroy", "tsvd_strerror")
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+class TSVDError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {tsvd_strerror(status)} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libtsvd.so (built by paper_2308_07641_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2308_07641_b200.build` "
+                              "(needs nvcc); there is no fallback implementation")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci, cu = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint
+        L.tsvd_pack.argtypes = [vp, vp, vp, ci, ci, ci, cu, ctypes.POINTER(vp)]
+        L.tsvd_pack.restype = ci
+        L.tsvd_forward.argtypes = [vp, vp, vp, ci, ci, vp]
+        L.tsvd_forward.restype = ci
+        L.tsvd_forward_ex.argtypes = [vp, vp, ci, vp, ci, ci, ci, cu, vp, vp]
+        L.tsvd_forward_ex.restype = ci
+        L.tsvd_forward_host.argtypes = [vp, vp, vp, ci, ci, cu, vp]
+        L.tsvd_forward_host.restype = ci
+        L.tsvd_last_status.argtypes = [vp]
+        L.tsvd_last_status.restype = ci
+        L.tsvd_info.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci),
+                                ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_double),
+                                ctypes.POINTER(ctypes.c_double)]
+        L.tsvd_info.restype = ci
+        L.tsvd_unpack.argtypes = [vp, vp, vp, vp]
+        L.tsvd_unpack.restype = ci
+        L.tsvd_profile_enable.argtypes = [vp, ci]
+        L.tsvd_profile_enable.restype = ci
+        L.tsvd_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(cu)]
+        L.tsvd_profile_read.restype = ci
+        L.tsvd_launch_count.argtypes = []
+        L.tsvd_launch_count.restype = ctypes.c_ulonglong
+        L.tsvd_destroy.argtypes = [vp]
+        L.tsvd_destroy.restype = None
+        L.tsvd_strerror.argtypes = [ci]
+        L.tsvd_strerror.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def tsvd_strerror(status: int) -> str:
+    return lib().tsvd_strerror(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != TSVD_OK:
+        raise TSVDError(status, what)
+
+
+def _np_ptr(a: Optional[np.ndarray]) -> Optional[int]:
+    return None if a is None else a.ctypes.data
+
+
+def tsvd_pack(U: np.ndarray, S: np.ndarray, V: np.ndarray, flags: int = 0) -> int:
+    """Pack host arrays U int8 [M,K], S float32 [K], V int8 [K,N]; returns the handle."""
+    U = np.ascontiguousarray(U, dtype=np.int8)
+    V = np.ascontiguousarray(V, dtype=np.int8)
+    S = np.ascontiguousarray(S, dtype=np.float32)
+    M, K = U.shape
+    K2, N = V.shape
+    if K2 != K or S.shape != (K,):
+        raise TSVDError(TSVD_E_SHAPE, "tsvd_pack")
+    h = ctypes.c_void_p()
+    _check(lib().tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, M, K, N, flags,
+                           ctypes.byref(h)), "tsvd_pack")
+    return h.value
+
+
+def tsvd_forward(h: int, x_ptr: int, y_ptr: int, B: int, dtype: int, stream: int = 0) -> None:
+    """Raw device pointers (e.g. torch.Tensor.data_ptr()) and a cudaStream_t value."""
+    _check(lib().tsvd_forward(h, x_ptr, y_ptr, B, dtype, stream or None), "tsvd_forward")
+
+
+def tsvd_forward_ex(h: int, x_ptr: int, ldx: int, y_ptr: int, ldy: int, B: int, dtype: int,
+                    flags: int = 0, z_out_ptr: int = 0, stream: int = 0) -> None:
+    _check(lib().tsvd_forward_ex(h, x_ptr, ldx, y_ptr, ldy, B, dtype, flags, z_out_ptr or None,
+                                 stream or None), "tsvd_forward_ex")
+
+
+def tsvd_forward_host(h: int, x_ptr: int, y_ptr: int, B: int, dtype: int, flags: int = 0,
+                      z_out_ptr: int = 0) -> None:
+    """Host pointers (numpy .ctypes.data or pinned torch tensors' data_ptr())."""
+    _check(lib().tsvd_forward_host(h, x_ptr, y_ptr, B, dtype, flags, z_out_ptr or None),
+           "tsvd_forward_host")
+
+
+def tsvd_last_status(h: int) -> int:
+    return int(lib().tsvd_last_status(h))
+
+
+def tsvd_info(h: int) -> dict:
+    M, K, N = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    pb = ctypes.c_size_t()
+    du, dv = ctypes.c_double(), ctypes.c_double()
+    _check(lib().tsvd_info(h, ctypes.byref(M), ctypes.byref(K), ctypes.byref(N), ctypes.byref(pb),
+                           ctypes.byref(du), ctypes.byref(dv)), "tsvd_info")
+    return {"M": M.value, "K": K.value, "N": N.value, "packed_bytes": pb.value,
+            "density_u": du.value, "density_v": dv.value}
+
+
+def tsvd_unpack(h: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    info = tsvd_info(h)
+    U = np.empty((info["M"], info["K"]), dtype=np.int8)
+    V = np.empty((info["K"], info["N"]), dtype=np.int8)
+    S = np.empty(info["K"], dtype=np.float32)
+    _check(lib().tsvd_unpack(h, U.ctypes.data, S.ctypes.data, V.ctypes.data), "tsvd_unpack")
+    return U, S, V
+
+
+N_STAGES = 4
+STAGE_NAMES = ("x_digits", "v_stage", "t_digits", "u_stage")
+
+
+def tsvd_profile_enable(h: int, on: bool) -> None:
+    _check(lib().tsvd_profile_enable(h, 1 if on else 0), "tsvd_profile_enable")
+
+
+def tsvd_profile_read(h: int):
+    """Returns ([ms summed per stage], [launches per stage]) since the last read."""
+    ms = (ctypes.c_float * N_STAGES)()
+    n = (ctypes.c_uint * N_STAGES)()
+    _check(lib().tsvd_profile_read(h, ms, n), "tsvd_profile_read")
+    return list(ms), list(n)
+
+
+def tsvd_launch_count() -> int:
+    return int(lib().tsvd_launch_count())
+
+
+def tsvd_destroy(h: int) -> None:
+    if h:
+        lib().tsvd_destroy(h)

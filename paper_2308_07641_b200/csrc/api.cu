@@ -1,0 +1,281 @@
+// The C ABI of libtsvd (see include/tsvd.h): argument validation, handle lifetime,
+// scratch management and dispatch.  No arithmetic of the map is done on the host.
+#include <atomic>
+#include <new>
+
+#include "tsvd_internal.cuh"
+
+static std::atomic<unsigned long long> g_launches{0};
+void tsvd_count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+extern "C" unsigned long long tsvd_launch_count(void) { return g_launches.load(); }
+
+extern "C" const char* tsvd_strerror(tsvd_status_t s)
+{
+    switch (s) {
+        case TSVD_OK: return "ok";
+        case TSVD_E_NULL: return "null pointer argument";
+        case TSVD_E_SHAPE: return "bad shape, batch or leading dimension";
+        case TSVD_E_VALUE: return "U or V holds a value outside {-1,0,+1}";
+        case TSVD_E_DTYPE: return "unknown dtype or unsupported flags";
+        case TSVD_E_ALIGN: return "pointer or leading dimension not aligned as required";
+        case TSVD_E_CUDA: return "CUDA runtime error (or no CUDA device)";
+        case TSVD_E_TIMEOUT: return "a bounded device-side wait gave up";
+        case TSVD_E_NOMEM: return "out of memory";
+    }
+    return "unknown status";
+}
+
+void StageProfiler::begin(int stage, cudaStream_t s)
+{
+    if (!on) return;
+    if (pending.size() >= 8192) drain();
+    Pair p;
+    p.stage = stage;
+    if (cudaEventCreate(&p.a) != cudaSuccess || cudaEventCreate(&p.b) != cudaSuccess) { (void)cudaGetLastError(); return; }
+    cudaEventRecord(p.a, s);
+    pending.push_back(p);
+}
+
+void StageProfiler::end(cudaStream_t s)
+{
+    if (!on || pending.empty()) return;
+    cudaEventRecord(pending.back().b, s);
+}
+
+void StageProfiler::drain()
+{
+    for (auto& p : pending) {
+        float t = 0.f;
+        if (cudaEventSynchronize(p.b) == cudaSuccess && cudaEventElapsedTime(&t, p.a, p.b) == cudaSuccess) {
+            ms[p.stage] += t;
+            launches[p.stage] += 1;
+        }
+        cudaEventDestroy(p.a);
+        cudaEventDestroy(p.b);
+    }
+    (void)cudaGetLastError();
+    pending.clear();
+}
+
+extern "C" tsvd_status_t tsvd_profile_enable(tsvd_handle_t h, int on)
+{
+    if (!h) return TSVD_E_NULL;
+    h->prof.drain();
+    for (int i = 0; i < TSVD_N_STAGES; ++i) { h->prof.ms[i] = 0.f; h->prof.launches[i] = 0; }
+    h->prof.on = on != 0;
+    return TSVD_OK;
+}
+
+extern "C" tsvd_status_t tsvd_profile_read(tsvd_handle_t h, float* ms_sum, unsigned* launches)
+{
+    if (!h || !ms_sum || !launches) return TSVD_E_NULL;
+    h->prof.drain();
+    for (int i = 0; i < TSVD_N_STAGES; ++i) {
+        ms_sum[i] = h->prof.ms[i];
+        launches[i] = h->prof.launches[i];
+        h->prof.ms[i] = 0.f;
+        h->prof.launches[i] = 0;
+    }
+    return TSVD_OK;
+}
+
+static void free_handle(tsvd_handle_s* h)
+{
+    if (!h) return;
+    h->prof.drain();
+    if (h->V.units) cudaFree(h->V.units);
+    if (h->U.units) cudaFree(h->U.units);
+    if (h->S) cudaFree(h->S);
+    if (h->ws) cudaFree(h->ws);
+    if (h->io) cudaFree(h->io);
+    if (h->dev_status) cudaFree(h->dev_status);
+    (void)cudaGetLastError();
+    delete h;
+}
+
+extern "C" void tsvd_destroy(tsvd_handle_t h)
+{
+    if (!h) return;
+    const int dev = h->device;
+    int prev = dev;
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) cudaSetDevice(dev);
+    cudaDeviceSynchronize();
+    free_handle(h);
+    if (prev != dev) cudaSetDevice(prev);
+}
+
+extern "C" tsvd_status_t tsvd_pack(const int8_t* U, const float* S, const int8_t* V, int M, int K, int N,
+                                   unsigned flags, tsvd_handle_t* out)
+{
+    if (!out) return TSVD_E_NULL;
+    *out = nullptr;
+    if (!U || !S || !V) return TSVD_E_NULL;
+    if (M < 1 || K < 1 || N < 1) return TSVD_E_SHAPE;
+    if (flags != 0) return TSVD_E_DTYPE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return TSVD_E_CUDA; }
+
+    tsvd_handle_s* h = new (std::nothrow) tsvd_handle_s();
+    if (!h) return TSVD_E_NOMEM;
+    h->device = dev;
+    h->M = M; h->K = K; h->N = N;
+
+    tsvd_status_t st = TSVD_OK;
+    do {
+        if (cudaMalloc(&h->dev_status, sizeof(int)) != cudaSuccess) { st = TSVD_E_NOMEM; break; }
+        if (cudaMemset(h->dev_status, 0, sizeof(int)) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+        if ((st = tsvd_pack_matrix(V, K, N, &h->V, h->dev_status)) != TSVD_OK) break;
+        if ((st = tsvd_pack_matrix(U, M, K, &h->U, h->dev_status)) != TSVD_OK) break;
+        int flag = 0;
+        if (cudaMemcpy(&flag, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+            st = TSVD_E_CUDA; break;
+        }
+        if (flag) { st = TSVD_E_VALUE; break; }
+        const size_t s_len = (size_t)h->V.R_pad;
+        if (cudaMalloc(&h->S, s_len * sizeof(float)) != cudaSuccess) { st = TSVD_E_NOMEM; break; }
+        if (cudaMemset(h->S, 0, s_len * sizeof(float)) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+        if (cudaMemcpy(h->S, S, (size_t)K * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+            st = TSVD_E_CUDA; break;
+        }
+        if (cudaMemset(h->dev_status, 0, sizeof(int)) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+    } while (0);
+    if (st != TSVD_OK) {
+        (void)cudaGetLastError();
+        free_handle(h);
+        return st;
+    }
+    *out = h;
+    return TSVD_OK;
+}
+
+extern "C" tsvd_status_t tsvd_info(tsvd_handle_t h, int* M, int* K, int* N, size_t* packed_bytes,
+                                   double* density_u, double* density_v)
+{
+    if (!h) return TSVD_E_NULL;
+    if (M) *M = h->M;
+    if (K) *K = h->K;
+    if (N) *N = h->N;
+    if (packed_bytes) *packed_bytes = h->U.bytes() + h->V.bytes() + (size_t)h->K * sizeof(float);
+    if (density_u) *density_u = (double)h->U.nnz / ((double)h->M * (double)h->K);
+    if (density_v) *density_v = (double)h->V.nnz / ((double)h->K * (double)h->N);
+    return TSVD_OK;
+}
+
+extern "C" tsvd_status_t tsvd_unpack(tsvd_handle_t h, int8_t* U, float* S, int8_t* V)
+{
+    if (!h) return TSVD_E_NULL;
+    tsvd_status_t st;
+    if (U && (st = tsvd_unpack_matrix(h->U, U)) != TSVD_OK) return st;
+    if (V && (st = tsvd_unpack_matrix(h->V, V)) != TSVD_OK) return st;
+    if (S) TSVD_CUDA_OK(cudaMemcpy(S, h->S, (size_t)h->K * sizeof(float), cudaMemcpyDeviceToHost));
+    return TSVD_OK;
+}
+
+extern "C" tsvd_status_t tsvd_last_status(tsvd_handle_t h)
+{
+    if (!h) return TSVD_E_NULL;
+    int word = 0;
+    TSVD_CUDA_OK(cudaMemcpy(&word, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (word) TSVD_CUDA_OK(cudaMemset(h->dev_status, 0, sizeof(int)));
+    return word ? TSVD_E_TIMEOUT : TSVD_OK;
+}
+
+static size_t dtype_size(tsvd_dtype_t d)
+{
+    switch (d) {
+        case TSVD_F32: return 4;
+        case TSVD_BF16: return 2;
+        case TSVD_I8: return 1;
+    }
+    return 0;
+}
+
+// Grow the handle's scratch to at least `bytes` (synchronises the device when it grows).
+static tsvd_status_t ensure_ws(tsvd_handle_s* h, size_t bytes)
+{
+    if (bytes <= h->ws_bytes) return TSVD_OK;
+    TSVD_CUDA_OK(cudaDeviceSynchronize());
+    if (h->ws) { cudaFree(h->ws); h->ws = nullptr; h->ws_bytes = 0; }
+    const size_t rounded = (bytes + 255) & ~(size_t)255;
+    if (cudaMalloc(&h->ws, rounded) != cudaSuccess) { (void)cudaGetLastError(); return TSVD_E_NOMEM; }
+    h->ws_bytes = rounded;
+    return TSVD_OK;
+}
+
+extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx, void* y, int ldy, int B,
+                                         tsvd_dtype_t dtype, unsigned flags, void* z_out, void* stream)
+{
+    if (!h || !x || !y) return TSVD_E_NULL;
+    if (B < 1) return TSVD_E_SHAPE;
+    const size_t xs = dtype_size(dtype);
+    if (xs == 0) return TSVD_E_DTYPE;
+    const unsigned known = TSVD_FLAG_OUT_F32 | TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR;
+    if (flags & ~known) return TSVD_E_DTYPE;
+    const unsigned path = flags & (TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR);
+    if (path & (path - 1)) return TSVD_E_DTYPE;  // at most one forced path
+    if (ldx < h->N || ldy < h->M) return TSVD_E_SHAPE;
+    if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)z_out & 3)) return TSVD_E_ALIGN;
+
+    int dev = 0;
+    TSVD_CUDA_OK(cudaGetDevice(&dev));
+    if (dev != h->device) return TSVD_E_CUDA;
+
+    ForwardArgs a;
+    a.h = h; a.x = x; a.ldx = ldx; a.y = y; a.ldy = ldy; a.B = B; a.dtype = dtype;
+    a.out_f32 = (flags & TSVD_FLAG_OUT_F32) != 0;
+    a.z_out = z_out;
+    a.stream = (cudaStream_t)stream;
+
+    tsvd_status_t st = ensure_ws(h, tsvd_simple_ws_bytes(h, B));
+    if (st != TSVD_OK) return st;
+    a.t = reinterpret_cast<float*>(h->ws);
+    a.t_ld = h->V.R_pad;
+    return tsvd_forward_simple(a);
+}
+
+extern "C" tsvd_status_t tsvd_forward(tsvd_handle_t h, const void* x, void* y, int B, tsvd_dtype_t dtype,
+                                      void* stream)
+{
+    if (!h) return TSVD_E_NULL;
+    return tsvd_forward_ex(h, x, h->N, y, h->M, B, dtype, 0u, nullptr, stream);
+}
+
+extern "C" tsvd_status_t tsvd_forward_host(tsvd_handle_t h, const void* x, void* y, int B,
+                                           tsvd_dtype_t dtype, unsigned flags, void* z_out)
+{
+    if (!h || !x || !y) return TSVD_E_NULL;
+    if (B < 1) return TSVD_E_SHAPE;
+    const size_t xs = dtype_size(dtype);
+    if (xs == 0) return TSVD_E_DTYPE;
+    const bool y_bf16 = (dtype == TSVD_BF16) && !(flags & TSVD_FLAG_OUT_F32);
+    const size_t x_bytes = (size_t)B * h->N * xs;
+    const size_t y_bytes = (size_t)B * h->M * (y_bf16 ? 2 : 4);
+    const size_t z_bytes = z_out ? (size_t)B * h->K * 4 : 0;
+    // staging buffers live in the handle and only grow
+    const size_t x_off = 0, y_off = (x_bytes + 255) & ~(size_t)255;
+    const size_t z_off = y_off + ((y_bytes + 255) & ~(size_t)255);
+    const size_t need = z_off + z_bytes;
+    if (need > h->io_bytes) {
+        TSVD_CUDA_OK(cudaDeviceSynchronize());
+        if (h->io) { cudaFree(h->io); h->io = nullptr; h->io_bytes = 0; }
+        if (cudaMalloc(&h->io, need) != cudaSuccess) { (void)cudaGetLastError(); return TSVD_E_NOMEM; }
+        h->io_bytes = need;
+    }
+    char* base = reinterpret_cast<char*>(h->io);
+    void *dx = base + x_off, *dy = base + y_off, *dz = z_out ? base + z_off : nullptr;
+    tsvd_status_t st = TSVD_OK;
+    cudaStream_t s = nullptr;
+    do {
+        if (cudaMemcpyAsync(dx, x, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+        st = tsvd_forward_ex(h, dx, h->N, dy, h->M, B, dtype, flags, dz, s);
+        if (st != TSVD_OK) break;
+        if (cudaMemcpyAsync(y, dy, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+        if (z_out && cudaMemcpyAsync(z_out, dz, z_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+            st = TSVD_E_CUDA; break;
+        }
+        if (cudaStreamSynchronize(s) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+    } while (0);
+    if (st != TSVD_OK) (void)cudaGetLastError();
+    return st;
+}

@@ -1,0 +1,127 @@
+// Internal definitions shared by the libtsvd translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <type_traits>
+#include <vector>
+
+#include "tsvd.h"
+
+// ---------------------------------------------------------------------------------------
+// Packed ternary format (2 bits per entry: bit0 = nonzero, bit1 = sign, code 2 never used;
+// +1 -> 1, -1 -> 3, 0 -> 0).  The paper fixes only "2 bits per element"; the arrangement
+// below is chosen for the kernels.
+//
+// A ternary matrix T [R, C] (R = output rows, C = contraction index; this is V [K,N]
+// and U [M,K] as they are) is padded to R_pad (multiple of 128) x C_pad (multiple of
+// 128) and cut into blocks of 128 rows x 64 columns.  Block (rt, cg) occupies 2 KiB at
+// unit index (rt * (C_pad/64) + cg) * 128; inside it row r (0..127) owns one 16-byte
+// unit = 4 words; word w covers columns cg*64 + 16*w .. +15.  Inside a word, entry e
+// (0..15) sits at bits [4e, 4e+1] for e < 8 and at bits [4(e-8)+2, 4(e-8)+3] for e >= 8,
+// so that (w & 0x33333333) and ((w >> 2) & 0x33333333) are directly byte-permute
+// selectors that expand eight entries each into int8 lanes.
+//
+// Consequences: a 128-row x 128-column MMA operand tile is 4 KiB contiguous; consecutive
+// rows of one 64-column group are consecutive 16-byte units (coalesced 128-bit loads when
+// a thread owns a row).
+// ---------------------------------------------------------------------------------------
+constexpr int TSVD_ROW_TILE = 128;
+constexpr int TSVD_COL_GROUP = 64;
+constexpr int TSVD_COL_PAD = 128;
+
+struct PackedMat {
+    uint4* units = nullptr;  // device
+    int R = 0, C = 0;        // logical
+    int R_pad = 0, C_pad = 0;
+    size_t n_units = 0;      // R_pad * C_pad / 64
+    unsigned long long nnz = 0;
+    size_t bytes() const { return n_units * sizeof(uint4); }
+};
+
+__host__ __device__ inline size_t tsvd_unit_index(int row, int col_group, int C_pad)
+{
+    return ((size_t)(row >> 7) * (size_t)(C_pad >> 6) + (size_t)col_group) * 128 + (size_t)(row & 127);
+}
+
+// bit position of entry e (0..15) inside its word
+__host__ __device__ inline int tsvd_entry_shift(int e) { return (e < 8) ? 4 * e : 4 * (e - 8) + 2; }
+
+// Expand eight 2-bit codes (selector nibbles, see above) to eight int8 values:
+// lo word = entries 0..3, hi word = entries 4..7 of the selector.
+__device__ __forceinline__ void tsvd_expand8(uint32_t sel, uint32_t& lo, uint32_t& hi)
+{
+    // byte table: code 0 -> 0x00, 1 -> 0x01, 2 -> 0x00, 3 -> 0xFF
+    const uint32_t table = 0xFF000100u;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(lo) : "r"(table), "r"(0u), "r"(sel));
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(table), "r"(0u), "r"(sel >> 16));
+}
+
+// Expand one packed word to sixteen int8 values (four 32-bit lanes, entries in order).
+__device__ __forceinline__ void tsvd_expand16(uint32_t w, uint32_t out[4])
+{
+    tsvd_expand8(w & 0x33333333u, out[0], out[1]);
+    tsvd_expand8((w >> 2) & 0x33333333u, out[2], out[3]);
+}
+
+// Event-pair recorder behind tsvd_profile_enable / tsvd_profile_read.
+struct StageProfiler {
+    bool on = false;
+    struct Pair { cudaEvent_t a, b; int stage; };
+    std::vector<Pair> pending;
+    float ms[TSVD_N_STAGES] = {0, 0, 0, 0};
+    unsigned launches[TSVD_N_STAGES] = {0, 0, 0, 0};
+    void begin(int stage, cudaStream_t s);
+    void end(cudaStream_t s);
+    void drain();
+};
+
+struct tsvd_handle_s {
+    int device = 0;
+    int M = 0, K = 0, N = 0;
+    PackedMat V;          // rows K, contraction N
+    PackedMat U;          // rows M, contraction K
+    float* S = nullptr;   // device, length V.R_pad (zero padded)
+    // scratch shared by all forwards on this handle
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    void* io = nullptr;   // device staging for the host-buffer entry point
+    size_t io_bytes = 0;
+    int* dev_status = nullptr;  // device error word
+    StageProfiler prof;
+};
+
+// launch accounting
+void tsvd_count_launch(unsigned n = 1);
+
+// pack.cu
+tsvd_status_t tsvd_pack_matrix(const int8_t* host, int R, int C, PackedMat* out, int* dev_flag);
+tsvd_status_t tsvd_unpack_matrix(const PackedMat& pm, int8_t* host);
+
+// simple.cu -- CUDA-core reference kernels
+struct ForwardArgs {
+    tsvd_handle_s* h;
+    const void* x;
+    int ldx;
+    void* y;
+    int ldy;
+    int B;
+    tsvd_dtype_t dtype;
+    bool out_f32;
+    void* z_out;
+    float* t;        // scratch [B][t_ld] fp32: S * (V x)
+    int t_ld;
+    cudaStream_t stream;
+};
+tsvd_status_t tsvd_forward_simple(const ForwardArgs& a);
+size_t tsvd_simple_ws_bytes(const tsvd_handle_s* h, int B);
+
+#define TSVD_CUDA_OK(expr)                            \
+    do {                                              \
+        cudaError_t _e = (expr);                      \
+        if (_e != cudaSuccess) {                      \
+            (void)cudaGetLastError();                 \
+            return (_e == cudaErrorMemoryAllocation) ? TSVD_E_NOMEM : TSVD_E_CUDA; \
+        }                                             \
+    } while (0)

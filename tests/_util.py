@@ -1,0 +1,92 @@
+"""Helpers for the GPU parity tests: run a case through the C ABI and compare with the CPU checker."""
+from __future__ import annotations
+
+import numpy as np
+
+import gen
+import oracle
+from gen import rng
+
+# Tolerances (stated for this map's outputs):
+#   int8 activations: z = V x bit-exact int32
+#   fp32 outputs:     max|y - y_ref| <= 1e-5 * max|y_ref|
+#   bf16 outputs:     |y - y_ref| <= 1e-2 * |y_ref| + 1e-3 per element
+F32_REL_MAX = 1e-5
+BF16_RTOL, BF16_ATOL = 1e-2, 1e-3
+
+
+def torch_x(case_x: np.ndarray, x_dtype: str):
+    import torch
+    if x_dtype == "bf16":
+        return torch.from_numpy(case_x.view(np.int16).copy()).cuda().view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(case_x)).cuda()
+
+
+def run_gpu(layer, x_np: np.ndarray, x_dtype: str, flags: int = 0, want_z: bool = True):
+    """Forward through TSVDLinear; returns (y as float64 numpy [B,M], z numpy or None, y_is_bf16)."""
+    import torch
+    from paper_2308_07641_b200 import TSVD_FLAG_OUT_F32
+    x = torch_x(x_np, x_dtype)
+    B = x.shape[0]
+    K = layer.info["K"]
+    z = None
+    if want_z:
+        z = torch.full((B, K), -12345, dtype=torch.int32 if x_dtype == "i8" else torch.float32,
+                       device="cuda")
+    y = layer.forward(x, flags=flags, z_out=z)
+    torch.cuda.synchronize()
+    y_bf16 = y.dtype == torch.bfloat16
+    y64 = y.float().double().cpu().numpy()
+    return y64, (z.cpu().numpy() if z is not None else None), y_bf16
+
+
+def oracle_x(x_np: np.ndarray, x_dtype: str) -> np.ndarray:
+    if x_dtype == "bf16":
+        return rng.bf16_bits_to_f32(x_np).astype(np.float64)
+    if x_dtype == "i8":
+        return x_np
+    return x_np.astype(np.float64)
+
+
+def check_outputs(y64: np.ndarray, z, ref: "oracle.OracleResult", x_dtype: str, y_bf16: bool, what=""):
+    """Apply the stated tolerances; returns a dict of error figures."""
+    err = np.abs(y64 - ref.y)
+    out = {}
+    if y_bf16:
+        tol = BF16_RTOL * np.abs(ref.y) + BF16_ATOL
+        bad = err > tol
+        out["violations"] = int(bad.sum())
+        out["worst_ratio"] = float((err / tol).max())
+        assert not bad.any(), (f"{what}: {bad.sum()} of {bad.size} bf16 outputs outside tolerance; "
+                               f"worst err/tol = {out['worst_ratio']:.3g}")
+    else:
+        scale = np.abs(ref.y).max()
+        out["max_err_over_max"] = float(err.max() / scale) if scale > 0 else float(err.max())
+        assert err.max() <= F32_REL_MAX * scale + (0.0 if scale > 0 else 0.0), \
+            f"{what}: max|y-y_ref| = {err.max():.3g} > 1e-5 * max|y_ref| = {F32_REL_MAX * scale:.3g}"
+    if z is not None:
+        if x_dtype == "i8":
+            assert z.dtype == np.int32
+            assert np.array_equal(z.astype(np.int64), ref.zraw), f"{what}: int32 z is not bit-exact"
+        else:
+            zs = max(1.0, np.abs(ref.zraw).max())
+            assert np.abs(z.astype(np.float64) - ref.zraw).max() <= 1e-6 * zs, f"{what}: z_out off"
+    return out
+
+
+def run_and_check(spec: "gen.CaseSpec", flags: int = 0, sample_tokens=None):
+    """Build the case, run it on the GPU at full batch, compare (all tokens, or a sample)."""
+    from paper_2308_07641_b200 import TSVDLinear
+    U, V, S = gen.make_weights(spec)
+    x = gen.make_x(spec)
+    layer = TSVDLinear(U, S, V)
+    try:
+        y64, z, y_bf16 = run_gpu(layer, x, spec.x_dtype, flags)
+    finally:
+        layer.close()
+    if sample_tokens is None:
+        idx = np.arange(spec.B)
+    else:
+        idx = np.asarray(sample_tokens)
+    ref = oracle.forward(U, S, V, oracle_x(x[idx], spec.x_dtype))
+    return check_outputs(y64[idx], None if z is None else z[idx], ref, spec.x_dtype, y_bf16, spec.name)

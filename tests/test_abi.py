@@ -1,0 +1,77 @@
+"""The C ABI without a GPU: the library loads, exports every declared symbol, and rejects bad
+arguments on the host before touching a device."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2308_07641_b200 import build
+    build.build()
+    from paper_2308_07641_b200 import binding as b
+    return b
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if not fn.endswith(".h"):
+            continue
+        text = open(os.path.join(ROOT, "include", fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(tsvd_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol(binding):
+    lib = binding.lib()
+    declared = _declared_symbols()
+    assert declared, "no declarations found"
+    for name in declared:
+        assert hasattr(lib, name), f"libtsvd.so does not export {name}"
+    assert declared == set(binding.EXPORTS)
+
+
+def test_strerror_covers_all_codes(binding):
+    seen = {binding.tsvd_strerror(i) for i in range(0, 9)}
+    assert len(seen) == 9 and "unknown status" not in seen
+    assert binding.tsvd_strerror(99) == "unknown status"
+
+
+def test_host_side_validation(binding):
+    lib = binding.lib()
+    h = ctypes.c_void_p()
+    U = np.zeros((2, 2), np.int8); S = np.zeros(2, np.float32); V = np.zeros((2, 2), np.int8)
+    assert lib.tsvd_pack(None, S.ctypes.data, V.ctypes.data, 2, 2, 2, 0, ctypes.byref(h)) == binding.TSVD_E_NULL
+    assert lib.tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, 2, 2, 2, 0, None) == binding.TSVD_E_NULL
+    assert lib.tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, 0, 2, 2, 0, ctypes.byref(h)) == binding.TSVD_E_SHAPE
+    assert lib.tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, 2, 2, 2, 7, ctypes.byref(h)) == binding.TSVD_E_DTYPE
+    assert h.value is None
+    assert lib.tsvd_forward(None, None, None, 1, 0, None) == binding.TSVD_E_NULL
+    assert lib.tsvd_info(None, None, None, None, None, None, None) == binding.TSVD_E_NULL
+    assert lib.tsvd_last_status(None) == binding.TSVD_E_NULL
+    lib.tsvd_destroy(None)  # no-op
+
+
+def test_no_cpu_fallback_without_device(binding):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    with pytest.raises(binding.TSVDError) as e:
+        binding.tsvd_pack(np.zeros((2, 2), np.int8), np.ones(2, np.float32), np.zeros((2, 2), np.int8))
+    assert e.value.status == binding.TSVD_E_CUDA
+
+
+def test_product_does_not_import_the_checker():
+    pkg = os.path.join(ROOT, "paper_2308_07641_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for fn in files:
+            if fn.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, fn)).read()
+                assert "oracle" not in text, f"{fn} mentions the checker"

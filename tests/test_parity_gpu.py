@@ -1,0 +1,172 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU checker on the same
+seeded inputs.  Small cases are compared element by element over every token; the full-size
+configurations are compared on sampled token columns (columns are independent, so the checker
+computes each sampled column completely)."""
+import numpy as np
+import pytest
+
+import gen
+import oracle
+from tests import _util
+
+pytestmark = pytest.mark.gpu
+
+C = gen.CONFIGS
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2308_07641_b200 import build
+    build.build()
+
+
+def test_pack_roundtrip_and_info():
+    from paper_2308_07641_b200 import binding
+    for (M, K, N, d) in [(1, 1, 1, 1.0), (130, 63, 345, 0.3), (256, 256, 256, 0.3), (1000, 2415, 96, 0.1)]:
+        spec = gen.scaled(C["cfg1"], M=M, K=K, N=N, B=1, density=d, seed=77)
+        U, V, S = gen.make_weights(spec)
+        h = binding.tsvd_pack(U, S, V)
+        try:
+            U2, S2, V2 = binding.tsvd_unpack(h)
+            assert np.array_equal(U, U2) and np.array_equal(V, V2) and np.array_equal(S, S2)
+            info = binding.tsvd_info(h)
+            assert (info["M"], info["K"], info["N"]) == (M, K, N)
+            assert abs(info["density_u"] - np.count_nonzero(U) / U.size) < 1e-12
+            assert abs(info["density_v"] - np.count_nonzero(V) / V.size) < 1e-12
+            rp = lambda v: (v + 127) // 128 * 128
+            assert info["packed_bytes"] == (rp(M) * rp(K) + rp(K) * rp(N)) // 4 + 4 * K
+        finally:
+            binding.tsvd_destroy(h)
+
+
+def test_pack_rejects_non_ternary():
+    from paper_2308_07641_b200 import binding
+    U = np.zeros((4, 4), np.int8); V = np.zeros((4, 4), np.int8); S = np.ones(4, np.float32)
+    V[2, 3] = 2
+    with pytest.raises(binding.TSVDError) as e:
+        binding.tsvd_pack(U, S, V)
+    assert e.value.status == binding.TSVD_E_VALUE
+    V[2, 3] = 0; U[0, 0] = -2
+    with pytest.raises(binding.TSVDError) as e:
+        binding.tsvd_pack(U, S, V)
+    assert e.value.status == binding.TSVD_E_VALUE
+
+
+def test_forward_argument_errors():
+    import torch
+    from paper_2308_07641_b200 import binding
+    U = np.zeros((4, 4), np.int8); V = np.zeros((4, 4), np.int8); S = np.ones(4, np.float32)
+    h = binding.tsvd_pack(U, S, V)
+    try:
+        x = torch.zeros(64, device="cuda"); y = torch.zeros(64, device="cuda")
+        L = binding.lib()
+        assert L.tsvd_forward(h, x.data_ptr(), y.data_ptr(), 0, 0, None) == binding.TSVD_E_SHAPE
+        assert L.tsvd_forward(h, x.data_ptr(), y.data_ptr(), 1, 9, None) == binding.TSVD_E_DTYPE
+        assert L.tsvd_forward(h, x.data_ptr() + 4, y.data_ptr(), 1, 0, None) == binding.TSVD_E_ALIGN
+        assert L.tsvd_forward_ex(h, x.data_ptr(), 3, y.data_ptr(), 4, 1, 0, 0, None, None) == binding.TSVD_E_SHAPE
+        assert L.tsvd_forward_ex(h, x.data_ptr(), 4, y.data_ptr(), 4, 1, 0, 0x30, None, None) == binding.TSVD_E_DTYPE
+        assert L.tsvd_forward(h, None, y.data_ptr(), 1, 0, None) == binding.TSVD_E_NULL
+        assert binding.tsvd_last_status(h) == binding.TSVD_OK
+    finally:
+        binding.tsvd_destroy(h)
+
+
+# ---- small cases, every element --------------------------------------------------------------
+SMALL = [
+    C["cfg1"],
+    gen.scaled(C["cfg1"], name="tiny_1x1x1", M=1, N=1, K=1, B=1, density=1.0),
+    gen.scaled(C["cfg1"], name="ragged_f32", M=300, N=333, K=200, B=13, seed=11),
+    gen.scaled(C["cfg2"], name="cfg2_small", M=384, N=200, K=130, B=70),
+    gen.scaled(C["cfg2"], name="ragged_bf16", M=1000, N=345, K=63, B=37, seed=12),
+    gen.scaled(C["cfg3_b4"], name="cfg3_small", M=512, N=640, K=384),
+    gen.scaled(C["cfg3_b1"], name="cfg3_small_b1", M=512, N=640, K=384),
+    gen.scaled(C["cfg4"], name="cfg4_small", M=640, N=256, K=256, B=160),
+    gen.scaled(C["cfg5_d05"], name="cfg5_small_d05", M=256, N=384, K=512, B=40),
+    gen.scaled(C["cfg5_d20"], name="cfg5_small_d20", M=256, N=384, K=512, B=40),
+    gen.scaled(C["cfg5_d50"], name="cfg5_small_d50", M=129, N=257, K=255, B=33),
+    gen.scaled(C["cfg2"], name="all_zero", M=140, N=130, K=150, B=9, density=0.0),
+    gen.scaled(C["cfg5_d50"], name="all_nonzero_i8", M=140, N=130, K=150, B=9, density=1.0),
+    gen.scaled(C["cfg2"], name="row_density_varies", M=260, N=300, K=280, B=20, row_density_spread=0.9),
+]
+
+
+@pytest.mark.parametrize("spec", SMALL, ids=lambda s: s.name)
+def test_small_cases_every_element(spec):
+    _util.run_and_check(spec)
+
+
+def test_out_f32_flag_and_strides():
+    """bf16 activations with fp32 output, and leading dimensions larger than the row length."""
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear, TSVD_FLAG_OUT_F32
+    spec = gen.scaled(C["cfg2"], name="strided", M=200, N=150, K=170, B=11, seed=21)
+    U, V, S = gen.make_weights(spec)
+    x = gen.make_x(spec)
+    layer = TSVDLinear(U, S, V)
+    try:
+        xt = _util.torch_x(x, "bf16")
+        xbig = torch.zeros((spec.B, spec.N + 10), dtype=torch.bfloat16, device="cuda")
+        xbig[:, :spec.N] = xt
+        ybig = torch.full((spec.B, spec.M + 24), 7.0, dtype=torch.float32, device="cuda")
+        layer.forward(xbig[:, :spec.N], out=ybig[:, :spec.M], flags=TSVD_FLAG_OUT_F32)
+        torch.cuda.synchronize()
+        ref = oracle.forward(U, S, V, _util.oracle_x(x, "bf16"))
+        y = ybig[:, :spec.M].double().cpu().numpy()
+        assert np.abs(y - ref.y).max() <= 1e-5 * np.abs(ref.y).max()
+        assert torch.all(ybig[:, spec.M:] == 7.0)          # padding untouched
+    finally:
+        layer.close()
+
+
+def test_repeatable_and_handle_reuse():
+    """Two calls on one handle with different batch sizes; int32 z identical run to run."""
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear
+    spec = gen.scaled(C["cfg5_d20"], name="reuse", M=200, N=300, K=260, B=50)
+    U, V, S = gen.make_weights(spec)
+    x = gen.make_x(spec)
+    layer = TSVDLinear(U, S, V)
+    try:
+        y1, z1, _ = _util.run_gpu(layer, x[:7], "i8")
+        y2, z2, _ = _util.run_gpu(layer, x, "i8")
+        y3, z3, _ = _util.run_gpu(layer, x, "i8")
+        assert np.array_equal(z2, z3) and np.array_equal(z1, z2[:7])
+        ref = oracle.forward(U, S, V, x)
+        _util.check_outputs(y2, z2, ref, "i8", False, "reuse")
+        assert np.abs(y1 - y2[:7]).max() <= 1e-5 * np.abs(ref.y).max()
+    finally:
+        layer.close()
+
+
+def test_host_buffer_entry_point():
+    from paper_2308_07641_b200 import binding
+    spec = gen.scaled(C["cfg1"], name="host", M=100, N=90, K=80, B=5, seed=31)
+    U, V, S = gen.make_weights(spec)
+    x = gen.make_x(spec)
+    h = binding.tsvd_pack(U, S, V)
+    try:
+        y = np.zeros((spec.B, spec.M), np.float32)
+        z = np.zeros((spec.B, spec.K), np.float32)
+        binding.tsvd_forward_host(h, x.ctypes.data, y.ctypes.data, spec.B, binding.TSVD_F32, 0, z.ctypes.data)
+        ref = oracle.forward(U, S, V, x.astype(np.float64))
+        _util.check_outputs(y.astype(np.float64), z, ref, "f32", False, "host")
+    finally:
+        binding.tsvd_destroy(h)
+
+
+# ---- full-size configurations, sampled token columns -------------------------------------------
+FULL = [
+    (C["cfg2"], [0, 1, 777, 2048, 4095]),
+    (C["cfg3_b1"], None),
+    (C["cfg3_b4"], None),
+    (C["cfg3_b16"], None),
+    (C["cfg4"], [0, 1023, 2047]),
+    (C["cfg5_d05"], [0, 100, 255]),
+    (C["cfg5_d20"], [0, 100, 255]),
+    (C["cfg5_d50"], [0, 100, 255]),
+]
+
+
+@pytest.mark.parametrize("spec,sample", FULL, ids=lambda v: v.name if hasattr(v, "name") else None)
+def test_full_size_sampled(spec, sample):
+    _util.run_and_check(spec, sample_tokens=sample)
