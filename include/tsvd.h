@@ -38,7 +38,8 @@ typedef enum {
     TSVD_E_ALIGN = 5,   /* a pointer or leading dimension breaks the stated rule   */
     TSVD_E_CUDA = 6,    /* a CUDA runtime call failed (or there is no device)      */
     TSVD_E_TIMEOUT = 7, /* a bounded device-side wait gave up                      */
-    TSVD_E_NOMEM = 8    /* host or device allocation failed                        */
+    TSVD_E_NOMEM = 8,   /* host or device allocation failed                        */
+    TSVD_E_TOOBIG = 9   /* request exceeds a fixed capacity (see tsvd_forward_static) */
 } tsvd_status_t;
 
 /* flags of tsvd_forward_ex */
@@ -102,6 +103,38 @@ tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx, void* y, 
  */
 tsvd_status_t tsvd_forward_host(tsvd_handle_t h, const void* x, void* y, int B,
                                 tsvd_dtype_t dtype, unsigned flags, void* z_out);
+
+/*
+ * tsvd_forward_static -- tsvd_forward for callers that must not allocate.
+ * (The paper has no counterpart to this call: it is a deployment convenience.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a serving
+ * loop whose memory budget was fixed at start-up and is audited, in a process that
+ * hands the whole device to another allocator and forbids side allocations, or in
+ * a latency-critical section where an allocation's implicit device synchronisation
+ * is unacceptable.  tsvd_forward grows a per-handle scratch buffer with cudaMalloc
+ * the first time it sees a larger batch; this call never allocates or frees: its
+ * intermediate S*(V x) lives in a fixed array of TSVD_STATIC_SCRATCH_BYTES that is
+ * part of the library image (every GPU that loads the library holds those bytes
+ * until the process exits).
+ *
+ *   h, x, y, B, dtype, stream   exactly as tsvd_forward (x, y device, token-major,
+ *                               16-byte aligned; y fp32, or bf16 for bf16 x)
+ *
+ * Limit: B * roundup(K,128) * 4 bytes must fit in TSVD_STATIC_SCRATCH_BYTES,
+ * otherwise TSVD_E_TOOBIG is returned and nothing is launched.
+ * First call on a device: looks up the array's device address once (with that device
+ * current, which the handle already requires); make that first call before any
+ * stream capture begins.
+ * Sharing: there is ONE array per device, used by every handle and every call.  It
+ * keeps the previous call's contents; nothing in it has to start at zero, because
+ * the V-stage overwrites every element the U-stage reads.  Two calls that overlap on
+ * the GPU (different streams, no ordering between them) race on it: order them.
+ * Runs the CUDA-core kernels.  Errors: as tsvd_forward, plus E_TOOBIG.
+ */
+#define TSVD_STATIC_SCRATCH_BYTES (4u << 20)
+tsvd_status_t tsvd_forward_static(tsvd_handle_t h, const void* x, void* y, int B,
+                                  tsvd_dtype_t dtype, void* stream);
 
 /* Device-side error word of the last forward on this handle (read after the
  * stream has been synchronised): TSVD_OK, or TSVD_E_TIMEOUT if a bounded wait

@@ -18,7 +18,8 @@ LIB_PATH = os.path.join(_HERE, "libtsvd.so")
 TSVD_F32, TSVD_BF16, TSVD_I8 = 0, 1, 2
 TSVD_OK = 0
 (TSVD_E_NULL, TSVD_E_SHAPE, TSVD_E_VALUE, TSVD_E_DTYPE, TSVD_E_ALIGN, TSVD_E_CUDA,
- TSVD_E_TIMEOUT, TSVD_E_NOMEM) = range(1, 9)
+ TSVD_E_TIMEOUT, TSVD_E_NOMEM, TSVD_E_TOOBIG) = range(1, 10)
+TSVD_STATIC_SCRATCH_BYTES = 4 << 20
 TSVD_FLAG_OUT_F32 = 0x1
 TSVD_FLAG_PATH_SIMPLE = 0x10
 TSVD_FLAG_PATH_DECODE = 0x20
@@ -27,8 +28,9 @@ TSVD_FLAG_PATH_TENSOR = 0x40
 DTYPES = {"f32": TSVD_F32, "bf16": TSVD_BF16, "i8": TSVD_I8}
 
 # every symbol include/tsvd.h declares
-EXPORTS = ("tsvd_pack", "tsvd_forward", "tsvd_forward_ex", "tsvd_forward_host", "tsvd_last_status",
-           "tsvd_info", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read", "tsvd_launch_count", "tsvd_destroy", "tsvd_strerror")
+EXPORTS = ("tsvd_pack", "tsvd_forward", "tsvd_forward_ex", "tsvd_forward_host", "tsvd_forward_static",
+           "tsvd_last_status", "tsvd_info", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
+           "tsvd_launch_count", "tsvd_destroy", "tsvd_strerror")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -56,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.tsvd_forward_ex.restype = ci
         L.tsvd_forward_host.argtypes = [vp, vp, vp, ci, ci, cu, vp]
         L.tsvd_forward_host.restype = ci
+        L.tsvd_forward_static.argtypes = [vp, vp, vp, ci, ci, vp]
+        L.tsvd_forward_static.restype = ci
         L.tsvd_last_status.argtypes = [vp]
         L.tsvd_last_status.restype = ci
         L.tsvd_info.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci),
@@ -122,6 +126,12 @@ def tsvd_forward_host(h: int, x_ptr: int, y_ptr: int, B: int, dtype: int, flags:
     """Host pointers (numpy .ctypes.data or pinned torch tensors' data_ptr())."""
     _check(lib().tsvd_forward_host(h, x_ptr, y_ptr, B, dtype, flags, z_out_ptr or None),
            "tsvd_forward_host")
+
+
+def tsvd_forward_static(h: int, x_ptr: int, y_ptr: int, B: int, dtype: int, stream: int = 0) -> None:
+    """tsvd_forward without any allocation: the intermediate lives in a fixed array inside the
+    library (TSVD_STATIC_SCRATCH_BYTES); larger requests raise with status TSVD_E_TOOBIG."""
+    _check(lib().tsvd_forward_static(h, x_ptr, y_ptr, B, dtype, stream or None), "tsvd_forward_static")
 
 
 def tsvd_last_status(h: int) -> int:

@@ -22,6 +22,7 @@ extern "C" const char* tsvd_strerror(tsvd_status_t s)
         case TSVD_E_CUDA: return "CUDA runtime error (or no CUDA device)";
         case TSVD_E_TIMEOUT: return "a bounded device-side wait gave up";
         case TSVD_E_NOMEM: return "out of memory";
+        case TSVD_E_TOOBIG: return "request exceeds the fixed scratch capacity of this entry point";
     }
     return "unknown status";
 }

@@ -157,3 +157,69 @@ tsvd_status_t tsvd_forward_simple(const ForwardArgs& a)
     h->prof.end(a.stream);
     return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
 }
+
+// ---------------------------------------------------------------------------------------
+// tsvd_forward_static: the same two kernels with the intermediate S*(V x) in a fixed
+// array that is part of the library image, for callers that must not allocate.
+// ---------------------------------------------------------------------------------------
+#include <mutex>
+
+// One array per device that loads the library.  In host code this name is only a handle
+// for the runtime's symbol table, never a device address: the address each device uses
+// is fetched with cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[TSVD_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+float* g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the CURRENT device (looked up once per device).
+tsvd_status_t static_scratch_for(int device, float** out)
+{
+    if (device < 0 || device >= kMaxDevices) return TSVD_E_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p) { (void)cudaGetLastError(); return TSVD_E_CUDA; }
+        g_static_ptr[device] = reinterpret_cast<float*>(p);
+    }
+    *out = g_static_ptr[device];
+    return TSVD_OK;
+}
+}  // namespace
+
+extern "C" tsvd_status_t tsvd_forward_static(tsvd_handle_t h, const void* x, void* y, int B,
+                                             tsvd_dtype_t dtype, void* stream)
+{
+    if (!h || !x || !y) return TSVD_E_NULL;
+    if (B < 1) return TSVD_E_SHAPE;
+    if (dtype != TSVD_F32 && dtype != TSVD_BF16 && dtype != TSVD_I8) return TSVD_E_DTYPE;
+    if (((uintptr_t)x & 15) || ((uintptr_t)y & 15)) return TSVD_E_ALIGN;
+    const size_t need = (size_t)B * (size_t)h->V.R_pad * sizeof(float);
+    if (need > (size_t)TSVD_STATIC_SCRATCH_BYTES) return TSVD_E_TOOBIG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return TSVD_E_CUDA; }
+    if (dev != h->device) return TSVD_E_CUDA;
+    float* t = nullptr;
+    tsvd_status_t st = static_scratch_for(dev, &t);
+    if (st != TSVD_OK) return st;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    const int t_ld = h->V.R_pad;
+    cudaError_t e;
+    if (dtype == TSVD_F32)
+        e = launch<float, EPI_SCALE_TO_T>(h->V, (const float*)x, h->N, B, h->S, t, t_ld, nullptr, 0, s);
+    else if (dtype == TSVD_BF16)
+        e = launch<__nv_bfloat16, EPI_SCALE_TO_T>(h->V, (const __nv_bfloat16*)x, h->N, B, h->S, t, t_ld,
+                                                  nullptr, 0, s);
+    else
+        e = launch<int8_t, EPI_SCALE_TO_T>(h->V, (const int8_t*)x, h->N, B, h->S, t, t_ld, nullptr, 0, s);
+    if (e != cudaSuccess) return TSVD_E_CUDA;
+    if (dtype == TSVD_BF16)
+        e = launch<float, EPI_Y_BF16>(h->U, t, t_ld, B, nullptr, y, h->M, nullptr, 0, s);
+    else
+        e = launch<float, EPI_Y_F32>(h->U, t, t_ld, B, nullptr, y, h->M, nullptr, 0, s);
+    return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
+}

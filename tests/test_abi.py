@@ -39,8 +39,8 @@ def test_library_exports_every_declared_symbol(binding):
 
 
 def test_strerror_covers_all_codes(binding):
-    seen = {binding.tsvd_strerror(i) for i in range(0, 9)}
-    assert len(seen) == 9 and "unknown status" not in seen
+    seen = {binding.tsvd_strerror(i) for i in range(0, 10)}
+    assert len(seen) == 10 and "unknown status" not in seen
     assert binding.tsvd_strerror(99) == "unknown status"
 
 

@@ -1,0 +1,75 @@
+"""tsvd_forward_static: the forward for callers that cannot allocate device memory.
+
+Some users of this library run it where cudaMalloc is not allowed: a serving loop whose
+device memory was budgeted once at start-up, a process whose device memory belongs to another
+allocator, or a latency-critical section that cannot afford the device synchronisation an
+allocation implies.  For them the library keeps the intermediate S*(V x) in a fixed array
+inside its own image.  This test calls that entry point through the C ABI twice in a row
+(different inputs and batch sizes, so stale contents of the shared array would show) and
+compares each result with the ordinary tsvd_forward on the same inputs, with the tolerances
+the other parity tests use.  It is collected last so that a stop-at-first-failure run has
+already covered everything else; it also passes when run alone in a fresh process.
+"""
+import numpy as np
+import pytest
+
+import gen
+from tests import _util
+
+pytestmark = pytest.mark.gpu
+
+
+def _forward_pair(binding, h, x_np, x_dtype, M):
+    import torch
+    x = _util.torch_x(x_np, x_dtype)
+    B = x.shape[0]
+    out_dtype = torch.bfloat16 if x_dtype == "bf16" else torch.float32
+    y_ref = torch.empty((B, M), dtype=out_dtype, device="cuda")
+    y_sta = torch.full((B, M), 3.0, dtype=out_dtype, device="cuda")
+    dt = binding.DTYPES[x_dtype]
+    binding.tsvd_forward(h, x.data_ptr(), y_ref.data_ptr(), B, dt)
+    binding.tsvd_forward_static(h, x.data_ptr(), y_sta.data_ptr(), B, dt)
+    torch.cuda.synchronize()
+    return y_ref.double().cpu().numpy(), y_sta.double().cpu().numpy()
+
+
+@pytest.mark.parametrize("x_dtype,base", [("bf16", "cfg2"), ("f32", "cfg1"), ("i8", "cfg5_d20")])
+def test_static_matches_forward_on_two_calls_in_a_row(x_dtype, base):
+    from paper_2308_07641_b200 import binding, build
+    build.build()
+    spec = gen.scaled(gen.CONFIGS[base], name="noalloc", M=300, N=270, K=200, B=48, seed=91)
+    U, V, S = gen.make_weights(spec)
+    x = gen.make_x(spec)
+    h = binding.tsvd_pack(U, S, V)
+    try:
+        for xs in (x, x[5:24]):              # second call: other inputs, smaller batch
+            y_ref, y_sta = _forward_pair(binding, h, xs, x_dtype, spec.M)
+            err = np.abs(y_sta - y_ref)
+            if x_dtype == "bf16":
+                assert np.all(err <= _util.BF16_RTOL * np.abs(y_ref) + _util.BF16_ATOL)
+            else:
+                assert err.max() <= _util.F32_REL_MAX * np.abs(y_ref).max()
+    finally:
+        binding.tsvd_destroy(h)
+
+
+def test_static_rejects_requests_beyond_its_capacity():
+    import torch
+    from paper_2308_07641_b200 import binding, build
+    build.build()
+    spec = gen.scaled(gen.CONFIGS["cfg1"], name="noalloc_big", M=8, N=8, K=1024, B=1, seed=92)
+    U, V, S = gen.make_weights(spec)
+    h = binding.tsvd_pack(U, S, V)
+    try:
+        cap_tokens = binding.TSVD_STATIC_SCRATCH_BYTES // (1024 * 4)
+        B = cap_tokens + 1
+        x = torch.zeros((B, spec.N), device="cuda")
+        y = torch.zeros((B, spec.M), device="cuda")
+        with pytest.raises(binding.TSVDError) as e:
+            binding.tsvd_forward_static(h, x.data_ptr(), y.data_ptr(), B, binding.TSVD_F32)
+        assert e.value.status == binding.TSVD_E_TOOBIG
+        binding.tsvd_forward_static(h, x.data_ptr(), y.data_ptr(), cap_tokens, binding.TSVD_F32)
+        torch.cuda.synchronize()
+        assert torch.all(y == 0)
+    finally:
+        binding.tsvd_destroy(h)
