@@ -228,6 +228,15 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     a.z_out = z_out;
     a.stream = (cudaStream_t)stream;
 
+    // dispatch: batches go to the tensor cores, a handful of columns to the CUDA-core kernels
+    bool use_tensor = B >= 32;
+    if (path == TSVD_FLAG_PATH_TENSOR) use_tensor = true;
+    if (path == TSVD_FLAG_PATH_SIMPLE || path == TSVD_FLAG_PATH_DECODE) use_tensor = false;
+    if (use_tensor) {
+        tsvd_status_t st = ensure_ws(h, tsvd_tensor_ws_bytes(h, B, dtype));
+        if (st != TSVD_OK) return st;
+        return tsvd_forward_tensor(a, h->ws);
+    }
     tsvd_status_t st = ensure_ws(h, tsvd_simple_ws_bytes(h, B));
     if (st != TSVD_OK) return st;
     a.t = reinterpret_cast<float*>(h->ws);

@@ -117,6 +117,10 @@ struct ForwardArgs {
 tsvd_status_t tsvd_forward_simple(const ForwardArgs& a);
 size_t tsvd_simple_ws_bytes(const tsvd_handle_s* h, int B);
 
+// tensor.cu -- tcgen05 path
+tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws);
+size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt);
+
 #define TSVD_CUDA_OK(expr)                            \
     do {                                              \
         cudaError_t _e = (expr);                      \

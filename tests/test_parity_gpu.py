@@ -90,9 +90,13 @@ SMALL = [
 ]
 
 
+PATHS = {"simple": 0x10, "tensor": 0x40}
+
+
+@pytest.mark.parametrize("path", sorted(PATHS))
 @pytest.mark.parametrize("spec", SMALL, ids=lambda s: s.name)
-def test_small_cases_every_element(spec):
-    _util.run_and_check(spec)
+def test_small_cases_every_element(spec, path):
+    _util.run_and_check(spec, flags=PATHS[path])
 
 
 def test_out_f32_flag_and_strides():
