@@ -289,22 +289,47 @@ def main():
 
     # roofline of the dominant kernel
     peaks, peaks_src = load_peaks()
+    plan = binding.tsvd_plan(layer.handle, spec.B, binding.DTYPES[spec.x_dtype], flags)
     dom = int(np.argmax(stage_ms))
     dom_ms = stage_ms[dom] / max(1, stage_n[dom])
-    rows, contr = ((spec.K, spec.N) if dom == 1 else (spec.M, spec.K))
-    # executed dense operations of that launch: 2 * rows * contraction * columns
-    dense_flop = 2.0 * rows * contr * spec.B
-    achieved_tf = dense_flop / (dom_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved_tf,
-                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"],
-                "traffic": None, "peak_source": f"bf16 burst, {peaks_src} (of measured)",
-                "ms_per_launch": dom_ms, "flop_per_launch": dense_flop,
-                "stage_ms_per_step": {n: m / args.steps for n, m in zip(binding.STAGE_NAMES, stage_ms)}}
+    pad = lambda v: (v + 127) // 128 * 128
+    if dom in (1, 3):
+        rows, contr = ((pad(spec.K), pad(spec.N)) if dom == 1 else (pad(spec.M), pad(spec.K)))
+        digits = max(1, plan["digits_x"] if dom == 1 else plan["digits_t"])
+        # executed dense operations of that launch: 2 * rows * contraction * tokens * digits
+        ops = 2.0 * rows * contr * spec.B * digits
+        if plan["path"] == "tensor":
+            peak, peak_note = peaks["bf16_tflops"] * INT8_OVER_BF16, "int8 = measured bf16 burst x 2 (nominal ratio)"
+        else:
+            peak, peak_note = peaks["bf16_tflops"], "measured bf16 burst"
+        achieved = ops / (dom_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved, "peak": peak,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "peak_source": f"{peak_note}; {peaks_src} (of measured)", "ops_per_launch": ops,
+                    "digits": digits}
+    else:
+        # a digit-conversion pass dominates: it is bound by HBM traffic (read values, write digits)
+        elems = spec.B * (pad(spec.N) if dom == 0 else pad(spec.K))
+        in_bytes = {"f32": 4, "bf16": 2, "i8": 1}[spec.x_dtype] if dom == 0 else 4
+        nd = plan["digits_x"] if dom == 0 else plan["digits_t"]
+        byts = float(elems) * (in_bytes + nd)
+        achieved = byts / (dom_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved,
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                    "traffic": None, "peak_source": f"{peaks_src} (of measured)", "bytes_per_launch": byts}
+    roofline["ms_per_launch"] = dom_ms
+    roofline["stage_ms_per_step"] = {n: m / args.steps for n, m in zip(binding.STAGE_NAMES, stage_ms)}
+    roofline["plan"] = plan
+    # whole-step tensor figure: all executed tensor operations over the whole step time
+    if plan["path"] == "tensor":
+        all_ops = 2.0 * spec.B * (pad(spec.K) * pad(spec.N) * plan["digits_x"] + pad(spec.M) * pad(spec.K) * plan["digits_t"])
+        roofline["step_tensor_frac"] = all_ops / (ms_per_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * INT8_OVER_BF16)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": {"f32": "f32", "bf16": "f32", "i8": "int32"}[spec.x_dtype], "data": "synthetic",
+            "dtype": "int32" if plan["path"] == "tensor" else {"f32": "f32", "bf16": "f32", "i8": "int32"}[spec.x_dtype],
+            "data": "synthetic",
             "config": workload_config(spec, "flushed between steps (256 MiB memset)"),
             "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks,
             "packed_bytes": info["packed_bytes"],

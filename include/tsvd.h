@@ -151,6 +151,17 @@ tsvd_status_t tsvd_info(tsvd_handle_t h, int* M, int* K, int* N, size_t* packed_
 tsvd_status_t tsvd_unpack(tsvd_handle_t h, int8_t* U, float* S, int8_t* V);
 
 /*
+ * tsvd_plan -- which kernels a forward with these arguments would run (no launch).
+ *   path  receives TSVD_FLAG_PATH_SIMPLE, _DECODE or _TENSOR
+ *   digits_x, digits_t  receive the number of signed 8-bit digits the tensor-core path
+ *   uses for the activations and for S*(V x) (0 on the other paths).  Executed tensor
+ *   operations per forward = 2*B*(K*N*digits_x + M*K*digits_t) on the padded shapes; the
+ *   paper's own count is additions at the nonzeros only (Table S1).
+ */
+tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, unsigned flags, unsigned* path,
+                        int* digits_x, int* digits_t);
+
+/*
  * Per-stage device timing (measurement support; the paper reports operation counts
  * per stage in Table S1 and no timings).  While enabled, every forward on the handle
  * records CUDA events on its own stream around each kernel it launches.

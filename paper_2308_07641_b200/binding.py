@@ -29,7 +29,7 @@ DTYPES = {"f32": TSVD_F32, "bf16": TSVD_BF16, "i8": TSVD_I8}
 
 # every symbol include/tsvd.h declares
 EXPORTS = ("tsvd_pack", "tsvd_forward", "tsvd_forward_ex", "tsvd_forward_host", "tsvd_forward_static",
-           "tsvd_last_status", "tsvd_info", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
+           "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
            "tsvd_launch_count", "tsvd_destroy", "tsvd_strerror")
 
 _lib: Optional[ctypes.CDLL] = None
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.tsvd_info.restype = ci
         L.tsvd_unpack.argtypes = [vp, vp, vp, vp]
         L.tsvd_unpack.restype = ci
+        L.tsvd_plan.argtypes = [vp, ci, ci, cu, ctypes.POINTER(cu), ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.tsvd_plan.restype = ci
         L.tsvd_profile_enable.argtypes = [vp, ci]
         L.tsvd_profile_enable.restype = ci
         L.tsvd_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(cu)]
@@ -155,6 +157,16 @@ def tsvd_unpack(h: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     S = np.empty(info["K"], dtype=np.float32)
     _check(lib().tsvd_unpack(h, U.ctypes.data, S.ctypes.data, V.ctypes.data), "tsvd_unpack")
     return U, S, V
+
+
+def tsvd_plan(h: int, B: int, dtype: int, flags: int = 0) -> dict:
+    """The dispatch decision for a forward with these arguments (nothing is launched)."""
+    path, dx, dt = ctypes.c_uint(), ctypes.c_int(), ctypes.c_int()
+    _check(lib().tsvd_plan(h, B, dtype, flags, ctypes.byref(path), ctypes.byref(dx), ctypes.byref(dt)),
+           "tsvd_plan")
+    name = {TSVD_FLAG_PATH_SIMPLE: "simple", TSVD_FLAG_PATH_DECODE: "decode",
+            TSVD_FLAG_PATH_TENSOR: "tensor"}[path.value]
+    return {"path": name, "digits_x": dx.value, "digits_t": dt.value}
 
 
 N_STAGES = 4

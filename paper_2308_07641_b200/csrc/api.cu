@@ -204,6 +204,30 @@ static tsvd_status_t ensure_ws(tsvd_handle_s* h, size_t bytes)
     return TSVD_OK;
 }
 
+// The dispatch rule shared by tsvd_plan and tsvd_forward_ex: batches go to the tensor cores,
+// a handful of columns to the CUDA-core kernels.
+static unsigned choose_path(int B, unsigned forced)
+{
+    if (forced == TSVD_FLAG_PATH_TENSOR) return TSVD_FLAG_PATH_TENSOR;
+    if (forced == TSVD_FLAG_PATH_SIMPLE || forced == TSVD_FLAG_PATH_DECODE) return TSVD_FLAG_PATH_SIMPLE;
+    return B >= 32 ? TSVD_FLAG_PATH_TENSOR : TSVD_FLAG_PATH_SIMPLE;
+}
+
+extern "C" tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, unsigned flags, unsigned* path,
+                                   int* digits_x, int* digits_t)
+{
+    if (!h) return TSVD_E_NULL;
+    if (B < 1) return TSVD_E_SHAPE;
+    if (dtype_size(dtype) == 0) return TSVD_E_DTYPE;
+    const unsigned forced = flags & (TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR);
+    if (forced & (forced - 1)) return TSVD_E_DTYPE;
+    const unsigned p = choose_path(B, forced);
+    if (path) *path = p;
+    if (digits_x) *digits_x = (p == TSVD_FLAG_PATH_TENSOR) ? tsvd_tensor_digits_x(dtype) : 0;
+    if (digits_t) *digits_t = (p == TSVD_FLAG_PATH_TENSOR) ? tsvd_tensor_digits_t() : 0;
+    return TSVD_OK;
+}
+
 extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx, void* y, int ldy, int B,
                                          tsvd_dtype_t dtype, unsigned flags, void* z_out, void* stream)
 {
@@ -228,11 +252,7 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     a.z_out = z_out;
     a.stream = (cudaStream_t)stream;
 
-    // dispatch: batches go to the tensor cores, a handful of columns to the CUDA-core kernels
-    bool use_tensor = B >= 32;
-    if (path == TSVD_FLAG_PATH_TENSOR) use_tensor = true;
-    if (path == TSVD_FLAG_PATH_SIMPLE || path == TSVD_FLAG_PATH_DECODE) use_tensor = false;
-    if (use_tensor) {
+    if (choose_path(B, path) == TSVD_FLAG_PATH_TENSOR) {
         tsvd_status_t st = ensure_ws(h, tsvd_tensor_ws_bytes(h, B, dtype));
         if (st != TSVD_OK) return st;
         return tsvd_forward_tensor(a, h->ws);

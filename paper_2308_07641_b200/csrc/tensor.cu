@@ -22,8 +22,8 @@ constexpr int BLOCK_R = 128;   // ternary rows per CTA tile = MMA M
 constexpr int BLOCK_C = 128;   // contraction elements per pipeline stage (one 128-byte swizzle row)
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
 constexpr int STAGES = 4;
-constexpr int TMEM_COLS = 256;
-constexpr int GEMM_THREADS = 192;  // warp 0: copies, warp 1: MMA issue, warps 2..5: expand + epilogue
+constexpr int TMEM_COLS = 512;   // two 256-column accumulator buffers
+constexpr int GEMM_THREADS = 320;  // warp 0: copies, 1: MMA issue, 2..5: expand, 6..9: epilogue
 
 // tokens per tile for nd digits: the MMA N extent is nd * tokens <= 256 and a multiple of 16
 __host__ __device__ constexpr int tokens_per_tile(int nd) { return nd == 1 ? 256 : nd == 2 ? 128 : nd == 3 ? 80 : 64; }
@@ -47,77 +47,109 @@ template <> __device__ __forceinline__ float to_float<float>(float v) { return v
 template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <> __device__ __forceinline__ float to_float<int8_t>(int8_t v) { return (float)v; }
 
-// One block per token slot b in [0, B_pad).  ND digits.  `amax_bits` (optional) holds the
-// precomputed max |value| of each token as float bits; otherwise the block reduces it.
-// For int8 input (ND == 1) the values are their own single digit and the scale is 1.
+// Load 16 consecutive values of a row as floats (vector loads when the chunk is whole and
+// 16-byte aligned, guarded scalar loads otherwise).
+template <typename IN_T>
+__device__ __forceinline__ void load16(const IN_T* __restrict__ row, int c0, int C, bool vec_ok, float (&v)[16])
+{
+    if (vec_ok && c0 + 16 <= C) {
+        if constexpr (sizeof(IN_T) == 4) {
+            const float4* p4 = reinterpret_cast<const float4*>(row + c0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 f = __ldg(p4 + i);
+                v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+            }
+        } else if constexpr (sizeof(IN_T) == 2) {
+            const uint4* p4 = reinterpret_cast<const uint4*>(row + c0);
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const uint4 u = __ldg(p4 + i);
+                const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {   // bf16 -> fp32 is a 16-bit shift
+                    v[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+                    v[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+                }
+            }
+        } else {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(row + c0));
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = (float)(int)(int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xFF);
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) v[e] = (c0 + e < C) ? to_float<IN_T>(row[c0 + e]) : 0.f;
+    }
+}
+
+// One warp per token slot b in [0, B_pad); 8 tokens per block.  ND digits.  `amax_bits`
+// (optional) holds the precomputed max |value| of each token as float bits; otherwise the warp
+// reduces it.  For int8 input (ND == 1) the values are their own single digit and the scale is 1.
 template <typename IN_T, int ND>
 __global__ void __launch_bounds__(256)
-digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int C, int KB,
+digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
                 unsigned* __restrict__ zero_me)
 {
     constexpr int TOK = tokens_per_tile(ND);
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
-    const int b = blockIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (b >= B_pad) return;
     const int jt = b / TOK, b_in = b % TOK;
     const bool live = b < B;
     const IN_T* row = in + (size_t)b * ld_in;
-    __shared__ float red[8];
-    __shared__ float s_qscale;
+    const bool vec_ok = ((((uintptr_t)in) | ((size_t)ld_in * sizeof(IN_T))) & 15) == 0;
+    const int n_chunks = KB * 8;
 
-    if (zero_me && threadIdx.x == 0) zero_me[b] = 0u;
+    if (zero_me && lane == 0) zero_me[b] = 0u;
 
+    float qscale = 1.f;
     if constexpr (!kInt) {
         float amax = 0.f;
         if (live) {
             if (amax_bits) {
                 amax = __uint_as_float(amax_bits[b]);
             } else {
-                for (int c = threadIdx.x; c < C; c += blockDim.x) amax = fmaxf(amax, fabsf(to_float<IN_T>(row[c])));
+                for (int ch = lane; ch < n_chunks; ch += 32) {
+                    float v[16];
+                    load16<IN_T>(row, ch * 16, C, vec_ok, v);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) amax = fmaxf(amax, fabsf(v[e]));
+                }
                 for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-                if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
-                __syncthreads();
-                amax = red[0];
-                for (int w = 1; w < (int)(blockDim.x >> 5); ++w) amax = fmaxf(amax, red[w]);
             }
         }
-        if (threadIdx.x == 0) {
-            // |v| <= amax < 2^E; quantise to q = rint(v * 2^(8ND-2-E)), so |q| <= 2^(8ND-2)
-            int E = -90;
-            if (amax > 0.f) {
-                int e;
-                (void)frexpf(amax, &e);
-                E = max(e, -90);
-            }
-            s_qscale = exp2f((float)(8 * ND - 2 - E));
-            scale_out[b] = exp2f((float)(E - (8 * ND - 2)));   // value = q * scale
+        // |v| <= amax < 2^E; quantise to q = rint(v * 2^(8ND-2-E)), so |q| <= 2^(8ND-2)
+        int E = -90;
+        if (amax > 0.f) {
+            int e;
+            (void)frexpf(amax, &e);
+            E = max(e, -90);
         }
-        __syncthreads();
+        qscale = exp2f((float)(8 * ND - 2 - E));
+        if (lane == 0) scale_out[b] = exp2f((float)(E - (8 * ND - 2)));   // value = q * scale
     } else {
-        if (threadIdx.x == 0) scale_out[b] = 1.f;
+        if (lane == 0) scale_out[b] = 1.f;
     }
-    const float qscale = kInt ? 1.f : s_qscale;
 
-    // each thread converts chunks of 16 consecutive contraction elements
-    const int n_chunks = KB * 8;
-    for (int ch = threadIdx.x; ch < n_chunks; ch += blockDim.x) {
+    // each lane converts chunks of 16 consecutive contraction elements
+    for (int ch = lane; ch < n_chunks; ch += 32) {
         const int kb = ch >> 3, cc = ch & 7;
-        const int c0 = ch * 16;
         uint32_t dig[ND][4];
 #pragma unroll
         for (int d = 0; d < ND; ++d)
 #pragma unroll
             for (int w = 0; w < 4; ++w) dig[d][w] = 0;
         if (live) {
+            float v[16];
+            load16<IN_T>(row, ch * 16, C, vec_ok, v);
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-                const int c = c0 + e;
-                int q = 0;
-                if (c < C) {
-                    if constexpr (kInt) q = (int)row[c];
-                    else q = __float2int_rn(to_float<IN_T>(row[c]) * qscale);
-                }
+                int q = __float2int_rn(v[e] * qscale);
 #pragma unroll
                 for (int d = 0; d < ND; ++d) {
                     int dv;
@@ -131,16 +163,18 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int C, int KB,
 #pragma unroll
         for (int d = 0; d < ND; ++d) {
             const int r = d * TOK + b_in;
-            uint4 v = make_uint4(dig[d][0], dig[d][1], dig[d][2], dig[d][3]);
-            *reinterpret_cast<uint4*>(tile + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+            uint4 v4 = make_uint4(dig[d][0], dig[d][1], dig[d][2], dig[d][3]);
+            *reinterpret_cast<uint4*>(tile + r * 128 + ((cc ^ (r & 7)) << 4)) = v4;
         }
     }
 }
 
 // ---------------------------------------------------------------------------------------
-// The contraction kernel.  CTA (rt, jt) computes the 128 x (ND*TOK) integer tile
+// The contraction kernel (persistent: one CTA per SM walks over the tiles).  Tile (rt, jt) is
+// the 128 x (ND*TOK) integer block
 //   acc[r, d*TOK + i] = sum_c T[rt*128 + r, c] * digit_d(token jt*TOK + i)[c]
-// in tensor memory, then combines the digits and applies the stage's epilogue.
+// accumulated in one of two tensor-memory buffers, so that the epilogue warps (combine the
+// digits, apply the stage's scaling, store) work on one tile while the next is contracted.
 // ---------------------------------------------------------------------------------------
 enum { EPI_V = 0, EPI_U_F32 = 1, EPI_U_BF16 = 2 };
 
@@ -161,6 +195,8 @@ struct GemmParams {
     void* y;              // EPI_U_*: out [B][ldy]
     int ldy;
     int* status;          // device error word
+    int row_tiles;        // tiles of 128 rows
+    int j_tiles;          // tiles of TOK tokens
 };
 
 template <int ND, int EPI>
@@ -178,16 +214,17 @@ ternary_mma_kernel(const GemmParams p)
     uint8_t* b_tiles = smem + STAGES * A_TILE_BYTES;           // STAGES x 32 KiB, 1024-aligned
     uint8_t* p_tiles = b_tiles + STAGES * B_TILE_BYTES_MAX;    // STAGES x 4 KiB
     uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + STAGES * P_TILE_BYTES);
-    uint64_t* full_bar = bars;                 // copies landed (packed codes + digit tile)
-    uint64_t* aready_bar = bars + STAGES;      // expanded operand written
-    uint64_t* empty_bar = bars + 2 * STAGES;   // MMAs that read the stage have completed
-    uint64_t* acc_bar = bars + 3 * STAGES;     // all MMAs of the tile have completed
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * STAGES + 1);
+    uint64_t* full_bar = bars;                   // copies landed (packed codes + digit tile)
+    uint64_t* aready_bar = bars + STAGES;        // expanded operand written
+    uint64_t* empty_bar = bars + 2 * STAGES;     // MMAs that read the stage have completed
+    uint64_t* accfull_bar = bars + 3 * STAGES;   // [2] all MMAs of a tile have completed
+    uint64_t* accempty_bar = accfull_bar + 2;    // [2] the epilogue has drained the accumulator
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accempty_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rt = blockIdx.x, jt = blockIdx.y;
     const int KB = p.KB;
+    const int n_tiles = p.row_tiles * p.j_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -195,7 +232,10 @@ ternary_mma_kernel(const GemmParams p)
             mbar_init(&aready_bar[s], 4);   // one arrival per expander warp
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(acc_bar, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&accfull_bar[i], 1);
+            mbar_init(&accempty_bar[i], 4);  // one arrival per epilogue warp
+        }
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -208,27 +248,33 @@ ternary_mma_kernel(const GemmParams p)
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Waiting for parity 1 on a barrier that has not completed a phase yet returns at once,
+    // which is what a consumer-release barrier needs on its first use.
     if (warp == 0) {
         // ---- copy producer: packed codes of the A tile and the digit tile, per stage ----
         if (lane == 0) {
-            const uint8_t* p_src = reinterpret_cast<const uint8_t*>(p.units) + (size_t)rt * KB * P_TILE_BYTES;
-            const int8_t* d_src = p.D + (size_t)jt * KB * B_TILE_BYTES;
-            int issued = 0;
-            for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t use = kb / STAGES;
-                if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1, abort_flag)) break;
-                issued = kb + 1;
-                mbar_arrive_expect_tx(&full_bar[s], P_TILE_BYTES + B_TILE_BYTES);
-                bulk_g2s(p_tiles + s * P_TILE_BYTES, p_src + (size_t)kb * P_TILE_BYTES, P_TILE_BYTES, &full_bar[s]);
-                bulk_g2s(b_tiles + s * B_TILE_BYTES_MAX, d_src + (size_t)kb * B_TILE_BYTES, B_TILE_BYTES,
-                         &full_bar[s]);
+            uint32_t it = 0;      // pipeline slot counter across all tiles of this CTA
+            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+                const int rt = tile % p.row_tiles, jt = tile / p.row_tiles;
+                const uint8_t* p_src = reinterpret_cast<const uint8_t*>(p.units) + (size_t)rt * KB * P_TILE_BYTES;
+                const int8_t* d_src = p.D + (size_t)jt * KB * B_TILE_BYTES;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abort_flag)) goto producer_done;
+                    mbar_arrive_expect_tx(&full_bar[s], P_TILE_BYTES + B_TILE_BYTES);
+                    bulk_g2s(p_tiles + s * P_TILE_BYTES, p_src + (size_t)kb * P_TILE_BYTES, P_TILE_BYTES,
+                             &full_bar[s]);
+                    bulk_g2s(b_tiles + s * B_TILE_BYTES_MAX, d_src + (size_t)kb * B_TILE_BYTES, B_TILE_BYTES,
+                             &full_bar[s]);
+                }
             }
+        producer_done:
             if (*abort_flag) {
                 // a wait gave up somewhere: let this CTA's own copies land before it exits (bounded)
-                for (int kb = max(0, issued - STAGES); kb < issued; ++kb) {
-                    uint64_t* bar = &full_bar[kb % STAGES];
-                    const uint32_t ph = (kb / STAGES) & 1;
+                const uint32_t first = it > (uint32_t)STAGES ? it - STAGES : 0u;
+                for (uint32_t j = first; j < it; ++j) {
+                    uint64_t* bar = &full_bar[j % STAGES];
+                    const uint32_t ph = (j / STAGES) & 1;
                     for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(bar, ph); ++spin) {}
                 }
             }
@@ -236,73 +282,95 @@ ternary_mma_kernel(const GemmParams p)
     } else if (warp == 1) {
         // ---- MMA issue: one thread ----
         if (lane == 0) {
-            for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (kb / STAGES) & 1;
-                if (!mbar_wait(&full_bar[s], ph, abort_flag)) break;
-                if (!mbar_wait(&aready_bar[s], ph, abort_flag)) break;
+            uint32_t it = 0, local = 0;
+            bool alive = true;
+            for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++local) {
+                const uint32_t buf = local & 1;
+                if (!mbar_wait(&accempty_bar[buf], ((local >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
-                const uint64_t a_desc = umma_desc_k_sw128(smem_u32(a_tiles + s * A_TILE_BYTES));
-                const uint64_t b_desc = umma_desc_k_sw128(smem_u32(b_tiles + s * B_TILE_BYTES_MAX));
+                const uint32_t d_tmem = tmem_base + buf * 256u;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(&full_bar[s], ph, abort_flag) || !mbar_wait(&aready_bar[s], ph, abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint64_t a_desc = umma_desc_k_sw128(smem_u32(a_tiles + s * A_TILE_BYTES));
+                    const uint64_t b_desc = umma_desc_k_sw128(smem_u32(b_tiles + s * B_TILE_BYTES_MAX));
 #pragma unroll
-                for (int k = 0; k < BLOCK_C / UMMA_K; ++k) {
-                    // advance both operands by 32 bytes inside the swizzled 128-byte rows
-                    umma_s8_ss(tmem_base, a_desc + (uint64_t)(k * (UMMA_K >> 4)),
-                               b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, (kb | k) != 0);
+                    for (int k = 0; k < BLOCK_C / UMMA_K; ++k) {
+                        // advance both operands by 32 bytes inside the swizzled 128-byte rows
+                        umma_s8_ss(d_tmem, a_desc + (uint64_t)(k * (UMMA_K >> 4)),
+                                   b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, (kb | k) != 0);
+                    }
+                    umma_commit(&empty_bar[s]);   // frees the stage when these MMAs are done
                 }
-                umma_commit(&empty_bar[s]);   // frees the stage when these MMAs are done
+                umma_commit(&accfull_bar[buf]);
             }
-            umma_commit(acc_bar);
         }
-    } else {
+    } else if (warp < 6) {
         // ---- expanders: thread = row of the tile ----
         const int r = threadIdx.x - 64;   // 0..127
-        for (int kb = 0; kb < KB; ++kb) {
-            const int s = kb % STAGES;
-            const uint32_t ph = (kb / STAGES) & 1;
-            if (!mbar_wait(&full_bar[s], ph, abort_flag)) break;
-            const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + s * P_TILE_BYTES);
-            uint8_t* a_row = a_tiles + s * A_TILE_BYTES + r * 128;
+        uint32_t it = 0;
+        bool alive = true;
+        for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
+            for (int kb = 0; kb < KB; ++kb, ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                if (!mbar_wait(&full_bar[s], ph, abort_flag)) { alive = false; break; }
+                const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + s * P_TILE_BYTES);
+                uint8_t* a_row = a_tiles + s * A_TILE_BYTES + r * 128;
 #pragma unroll
-            for (int g = 0; g < 2; ++g) {
-                const uint4 u = packed[g * 128 + r];
-                const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+                for (int g = 0; g < 2; ++g) {
+                    const uint4 u = packed[g * 128 + r];
+                    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
-                for (int wi = 0; wi < 4; ++wi) {
-                    uint32_t o[4];
-                    tsvd_expand16(w[wi], o);
-                    const int chunk = g * 4 + wi;
-                    *reinterpret_cast<uint4*>(a_row + ((chunk ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    for (int wi = 0; wi < 4; ++wi) {
+                        uint32_t o[4];
+                        tsvd_expand16(w[wi], o);
+                        const int chunk = g * 4 + wi;
+                        *reinterpret_cast<uint4*>(a_row + ((chunk ^ (r & 7)) << 4)) =
+                            make_uint4(o[0], o[1], o[2], o[3]);
+                    }
                 }
+                fence_proxy_async_smem();   // generic-proxy stores -> visible to the MMA's async reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&aready_bar[s]);
             }
-            fence_proxy_async_smem();   // generic-proxy stores -> visible to the MMA's async reads
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&aready_bar[s]);
         }
-
+    } else {
         // ---- epilogue: this warp owns tensor-memory lanes 32*(warp%4) .. +31 ----
         const int lane_grp = warp & 3;
         const int row_in = lane_grp * 32 + lane;
-        const int row = rt * BLOCK_R + row_in;
-        const bool ok = mbar_wait(acc_bar, 0, abort_flag);
-        tc_fence_after_sync();
-        if (ok) {
-            const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
+        uint32_t local = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++local) {
+            const int rt = tile % p.row_tiles, jt = tile / p.row_tiles;
+            const int row = rt * BLOCK_R + row_in;
+            const uint32_t buf = local & 1;
+            if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
+            tc_fence_after_sync();
+            const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(lane_grp * 32) << 16);
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             for (int g = 0; g < TOK / 16; ++g) {
                 uint32_t acc[ND][16];
 #pragma unroll
                 for (int d = 0; d < ND; ++d) tmem_ld16(t_lane + (uint32_t)(d * TOK + g * 16), acc[d]);
+                const int b0 = jt * TOK + g * 16;
+                // lane i < 16 fetches the scale of token b0 + i (0 beyond the batch)
+                float my_scale = 0.f;
+                if (lane < 16 && b0 + lane < p.B) my_scale = p.scale[b0 + lane];
                 tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const int b = jt * TOK + g * 16 + i;
+                    const int b = b0 + i;
                     long long v = (long long)(int)acc[0][i];
 #pragma unroll
                     for (int d = 1; d < ND; ++d) v += (long long)(int)acc[d][i] << (8 * d);
                     const bool live = b < p.B;   // uniform across the warp
-                    const float sc = live ? p.scale[b] : 0.f;
+                    const float sc = __shfl_sync(0xffffffffu, my_scale, i);
                     const float val = __ll2float_rn(v) * sc;   // sc is a power of two: one rounding
                     if constexpr (EPI == EPI_V) {
                         const float tv = s_row * val;           // the K multiplications (Table S1)
@@ -323,6 +391,10 @@ ternary_mma_kernel(const GemmParams p)
                     }
                 }
             }
+            // all tensor-memory reads of this buffer are done: hand it back to the MMA thread
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&accempty_bar[buf]);
         }
     }
 
@@ -342,7 +414,8 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
 {
     constexpr int TOK = tokens_per_tile(ND);
     const int B_pad = (B + TOK - 1) / TOK * TOK;
-    digitise_kernel<IN_T, ND><<<B_pad, 256, 0, stream>>>(in, ld_in, B, C, KB, amax_bits, D, scale, zero_me);
+    digitise_kernel<IN_T, ND><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D, scale,
+                                                                   zero_me);
     tsvd_count_launch();
     if (B_pad_out) *B_pad_out = B_pad;
     return cudaGetLastError();
@@ -362,8 +435,14 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    dim3 grid(row_tiles, (p.B + TOK - 1) / TOK);
-    ternary_mma_kernel<ND, EPI><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(p);
+    GemmParams q = p;
+    q.row_tiles = row_tiles;
+    q.j_tiles = (p.B + TOK - 1) / TOK;
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int n_tiles = q.row_tiles * q.j_tiles;
+    const int grid = n_tiles < sms ? n_tiles : sms;
+    ternary_mma_kernel<ND, EPI><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
     tsvd_count_launch();
     return cudaGetLastError();
 }
@@ -409,6 +488,9 @@ TensorWs carve(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, void* base)
 }
 
 }  // namespace
+
+int tsvd_tensor_digits_x(tsvd_dtype_t dt) { return digits_for_x(dt); }
+int tsvd_tensor_digits_t() { return ND_T; }
 
 size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt)
 {
