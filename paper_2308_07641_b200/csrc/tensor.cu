@@ -23,7 +23,8 @@ constexpr int BLOCK_C = 128;   // contraction elements per pipeline stage (one 1
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
 constexpr int STAGES = 4;
 constexpr int TMEM_COLS = 512;   // two 256-column accumulator buffers
-constexpr int GEMM_THREADS = 320;  // warp 0: copies, 1: MMA issue, 2..5: expand, 6..9: epilogue
+constexpr int GEMM_THREADS = 448;  // warp 0: copies, 1: MMA issue, 2..5: expand, 6..13: epilogue
+constexpr int EPI_WARP0 = 6;
 
 // tokens per tile for nd digits: the MMA N extent is nd * tokens <= 256 and a multiple of 16
 __host__ __device__ constexpr int tokens_per_tile(int nd) { return nd == 1 ? 256 : nd == 2 ? 128 : nd == 3 ? 80 : 64; }
@@ -188,7 +189,6 @@ struct GemmParams {
     const float* S;       // EPI_V: S padded to R_pad
     float* t;             // EPI_V: out [B][t_ld]
     int t_ld;
-    unsigned* tmax;       // EPI_V: per-token max |t| as float bits (atomicMax)
     void* z_out;          // EPI_V: optional [B][z_ld]: int32 when z_int, else fp32
     int z_ld;
     int z_int;
@@ -199,7 +199,22 @@ struct GemmParams {
     int j_tiles;          // tiles of TOK tokens
 };
 
-template <int ND, int EPI>
+// int32 -> fp32.  The conversion instruction runs at a small fraction of the add rate on this
+// part, so when |v| < 2^22 is guaranteed (FAST) the value is placed in the mantissa of
+// 1.5*2^23 and that constant is subtracted: both steps are exact.
+template <bool FAST> __device__ __forceinline__ float cvt_i2f(int v)
+{
+    if constexpr (FAST) return __int_as_float(0x4B400000 + v) - 12582912.f;
+    else return (float)v;
+}
+// fp32 -> bf16 bits, round to nearest even (finite inputs), with integer adds.
+__device__ __forceinline__ uint16_t bf16_bits_rn(float x)
+{
+    const uint32_t u = __float_as_uint(x);
+    return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+
+template <int ND, int EPI, bool FAST>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 ternary_mma_kernel(const GemmParams p)
 {
@@ -234,7 +249,7 @@ ternary_mma_kernel(const GemmParams p)
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&accfull_bar[i], 1);
-            mbar_init(&accempty_bar[i], 4);  // one arrival per epilogue warp
+            mbar_init(&accempty_bar[i], 8);  // one arrival per epilogue warp
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -341,8 +356,10 @@ ternary_mma_kernel(const GemmParams p)
             }
         }
     } else {
-        // ---- epilogue: this warp owns tensor-memory lanes 32*(warp%4) .. +31 ----
+        // ---- epilogue: eight warps; warp w reads tensor-memory lanes 32*(w%4) .. +31 and takes
+        //      every second group of 16 tokens ----
         const int lane_grp = warp & 3;
+        const int half = (warp - EPI_WARP0) >> 2;
         const int row_in = lane_grp * 32 + lane;
         uint32_t local = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++local) {
@@ -354,7 +371,8 @@ ternary_mma_kernel(const GemmParams p)
             const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(lane_grp * 32) << 16);
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
-            for (int g = 0; g < TOK / 16; ++g) {
+            const bool row_ok = row < p.R;
+            for (int g = half; g < TOK / 16; g += 2) {
                 uint32_t acc[ND][16];
 #pragma unroll
                 for (int d = 0; d < ND; ++d) tmem_ld16(t_lane + (uint32_t)(d * TOK + g * 16), acc[d]);
@@ -363,31 +381,29 @@ ternary_mma_kernel(const GemmParams p)
                 float my_scale = 0.f;
                 if (lane < 16 && b0 + lane < p.B) my_scale = p.scale[b0 + lane];
                 tmem_ld_wait();
+                const int n_live = min(16, p.B - b0);   // uniform across the warp
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const int b = b0 + i;
-                    long long v = (long long)(int)acc[0][i];
+                    // digits -> fp32: each digit sum converts exactly, the three fused multiply-adds
+                    // round at 2^-24 of their partial sums.
+                    float f = cvt_i2f<FAST>((int)acc[ND - 1][i]);
 #pragma unroll
-                    for (int d = 1; d < ND; ++d) v += (long long)(int)acc[d][i] << (8 * d);
-                    const bool live = b < p.B;   // uniform across the warp
+                    for (int d = ND - 2; d >= 0; --d) f = fmaf(f, 256.f, cvt_i2f<FAST>((int)acc[d][i]));
                     const float sc = __shfl_sync(0xffffffffu, my_scale, i);
-                    const float val = __ll2float_rn(v) * sc;   // sc is a power of two: one rounding
-                    if constexpr (EPI == EPI_V) {
-                        const float tv = s_row * val;           // the K multiplications (Table S1)
-                        if (live) {
-                            p.t[(size_t)b * p.t_ld + row] = tv;
-                            if (p.z_out && row < p.R) {
-                                if (p.z_int) reinterpret_cast<int*>(p.z_out)[(size_t)b * p.z_ld + row] = (int)v;
+                    const float val = f * sc;   // sc is a power of two: exact
+                    if (i < n_live) {
+                        const int b = b0 + i;
+                        if constexpr (EPI == EPI_V) {
+                            p.t[(size_t)b * p.t_ld + row] = s_row * val;   // the K multiplications (Table S1)
+                            if (p.z_out && row_ok) {
+                                if (p.z_int) reinterpret_cast<int*>(p.z_out)[(size_t)b * p.z_ld + row] = (int)acc[0][i];
                                 else reinterpret_cast<float*>(p.z_out)[(size_t)b * p.z_ld + row] = val;
                             }
-                            const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(tv)));
-                            if (lane == 0) atomicMax(&p.tmax[b], m);
+                        } else if constexpr (EPI == EPI_U_F32) {
+                            if (row_ok) reinterpret_cast<float*>(p.y)[(size_t)b * p.ldy + row] = val;
+                        } else {
+                            if (row_ok) reinterpret_cast<uint16_t*>(p.y)[(size_t)b * p.ldy + row] = bf16_bits_rn(val);
                         }
-                    } else if constexpr (EPI == EPI_U_F32) {
-                        if (live && row < p.R) reinterpret_cast<float*>(p.y)[(size_t)b * p.ldy + row] = val;
-                    } else {
-                        if (live && row < p.R)
-                            reinterpret_cast<__nv_bfloat16*>(p.y)[(size_t)b * p.ldy + row] = __float2bfloat16_rn(val);
                     }
                 }
             }
@@ -421,8 +437,8 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
     return cudaGetLastError();
 }
 
-template <int ND, int EPI>
-cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
+template <int ND, int EPI, bool FAST>
+cudaError_t launch_gemm_impl(const GemmParams& p, int row_tiles, cudaStream_t stream)
 {
     constexpr int TOK = tokens_per_tile(ND);
     static bool attr_set[64] = {};   // per instantiation and device
@@ -430,7 +446,7 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
     cudaError_t e0 = cudaGetDevice(&dev);
     if (e0 != cudaSuccess) return e0;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(ternary_mma_kernel<ND, EPI>,
+        cudaError_t e = cudaFuncSetAttribute(ternary_mma_kernel<ND, EPI, FAST>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -442,9 +458,17 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int n_tiles = q.row_tiles * q.j_tiles;
     const int grid = n_tiles < sms ? n_tiles : sms;
-    ternary_mma_kernel<ND, EPI><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
+    ternary_mma_kernel<ND, EPI, FAST><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
     tsvd_count_launch();
     return cudaGetLastError();
+}
+
+// Digit sums are bounded by 128 * (contraction length): below 2^22 up to 32768 columns.
+template <int ND, int EPI>
+cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
+{
+    if (p.KB * BLOCK_C <= 32768) return launch_gemm_impl<ND, EPI, true>(p, row_tiles, stream);
+    return launch_gemm_impl<ND, EPI, false>(p, row_tiles, stream);
 }
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -505,20 +529,20 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     cudaStream_t st = a.stream;
     cudaError_t e;
 
-    // stage 0: activations -> digits (also clears the per-token max of t)
+    // stage 0: activations -> digits
     h->prof.begin(0, st);
     switch (a.dtype) {
         case TSVD_F32:
-            e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, w.tmax,
+            e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, nullptr,
                                           nullptr, st);
             break;
         case TSVD_BF16:
             e = launch_digitise<__nv_bfloat16, 3>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
-                                                  w.scale_x, w.tmax, nullptr, st);
+                                                  w.scale_x, nullptr, nullptr, st);
             break;
         case TSVD_I8:
             e = launch_digitise<int8_t, 1>((const int8_t*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                           w.tmax, nullptr, st);
+                                           nullptr, nullptr, st);
             break;
         default:
             return TSVD_E_DTYPE;
@@ -528,7 +552,7 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     // stage 1: V-stage + S scale
     GemmParams p{};
     p.units = h->V.units; p.KB = KBv; p.R = h->K; p.D = w.Dx; p.scale = w.scale_x; p.B = a.B;
-    p.S = h->S; p.t = w.t; p.t_ld = h->V.R_pad; p.tmax = w.tmax;
+    p.S = h->S; p.t = w.t; p.t_ld = h->V.R_pad;
     p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
     p.status = h->dev_status;
     const int v_tiles = h->V.R_pad / BLOCK_R;
@@ -539,9 +563,9 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
-    // stage 2: t -> digits, using the per-token max gathered by the V-stage epilogue
+    // stage 2: t -> digits (each token's scale comes from its own max |t|)
     h->prof.begin(2, st);
-    e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, w.tmax, w.Dt, w.scale_t, nullptr, nullptr, st);
+    e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, nullptr, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
