@@ -21,10 +21,14 @@ using namespace ptx;
 constexpr int BLOCK_R = 128;   // ternary rows per CTA tile = MMA M
 constexpr int BLOCK_C = 128;   // contraction elements per pipeline stage (one 128-byte swizzle row)
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
-constexpr int STAGES = 4;
+constexpr int NP = 6;          // ring depth of the packed codes
+constexpr int NS = 4;          // ring depth shared by the expanded operand and the digit tiles
 constexpr int TMEM_COLS = 512;   // two 256-column accumulator buffers
-constexpr int GEMM_THREADS = 448;  // warp 0: copies, 1: MMA issue, 2..5: expand, 6..13: epilogue
-constexpr int EPI_WARP0 = 6;
+// warp 0: digit-tile copies, 1: MMA issue, 2: packed-code copies, 3: idle,
+// 4..11: expand (two groups of four that take alternate contraction blocks), 12..19: epilogue
+constexpr int GEMM_THREADS = 640;
+constexpr int EXP_WARP0 = 4;
+constexpr int EPI_WARP0 = 12;
 
 // tokens per tile for nd digits: the MMA N extent is nd * tokens <= 256 and a multiple of 16
 __host__ __device__ constexpr int tokens_per_tile(int nd) { return nd == 1 ? 256 : nd == 2 ? 128 : nd == 3 ? 80 : 64; }
@@ -32,8 +36,8 @@ __host__ __device__ constexpr int tokens_per_tile(int nd) { return nd == 1 ? 256
 constexpr int A_TILE_BYTES = BLOCK_R * BLOCK_C;          // expanded int8 operand, 16 KiB
 constexpr int P_TILE_BYTES = BLOCK_R * BLOCK_C / 4;      // packed codes of that tile, 4 KiB
 constexpr int B_TILE_BYTES_MAX = 256 * BLOCK_C;          // digit rows, up to 32 KiB
-constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES_MAX + P_TILE_BYTES;
-constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int GEMM_SMEM_BYTES = NS * A_TILE_BYTES + NS * B_TILE_BYTES_MAX + NP * P_TILE_BYTES +
+                                1024 /*alignment slack*/ + 512 /*barriers*/;
 
 // ---------------------------------------------------------------------------------------
 // Digit matrix layout (scratch written by digitise_kernel, read by bulk copies):
@@ -199,22 +203,7 @@ struct GemmParams {
     int j_tiles;          // tiles of TOK tokens
 };
 
-// int32 -> fp32.  The conversion instruction runs at a small fraction of the add rate on this
-// part, so when |v| < 2^22 is guaranteed (FAST) the value is placed in the mantissa of
-// 1.5*2^23 and that constant is subtracted: both steps are exact.
-template <bool FAST> __device__ __forceinline__ float cvt_i2f(int v)
-{
-    if constexpr (FAST) return __int_as_float(0x4B400000 + v) - 12582912.f;
-    else return (float)v;
-}
-// fp32 -> bf16 bits, round to nearest even (finite inputs), with integer adds.
-__device__ __forceinline__ uint16_t bf16_bits_rn(float x)
-{
-    const uint32_t u = __float_as_uint(x);
-    return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
-}
-
-template <int ND, int EPI, bool FAST>
+template <int ND, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 ternary_mma_kernel(const GemmParams p)
 {
@@ -223,17 +212,25 @@ ternary_mma_kernel(const GemmParams p)
     constexpr uint32_t B_TILE_BYTES = NT * BLOCK_C;
     constexpr uint32_t IDESC = umma_idesc_s8(BLOCK_R, NT);
 
+    // Three rings, because their contents live for different times:
+    //   P: packed codes (4 KiB), copied far ahead, freed as soon as the expanders have read them
+    //   A: expanded int8 operand (16 KiB), lives from expansion to the end of its MMAs
+    //   B: digit tiles (32 KiB), live from the copy's issue to the end of their MMAs
+    // A and B share one depth and one "MMAs done" barrier per slot: every tcgen05.commit
+    // between MMAs costs issue time, so there is exactly one per contraction block.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* a_tiles = smem;                                   // STAGES x 16 KiB, 1024-aligned
-    uint8_t* b_tiles = smem + STAGES * A_TILE_BYTES;           // STAGES x 32 KiB, 1024-aligned
-    uint8_t* p_tiles = b_tiles + STAGES * B_TILE_BYTES_MAX;    // STAGES x 4 KiB
-    uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + STAGES * P_TILE_BYTES);
-    uint64_t* full_bar = bars;                   // copies landed (packed codes + digit tile)
-    uint64_t* aready_bar = bars + STAGES;        // expanded operand written
-    uint64_t* empty_bar = bars + 2 * STAGES;     // MMAs that read the stage have completed
-    uint64_t* accfull_bar = bars + 3 * STAGES;   // [2] all MMAs of a tile have completed
-    uint64_t* accempty_bar = accfull_bar + 2;    // [2] the epilogue has drained the accumulator
+    uint8_t* a_tiles = smem;                                 // NS x 16 KiB, 1024-aligned
+    uint8_t* b_tiles = a_tiles + NS * A_TILE_BYTES;          // NS x 32 KiB, 1024-aligned
+    uint8_t* p_tiles = b_tiles + NS * B_TILE_BYTES_MAX;      // NP x 4 KiB
+    uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + NP * P_TILE_BYTES);
+    uint64_t* pfull_bar = bars;                      // [NP] packed codes landed
+    uint64_t* pempty_bar = pfull_bar + NP;           // [NP] expanders have read them
+    uint64_t* afull_bar = pempty_bar + NP;           // [NS] expanded operand written
+    uint64_t* bfull_bar = afull_bar + NS;            // [NS] digit tile landed
+    uint64_t* done_bar = bfull_bar + NS;             // [NS] the MMAs reading slot s (A and B) have completed
+    uint64_t* accfull_bar = done_bar + NS;           // [2] all MMAs of a tile have completed
+    uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accempty_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -242,10 +239,11 @@ ternary_mma_kernel(const GemmParams p)
     const int n_tiles = p.row_tiles * p.j_tiles;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full_bar[s], 1);
-            mbar_init(&aready_bar[s], 4);   // one arrival per expander warp
-            mbar_init(&empty_bar[s], 1);
+        for (int s = 0; s < NP; ++s) { mbar_init(&pfull_bar[s], 1); mbar_init(&pempty_bar[s], 4); }
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(&afull_bar[s], 4);   // one arrival per expander warp of the group
+            mbar_init(&bfull_bar[s], 1);
+            mbar_init(&done_bar[s], 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&accfull_bar[i], 1);
@@ -265,31 +263,34 @@ ternary_mma_kernel(const GemmParams p)
 
     // Waiting for parity 1 on a barrier that has not completed a phase yet returns at once,
     // which is what a consumer-release barrier needs on its first use.
-    if (warp == 0) {
-        // ---- copy producer: packed codes of the A tile and the digit tile, per stage ----
+    if (warp == 0 || warp == 2) {
+        // ---- copy producers: warp 0 streams the digit tiles, warp 2 the packed codes ----
         if (lane == 0) {
+            const bool is_b = warp == 0;
+            const int depth = is_b ? NS : NP;
+            uint64_t* full = is_b ? bfull_bar : pfull_bar;
+            uint64_t* empty = is_b ? done_bar : pempty_bar;
+            const uint32_t bytes = is_b ? B_TILE_BYTES : (uint32_t)P_TILE_BYTES;
             uint32_t it = 0;      // pipeline slot counter across all tiles of this CTA
-            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+            bool alive = true;
+            for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
                 const int rt = tile % p.row_tiles, jt = tile / p.row_tiles;
-                const uint8_t* p_src = reinterpret_cast<const uint8_t*>(p.units) + (size_t)rt * KB * P_TILE_BYTES;
-                const int8_t* d_src = p.D + (size_t)jt * KB * B_TILE_BYTES;
+                const uint8_t* src = is_b ? reinterpret_cast<const uint8_t*>(p.D) + (size_t)jt * KB * B_TILE_BYTES
+                                          : reinterpret_cast<const uint8_t*>(p.units) + (size_t)rt * KB * P_TILE_BYTES;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abort_flag)) goto producer_done;
-                    mbar_arrive_expect_tx(&full_bar[s], P_TILE_BYTES + B_TILE_BYTES);
-                    bulk_g2s(p_tiles + s * P_TILE_BYTES, p_src + (size_t)kb * P_TILE_BYTES, P_TILE_BYTES,
-                             &full_bar[s]);
-                    bulk_g2s(b_tiles + s * B_TILE_BYTES_MAX, d_src + (size_t)kb * B_TILE_BYTES, B_TILE_BYTES,
-                             &full_bar[s]);
+                    const int s = it % depth;
+                    if (!mbar_wait(&empty[s], ((it / depth) & 1) ^ 1, abort_flag)) { alive = false; break; }
+                    mbar_arrive_expect_tx(&full[s], bytes);
+                    uint8_t* dst = is_b ? b_tiles + s * B_TILE_BYTES_MAX : p_tiles + s * P_TILE_BYTES;
+                    bulk_g2s(dst, src + (size_t)kb * bytes, bytes, &full[s]);
                 }
             }
-        producer_done:
             if (*abort_flag) {
                 // a wait gave up somewhere: let this CTA's own copies land before it exits (bounded)
-                const uint32_t first = it > (uint32_t)STAGES ? it - STAGES : 0u;
+                const uint32_t first = it > (uint32_t)depth ? it - depth : 0u;
                 for (uint32_t j = first; j < it; ++j) {
-                    uint64_t* bar = &full_bar[j % STAGES];
-                    const uint32_t ph = (j / STAGES) & 1;
+                    uint64_t* bar = &full[j % depth];
+                    const uint32_t ph = (j / depth) & 1;
                     for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(bar, ph); ++spin) {}
                 }
             }
@@ -305,9 +306,9 @@ ternary_mma_kernel(const GemmParams p)
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * 256u;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t ph = (it / STAGES) & 1;
-                    if (!mbar_wait(&full_bar[s], ph, abort_flag) || !mbar_wait(&aready_bar[s], ph, abort_flag)) {
+                    const int s = it % NS;
+                    const uint32_t ph = (it / NS) & 1;
+                    if (!mbar_wait(&bfull_bar[s], ph, abort_flag) || !mbar_wait(&afull_bar[s], ph, abort_flag)) {
                         alive = false;
                         break;
                     }
@@ -320,42 +321,48 @@ ternary_mma_kernel(const GemmParams p)
                         umma_s8_ss(d_tmem, a_desc + (uint64_t)(k * (UMMA_K >> 4)),
                                    b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, (kb | k) != 0);
                     }
-                    umma_commit(&empty_bar[s]);   // frees the stage when these MMAs are done
+                    umma_commit(&done_bar[s]);   // slot s of A and of B is free when these MMAs are done
                 }
                 umma_commit(&accfull_bar[buf]);
             }
         }
-    } else if (warp < 6) {
-        // ---- expanders: thread = row of the tile ----
-        const int r = threadIdx.x - 64;   // 0..127
+    } else if (warp >= EXP_WARP0 && warp < EXP_WARP0 + 8) {
+        // ---- expanders: thread = row of the tile; the two groups of four warps take alternate
+        //      contraction blocks, so that the barrier and shared-memory latencies of one block
+        //      overlap with the work on the next ----
+        const int r = (threadIdx.x - EXP_WARP0 * 32) & 127;   // 0..127
+        const uint32_t group = (uint32_t)(warp - EXP_WARP0) >> 2;
         uint32_t it = 0;
         bool alive = true;
         for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
             for (int kb = 0; kb < KB; ++kb, ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
-                if (!mbar_wait(&full_bar[s], ph, abort_flag)) { alive = false; break; }
-                const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + s * P_TILE_BYTES);
-                uint8_t* a_row = a_tiles + s * A_TILE_BYTES + r * 128;
+                if ((it & 1u) != group) continue;
+                const int sp = it % NP, sa = it % NS;
+                if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
+                const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_TILE_BYTES);
+                uint32_t o[8][4];
 #pragma unroll
                 for (int g = 0; g < 2; ++g) {
                     const uint4 u = packed[g * 128 + r];
-                    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-                    for (int wi = 0; wi < 4; ++wi) {
-                        uint32_t o[4];
-                        tsvd_expand16(w[wi], o);
-                        const int chunk = g * 4 + wi;
-                        *reinterpret_cast<uint4*>(a_row + ((chunk ^ (r & 7)) << 4)) =
-                            make_uint4(o[0], o[1], o[2], o[3]);
-                    }
+                    tsvd_expand16(u.x, o[g * 4 + 0]);
+                    tsvd_expand16(u.y, o[g * 4 + 1]);
+                    tsvd_expand16(u.z, o[g * 4 + 2]);
+                    tsvd_expand16(u.w, o[g * 4 + 3]);
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // codes are in registers: slot reusable
+                if (!mbar_wait(&done_bar[sa], ((it / NS) & 1) ^ 1, abort_flag)) { alive = false; break; }
+                uint8_t* a_row = a_tiles + sa * A_TILE_BYTES + r * 128;
+#pragma unroll
+                for (int chunk = 0; chunk < 8; ++chunk)
+                    *reinterpret_cast<uint4*>(a_row + ((chunk ^ (r & 7)) << 4)) =
+                        make_uint4(o[chunk][0], o[chunk][1], o[chunk][2], o[chunk][3]);
                 fence_proxy_async_smem();   // generic-proxy stores -> visible to the MMA's async reads
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&aready_bar[s]);
+                if (lane == 0) mbar_arrive(&afull_bar[sa]);
             }
         }
-    } else {
+    } else if (warp >= EPI_WARP0) {
         // ---- epilogue: eight warps; warp w reads tensor-memory lanes 32*(w%4) .. +31 and takes
         //      every second group of 16 tokens ----
         const int lane_grp = warp & 3;
@@ -366,44 +373,80 @@ ternary_mma_kernel(const GemmParams p)
             const int rt = tile % p.row_tiles, jt = tile / p.row_tiles;
             const int row = rt * BLOCK_R + row_in;
             const uint32_t buf = local & 1;
-            if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
-            tc_fence_after_sync();
-            const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(lane_grp * 32) << 16);
+            // fetch the per-token scales of this warp's groups while the tile is still being
+            // contracted: lane i holds the scale of token 16*g + (i & 15) (0 beyond the batch)
+            constexpr int MY_GROUPS = (TOK / 16 + 1) / 2;
+            float scales[MY_GROUPS];
+#pragma unroll
+            for (int k = 0; k < MY_GROUPS; ++k) {
+                const int bb = jt * TOK + (half + 2 * k) * 16 + (lane & 15);
+                scales[k] = (half + 2 * k < TOK / 16 && bb < p.B) ? __ldg(p.scale + bb) : 0.f;
+            }
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             const bool row_ok = row < p.R;
-            for (int g = half; g < TOK / 16; g += 2) {
+            if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
+            tc_fence_after_sync();
+            const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(lane_grp * 32) << 16);
+#pragma unroll
+            for (int k = 0; k < MY_GROUPS; ++k) {
+                const int g = half + 2 * k;
+                if (g >= TOK / 16) break;
                 uint32_t acc[ND][16];
 #pragma unroll
                 for (int d = 0; d < ND; ++d) tmem_ld16(t_lane + (uint32_t)(d * TOK + g * 16), acc[d]);
                 const int b0 = jt * TOK + g * 16;
-                // lane i < 16 fetches the scale of token b0 + i (0 beyond the batch)
-                float my_scale = 0.f;
-                if (lane < 16 && b0 + lane < p.B) my_scale = p.scale[b0 + lane];
+                const float my_scale = scales[k];
                 tmem_ld_wait();
                 const int n_live = min(16, p.B - b0);   // uniform across the warp
+                // digits -> fp32: lo and hi are exact 32-bit integers; their conversions and the
+                // fused multiply-add round at 2^-24 of |hi|*65536 and |lo|.  (64-bit integer and
+                // double conversions are far too slow on this part to sit in this loop.)
+                float val[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    // digits -> fp32: each digit sum converts exactly, the three fused multiply-adds
-                    // round at 2^-24 of their partial sums.
-                    float f = cvt_i2f<FAST>((int)acc[ND - 1][i]);
+                    float f;
+                    if constexpr (ND == 1) {
+                        f = (float)(int)acc[0][i];
+                    } else if constexpr (ND == 2) {
+                        f = (float)((int)acc[0][i] + ((int)acc[1][i] << 8));
+                    } else {
+                        const int lo = (int)acc[0][i] + ((int)acc[1][i] << 8);
+                        int hi = (int)acc[2][i];
+                        if constexpr (ND == 4) hi += (int)acc[3][i] << 8;
+                        f = fmaf((float)hi, 65536.f, (float)lo);
+                    }
+                    val[i] = f * __shfl_sync(0xffffffffu, my_scale, i);   // a power of two: exact
+                }
+                if constexpr (EPI == EPI_V) {
+                    float* tp = p.t + (size_t)b0 * p.t_ld + row;
 #pragma unroll
-                    for (int d = ND - 2; d >= 0; --d) f = fmaf(f, 256.f, cvt_i2f<FAST>((int)acc[d][i]));
-                    const float sc = __shfl_sync(0xffffffffu, my_scale, i);
-                    const float val = f * sc;   // sc is a power of two: exact
-                    if (i < n_live) {
-                        const int b = b0 + i;
-                        if constexpr (EPI == EPI_V) {
-                            p.t[(size_t)b * p.t_ld + row] = s_row * val;   // the K multiplications (Table S1)
-                            if (p.z_out && row_ok) {
-                                if (p.z_int) reinterpret_cast<int*>(p.z_out)[(size_t)b * p.z_ld + row] = (int)acc[0][i];
-                                else reinterpret_cast<float*>(p.z_out)[(size_t)b * p.z_ld + row] = val;
+                    for (int i = 0; i < 16; ++i)
+                        if (i < n_live) tp[(size_t)i * p.t_ld] = s_row * val[i];   // the K multiplications (Table S1)
+                    if (p.z_out && row_ok) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            if (i < n_live) {
+                                const size_t o = (size_t)(b0 + i) * p.z_ld + row;
+                                if (p.z_int) reinterpret_cast<int*>(p.z_out)[o] = (int)acc[0][i];
+                                else reinterpret_cast<float*>(p.z_out)[o] = val[i];
                             }
-                        } else if constexpr (EPI == EPI_U_F32) {
-                            if (row_ok) reinterpret_cast<float*>(p.y)[(size_t)b * p.ldy + row] = val;
-                        } else {
-                            if (row_ok) reinterpret_cast<uint16_t*>(p.y)[(size_t)b * p.ldy + row] = bf16_bits_rn(val);
                         }
+                    }
+                } else if constexpr (EPI == EPI_U_F32) {
+                    float* yp = reinterpret_cast<float*>(p.y) + (size_t)b0 * p.ldy + row;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (row_ok && i < n_live) yp[(size_t)i * p.ldy] = val[i];
+                } else {
+                    uint16_t* yp = reinterpret_cast<uint16_t*>(p.y) + (size_t)b0 * p.ldy + row;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) {
+                        // one conversion instruction rounds two values (to nearest even)
+                        const __nv_bfloat162 pr = __floats2bfloat162_rn(val[i], val[i + 1]);
+                        const uint32_t u = *reinterpret_cast<const uint32_t*>(&pr);
+                        if (row_ok && i < n_live) yp[(size_t)i * p.ldy] = (uint16_t)(u & 0xFFFFu);
+                        if (row_ok && i + 1 < n_live) yp[(size_t)(i + 1) * p.ldy] = (uint16_t)(u >> 16);
                     }
                 }
             }
@@ -437,8 +480,8 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
     return cudaGetLastError();
 }
 
-template <int ND, int EPI, bool FAST>
-cudaError_t launch_gemm_impl(const GemmParams& p, int row_tiles, cudaStream_t stream)
+template <int ND, int EPI>
+cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
 {
     constexpr int TOK = tokens_per_tile(ND);
     static bool attr_set[64] = {};   // per instantiation and device
@@ -446,7 +489,7 @@ cudaError_t launch_gemm_impl(const GemmParams& p, int row_tiles, cudaStream_t st
     cudaError_t e0 = cudaGetDevice(&dev);
     if (e0 != cudaSuccess) return e0;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(ternary_mma_kernel<ND, EPI, FAST>,
+        cudaError_t e = cudaFuncSetAttribute(ternary_mma_kernel<ND, EPI>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -458,17 +501,9 @@ cudaError_t launch_gemm_impl(const GemmParams& p, int row_tiles, cudaStream_t st
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int n_tiles = q.row_tiles * q.j_tiles;
     const int grid = n_tiles < sms ? n_tiles : sms;
-    ternary_mma_kernel<ND, EPI, FAST><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
+    ternary_mma_kernel<ND, EPI><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
     tsvd_count_launch();
     return cudaGetLastError();
-}
-
-// Digit sums are bounded by 128 * (contraction length): below 2^22 up to 32768 columns.
-template <int ND, int EPI>
-cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
-{
-    if (p.KB * BLOCK_C <= 32768) return launch_gemm_impl<ND, EPI, true>(p, row_tiles, stream);
-    return launch_gemm_impl<ND, EPI, false>(p, row_tiles, stream);
 }
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
