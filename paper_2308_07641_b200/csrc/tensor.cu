@@ -21,22 +21,28 @@ using namespace ptx;
 constexpr int BLOCK_R = 128;   // ternary rows per CTA tile = MMA M
 constexpr int BLOCK_C = 128;   // contraction elements per pipeline stage (one 128-byte swizzle row)
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
-constexpr int NP = 6;          // ring depth of the packed codes
-constexpr int NS = 4;          // ring depth shared by the expanded operand and the digit tiles
-constexpr int TMEM_COLS = 512;   // two 256-column accumulator buffers
+constexpr int NT_MAX = 192;    // MMA N extent: digit rows per tile
+constexpr int NP = 6;          // ring depth of the packed codes (shared memory)
+constexpr int NB = 6;          // ring depth of the digit tiles (shared memory)
+constexpr int NA = 4;          // ring depth of the expanded operand (tensor memory)
+// tensor memory: two accumulator buffers of 192 columns, then four 32-column slots that hold
+// the expanded ternary operand (128 rows x 128 int8 = 32 columns of 32 bits per row)
+constexpr int TMEM_COLS = 512;
+constexpr int ACC_COLS = NT_MAX;
+constexpr int A_COL0 = 2 * ACC_COLS;
+constexpr int A_SLOT_COLS = BLOCK_C / 4;
 // warp 0: digit-tile copies, 1: MMA issue, 2: packed-code copies, 3: idle,
 // 4..11: expand (two groups of four that take alternate contraction blocks), 12..19: epilogue
 constexpr int GEMM_THREADS = 640;
 constexpr int EXP_WARP0 = 4;
 constexpr int EPI_WARP0 = 12;
 
-// tokens per tile for nd digits: the MMA N extent is nd * tokens <= 256 and a multiple of 16
-__host__ __device__ constexpr int tokens_per_tile(int nd) { return nd == 1 ? 256 : nd == 2 ? 128 : nd == 3 ? 80 : 64; }
+// tokens per tile for nd digits: the MMA N extent is nd * tokens = 192 for every nd
+__host__ __device__ constexpr int tokens_per_tile(int nd) { return 192 / nd; }
 
-constexpr int A_TILE_BYTES = BLOCK_R * BLOCK_C;          // expanded int8 operand, 16 KiB
 constexpr int P_TILE_BYTES = BLOCK_R * BLOCK_C / 4;      // packed codes of that tile, 4 KiB
-constexpr int B_TILE_BYTES_MAX = 256 * BLOCK_C;          // digit rows, up to 32 KiB
-constexpr int GEMM_SMEM_BYTES = NS * A_TILE_BYTES + NS * B_TILE_BYTES_MAX + NP * P_TILE_BYTES +
+constexpr int B_TILE_BYTES_MAX = NT_MAX * BLOCK_C;       // digit rows, 24 KiB
+constexpr int GEMM_SMEM_BYTES = NB * B_TILE_BYTES_MAX + NP * P_TILE_BYTES +
                                 1024 /*alignment slack*/ + 512 /*barriers*/;
 
 // ---------------------------------------------------------------------------------------
@@ -213,23 +219,24 @@ ternary_mma_kernel(const GemmParams p)
     constexpr uint32_t IDESC = umma_idesc_s8(BLOCK_R, NT);
 
     // Three rings, because their contents live for different times:
-    //   P: packed codes (4 KiB), copied far ahead, freed as soon as the expanders have read them
-    //   A: expanded int8 operand (16 KiB), lives from expansion to the end of its MMAs
-    //   B: digit tiles (32 KiB), live from the copy's issue to the end of their MMAs
-    // A and B share one depth and one "MMAs done" barrier per slot: every tcgen05.commit
-    // between MMAs costs issue time, so there is exactly one per contraction block.
+    //   P: packed codes (4 KiB, shared memory), copied far ahead, freed once the expanders read them
+    //   A: expanded int8 operand (tensor memory), lives from expansion to the end of its MMAs;
+    //      it never touches shared memory, whose bandwidth the digit tiles need
+    //   B: digit tiles (24 KiB, shared memory), live from the copy's issue to the end of their MMAs
+    // One "MMAs done" barrier per contraction block serves both A and B (every tcgen05.commit
+    // between MMAs costs issue time): block `it` signals done_bar[it % NB], and an A slot is
+    // free again when block it - NA has signalled.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* a_tiles = smem;                                 // NS x 16 KiB, 1024-aligned
-    uint8_t* b_tiles = a_tiles + NS * A_TILE_BYTES;          // NS x 32 KiB, 1024-aligned
-    uint8_t* p_tiles = b_tiles + NS * B_TILE_BYTES_MAX;      // NP x 4 KiB
+    uint8_t* b_tiles = smem;                                 // NB x 24 KiB, 1024-aligned
+    uint8_t* p_tiles = b_tiles + NB * B_TILE_BYTES_MAX;      // NP x 4 KiB
     uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + NP * P_TILE_BYTES);
     uint64_t* pfull_bar = bars;                      // [NP] packed codes landed
     uint64_t* pempty_bar = pfull_bar + NP;           // [NP] expanders have read them
-    uint64_t* afull_bar = pempty_bar + NP;           // [NS] expanded operand written
-    uint64_t* bfull_bar = afull_bar + NS;            // [NS] digit tile landed
-    uint64_t* done_bar = bfull_bar + NS;             // [NS] the MMAs reading slot s (A and B) have completed
-    uint64_t* accfull_bar = done_bar + NS;           // [2] all MMAs of a tile have completed
+    uint64_t* afull_bar = pempty_bar + NP;           // [NA] expanded operand written
+    uint64_t* bfull_bar = afull_bar + NA;            // [NB] digit tile landed
+    uint64_t* done_bar = bfull_bar + NB;             // [NB] the MMAs of a contraction block have completed
+    uint64_t* accfull_bar = done_bar + NB;           // [2] all MMAs of a tile have completed
     uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accempty_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -240,11 +247,8 @@ ternary_mma_kernel(const GemmParams p)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NP; ++s) { mbar_init(&pfull_bar[s], 1); mbar_init(&pempty_bar[s], 4); }
-        for (int s = 0; s < NS; ++s) {
-            mbar_init(&afull_bar[s], 4);   // one arrival per expander warp of the group
-            mbar_init(&bfull_bar[s], 1);
-            mbar_init(&done_bar[s], 1);
-        }
+        for (int s = 0; s < NA; ++s) mbar_init(&afull_bar[s], 4);   // one arrival per expander warp of the group
+        for (int s = 0; s < NB; ++s) { mbar_init(&bfull_bar[s], 1); mbar_init(&done_bar[s], 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&accfull_bar[i], 1);
             mbar_init(&accempty_bar[i], 8);  // one arrival per epilogue warp
@@ -267,7 +271,7 @@ ternary_mma_kernel(const GemmParams p)
         // ---- copy producers: warp 0 streams the digit tiles, warp 2 the packed codes ----
         if (lane == 0) {
             const bool is_b = warp == 0;
-            const int depth = is_b ? NS : NP;
+            const int depth = is_b ? NB : NP;
             uint64_t* full = is_b ? bfull_bar : pfull_bar;
             uint64_t* empty = is_b ? done_bar : pempty_bar;
             const uint32_t bytes = is_b ? B_TILE_BYTES : (uint32_t)P_TILE_BYTES;
@@ -304,32 +308,33 @@ ternary_mma_kernel(const GemmParams p)
                 const uint32_t buf = local & 1;
                 if (!mbar_wait(&accempty_bar[buf], ((local >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + buf * 256u;
+                const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % NS;
-                    const uint32_t ph = (it / NS) & 1;
-                    if (!mbar_wait(&bfull_bar[s], ph, abort_flag) || !mbar_wait(&afull_bar[s], ph, abort_flag)) {
+                    const int sa = it % NA, sb = it % NB;
+                    if (!mbar_wait(&bfull_bar[sb], (it / NB) & 1, abort_flag) ||
+                        !mbar_wait(&afull_bar[sa], (it / NA) & 1, abort_flag)) {
                         alive = false;
                         break;
                     }
                     tc_fence_after_sync();
-                    const uint64_t a_desc = umma_desc_k_sw128(smem_u32(a_tiles + s * A_TILE_BYTES));
-                    const uint64_t b_desc = umma_desc_k_sw128(smem_u32(b_tiles + s * B_TILE_BYTES_MAX));
+                    const uint32_t a_tmem = tmem_base + (uint32_t)(A_COL0 + sa * A_SLOT_COLS);
+                    const uint64_t b_desc = umma_desc_k_sw128(smem_u32(b_tiles + sb * B_TILE_BYTES_MAX));
 #pragma unroll
                     for (int k = 0; k < BLOCK_C / UMMA_K; ++k) {
-                        // advance both operands by 32 bytes inside the swizzled 128-byte rows
-                        umma_s8_ss(d_tmem, a_desc + (uint64_t)(k * (UMMA_K >> 4)),
+                        // 32 contraction elements per instruction: 8 columns of A, 32 bytes of the
+                        // swizzled 128-byte rows of B
+                        umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)),
                                    b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, (kb | k) != 0);
                     }
-                    umma_commit(&done_bar[s]);   // slot s of A and of B is free when these MMAs are done
+                    umma_commit(&done_bar[sb]);   // block `it` is done: frees B slot sb and A slot sa
                 }
                 umma_commit(&accfull_bar[buf]);
             }
         }
     } else if (warp >= EXP_WARP0 && warp < EXP_WARP0 + 8) {
-        // ---- expanders: thread = row of the tile; the two groups of four warps take alternate
-        //      contraction blocks, so that the barrier and shared-memory latencies of one block
-        //      overlap with the work on the next ----
+        // ---- expanders: thread = row of the tile = tensor-memory lane (warp w may touch lanes
+        //      32*(w%4)..+31); the two groups of four warps take alternate contraction blocks, so
+        //      that the barrier and memory latencies of one block overlap with work on the next ----
         const int r = (threadIdx.x - EXP_WARP0 * 32) & 127;   // 0..127
         const uint32_t group = (uint32_t)(warp - EXP_WARP0) >> 2;
         uint32_t it = 0;
@@ -337,34 +342,35 @@ ternary_mma_kernel(const GemmParams p)
         for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 if ((it & 1u) != group) continue;
-                const int sp = it % NP, sa = it % NS;
+                const int sp = it % NP, sa = it % NA;
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_TILE_BYTES);
-                uint32_t o[8][4];
+                uint32_t o[32];   // the row's 128 int8 values, four per 32-bit column
 #pragma unroll
                 for (int g = 0; g < 2; ++g) {
                     const uint4 u = packed[g * 128 + r];
-                    tsvd_expand16(u.x, o[g * 4 + 0]);
-                    tsvd_expand16(u.y, o[g * 4 + 1]);
-                    tsvd_expand16(u.z, o[g * 4 + 2]);
-                    tsvd_expand16(u.w, o[g * 4 + 3]);
+                    tsvd_expand16(u.x, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 0]));
+                    tsvd_expand16(u.y, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 4]));
+                    tsvd_expand16(u.z, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 8]));
+                    tsvd_expand16(u.w, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 12]));
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // codes are in registers: slot reusable
-                if (!mbar_wait(&done_bar[sa], ((it / NS) & 1) ^ 1, abort_flag)) { alive = false; break; }
-                uint8_t* a_row = a_tiles + sa * A_TILE_BYTES + r * 128;
-#pragma unroll
-                for (int chunk = 0; chunk < 8; ++chunk)
-                    *reinterpret_cast<uint4*>(a_row + ((chunk ^ (r & 7)) << 4)) =
-                        make_uint4(o[chunk][0], o[chunk][1], o[chunk][2], o[chunk][3]);
-                fence_proxy_async_smem();   // generic-proxy stores -> visible to the MMA's async reads
+                if (it >= (uint32_t)NA) {   // the A slot is free once block it - NA has completed
+                    const uint32_t j = it - NA;
+                    if (!mbar_wait(&done_bar[j % NB], (j / NB) & 1, abort_flag)) { alive = false; break; }
+                    tc_fence_after_sync();
+                }
+                tmem_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS), o);
+                tmem_st_wait();
+                tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&afull_bar[sa]);
             }
         }
     } else if (warp >= EPI_WARP0) {
         // ---- epilogue: eight warps; warp w reads tensor-memory lanes 32*(w%4) .. +31 and takes
-        //      every second group of 16 tokens ----
+        //      every second group of 8 tokens ----
         const int lane_grp = warp & 3;
         const int half = (warp - EPI_WARP0) >> 2;
         const int row_in = lane_grp * 32 + lane;
@@ -373,38 +379,39 @@ ternary_mma_kernel(const GemmParams p)
             const int rt = tile % p.row_tiles, jt = tile / p.row_tiles;
             const int row = rt * BLOCK_R + row_in;
             const uint32_t buf = local & 1;
-            // fetch the per-token scales of this warp's groups while the tile is still being
-            // contracted: lane i holds the scale of token 16*g + (i & 15) (0 beyond the batch)
-            constexpr int MY_GROUPS = (TOK / 16 + 1) / 2;
+            // fetch the per-token scales of this warp's groups (8 tokens each; this warp takes
+            // every second group) while the tile is still being contracted: lane i holds the
+            // scale of token 8*g + (i & 7), 0 beyond the batch
+            constexpr int N_GROUPS = TOK / 8;
+            constexpr int MY_GROUPS = N_GROUPS / 2;
             float scales[MY_GROUPS];
 #pragma unroll
             for (int k = 0; k < MY_GROUPS; ++k) {
-                const int bb = jt * TOK + (half + 2 * k) * 16 + (lane & 15);
-                scales[k] = (half + 2 * k < TOK / 16 && bb < p.B) ? __ldg(p.scale + bb) : 0.f;
+                const int bb = jt * TOK + (half + 2 * k) * 8 + (lane & 7);
+                scales[k] = bb < p.B ? __ldg(p.scale + bb) : 0.f;
             }
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             const bool row_ok = row < p.R;
             if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
             tc_fence_after_sync();
-            const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(lane_grp * 32) << 16);
+            const uint32_t t_lane = tmem_base + buf * (uint32_t)ACC_COLS + ((uint32_t)(lane_grp * 32) << 16);
 #pragma unroll
             for (int k = 0; k < MY_GROUPS; ++k) {
                 const int g = half + 2 * k;
-                if (g >= TOK / 16) break;
-                uint32_t acc[ND][16];
+                uint32_t acc[ND][8];
 #pragma unroll
-                for (int d = 0; d < ND; ++d) tmem_ld16(t_lane + (uint32_t)(d * TOK + g * 16), acc[d]);
-                const int b0 = jt * TOK + g * 16;
+                for (int d = 0; d < ND; ++d) tmem_ld8(t_lane + (uint32_t)(d * TOK + g * 8), acc[d]);
+                const int b0 = jt * TOK + g * 8;
                 const float my_scale = scales[k];
                 tmem_ld_wait();
-                const int n_live = min(16, p.B - b0);   // uniform across the warp
+                const int n_live = min(8, p.B - b0);   // uniform across the warp
                 // digits -> fp32: lo and hi are exact 32-bit integers; their conversions and the
                 // fused multiply-add round at 2^-24 of |hi|*65536 and |lo|.  (64-bit integer and
                 // double conversions are far too slow on this part to sit in this loop.)
-                float val[16];
+                float val[8];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
+                for (int i = 0; i < 8; ++i) {
                     float f;
                     if constexpr (ND == 1) {
                         f = (float)(int)acc[0][i];
@@ -421,11 +428,11 @@ ternary_mma_kernel(const GemmParams p)
                 if constexpr (EPI == EPI_V) {
                     float* tp = p.t + (size_t)b0 * p.t_ld + row;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
+                    for (int i = 0; i < 8; ++i)
                         if (i < n_live) tp[(size_t)i * p.t_ld] = s_row * val[i];   // the K multiplications (Table S1)
                     if (p.z_out && row_ok) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
+                        for (int i = 0; i < 8; ++i) {
                             if (i < n_live) {
                                 const size_t o = (size_t)(b0 + i) * p.z_ld + row;
                                 if (p.z_int) reinterpret_cast<int*>(p.z_out)[o] = (int)acc[0][i];
@@ -436,12 +443,12 @@ ternary_mma_kernel(const GemmParams p)
                 } else if constexpr (EPI == EPI_U_F32) {
                     float* yp = reinterpret_cast<float*>(p.y) + (size_t)b0 * p.ldy + row;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
+                    for (int i = 0; i < 8; ++i)
                         if (row_ok && i < n_live) yp[(size_t)i * p.ldy] = val[i];
                 } else {
                     uint16_t* yp = reinterpret_cast<uint16_t*>(p.y) + (size_t)b0 * p.ldy + row;
 #pragma unroll
-                    for (int i = 0; i < 16; i += 2) {
+                    for (int i = 0; i < 8; i += 2) {
                         // one conversion instruction rounds two values (to nearest even)
                         const __nv_bfloat162 pr = __floats2bfloat162_rn(val[i], val[i + 1]);
                         const uint32_t u = *reinterpret_cast<const uint32_t*>(&pr);
