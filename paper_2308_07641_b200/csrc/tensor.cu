@@ -23,8 +23,8 @@ constexpr int BLOCK_C = 128;   // contraction elements per pipeline stage (one 1
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
 constexpr int NT_MAX = 192;    // MMA N extent: digit rows per tile
 constexpr int NP = 6;          // ring depth of the packed codes (shared memory)
-constexpr int NB = 6;          // ring depth of the digit tiles (shared memory)
-constexpr int NA = 4;          // ring depth of the expanded operand (tensor memory)
+constexpr int NS = 4;          // ring depth of the operand slots: digit tile (shared memory) + expanded
+                               // ternary tile (tensor memory)
 // tensor memory: two accumulator buffers of 192 columns, then four 32-column slots that hold
 // the expanded ternary operand (128 rows x 128 int8 = 32 columns of 32 bits per row)
 constexpr int TMEM_COLS = 512;
@@ -42,7 +42,7 @@ __host__ __device__ constexpr int tokens_per_tile(int nd) { return 192 / nd; }
 
 constexpr int P_TILE_BYTES = BLOCK_R * BLOCK_C / 4;      // packed codes of that tile, 4 KiB
 constexpr int B_TILE_BYTES_MAX = NT_MAX * BLOCK_C;       // digit rows, 24 KiB
-constexpr int GEMM_SMEM_BYTES = NB * B_TILE_BYTES_MAX + NP * P_TILE_BYTES +
+constexpr int GEMM_SMEM_BYTES = NS * B_TILE_BYTES_MAX + NP * P_TILE_BYTES +
                                 1024 /*alignment slack*/ + 512 /*barriers*/;
 
 // ---------------------------------------------------------------------------------------
@@ -223,20 +223,20 @@ ternary_mma_kernel(const GemmParams p)
     //   A: expanded int8 operand (tensor memory), lives from expansion to the end of its MMAs;
     //      it never touches shared memory, whose bandwidth the digit tiles need
     //   B: digit tiles (24 KiB, shared memory), live from the copy's issue to the end of their MMAs
-    // One "MMAs done" barrier per contraction block serves both A and B (every tcgen05.commit
-    // between MMAs costs issue time): block `it` signals done_bar[it % NB], and an A slot is
-    // free again when block it - NA has signalled.
+    // A and B share their slot index: one "operands ready" barrier per slot (the copy's byte count
+    // plus one arrival per expander warp) and one "MMAs done" barrier, so that the single thread
+    // that issues the MMAs does one wait and one commit per contraction block; that thread's
+    // instruction stream is the critical path of the kernel.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* b_tiles = smem;                                 // NB x 24 KiB, 1024-aligned
-    uint8_t* p_tiles = b_tiles + NB * B_TILE_BYTES_MAX;      // NP x 4 KiB
+    uint8_t* b_tiles = smem;                                 // NS x 24 KiB, 1024-aligned
+    uint8_t* p_tiles = b_tiles + NS * B_TILE_BYTES_MAX;      // NP x 4 KiB
     uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + NP * P_TILE_BYTES);
     uint64_t* pfull_bar = bars;                      // [NP] packed codes landed
     uint64_t* pempty_bar = pfull_bar + NP;           // [NP] expanders have read them
-    uint64_t* afull_bar = pempty_bar + NP;           // [NA] expanded operand written
-    uint64_t* bfull_bar = afull_bar + NA;            // [NB] digit tile landed
-    uint64_t* done_bar = bfull_bar + NB;             // [NB] the MMAs of a contraction block have completed
-    uint64_t* accfull_bar = done_bar + NB;           // [2] all MMAs of a tile have completed
+    uint64_t* ready_bar = pempty_bar + NP;           // [NS] digit tile landed and expanded operand written
+    uint64_t* done_bar = ready_bar + NS;             // [NS] the MMAs reading the slot have completed
+    uint64_t* accfull_bar = done_bar + NS;           // [2] all MMAs of a tile have completed
     uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accempty_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -247,8 +247,10 @@ ternary_mma_kernel(const GemmParams p)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NP; ++s) { mbar_init(&pfull_bar[s], 1); mbar_init(&pempty_bar[s], 4); }
-        for (int s = 0; s < NA; ++s) mbar_init(&afull_bar[s], 4);   // one arrival per expander warp of the group
-        for (int s = 0; s < NB; ++s) { mbar_init(&bfull_bar[s], 1); mbar_init(&done_bar[s], 1); }
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(&ready_bar[s], 5);   // the copy's expect-tx arrival + one per expander warp of the group
+            mbar_init(&done_bar[s], 1);
+        }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&accfull_bar[i], 1);
             mbar_init(&accempty_bar[i], 8);  // one arrival per epilogue warp
@@ -271,8 +273,8 @@ ternary_mma_kernel(const GemmParams p)
         // ---- copy producers: warp 0 streams the digit tiles, warp 2 the packed codes ----
         if (lane == 0) {
             const bool is_b = warp == 0;
-            const int depth = is_b ? NB : NP;
-            uint64_t* full = is_b ? bfull_bar : pfull_bar;
+            const int depth = is_b ? NS : NP;
+            uint64_t* full = is_b ? ready_bar : pfull_bar;
             uint64_t* empty = is_b ? done_bar : pempty_bar;
             const uint32_t bytes = is_b ? B_TILE_BYTES : (uint32_t)P_TILE_BYTES;
             uint32_t it = 0;      // pipeline slot counter across all tiles of this CTA
@@ -302,31 +304,30 @@ ternary_mma_kernel(const GemmParams p)
     } else if (warp == 1) {
         // ---- MMA issue: one thread ----
         if (lane == 0) {
-            uint32_t it = 0, local = 0;
+            // slot index and phase are carried as counters, descriptors are precomputed: this loop
+            // must issue a contraction block in fewer cycles than the block takes to execute
+            uint32_t slot = 0, phase = 0, local = 0;
+            const uint64_t b_desc0 = umma_desc_k_sw128(smem_u32(b_tiles));
             bool alive = true;
             for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++local) {
                 const uint32_t buf = local & 1;
                 if (!mbar_wait(&accempty_bar[buf], ((local >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
-                for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int sa = it % NA, sb = it % NB;
-                    if (!mbar_wait(&bfull_bar[sb], (it / NB) & 1, abort_flag) ||
-                        !mbar_wait(&afull_bar[sa], (it / NA) & 1, abort_flag)) {
-                        alive = false;
-                        break;
-                    }
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait(&ready_bar[slot], phase, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a_tmem = tmem_base + (uint32_t)(A_COL0 + sa * A_SLOT_COLS);
-                    const uint64_t b_desc = umma_desc_k_sw128(smem_u32(b_tiles + sb * B_TILE_BYTES_MAX));
+                    const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + slot * (uint32_t)A_SLOT_COLS;
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_TILE_BYTES_MAX >> 4));
+                    // 32 contraction elements per instruction: 8 columns of A, 32 bytes of the
+                    // swizzled 128-byte rows of B
+                    umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != 0);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_C / UMMA_K; ++k) {
-                        // 32 contraction elements per instruction: 8 columns of A, 32 bytes of the
-                        // swizzled 128-byte rows of B
+                    for (int k = 1; k < BLOCK_C / UMMA_K; ++k)
                         umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)),
-                                   b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, (kb | k) != 0);
-                    }
-                    umma_commit(&done_bar[sb]);   // block `it` is done: frees B slot sb and A slot sa
+                                   b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, true);
+                    umma_commit(&done_bar[slot]);   // the slot (A and B) is free when these MMAs are done
+                    if (++slot == NS) { slot = 0; phase ^= 1; }
                 }
                 umma_commit(&accfull_bar[buf]);
             }
@@ -342,7 +343,7 @@ ternary_mma_kernel(const GemmParams p)
         for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 if ((it & 1u) != group) continue;
-                const int sp = it % NP, sa = it % NA;
+                const int sp = it % NP, sa = it % NS;
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_TILE_BYTES);
                 uint32_t o[32];   // the row's 128 int8 values, four per 32-bit column
@@ -356,16 +357,13 @@ ternary_mma_kernel(const GemmParams p)
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // codes are in registers: slot reusable
-                if (it >= (uint32_t)NA) {   // the A slot is free once block it - NA has completed
-                    const uint32_t j = it - NA;
-                    if (!mbar_wait(&done_bar[j % NB], (j / NB) & 1, abort_flag)) { alive = false; break; }
-                    tc_fence_after_sync();
-                }
+                if (!mbar_wait(&done_bar[sa], ((it / NS) & 1) ^ 1, abort_flag)) { alive = false; break; }
+                tc_fence_after_sync();
                 tmem_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS), o);
                 tmem_st_wait();
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&afull_bar[sa]);
+                if (lane == 0) mbar_arrive(&ready_bar[sa]);
             }
         }
     } else if (warp >= EPI_WARP0) {
