@@ -22,9 +22,9 @@ constexpr int BLOCK_R = 128;   // ternary rows per CTA tile = MMA M
 constexpr int BLOCK_C = 128;   // contraction elements per pipeline stage (one 128-byte swizzle row)
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
 constexpr int NT_MAX = 192;    // MMA N extent: digit rows per tile
-constexpr int NP = 6;          // ring depth of the packed codes (shared memory)
-constexpr int NS = 4;          // ring depth of the operand slots: digit tile (shared memory) + expanded
-                               // ternary tile (tensor memory)
+constexpr int NP = 8;          // ring depth of the packed codes (shared memory)
+constexpr int NB = 8;          // ring depth of the digit tiles (shared memory) and of the per-block barriers
+constexpr int NA = 4;          // ring depth of the expanded ternary operand (tensor memory)
 // tensor memory: two accumulator buffers of 192 columns, then four 32-column slots that hold
 // the expanded ternary operand (128 rows x 128 int8 = 32 columns of 32 bits per row)
 constexpr int TMEM_COLS = 512;
@@ -42,7 +42,7 @@ __host__ __device__ constexpr int tokens_per_tile(int nd) { return 192 / nd; }
 
 constexpr int P_TILE_BYTES = BLOCK_R * BLOCK_C / 4;      // packed codes of that tile, 4 KiB
 constexpr int B_TILE_BYTES_MAX = NT_MAX * BLOCK_C;       // digit rows, 24 KiB
-constexpr int GEMM_SMEM_BYTES = NS * B_TILE_BYTES_MAX + NP * P_TILE_BYTES +
+constexpr int GEMM_SMEM_BYTES = NB * B_TILE_BYTES_MAX + NP * P_TILE_BYTES +
                                 1024 /*alignment slack*/ + 512 /*barriers*/;
 
 // ---------------------------------------------------------------------------------------
@@ -223,20 +223,21 @@ ternary_mma_kernel(const GemmParams p)
     //   A: expanded int8 operand (tensor memory), lives from expansion to the end of its MMAs;
     //      it never touches shared memory, whose bandwidth the digit tiles need
     //   B: digit tiles (24 KiB, shared memory), live from the copy's issue to the end of their MMAs
-    // A and B share their slot index: one "operands ready" barrier per slot (the copy's byte count
-    // plus one arrival per expander warp) and one "MMAs done" barrier, so that the single thread
-    // that issues the MMAs does one wait and one commit per contraction block; that thread's
-    // instruction stream is the critical path of the kernel.
+    // Contraction block `it` uses barrier pair it % NB: "operands ready" (the digit copy's byte
+    // count plus one arrival per expander warp) and "MMAs done", so that the warp that issues
+    // the MMAs does one wait and one commit per block; its instruction stream is the critical
+    // path of the kernel.  The digit tile sits in slot it % NB, the expanded operand in tensor-
+    // memory slot it % NA, which is free again once block it - NA is done.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* b_tiles = smem;                                 // NS x 24 KiB, 1024-aligned
-    uint8_t* p_tiles = b_tiles + NS * B_TILE_BYTES_MAX;      // NP x 4 KiB
+    uint8_t* b_tiles = smem;                                 // NB x 24 KiB, 1024-aligned
+    uint8_t* p_tiles = b_tiles + NB * B_TILE_BYTES_MAX;      // NP x 4 KiB
     uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + NP * P_TILE_BYTES);
     uint64_t* pfull_bar = bars;                      // [NP] packed codes landed
     uint64_t* pempty_bar = pfull_bar + NP;           // [NP] expanders have read them
-    uint64_t* ready_bar = pempty_bar + NP;           // [NS] digit tile landed and expanded operand written
-    uint64_t* done_bar = ready_bar + NS;             // [NS] the MMAs reading the slot have completed
-    uint64_t* accfull_bar = done_bar + NS;           // [2] all MMAs of a tile have completed
+    uint64_t* ready_bar = pempty_bar + NP;           // [NB] digit tile landed and expanded operand written
+    uint64_t* done_bar = ready_bar + NB;             // [NB] the MMAs of the block have completed
+    uint64_t* accfull_bar = done_bar + NB;           // [2] all MMAs of a tile have completed
     uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accempty_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -247,7 +248,7 @@ ternary_mma_kernel(const GemmParams p)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NP; ++s) { mbar_init(&pfull_bar[s], 1); mbar_init(&pempty_bar[s], 4); }
-        for (int s = 0; s < NS; ++s) {
+        for (int s = 0; s < NB; ++s) {
             mbar_init(&ready_bar[s], 5);   // the copy's expect-tx arrival + one per expander warp of the group
             mbar_init(&done_bar[s], 1);
         }
@@ -270,31 +271,36 @@ ternary_mma_kernel(const GemmParams p)
     // Waiting for parity 1 on a barrier that has not completed a phase yet returns at once,
     // which is what a consumer-release barrier needs on its first use.
     if (warp == 0 || warp == 2) {
-        // ---- copy producers: warp 0 streams the digit tiles, warp 2 the packed codes ----
-        if (lane == 0) {
+        // ---- copy producers: warp 0 streams the digit tiles, warp 2 the packed codes.  The whole
+        //      warp runs the loop (uniform control flow); one elected lane issues the copies ----
+        {
             const bool is_b = warp == 0;
-            const int depth = is_b ? NS : NP;
+            const uint32_t depth = is_b ? NB : NP;
             uint64_t* full = is_b ? ready_bar : pfull_bar;
             uint64_t* empty = is_b ? done_bar : pempty_bar;
             const uint32_t bytes = is_b ? B_TILE_BYTES : (uint32_t)P_TILE_BYTES;
-            uint32_t it = 0;      // pipeline slot counter across all tiles of this CTA
+            const uint32_t slot_bytes = is_b ? (uint32_t)B_TILE_BYTES_MAX : (uint32_t)P_TILE_BYTES;
+            uint8_t* ring = is_b ? b_tiles : p_tiles;
+            uint32_t slot = 0, phase = 0, issued = 0;
             bool alive = true;
             for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
                 const int rt = tile % p.row_tiles, jt = tile / p.row_tiles;
                 const uint8_t* src = is_b ? reinterpret_cast<const uint8_t*>(p.D) + (size_t)jt * KB * B_TILE_BYTES
                                           : reinterpret_cast<const uint8_t*>(p.units) + (size_t)rt * KB * P_TILE_BYTES;
-                for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % depth;
-                    if (!mbar_wait(&empty[s], ((it / depth) & 1) ^ 1, abort_flag)) { alive = false; break; }
-                    mbar_arrive_expect_tx(&full[s], bytes);
-                    uint8_t* dst = is_b ? b_tiles + s * B_TILE_BYTES_MAX : p_tiles + s * P_TILE_BYTES;
-                    bulk_g2s(dst, src + (size_t)kb * bytes, bytes, &full[s]);
+                for (int kb = 0; kb < KB; ++kb, ++issued) {
+                    if (!mbar_wait(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
+                    if (elect_one()) {
+                        mbar_arrive_expect_tx(&full[slot], bytes);
+                        bulk_g2s(ring + slot * slot_bytes, src + (size_t)kb * bytes, bytes, &full[slot]);
+                    }
+                    __syncwarp();
+                    if (++slot == depth) { slot = 0; phase ^= 1; }
                 }
             }
-            if (*abort_flag) {
+            if (*abort_flag && lane == 0) {
                 // a wait gave up somewhere: let this CTA's own copies land before it exits (bounded)
-                const uint32_t first = it > (uint32_t)depth ? it - depth : 0u;
-                for (uint32_t j = first; j < it; ++j) {
+                const uint32_t first = issued > depth ? issued - depth : 0u;
+                for (uint32_t j = first; j < issued; ++j) {
                     uint64_t* bar = &full[j % depth];
                     const uint32_t ph = (j / depth) & 1;
                     for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(bar, ph); ++spin) {}
@@ -302,12 +308,15 @@ ternary_mma_kernel(const GemmParams p)
             }
         }
     } else if (warp == 1) {
-        // ---- MMA issue: one thread ----
-        if (lane == 0) {
-            // slot index and phase are carried as counters, descriptors are precomputed: this loop
-            // must issue a contraction block in fewer cycles than the block takes to execute
-            uint32_t slot = 0, phase = 0, local = 0;
+        // ---- MMA issue.  The whole warp runs the loop so that slot, phase and the operand
+        //      descriptors stay warp-uniform (the MMA instructions take them from the uniform
+        //      register file); one elected lane issues the MMAs and commits. ----
+        {
+            uint32_t slot = 0, phase = 0, aslot = 0, local = 0;
             const uint64_t b_desc0 = umma_desc_k_sw128(smem_u32(b_tiles));
+            // readiness of the next slot is tested (without blocking) while the current block's
+            // MMAs are being issued, so that the barrier's latency is off the issue path
+            bool ready = mbar_test_wait(&ready_bar[0], 0);
             bool alive = true;
             for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++local) {
                 const uint32_t buf = local & 1;
@@ -315,21 +324,28 @@ ternary_mma_kernel(const GemmParams p)
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
                 for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait(&ready_bar[slot], phase, abort_flag)) { alive = false; break; }
+                    if (!ready && !mbar_wait(&ready_bar[slot], phase, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + slot * (uint32_t)A_SLOT_COLS;
+                    const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
                     const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_TILE_BYTES_MAX >> 4));
-                    // 32 contraction elements per instruction: 8 columns of A, 32 bytes of the
-                    // swizzled 128-byte rows of B
-                    umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != 0);
+                    const uint32_t cur = slot;
+                    if (++slot == NB) { slot = 0; phase ^= 1; }
+                    aslot = (aslot + 1) & (NA - 1);
+                    if (elect_one()) {
+                        // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
+                        // the swizzled 128-byte rows of B
+                        umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != 0);
 #pragma unroll
-                    for (int k = 1; k < BLOCK_C / UMMA_K; ++k)
-                        umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)),
-                                   b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, true);
-                    umma_commit(&done_bar[slot]);   // the slot (A and B) is free when these MMAs are done
-                    if (++slot == NS) { slot = 0; phase ^= 1; }
+                        for (int k = 1; k < BLOCK_C / UMMA_K; ++k)
+                            umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)),
+                                       b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, true);
+                        umma_commit(&done_bar[cur]);   // frees the digit slot and, NA blocks on, the A slot
+                    }
+                    __syncwarp();
+                    ready = mbar_test_wait(&ready_bar[slot], phase);
                 }
-                umma_commit(&accfull_bar[buf]);
+                if (elect_one()) umma_commit(&accfull_bar[buf]);
+                __syncwarp();
             }
         }
     } else if (warp >= EXP_WARP0 && warp < EXP_WARP0 + 8) {
@@ -343,7 +359,7 @@ ternary_mma_kernel(const GemmParams p)
         for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 if ((it & 1u) != group) continue;
-                const int sp = it % NP, sa = it % NS;
+                const int sp = it % NP, sa = it % NA, sb = it % NB;
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_TILE_BYTES);
                 uint32_t o[32];   // the row's 128 int8 values, four per 32-bit column
@@ -357,13 +373,16 @@ ternary_mma_kernel(const GemmParams p)
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // codes are in registers: slot reusable
-                if (!mbar_wait(&done_bar[sa], ((it / NS) & 1) ^ 1, abort_flag)) { alive = false; break; }
-                tc_fence_after_sync();
+                if (it >= (uint32_t)NA) {   // the A slot is free once block it - NA is done
+                    const uint32_t j = it - NA;
+                    if (!mbar_wait(&done_bar[j % NB], (j / NB) & 1, abort_flag)) { alive = false; break; }
+                    tc_fence_after_sync();
+                }
                 tmem_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS), o);
                 tmem_st_wait();
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&ready_bar[sa]);
+                if (lane == 0) mbar_arrive(&ready_bar[sb]);
             }
         }
     } else if (warp >= EPI_WARP0) {
