@@ -497,6 +497,15 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
 {
     constexpr int TOK = tokens_per_tile(ND);
     const int B_pad = (B + TOK - 1) / TOK * TOK;
+    // ask for the same shared-memory carve-out as the contraction kernels that run before and
+    // after this one, so that the SMs are not reconfigured between the launches of a forward
+    static bool carveout_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !carveout_set[dev]) {
+        cudaFuncSetAttribute(digitise_kernel<IN_T, ND>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared);
+        carveout_set[dev] = true;
+    }
     digitise_kernel<IN_T, ND><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D, scale,
                                                                    zero_me);
     tsvd_count_launch();
