@@ -204,13 +204,15 @@ static tsvd_status_t ensure_ws(tsvd_handle_s* h, size_t bytes)
     return TSVD_OK;
 }
 
-// The dispatch rule shared by tsvd_plan and tsvd_forward_ex: batches go to the tensor cores,
-// a handful of columns to the CUDA-core kernels.
+// The dispatch rule shared by tsvd_plan and tsvd_forward_ex.  The tensor-core kernels serve every
+// batch size (a small batch leaves most of a tile's columns empty, yet still streams the packed
+// codes several times faster than the CUDA-core kernels); the CUDA-core kernels remain as the
+// plain reference path, on request.
 static unsigned choose_path(int B, unsigned forced)
 {
-    if (forced == TSVD_FLAG_PATH_TENSOR) return TSVD_FLAG_PATH_TENSOR;
-    if (forced == TSVD_FLAG_PATH_SIMPLE || forced == TSVD_FLAG_PATH_DECODE) return TSVD_FLAG_PATH_SIMPLE;
-    return B >= 32 ? TSVD_FLAG_PATH_TENSOR : TSVD_FLAG_PATH_SIMPLE;
+    (void)B;
+    if (forced == TSVD_FLAG_PATH_SIMPLE) return TSVD_FLAG_PATH_SIMPLE;
+    return TSVD_FLAG_PATH_TENSOR;
 }
 
 extern "C" tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, unsigned flags, unsigned* path,

@@ -95,10 +95,12 @@ __device__ __forceinline__ void load16(const IN_T* __restrict__ row, int c0, int
     }
 }
 
-// One warp per token slot b in [0, B_pad); 8 tokens per block.  ND digits.  `amax_bits`
-// (optional) holds the precomputed max |value| of each token as float bits; otherwise the warp
-// reduces it.  For int8 input (ND == 1) the values are their own single digit and the scale is 1.
-template <typename IN_T, int ND>
+// TPT threads per token slot b in [0, B_pad): one warp (8 tokens per block) for large batches,
+// a whole block of 256 for small ones, where a row must be spread over more threads to hide
+// latency.  ND digits.  `amax_bits` (optional) holds the precomputed max |value| of each token
+// as float bits; otherwise the token's threads reduce it.  For int8 input (ND == 1) the
+// values are their own single digit and the scale is 1.
+template <typename IN_T, int ND, int TPT>
 __global__ void __launch_bounds__(256)
 digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
@@ -107,9 +109,11 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     constexpr int TOK = tokens_per_tile(ND);
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
-    const int lane = threadIdx.x & 31;
-    const int b = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (b >= B_pad) return;
+    static_assert(TPT == 32 || TPT == 256, "one warp or one block per token");
+    const int lane = threadIdx.x % TPT;                       // index among the token's threads
+    const int b = blockIdx.x * (256 / TPT) + threadIdx.x / TPT;
+    if (b >= B_pad) return;                                   // (whole block when TPT == 256)
+    __shared__ float red[8];
     const int jt = b / TOK, b_in = b % TOK;
     const bool live = b < B;
     const IN_T* row = in + (size_t)b * ld_in;
@@ -125,7 +129,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
             if (amax_bits) {
                 amax = __uint_as_float(amax_bits[b]);
             } else {
-                for (int ch = lane; ch < n_chunks; ch += 32) {
+                for (int ch = lane; ch < n_chunks; ch += TPT) {
                     float v[16];
                     load16<IN_T>(row, ch * 16, C, vec_ok, v);
 #pragma unroll
@@ -133,6 +137,12 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
                 }
                 for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
             }
+        }
+        if constexpr (TPT == 256) {   // block-wide maximum (every thread of the block is here)
+            if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+            __syncthreads();
+#pragma unroll
+            for (int w = 0; w < 8; ++w) amax = fmaxf(amax, red[w]);
         }
         // |v| <= amax < 2^E; quantise to q = rint(v * 2^(8ND-2-E)), so |q| <= 2^(8ND-2)
         int E = -90;
@@ -148,7 +158,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     }
 
     // each lane converts chunks of 16 consecutive contraction elements
-    for (int ch = lane; ch < n_chunks; ch += 32) {
+    for (int ch = lane; ch < n_chunks; ch += TPT) {
         const int kb = ch >> 3, cc = ch & 7;
         uint32_t dig[ND][4];
 #pragma unroll
@@ -497,17 +507,12 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
 {
     constexpr int TOK = tokens_per_tile(ND);
     const int B_pad = (B + TOK - 1) / TOK * TOK;
-    // ask for the same shared-memory carve-out as the contraction kernels that run before and
-    // after this one, so that the SMs are not reconfigured between the launches of a forward
-    static bool carveout_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !carveout_set[dev]) {
-        cudaFuncSetAttribute(digitise_kernel<IN_T, ND>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             cudaSharedmemCarveoutMaxShared);
-        carveout_set[dev] = true;
-    }
-    digitise_kernel<IN_T, ND><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D, scale,
-                                                                   zero_me);
+    if (B_pad * 32 >= 148 * 1024 || KB < 8)   // enough warps to fill the GPU, or short rows
+        digitise_kernel<IN_T, ND, 32><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D,
+                                                                           scale, zero_me);
+    else
+        digitise_kernel<IN_T, ND, 256><<<B_pad, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D, scale,
+                                                                  zero_me);
     tsvd_count_launch();
     if (B_pad_out) *B_pad_out = B_pad;
     return cudaGetLastError();
