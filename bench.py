@@ -38,6 +38,48 @@ PEAKS_COPY = {"hbm_gbs": 6524.9, "bf16_tflops": 1681.0, "bf16_tflops_sustained":
 INT8_OVER_BF16 = 2.0  # nominal dense tensor ratio (4.5 / 2.25 PFLOP/s)
 
 
+def max_over_ranks(dist, value, device):
+    """Max of a per-rank scalar over all ranks (the time every N-GPU number is taken on)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(world, tokens_per_rank, ms_per_step_max):
+    """Whole-job throughput of `world` replicas that each process their own tokens per step."""
+    return world * tokens_per_rank / (ms_per_step_max * 1e-3)
+
+
+def rank_spec(spec, rank):
+    """Rank r works on its own tokens of the same layer (weak scaling: same B per rank)."""
+    return gen.scaled(spec, seed=spec.seed + 1000 * rank) if rank else spec
+
+
+def kernel_source_sha1():
+    import hashlib
+    h = hashlib.sha1()
+    for name in ("tensor.cu", "sm100_ptx.cuh", "tsvd_internal.cuh"):
+        with open(os.path.join(ROOT, "paper_2308_07641_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def recorded_traffic(workload, stage):
+    """DRAM bytes per launch from the committed ncu capture, or None when the kernel sources have
+    changed since that capture was taken (profiles/dram_traffic.txt holds JSON)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            d = json.load(f)
+        if d.get("kernel_source_sha1") != kernel_source_sha1():
+            return None
+        return d["bytes_per_launch"][workload][stage]
+    except Exception:
+        return None
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -213,7 +255,7 @@ def main():
     flags = {"auto": 0, "simple": TSVD_FLAG_PATH_SIMPLE, "decode": TSVD_FLAG_PATH_DECODE,
              "tensor": TSVD_FLAG_PATH_TENSOR}[args.path]
     U, V, S = gen.make_weights(spec)
-    x_np = gen.make_x(gen.scaled(spec, seed=spec.seed + 1000 * rank) if rank else spec)
+    x_np = gen.make_x(rank_spec(spec, rank))
     layer = TSVDLinear(U, S, V)
     info = layer.info
     from tests._util import torch_x
@@ -260,12 +302,9 @@ def main():
     stage_ms, stage_n = binding.tsvd_profile_read(layer.handle)
     binding.tsvd_profile_enable(layer.handle, False)
     clocks = sampler.stop() if rank == 0 else None
-    if dist:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(dist, total_ms, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * spec.B / (ms_per_step * 1e-3)
+    value = aggregate_tokens_per_s(world, spec.B, ms_per_step)
 
     # end to end: host buffers, copies inside the timed region
     x_host = torch.from_numpy(x_np.view(np.int16) if spec.x_dtype == "bf16" else x_np).pin_memory()
@@ -281,11 +320,8 @@ def main():
         binding.tsvd_forward_host(layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if dist:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * spec.B / e2e_s, "unit": UNIT,
+    e2e_s = max_over_ranks(dist, e2e_s, "cuda")
+    e2e = {"value": aggregate_tokens_per_s(world, spec.B, e2e_s * 1e3), "unit": UNIT,
            "h2d_bytes_per_step": int(x_host.numel() * x_host.element_size()),
            "d2h_bytes_per_step": int(y_host.numel() * y_host.element_size()), "steps": e2e_steps}
 
@@ -311,7 +347,8 @@ def main():
             peak, peak_note = peaks["bf16_tflops"], "measured bf16 burst"
         achieved = ops / (dom_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved, "peak": peak,
-                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": recorded_traffic(spec.name, binding.STAGE_NAMES[dom]),
                     "peak_source": f"{peak_note}; {peaks_src} (of measured)", "ops_per_launch": ops,
                     "digits": digits}
     else:
