@@ -100,13 +100,12 @@ __device__ __forceinline__ void load16(const IN_T* __restrict__ row, int c0, int
 // latency.  ND digits.  `amax_bits` (optional) holds the precomputed max |value| of each token
 // as float bits; otherwise the token's threads reduce it.  For int8 input (ND == 1) the
 // values are their own single digit and the scale is 1.
-template <typename IN_T, int ND, int TPT>
+template <typename IN_T, int ND, int TPT, int TOK>
 __global__ void __launch_bounds__(256)
 digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
-                unsigned* __restrict__ zero_me)
+                int* __restrict__ zero_buf, int zero_per_token)
 {
-    constexpr int TOK = tokens_per_tile(ND);
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
     static_assert(TPT == 32 || TPT == 256, "one warp or one block per token");
@@ -120,7 +119,8 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     const bool vec_ok = ((((uintptr_t)in) | ((size_t)ld_in * sizeof(IN_T))) & 15) == 0;
     const int n_chunks = KB * 8;
 
-    if (zero_me && lane == 0) zero_me[b] = 0u;
+    if (zero_buf)   // clear this token's slice of the accumulators a later kernel adds into
+        for (int i = lane; i < zero_per_token; i += TPT) zero_buf[(size_t)b * zero_per_token + i] = 0;
 
     float qscale = 1.f;
     if constexpr (!kInt) {
@@ -197,7 +197,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
 // accumulated in one of two tensor-memory buffers, so that the epilogue warps (combine the
 // digits, apply the stage's scaling, store) work on one tile while the next is contracted.
 // ---------------------------------------------------------------------------------------
-enum { EPI_V = 0, EPI_U_F32 = 1, EPI_U_BF16 = 2 };
+enum { EPI_V = 0, EPI_U_F32 = 1, EPI_U_BF16 = 2, EPI_ACC = 3 };
 
 struct GemmParams {
     const uint4* units;   // packed ternary operand
@@ -217,14 +217,32 @@ struct GemmParams {
     int* status;          // device error word
     int row_tiles;        // tiles of 128 rows
     int j_tiles;          // tiles of TOK tokens
+    int ksplit;           // the contraction is cut into this many parts, one tile each (EPI_ACC when > 1)
+    int* acc;             // EPI_ACC: int32 digit sums [B][ND][acc_ld], added to atomically
+    int acc_ld;
 };
 
-template <int ND, int EPI>
+// Tile index -> (row tile, token tile, contraction part); parts of one output tile are adjacent
+// so that they run at the same time.
+struct TileCoord { int rt, jt, kb0, kb1; };
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile)
+{
+    TileCoord c;
+    const int ks = tile % p.ksplit;
+    const int rest = tile / p.ksplit;
+    c.rt = rest % p.row_tiles;
+    c.jt = rest / p.row_tiles;
+    c.kb0 = (int)((long long)ks * p.KB / p.ksplit);
+    c.kb1 = (int)((long long)(ks + 1) * p.KB / p.ksplit);
+    return c;
+}
+
+template <int ND, int EPI, int TOK>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 ternary_mma_kernel(const GemmParams p)
 {
-    constexpr int TOK = tokens_per_tile(ND);
     constexpr int NT = ND * TOK;
+    static_assert(NT % 16 == 0 && NT <= NT_MAX && TOK % 16 == 0, "tile shape");
     constexpr uint32_t B_TILE_BYTES = NT * BLOCK_C;
     constexpr uint32_t IDESC = umma_idesc_s8(BLOCK_R, NT);
 
@@ -254,7 +272,7 @@ ternary_mma_kernel(const GemmParams p)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = p.KB;
-    const int n_tiles = p.row_tiles * p.j_tiles;
+    const int n_tiles = p.row_tiles * p.j_tiles * p.ksplit;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NP; ++s) { mbar_init(&pfull_bar[s], 1); mbar_init(&pempty_bar[s], 4); }
@@ -294,10 +312,10 @@ ternary_mma_kernel(const GemmParams p)
             uint32_t slot = 0, phase = 0, issued = 0;
             bool alive = true;
             for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
-                const int rt = tile % p.row_tiles, jt = tile / p.row_tiles;
-                const uint8_t* src = is_b ? reinterpret_cast<const uint8_t*>(p.D) + (size_t)jt * KB * B_TILE_BYTES
-                                          : reinterpret_cast<const uint8_t*>(p.units) + (size_t)rt * KB * P_TILE_BYTES;
-                for (int kb = 0; kb < KB; ++kb, ++issued) {
+                const TileCoord tc = tile_coord(p, tile);
+                const uint8_t* src = is_b ? reinterpret_cast<const uint8_t*>(p.D) + (size_t)tc.jt * KB * B_TILE_BYTES
+                                          : reinterpret_cast<const uint8_t*>(p.units) + (size_t)tc.rt * KB * P_TILE_BYTES;
+                for (int kb = tc.kb0; kb < tc.kb1; ++kb, ++issued) {
                     if (!mbar_wait(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
                     if (elect_one()) {
                         mbar_arrive_expect_tx(&full[slot], bytes);
@@ -333,7 +351,8 @@ ternary_mma_kernel(const GemmParams p)
                 if (!mbar_wait(&accempty_bar[buf], ((local >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
-                for (int kb = 0; kb < KB; ++kb) {
+                const TileCoord tc = tile_coord(p, tile);
+                for (int kb = tc.kb0; kb < tc.kb1; ++kb) {
                     if (!ready && !mbar_wait(&ready_bar[slot], phase, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
                     const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
@@ -344,7 +363,7 @@ ternary_mma_kernel(const GemmParams p)
                     if (elect_one()) {
                         // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
                         // the swizzled 128-byte rows of B
-                        umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != 0);
+                        umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != tc.kb0);
 #pragma unroll
                         for (int k = 1; k < BLOCK_C / UMMA_K; ++k)
                             umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)),
@@ -367,7 +386,8 @@ ternary_mma_kernel(const GemmParams p)
         uint32_t it = 0;
         bool alive = true;
         for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
-            for (int kb = 0; kb < KB; ++kb, ++it) {
+            const TileCoord tc = tile_coord(p, tile);
+            for (int kb = tc.kb0; kb < tc.kb1; ++kb, ++it) {
                 if ((it & 1u) != group) continue;
                 const int sp = it % NP, sa = it % NA, sb = it % NB;
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
@@ -403,7 +423,8 @@ ternary_mma_kernel(const GemmParams p)
         const int row_in = lane_grp * 32 + lane;
         uint32_t local = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++local) {
-            const int rt = tile % p.row_tiles, jt = tile / p.row_tiles;
+            const TileCoord tc = tile_coord(p, tile);
+            const int rt = tc.rt, jt = tc.jt;
             const int row = rt * BLOCK_R + row_in;
             const uint32_t buf = local & 1;
             // fetch the per-token scales of this warp's groups (8 tokens each; this warp takes
@@ -411,11 +432,13 @@ ternary_mma_kernel(const GemmParams p)
             // scale of token 8*g + (i & 7), 0 beyond the batch
             constexpr int N_GROUPS = TOK / 8;
             constexpr int MY_GROUPS = N_GROUPS / 2;
+            static_assert(N_GROUPS % 2 == 0, "two epilogue warps per lane group share the token groups");
             float scales[MY_GROUPS];
 #pragma unroll
             for (int k = 0; k < MY_GROUPS; ++k) {
                 const int bb = jt * TOK + (half + 2 * k) * 8 + (lane & 7);
-                scales[k] = bb < p.B ? __ldg(p.scale + bb) : 0.f;
+                scales[k] = 0.f;
+                if constexpr (EPI != EPI_ACC) scales[k] = bb < p.B ? __ldg(p.scale + bb) : 0.f;
             }
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
@@ -433,6 +456,18 @@ ternary_mma_kernel(const GemmParams p)
                 const float my_scale = scales[k];
                 tmem_ld_wait();
                 const int n_live = min(8, p.B - b0);   // uniform across the warp
+                if constexpr (EPI == EPI_ACC) {
+                    // part of a split contraction: add the raw digit sums to the global accumulators
+                    // (integer adds commute exactly, so the result does not depend on arrival order)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (i < n_live) {
+#pragma unroll
+                            for (int d = 0; d < ND; ++d)
+                                atomicAdd(p.acc + ((size_t)(b0 + i) * ND + d) * p.acc_ld + row, (int)acc[d][i]);
+                        }
+                    }
+                } else {
                 // digits -> fp32: lo and hi are exact 32-bit integers; their conversions and the
                 // fused multiply-add round at 2^-24 of |hi|*65536 and |lo|.  (64-bit integer and
                 // double conversions are far too slow on this part to sit in this loop.)
@@ -483,6 +518,7 @@ ternary_mma_kernel(const GemmParams p)
                         if (row_ok && i + 1 < n_live) yp[(size_t)(i + 1) * p.ldy] = (uint16_t)(u >> 16);
                     }
                 }
+                }   // EPI != EPI_ACC
             }
             // all tensor-memory reads of this buffer are done: hand it back to the MMA thread
             tc_fence_before_sync();
@@ -501,33 +537,145 @@ ternary_mma_kernel(const GemmParams p)
     }
 }
 
-template <typename IN_T, int ND>
-cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, const unsigned* amax_bits,
-                            int8_t* D, float* scale, unsigned* zero_me, int* B_pad_out, cudaStream_t stream)
+// ---------------------------------------------------------------------------------------
+// Small batches: the contraction is split over several CTAs that add raw int32 digit sums into
+// a global accumulator acc[b][d][row]; these two kernels pick the sums up.
+// ---------------------------------------------------------------------------------------
+template <int ND> __device__ __forceinline__ float combine_digits(const int* __restrict__ a, int stride)
 {
-    constexpr int TOK = tokens_per_tile(ND);
+    if constexpr (ND == 1) return (float)a[0];
+    else if constexpr (ND == 2) return (float)(a[0] + (a[stride] << 8));
+    else {
+        const int lo = a[0] + (a[stride] << 8);
+        int hi = a[2 * stride];
+        if constexpr (ND == 4) hi += a[3 * stride] << 8;
+        return fmaf((float)hi, 65536.f, (float)lo);
+    }
+}
+
+// One block per token slot: v[k] = digits(acc_in[b][.][k]) * scale_in[b] * (S ? S[k] : 1), then the
+// same fixed-point split as digitise_kernel into ND_OUT digits.  Optionally writes V x before the
+// S scale (z_out) and clears the next accumulator.
+template <int ND_IN, int ND_OUT, int TOK>
+__global__ void __launch_bounds__(256)
+digitise_acc_kernel(const int* __restrict__ acc_in, int acc_ld, const float* __restrict__ scale_in,
+                    const float* __restrict__ S, int B, int C, int KB, int8_t* __restrict__ D,
+                    float* __restrict__ scale_out, void* __restrict__ z_out, int z_ld, int z_int,
+                    int* __restrict__ zero_buf, int zero_per_token)
+{
+    constexpr int NT = ND_OUT * TOK;
+    const int b = blockIdx.x;
+    const int jt = b / TOK, b_in = b % TOK;
+    const bool live = b < B;
+    const int* a = acc_in + (size_t)b * ND_IN * acc_ld;
+    const float sc_in = live ? scale_in[b] : 0.f;
+    __shared__ float red[8];
+
+    if (zero_buf)
+        for (int i = threadIdx.x; i < zero_per_token; i += 256) zero_buf[(size_t)b * zero_per_token + i] = 0;
+
+    float amax = 0.f;
+    if (live) {
+        for (int c = threadIdx.x; c < C; c += 256) {
+            const float z = combine_digits<ND_IN>(a + c, acc_ld) * sc_in;
+            if (z_out) {
+                if (z_int) reinterpret_cast<int*>(z_out)[(size_t)b * z_ld + c] = a[c];
+                else reinterpret_cast<float*>(z_out)[(size_t)b * z_ld + c] = z;
+            }
+            amax = fmaxf(amax, fabsf(S ? S[c] * z : z));
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < 8; ++w) amax = fmaxf(amax, red[w]);
+    int E = -90;
+    if (amax > 0.f) {
+        int e;
+        (void)frexpf(amax, &e);
+        E = max(e, -90);
+    }
+    const float qscale = exp2f((float)(8 * ND_OUT - 2 - E));
+    if (threadIdx.x == 0) scale_out[b] = exp2f((float)(E - (8 * ND_OUT - 2)));
+
+    const int n_chunks = KB * 8;
+    for (int ch = threadIdx.x; ch < n_chunks; ch += 256) {
+        const int kb = ch >> 3, cc = ch & 7;
+        uint32_t dig[ND_OUT][4];
+#pragma unroll
+        for (int d = 0; d < ND_OUT; ++d)
+#pragma unroll
+            for (int w = 0; w < 4; ++w) dig[d][w] = 0;
+        if (live) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                const int c = ch * 16 + e;
+                float v = 0.f;
+                if (c < C) {
+                    v = combine_digits<ND_IN>(a + c, acc_ld) * sc_in;
+                    if (S) v *= S[c];   // the K multiplications (Table S1, row "diag(s)(.)")
+                }
+                int q = __float2int_rn(v * qscale);
+#pragma unroll
+                for (int d = 0; d < ND_OUT; ++d) {
+                    int dv;
+                    if (d == ND_OUT - 1) dv = q;
+                    else { dv = (int)(int8_t)(q & 0xFF); q = (q - dv) >> 8; }
+                    dig[d][e >> 2] |= (uint32_t)(dv & 0xFF) << (8 * (e & 3));
+                }
+            }
+        }
+        int8_t* tile = D + ((size_t)jt * KB + kb) * (size_t)(NT * 128);
+#pragma unroll
+        for (int d = 0; d < ND_OUT; ++d) {
+            const int r = d * TOK + b_in;
+            *reinterpret_cast<uint4*>(tile + r * 128 + ((cc ^ (r & 7)) << 4)) =
+                make_uint4(dig[d][0], dig[d][1], dig[d][2], dig[d][3]);
+        }
+    }
+}
+
+// y[b][m] = digits(acc[b][.][m]) * scale[b], stored as fp32 or (one rounding to nearest even) bf16.
+template <int ND, bool BF16_OUT>
+__global__ void __launch_bounds__(256)
+finish_kernel(const int* __restrict__ acc, int acc_ld, const float* __restrict__ scale, int B, int M,
+              void* __restrict__ y, int ldy)
+{
+    const int b = blockIdx.y;
+    const int m = blockIdx.x * 256 + threadIdx.x;
+    if (b >= B || m >= M) return;
+    const float v = combine_digits<ND>(acc + (size_t)b * ND * acc_ld + m, acc_ld) * scale[b];
+    if constexpr (BF16_OUT) reinterpret_cast<__nv_bfloat16*>(y)[(size_t)b * ldy + m] = __float2bfloat16_rn(v);
+    else reinterpret_cast<float*>(y)[(size_t)b * ldy + m] = v;
+}
+
+template <typename IN_T, int ND, int TOK = tokens_per_tile(ND)>
+cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, const unsigned* amax_bits,
+                            int8_t* D, float* scale, int* zero_buf, int zero_per_token, int* B_pad_out,
+                            cudaStream_t stream)
+{
     const int B_pad = (B + TOK - 1) / TOK * TOK;
     if (B_pad * 32 >= 148 * 1024 || KB < 8)   // enough warps to fill the GPU, or short rows
-        digitise_kernel<IN_T, ND, 32><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                                                                           scale, zero_me);
+        digitise_kernel<IN_T, ND, 32, TOK><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits,
+                                                                                D, scale, zero_buf, zero_per_token);
     else
-        digitise_kernel<IN_T, ND, 256><<<B_pad, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D, scale,
-                                                                  zero_me);
+        digitise_kernel<IN_T, ND, 256, TOK><<<B_pad, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D,
+                                                                       scale, zero_buf, zero_per_token);
     tsvd_count_launch();
     if (B_pad_out) *B_pad_out = B_pad;
     return cudaGetLastError();
 }
 
-template <int ND, int EPI>
+template <int ND, int EPI, int TOK = tokens_per_tile(ND)>
 cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
 {
-    constexpr int TOK = tokens_per_tile(ND);
     static bool attr_set[64] = {};   // per instantiation and device
     int dev = 0;
     cudaError_t e0 = cudaGetDevice(&dev);
     if (e0 != cudaSuccess) return e0;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(ternary_mma_kernel<ND, EPI>,
+        cudaError_t e = cudaFuncSetAttribute(ternary_mma_kernel<ND, EPI, TOK>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -535,11 +683,12 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
     GemmParams q = p;
     q.row_tiles = row_tiles;
     q.j_tiles = (p.B + TOK - 1) / TOK;
+    if (q.ksplit < 1) q.ksplit = 1;
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int n_tiles = q.row_tiles * q.j_tiles;
+    const int n_tiles = q.row_tiles * q.j_tiles * q.ksplit;
     const int grid = n_tiles < sms ? n_tiles : sms;
-    ternary_mma_kernel<ND, EPI><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
+    ternary_mma_kernel<ND, EPI, TOK><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
     tsvd_count_launch();
     return cudaGetLastError();
 }
@@ -586,17 +735,134 @@ TensorWs carve(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, void* base)
 
 }  // namespace
 
+namespace {
+
+constexpr int SMALL_TOK = 16;        // tokens per tile on the small-batch path
+constexpr int SMALL_MAX_B = 64;
+
+struct SmallWs {
+    int8_t* Dx; float* scale_x; int* zacc; int8_t* Dt; float* scale_t; int* yacc;
+    size_t total;
+};
+
+SmallWs carve_small(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, void* base)
+{
+    const int ndx = digits_for_x(dt);
+    const size_t Bp = align_up(B, SMALL_TOK);
+    const size_t KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+    const size_t o_dx = take(Bp * ndx * KBv * 128);
+    const size_t o_sx = take(Bp * sizeof(float));
+    const size_t o_za = take(Bp * ndx * (size_t)h->V.R_pad * sizeof(int));
+    const size_t o_dt = take(Bp * ND_T * KBu * 128);
+    const size_t o_st = take(Bp * sizeof(float));
+    const size_t o_ya = take(Bp * ND_T * (size_t)h->U.R_pad * sizeof(int));
+    SmallWs w;
+    char* b = reinterpret_cast<char*>(base);
+    w.Dx = reinterpret_cast<int8_t*>(b + o_dx);
+    w.scale_x = reinterpret_cast<float*>(b + o_sx);
+    w.zacc = reinterpret_cast<int*>(b + o_za);
+    w.Dt = reinterpret_cast<int8_t*>(b + o_dt);
+    w.scale_t = reinterpret_cast<float*>(b + o_st);
+    w.yacc = reinterpret_cast<int*>(b + o_ya);
+    w.total = off;
+    return w;
+}
+
+// how many parts to cut the contraction into so that the tiles about fill the GPU
+int pick_ksplit(int out_tiles, int KB)
+{
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int ks = sms / (out_tiles > 0 ? out_tiles : 1);
+    if (ks > KB) ks = KB;
+    if (ks > 16) ks = 16;
+    return ks < 1 ? 1 : ks;
+}
+
+template <typename IN_T, int NDX>
+tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
+{
+    tsvd_handle_s* h = a.h;
+    const int KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
+    const int Bp = (a.B + SMALL_TOK - 1) / SMALL_TOK * SMALL_TOK;
+    const int j_tiles = Bp / SMALL_TOK;
+    cudaStream_t st = a.stream;
+    cudaError_t e;
+
+    // activations -> digits; clears the V-stage accumulators
+    h->prof.begin(0, st);
+    e = launch_digitise<IN_T, NDX, SMALL_TOK>((const IN_T*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
+                                              w.zacc, NDX * h->V.R_pad, nullptr, st);
+    h->prof.end(st);
+    if (e != cudaSuccess) return TSVD_E_CUDA;
+
+    // V-stage, contraction split across CTAs
+    GemmParams p{};
+    p.units = h->V.units; p.KB = KBv; p.R = h->K; p.D = w.Dx; p.B = a.B; p.status = h->dev_status;
+    p.acc = w.zacc; p.acc_ld = h->V.R_pad;
+    const int v_tiles = h->V.R_pad / BLOCK_R;
+    p.ksplit = pick_ksplit(v_tiles * j_tiles, KBv);
+    h->prof.begin(1, st);
+    e = launch_gemm<NDX, EPI_ACC, SMALL_TOK>(p, v_tiles, st);
+    h->prof.end(st);
+    if (e != cudaSuccess) return TSVD_E_CUDA;
+
+    // z = sums * 2^e (optional z_out), t = S*z -> digits; clears the U-stage accumulators
+    h->prof.begin(2, st);
+    digitise_acc_kernel<NDX, ND_T, SMALL_TOK><<<Bp, 256, 0, st>>>(
+        w.zacc, h->V.R_pad, w.scale_x, h->S, a.B, h->K, KBu, w.Dt, w.scale_t, a.z_out, h->K,
+        a.dtype == TSVD_I8 ? 1 : 0, w.yacc, ND_T * h->U.R_pad);
+    tsvd_count_launch();
+    e = cudaGetLastError();
+    h->prof.end(st);
+    if (e != cudaSuccess) return TSVD_E_CUDA;
+
+    // U-stage, split likewise, then the final conversion
+    GemmParams q{};
+    q.units = h->U.units; q.KB = KBu; q.R = h->M; q.D = w.Dt; q.B = a.B; q.status = h->dev_status;
+    q.acc = w.yacc; q.acc_ld = h->U.R_pad;
+    const int u_tiles = h->U.R_pad / BLOCK_R;
+    q.ksplit = pick_ksplit(u_tiles * j_tiles, KBu);
+    h->prof.begin(3, st);
+    e = launch_gemm<ND_T, EPI_ACC, SMALL_TOK>(q, u_tiles, st);
+    if (e == cudaSuccess) {
+        const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;
+        dim3 grid((h->M + 255) / 256, a.B);
+        if (bf16_out) finish_kernel<ND_T, true><<<grid, 256, 0, st>>>(w.yacc, h->U.R_pad, w.scale_t, a.B, h->M, a.y, a.ldy);
+        else finish_kernel<ND_T, false><<<grid, 256, 0, st>>>(w.yacc, h->U.R_pad, w.scale_t, a.B, h->M, a.y, a.ldy);
+        tsvd_count_launch();
+        e = cudaGetLastError();
+    }
+    h->prof.end(st);
+    return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
+}
+
+}  // namespace
+
 int tsvd_tensor_digits_x(tsvd_dtype_t dt) { return digits_for_x(dt); }
 int tsvd_tensor_digits_t() { return ND_T; }
 
 size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt)
 {
+    if (B <= SMALL_MAX_B) return carve_small(h, B, dt, nullptr).total;
     return carve(h, B, dt, nullptr).total;
 }
 
 tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
 {
     tsvd_handle_s* h = a.h;
+    if (a.B <= SMALL_MAX_B) {
+        // small batches: 16-token tiles, the contraction split across CTAs
+        const SmallWs sw = carve_small(h, a.B, a.dtype, ws);
+        switch (a.dtype) {
+            case TSVD_F32: return forward_small<float, 4>(a, sw);
+            case TSVD_BF16: return forward_small<__nv_bfloat16, 3>(a, sw);
+            case TSVD_I8: return forward_small<int8_t, 1>(a, sw);
+            default: return TSVD_E_DTYPE;
+        }
+    }
     const TensorWs w = carve(h, a.B, a.dtype, ws);
     const int KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
     cudaStream_t st = a.stream;
@@ -606,16 +872,16 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     h->prof.begin(0, st);
     switch (a.dtype) {
         case TSVD_F32:
-            e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, nullptr,
+            e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, nullptr, 0,
                                           nullptr, st);
             break;
         case TSVD_BF16:
             e = launch_digitise<__nv_bfloat16, 3>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
-                                                  w.scale_x, nullptr, nullptr, st);
+                                                  w.scale_x, nullptr, 0, nullptr, st);
             break;
         case TSVD_I8:
             e = launch_digitise<int8_t, 1>((const int8_t*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                           nullptr, nullptr, st);
+                                           nullptr, 0, nullptr, st);
             break;
         default:
             return TSVD_E_DTYPE;
@@ -638,7 +904,7 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
 
     // stage 2: t -> digits (each token's scale comes from its own max |t|)
     h->prof.begin(2, st);
-    e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, nullptr, st);
+    e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, 0, nullptr, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
