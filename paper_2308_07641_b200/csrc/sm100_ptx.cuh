@@ -24,13 +24,6 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 
-// ---- programmatic dependent launch ------------------------------------------------------
-// A kernel launched with the programmatic-serialization attribute may start while its
-// predecessor in the stream is still running; grid_dep_wait() blocks until that predecessor
-// has completed and its writes are visible.  grid_dep_launch() lets the successor start.
-__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
 // ---- mbarrier -------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
 {

@@ -18,26 +18,6 @@ namespace {
 
 using namespace ptx;
 
-// Every kernel of a forward is launched with programmatic stream serialization: its CTAs may
-// be scheduled, and run their set-up, while the previous kernel drains; each kernel calls
-// grid_dep_wait() before it touches anything the previous one wrote.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                       Args... args)
-{
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
 constexpr int BLOCK_R = 128;   // ternary rows per CTA tile = MMA M
 constexpr int BLOCK_C = 128;   // contraction elements per pipeline stage (one 128-byte swizzle row)
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
@@ -129,8 +109,6 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
     static_assert(TPT == 32 || TPT == 256, "one warp or one block per token");
-    grid_dep_launch();
-    grid_dep_wait();   // the input (and the scratch this kernel overwrites) belongs to earlier kernels
     const int lane = threadIdx.x % TPT;                       // index among the token's threads
     const int b = blockIdx.x * (256 / TPT) + threadIdx.x / TPT;
     if (b >= B_pad) return;                                   // (whole block when TPT == 256)
@@ -317,10 +295,6 @@ ternary_mma_kernel(const GemmParams p)
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    // set-up done (barriers, tensor memory): let the next kernel's CTAs be scheduled as this one
-    // drains, and wait for the previous kernel's results before reading or writing global memory
-    grid_dep_launch();
-    grid_dep_wait();
 
     // Waiting for parity 1 on a barrier that has not completed a phase yet returns at once,
     // which is what a consumer-release barrier needs on its first use.
@@ -590,8 +564,6 @@ digitise_acc_kernel(const int* __restrict__ acc_in, int acc_ld, const float* __r
                     int* __restrict__ zero_buf, int zero_per_token)
 {
     constexpr int NT = ND_OUT * TOK;
-    grid_dep_launch();
-    grid_dep_wait();
     const int b = blockIdx.x;
     const int jt = b / TOK, b_in = b % TOK;
     const bool live = b < B;
@@ -670,8 +642,6 @@ __global__ void __launch_bounds__(256)
 finish_kernel(const int* __restrict__ acc, int acc_ld, const float* __restrict__ scale, int B, int M,
               void* __restrict__ y, int ldy)
 {
-    grid_dep_launch();
-    grid_dep_wait();
     const int b = blockIdx.y;
     const int m = blockIdx.x * 256 + threadIdx.x;
     if (b >= B || m >= M) return;
@@ -686,16 +656,15 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
                             cudaStream_t stream)
 {
     const int B_pad = (B + TOK - 1) / TOK * TOK;
-    cudaError_t e;
     if (B_pad * 32 >= 148 * 1024 || KB < 8)   // enough warps to fill the GPU, or short rows
-        e = launch_pdl(digitise_kernel<IN_T, ND, 32, TOK>, dim3((B_pad + 7) / 8), dim3(256), 0, stream, in, ld_in, B,
-                       B_pad, C, KB, amax_bits, D, scale, zero_buf, zero_per_token);
+        digitise_kernel<IN_T, ND, 32, TOK><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits,
+                                                                                D, scale, zero_buf, zero_per_token);
     else
-        e = launch_pdl(digitise_kernel<IN_T, ND, 256, TOK>, dim3(B_pad), dim3(256), 0, stream, in, ld_in, B, B_pad, C,
-                       KB, amax_bits, D, scale, zero_buf, zero_per_token);
+        digitise_kernel<IN_T, ND, 256, TOK><<<B_pad, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D,
+                                                                       scale, zero_buf, zero_per_token);
     tsvd_count_launch();
     if (B_pad_out) *B_pad_out = B_pad;
-    return e != cudaSuccess ? e : cudaGetLastError();
+    return cudaGetLastError();
 }
 
 template <int ND, int EPI, int TOK = tokens_per_tile(ND)>
@@ -719,10 +688,9 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int n_tiles = q.row_tiles * q.j_tiles * q.ksplit;
     const int grid = n_tiles < sms ? n_tiles : sms;
-    cudaError_t e = launch_pdl(ternary_mma_kernel<ND, EPI, TOK>, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES,
-                               stream, q);
+    ternary_mma_kernel<ND, EPI, TOK><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
     tsvd_count_launch();
-    return e != cudaSuccess ? e : cudaGetLastError();
+    return cudaGetLastError();
 }
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -843,11 +811,11 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
 
     // z = sums * 2^e (optional z_out), t = S*z -> digits; clears the U-stage accumulators
     h->prof.begin(2, st);
-    e = launch_pdl(digitise_acc_kernel<NDX, ND_T, SMALL_TOK>, dim3(Bp), dim3(256), 0, st, w.zacc, h->V.R_pad, w.scale_x,
-                   h->S, a.B, h->K, KBu, w.Dt, w.scale_t, a.z_out, h->K, a.dtype == TSVD_I8 ? 1 : 0, w.yacc,
-                   ND_T * h->U.R_pad);
+    digitise_acc_kernel<NDX, ND_T, SMALL_TOK><<<Bp, 256, 0, st>>>(
+        w.zacc, h->V.R_pad, w.scale_x, h->S, a.B, h->K, KBu, w.Dt, w.scale_t, a.z_out, h->K,
+        a.dtype == TSVD_I8 ? 1 : 0, w.yacc, ND_T * h->U.R_pad);
     tsvd_count_launch();
-    if (e == cudaSuccess) e = cudaGetLastError();
+    e = cudaGetLastError();
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
@@ -862,14 +830,10 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
     if (e == cudaSuccess) {
         const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;
         dim3 grid((h->M + 255) / 256, a.B);
-        if (bf16_out)
-            e = launch_pdl(finish_kernel<ND_T, true>, grid, dim3(256), 0, st, w.yacc, h->U.R_pad, w.scale_t, a.B, h->M,
-                           a.y, a.ldy);
-        else
-            e = launch_pdl(finish_kernel<ND_T, false>, grid, dim3(256), 0, st, w.yacc, h->U.R_pad, w.scale_t, a.B, h->M,
-                           a.y, a.ldy);
+        if (bf16_out) finish_kernel<ND_T, true><<<grid, 256, 0, st>>>(w.yacc, h->U.R_pad, w.scale_t, a.B, h->M, a.y, a.ldy);
+        else finish_kernel<ND_T, false><<<grid, 256, 0, st>>>(w.yacc, h->U.R_pad, w.scale_t, a.B, h->M, a.y, a.ldy);
         tsvd_count_launch();
-        if (e == cudaSuccess) e = cudaGetLastError();
+        e = cudaGetLastError();
     }
     h->prof.end(st);
     return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
