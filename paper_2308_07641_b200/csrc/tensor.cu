@@ -122,12 +122,26 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     if (zero_buf)   // clear this token's slice of the accumulators a later kernel adds into
         for (int i = lane; i < zero_per_token; i += TPT) zero_buf[(size_t)b * zero_per_token + i] = 0;
 
+    // Rows of up to two chunks per thread (C <= 1024 with one warp per token, <= 8192 with a
+    // block) are loaded once and kept in registers for both passes.
+    const bool cached = n_chunks <= 2 * TPT;
+    float keep[2][16];
     float qscale = 1.f;
     if constexpr (!kInt) {
         float amax = 0.f;
         if (live) {
             if (amax_bits) {
                 amax = __uint_as_float(amax_bits[b]);
+            } else if (cached) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int ch = lane + j * TPT;
+                    if (ch < n_chunks) {
+                        load16<IN_T>(row, ch * 16, C, vec_ok, keep[j]);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) amax = fmaxf(amax, fabsf(keep[j][e]));
+                    }
+                }
             } else {
                 for (int ch = lane; ch < n_chunks; ch += TPT) {
                     float v[16];
@@ -167,7 +181,13 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
             for (int w = 0; w < 4; ++w) dig[d][w] = 0;
         if (live) {
             float v[16];
-            load16<IN_T>(row, ch * 16, C, vec_ok, v);
+            const int j = ch >= TPT ? 1 : 0;          // ch = lane + j * TPT
+            if (!kInt && cached && !amax_bits) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = j ? keep[1][e] : keep[0][e];
+            } else {
+                load16<IN_T>(row, ch * 16, C, vec_ok, v);
+            }
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
                 int q = __float2int_rn(v[e] * qscale);
@@ -232,8 +252,8 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile)
     const int rest = tile / p.ksplit;
     c.rt = rest % p.row_tiles;
     c.jt = rest / p.row_tiles;
-    c.kb0 = (int)((long long)ks * p.KB / p.ksplit);
-    c.kb1 = (int)((long long)(ks + 1) * p.KB / p.ksplit);
+    c.kb0 = ks * p.KB / p.ksplit;          // ksplit <= 16 and KB < 2^20: no overflow
+    c.kb1 = (ks + 1) * p.KB / p.ksplit;
     return c;
 }
 
