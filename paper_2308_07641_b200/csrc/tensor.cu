@@ -149,8 +149,9 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
 #pragma unroll
                     for (int e = 0; e < 16; ++e) amax = fmaxf(amax, fabsf(v[e]));
                 }
-                for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
             }
+            // warp-wide maximum (live is uniform across the warp)
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
         }
         if constexpr (TPT == 256) {   // block-wide maximum (every thread of the block is here)
             if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
