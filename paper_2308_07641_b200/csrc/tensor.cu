@@ -58,6 +58,27 @@ template <> __device__ __forceinline__ float to_float<float>(float v) { return v
 template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <> __device__ __forceinline__ float to_float<int8_t>(int8_t v) { return (float)v; }
 
+// Balanced radix-256 digits of sixteen fixed-point integers, as ND words of four int8 each per
+// group of four values (dig[d][g] = digit d of values 4g..4g+3).  With q = sum_d digit_d*256^d
+// and digits in [-128,127], digit d is byte d of q + 0x80 + 0x8000 + ... (d terms): adding half
+// the radix at every lower position turns the floor of the arithmetic shift into rounding.
+// The top digit is what is left; it fits because |q| <= 2^(8ND-2).
+template <int ND>
+__device__ __forceinline__ void digits_of_16(const int (&q)[16], uint32_t (&dig)[ND][4])
+{
+#pragma unroll
+    for (int d = 0; d < ND; ++d) {
+        const uint32_t off = d == 0 ? 0u : d == 1 ? 0x80u : d == 2 ? 0x8080u : 0x808080u;
+        const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);   // byte d of a, byte d of b
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const uint32_t lo = __byte_perm((uint32_t)q[4 * g] + off, (uint32_t)q[4 * g + 1] + off, sel);
+            const uint32_t hi = __byte_perm((uint32_t)q[4 * g + 2] + off, (uint32_t)q[4 * g + 3] + off, sel);
+            dig[d][g] = __byte_perm(lo, hi, 0x5410);
+        }
+    }
+}
+
 // Load 16 consecutive values of a row as floats (vector loads when the chunk is whole and
 // 16-byte aligned, guarded scalar loads otherwise).
 template <typename IN_T>
@@ -189,17 +210,10 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
             } else {
                 load16<IN_T>(row, ch * 16, C, vec_ok, v);
             }
+            int q[16];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                int q = __float2int_rn(v[e] * qscale);
-#pragma unroll
-                for (int d = 0; d < ND; ++d) {
-                    int dv;
-                    if (d == ND - 1) dv = q;                       // top digit: what is left
-                    else { dv = (int)(int8_t)(q & 0xFF); q = (q - dv) >> 8; }
-                    dig[d][e >> 2] |= (uint32_t)(dv & 0xFF) << (8 * (e & 3));
-                }
-            }
+            for (int e = 0; e < 16; ++e) q[e] = __float2int_rn(v[e] * qscale);
+            digits_of_16<ND>(q, dig);
         }
         int8_t* tile = D + ((size_t)jt * KB + kb) * (size_t)(NT * 128);
 #pragma unroll
@@ -249,13 +263,29 @@ struct TileCoord { int rt, jt, kb0, kb1; };
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile)
 {
     TileCoord c;
-    const int ks = tile % p.ksplit;
-    const int rest = tile / p.ksplit;
+    int rest = tile;
+    c.kb0 = 0;
+    c.kb1 = p.KB;
+    if (p.ksplit > 1) {
+        const int ks = tile % p.ksplit;
+        rest = tile / p.ksplit;
+        c.kb0 = ks * p.KB / p.ksplit;          // ksplit <= 16 and KB < 2^20: no overflow
+        c.kb1 = (ks + 1) * p.KB / p.ksplit;
+    }
     c.rt = rest % p.row_tiles;
     c.jt = rest / p.row_tiles;
-    c.kb0 = ks * p.KB / p.ksplit;          // ksplit <= 16 and KB < 2^20: no overflow
-    c.kb1 = (ks + 1) * p.KB / p.ksplit;
     return c;
+}
+// The contraction range alone (no divisions when the contraction is not split).
+__device__ __forceinline__ void tile_kb_range(const GemmParams& p, int tile, int& kb0, int& kb1)
+{
+    kb0 = 0;
+    kb1 = p.KB;
+    if (p.ksplit > 1) {
+        const int ks = tile % p.ksplit;
+        kb0 = ks * p.KB / p.ksplit;
+        kb1 = (ks + 1) * p.KB / p.ksplit;
+    }
 }
 
 template <int ND, int EPI, int TOK>
@@ -372,8 +402,9 @@ ternary_mma_kernel(const GemmParams p)
                 if (!mbar_wait(&accempty_bar[buf], ((local >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
-                const TileCoord tc = tile_coord(p, tile);
-                for (int kb = tc.kb0; kb < tc.kb1; ++kb) {
+                int kb0, kb1;
+                tile_kb_range(p, tile, kb0, kb1);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!ready && !mbar_wait(&ready_bar[slot], phase, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
                     const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
@@ -384,7 +415,7 @@ ternary_mma_kernel(const GemmParams p)
                     if (elect_one()) {
                         // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
                         // the swizzled 128-byte rows of B
-                        umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != tc.kb0);
+                        umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != kb0);
 #pragma unroll
                         for (int k = 1; k < BLOCK_C / UMMA_K; ++k)
                             umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)),
@@ -407,8 +438,9 @@ ternary_mma_kernel(const GemmParams p)
         uint32_t it = 0;
         bool alive = true;
         for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
-            const TileCoord tc = tile_coord(p, tile);
-            for (int kb = tc.kb0; kb < tc.kb1; ++kb, ++it) {
+            int kb0, kb1;
+            tile_kb_range(p, tile, kb0, kb1);
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
                 if ((it & 1u) != group) continue;
                 const int sp = it % NP, sa = it % NA, sb = it % NB;
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
@@ -629,6 +661,7 @@ digitise_acc_kernel(const int* __restrict__ acc_in, int acc_ld, const float* __r
 #pragma unroll
             for (int w = 0; w < 4; ++w) dig[d][w] = 0;
         if (live) {
+            int q[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
                 const int c = ch * 16 + e;
@@ -637,15 +670,9 @@ digitise_acc_kernel(const int* __restrict__ acc_in, int acc_ld, const float* __r
                     v = combine_digits<ND_IN>(a + c, acc_ld) * sc_in;
                     if (S) v *= S[c];   // the K multiplications (Table S1, row "diag(s)(.)")
                 }
-                int q = __float2int_rn(v * qscale);
-#pragma unroll
-                for (int d = 0; d < ND_OUT; ++d) {
-                    int dv;
-                    if (d == ND_OUT - 1) dv = q;
-                    else { dv = (int)(int8_t)(q & 0xFF); q = (q - dv) >> 8; }
-                    dig[d][e >> 2] |= (uint32_t)(dv & 0xFF) << (8 * (e & 3));
-                }
+                q[e] = __float2int_rn(v * qscale);
             }
+            digits_of_16<ND_OUT>(q, dig);
         }
         int8_t* tile = D + ((size_t)jt * KB + kb) * (size_t)(NT * 128);
 #pragma unroll
