@@ -122,7 +122,7 @@ __device__ __forceinline__ void load16(const IN_T* __restrict__ row, int c0, int
 // as float bits; otherwise the token's threads reduce it.  For int8 input (ND == 1) the
 // values are their own single digit and the scale is 1.
 template <typename IN_T, int ND, int TPT, int TOK>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)   // <= 64 registers: a batch of 4096 tokens is then one wave
 digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
                 int* __restrict__ zero_buf, int zero_per_token)
