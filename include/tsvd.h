@@ -47,6 +47,12 @@ typedef enum {
 #define TSVD_FLAG_PATH_SIMPLE 0x10u /* force the CUDA-core reference kernels               */
 #define TSVD_FLAG_PATH_DECODE 0x20u /* force the small-batch streaming kernels             */
 #define TSVD_FLAG_PATH_TENSOR 0x40u /* force the tcgen05 tensor-core kernels               */
+/* Test hook for the bounded device-side waits: with B > 64 the V-stage kernel's copy
+ * producer withholds the activation digits, so every wait on them runs out (after a few
+ * milliseconds instead of the usual ~2 s); all CTAs then leave through their normal exit,
+ * y is unspecified, and tsvd_last_status reports TSVD_E_TIMEOUT.  No fault, no hang: the
+ * context and the handle stay usable. */
+#define TSVD_FLAG_TEST_STALL 0x100u
 
 /*
  * tsvd_pack -- store U and V in the 2-bit sign/nonzero form (the paper: "we only

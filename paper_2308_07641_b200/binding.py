@@ -24,6 +24,7 @@ TSVD_FLAG_OUT_F32 = 0x1
 TSVD_FLAG_PATH_SIMPLE = 0x10
 TSVD_FLAG_PATH_DECODE = 0x20
 TSVD_FLAG_PATH_TENSOR = 0x40
+TSVD_FLAG_TEST_STALL = 0x100
 
 DTYPES = {"f32": TSVD_F32, "bf16": TSVD_BF16, "i8": TSVD_I8}
 

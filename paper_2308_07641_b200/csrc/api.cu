@@ -237,7 +237,8 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     if (B < 1) return TSVD_E_SHAPE;
     const size_t xs = dtype_size(dtype);
     if (xs == 0) return TSVD_E_DTYPE;
-    const unsigned known = TSVD_FLAG_OUT_F32 | TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR;
+    const unsigned known = TSVD_FLAG_OUT_F32 | TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR |
+                           TSVD_FLAG_TEST_STALL;
     if (flags & ~known) return TSVD_E_DTYPE;
     const unsigned path = flags & (TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR);
     if (path & (path - 1)) return TSVD_E_DTYPE;  // at most one forced path
@@ -252,6 +253,7 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     a.h = h; a.x = x; a.ldx = ldx; a.y = y; a.ldy = ldy; a.B = B; a.dtype = dtype;
     a.out_f32 = (flags & TSVD_FLAG_OUT_F32) != 0;
     a.z_out = z_out;
+    a.test_stall = (flags & TSVD_FLAG_TEST_STALL) != 0;
     a.stream = (cudaStream_t)stream;
 
     if (choose_path(B, path) == TSVD_FLAG_PATH_TENSOR) {

@@ -69,21 +69,24 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after `limit_cycles` SM clocks, or at once when *abort is already
-// set (another wait of this CTA gave up).  On giving up it sets *abort and returns false;
-// the caller carries on to the kernel's normal exit so that tensor memory is released.
-constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag)
+// Bounded wait.  `ctl` points at two ints in shared memory: ctl[0] is the CTA's abort flag,
+// ctl[1] the wait limit in units of 2^20 SM clocks.  The wait gives up after that many clocks,
+// or at once when the abort flag is already set (another wait of this CTA gave up).  On giving
+// up it sets the flag and returns false; the caller carries on to the kernel's normal exit so
+// that tensor memory is released.
+constexpr int kWaitLimitDefault = 4096;  // 2^32 clocks, about two seconds
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
+    const long long limit = (long long)ctl[1] << 20;
     unsigned spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
-                *abort_flag = 1;
+            if (ctl[0]) return false;
+            if (clock64() - t0 > limit) {
+                ctl[0] = 1;
                 return false;
             }
         }

@@ -255,6 +255,8 @@ struct GemmParams {
     int ksplit;           // the contraction is cut into this many parts, one tile each (EPI_ACC when > 1)
     int* acc;             // EPI_ACC: int32 digit sums [B][ND][acc_ld], added to atomically
     int acc_ld;
+    int wait_limit;       // bound of every barrier wait in units of 2^20 clocks (0: default, ~2 s)
+    int test_stall;       // test hook: the digit tiles are never copied, so the waits must give up
 };
 
 // Tile index -> (row tile, token tile, contraction part); parts of one output tile are adjacent
@@ -335,7 +337,8 @@ ternary_mma_kernel(const GemmParams p)
             mbar_init(&accfull_bar[i], 1);
             mbar_init(&accempty_bar[i], 8);  // one arrival per epilogue warp
         }
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = p.wait_limit > 0 ? p.wait_limit : kWaitLimitDefault;
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -368,6 +371,7 @@ ternary_mma_kernel(const GemmParams p)
                                           : reinterpret_cast<const uint8_t*>(p.units) + (size_t)tc.rt * KB * P_TILE_BYTES;
                 for (int kb = tc.kb0; kb < tc.kb1; ++kb, ++issued) {
                     if (!mbar_wait(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
+                    if (is_b && p.test_stall) { alive = false; break; }   // nothing will ever land
                     if (elect_one()) {
                         mbar_arrive_expect_tx(&full[slot], bytes);
                         bulk_g2s(ring + slot * slot_bytes, src + (size_t)kb * bytes, bytes, &full[slot]);
@@ -942,6 +946,7 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     p.S = h->S; p.t = w.t; p.t_ld = h->V.R_pad;
     p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
     p.status = h->dev_status;
+    if (a.test_stall) { p.test_stall = 1; p.wait_limit = 16; }   // ~8 ms instead of ~2 s
     const int v_tiles = h->V.R_pad / BLOCK_R;
     h->prof.begin(1, st);
     if (a.dtype == TSVD_F32) e = launch_gemm<4, EPI_V>(p, v_tiles, st);

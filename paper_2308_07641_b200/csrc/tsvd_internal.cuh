@@ -110,6 +110,7 @@ struct ForwardArgs {
     tsvd_dtype_t dtype;
     bool out_f32;
     void* z_out;
+    bool test_stall = false;   // TSVD_FLAG_TEST_STALL
     float* t;        // scratch [B][t_ld] fp32: S * (V x)
     int t_ld;
     cudaStream_t stream;

@@ -174,3 +174,31 @@ FULL = [
 @pytest.mark.parametrize("spec,sample", FULL, ids=lambda v: v.name if hasattr(v, "name") else None)
 def test_full_size_sampled(spec, sample):
     _util.run_and_check(spec, sample_tokens=sample)
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """Failure detection without a fault: a forward whose copy producer withholds its data (test
+    hook) must end by itself, report TSVD_E_TIMEOUT through the handle's status word, and leave
+    the context and the handle usable for a correct forward right after."""
+    import time
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear, binding
+    spec = gen.scaled(C["cfg2"], name="stall", M=256, N=256, K=256, B=200, seed=41)
+    U, V, S = gen.make_weights(spec)
+    x = gen.make_x(spec)
+    layer = TSVDLinear(U, S, V)
+    try:
+        xt = _util.torch_x(x, "bf16")
+        assert binding.tsvd_last_status(layer.handle) == binding.TSVD_OK
+        t0 = time.perf_counter()
+        layer.forward(xt, flags=binding.TSVD_FLAG_TEST_STALL)
+        torch.cuda.synchronize()
+        assert time.perf_counter() - t0 < 5.0                      # bounded, not the default 2 s per wait chain
+        assert binding.tsvd_last_status(layer.handle) == binding.TSVD_E_TIMEOUT
+        assert binding.tsvd_last_status(layer.handle) == binding.TSVD_OK   # reading resets the word
+        y64, z, y_bf16 = _util.run_gpu(layer, x, "bf16")
+        ref = oracle.forward(U, S, V, _util.oracle_x(x, "bf16"))
+        _util.check_outputs(y64, z, ref, "bf16", y_bf16, "after a timed-out forward")
+        assert binding.tsvd_last_status(layer.handle) == binding.TSVD_OK
+    finally:
+        layer.close()
