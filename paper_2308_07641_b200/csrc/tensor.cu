@@ -125,7 +125,7 @@ template <typename IN_T, int ND, int TPT, int TOK>
 __global__ void __launch_bounds__(256, 4)   // <= 64 registers: a batch of 4096 tokens is then one wave
 digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
-                int* __restrict__ zero_buf, int zero_per_token)
+                int* __restrict__ zero_buf, int zero_per_token, int zero_total)
 {
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
@@ -141,7 +141,8 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     const int n_chunks = KB * 8;
 
     if (zero_buf)   // clear this token's slice of the accumulators a later kernel adds into
-        for (int i = lane; i < zero_per_token; i += TPT) zero_buf[(size_t)b * zero_per_token + i] = 0;
+        for (int i = lane; i < zero_per_token; i += TPT)
+            if ((size_t)b * zero_per_token + i < (size_t)zero_total) zero_buf[(size_t)b * zero_per_token + i] = 0;
 
     // Rows of up to two chunks per thread (C <= 1024 with one warp per token, <= 8192 with a
     // block) are loaded once and kept in registers for both passes.
@@ -233,6 +234,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
 // digits, apply the stage's scaling, store) work on one tile while the next is contracted.
 // ---------------------------------------------------------------------------------------
 enum { EPI_V = 0, EPI_U_F32 = 1, EPI_U_BF16 = 2, EPI_ACC = 3 };
+enum { TAIL_T = 1, TAIL_Y = 2 };
 
 struct GemmParams {
     const uint4* units;   // packed ternary operand
@@ -255,6 +257,12 @@ struct GemmParams {
     int ksplit;           // the contraction is cut into this many parts, one tile each (EPI_ACC when > 1)
     int* acc;             // EPI_ACC: int32 digit sums [B][ND][acc_ld], added to atomically
     int acc_ld;
+    int* tile_done;       // EPI_ACC: per output tile, how many contraction parts have added their sums
+    int tail;             // EPI_ACC: what the last part to finish does with the complete sums:
+                          //   TAIL_T: t = S*z*scale -> p.t (+ z_out, per-token max |t| -> p.tmax)
+                          //   TAIL_Y: y = sums*scale -> p.y (bf16 when p.y_bf16)
+    unsigned* tmax;       // TAIL_T: per-token max |t| as float bits
+    int y_bf16;
     int wait_limit;       // bound of every barrier wait in units of 2^20 clocks (0: default, ~2 s)
     int test_stall;       // test hook: the digit tiles are never copied, so the waits must give up
 };
@@ -320,8 +328,10 @@ ternary_mma_kernel(const GemmParams p)
     uint64_t* done_bar = ready_bar + NB;             // [NB] the MMAs of the block have completed
     uint64_t* accfull_bar = done_bar + NB;           // [2] all MMAs of a tile have completed
     uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accempty_bar + 2);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint64_t* tail_bar = accempty_bar + 2;           // [2] split contraction: epilogue warps meet, verdict is in
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [2]: flag, wait limit
+    volatile int* tail_last = abort_flag + 2;        // whether this CTA finished its output tile last
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = p.KB;
@@ -337,6 +347,8 @@ ternary_mma_kernel(const GemmParams p)
             mbar_init(&accfull_bar[i], 1);
             mbar_init(&accempty_bar[i], 8);  // one arrival per epilogue warp
         }
+        mbar_init(&tail_bar[0], 8);
+        mbar_init(&tail_bar[1], 1);
         abort_flag[0] = 0;
         abort_flag[1] = p.wait_limit > 0 ? p.wait_limit : kWaitLimitDefault;
         fence_mbar_init();
@@ -581,6 +593,63 @@ ternary_mma_kernel(const GemmParams p)
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&accempty_bar[buf]);
+
+            if constexpr (EPI == EPI_ACC) {
+                // Split contraction: the part that finishes an output tile last turns the complete
+                // sums into the stage's result.  (Sums were added with device-scope atomics; the
+                // fence orders them before the counter.)
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tail_bar[0]);
+                if (!mbar_wait(&tail_bar[0], local & 1, abort_flag)) break;
+                if (warp == EPI_WARP0 && lane == 0) {
+                    const int out_tile = jt * p.row_tiles + rt;
+                    *tail_last = atomicAdd(p.tile_done + out_tile, 1) == p.ksplit - 1;
+                    __threadfence();
+                    mbar_arrive(&tail_bar[1]);
+                }
+                if (!mbar_wait(&tail_bar[1], local & 1, abort_flag)) break;
+                if (*tail_last) {
+                    // this warp: rows 32*(warp%4).. and the 8 tokens of group `half` (TOK == 16)
+                    static_assert(TOK == 16, "the tail assumes two token groups");
+                    const int b0 = jt * TOK + half * 8;
+                    const bool row_ok = row < p.R;
+                    const float s_row = p.tail == TAIL_T ? p.S[row] : 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int b = b0 + i;
+                        if (b >= p.B) break;                         // uniform across the warp
+                        int a[ND];
+#pragma unroll
+                        for (int d = 0; d < ND; ++d) a[d] = __ldcg(p.acc + ((size_t)b * ND + d) * p.acc_ld + row);
+                        float f;
+                        if constexpr (ND == 1) f = (float)a[0];
+                        else if constexpr (ND == 2) f = (float)(a[0] + (a[1] << 8));
+                        else {
+                            const int lo = a[0] + (a[1] << 8);
+                            int hi = a[2];
+                            if constexpr (ND == 4) hi += a[3] << 8;
+                            f = fmaf((float)hi, 65536.f, (float)lo);
+                        }
+                        const float val = f * __ldg(p.scale + b);
+                        if (p.tail == TAIL_T) {
+                            const float tv = s_row * val;             // the K multiplications (Table S1)
+                            p.t[(size_t)b * p.t_ld + row] = tv;
+                            if (p.z_out && row_ok) {
+                                if (p.z_int) reinterpret_cast<int*>(p.z_out)[(size_t)b * p.z_ld + row] = a[0];
+                                else reinterpret_cast<float*>(p.z_out)[(size_t)b * p.z_ld + row] = val;
+                            }
+                            const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(tv)));
+                            if (lane == 0) atomicMax(p.tmax + b, m);
+                        } else if (row_ok) {
+                            if (p.y_bf16)
+                                reinterpret_cast<__nv_bfloat16*>(p.y)[(size_t)b * p.ldy + row] = __float2bfloat16_rn(val);
+                            else
+                                reinterpret_cast<float*>(p.y)[(size_t)b * p.ldy + row] = val;
+                        }
+                    }
+                }
+            }
         }
     }
 
@@ -594,126 +663,19 @@ ternary_mma_kernel(const GemmParams p)
     }
 }
 
-// ---------------------------------------------------------------------------------------
-// Small batches: the contraction is split over several CTAs that add raw int32 digit sums into
-// a global accumulator acc[b][d][row]; these two kernels pick the sums up.
-// ---------------------------------------------------------------------------------------
-template <int ND> __device__ __forceinline__ float combine_digits(const int* __restrict__ a, int stride)
-{
-    if constexpr (ND == 1) return (float)a[0];
-    else if constexpr (ND == 2) return (float)(a[0] + (a[stride] << 8));
-    else {
-        const int lo = a[0] + (a[stride] << 8);
-        int hi = a[2 * stride];
-        if constexpr (ND == 4) hi += a[3 * stride] << 8;
-        return fmaf((float)hi, 65536.f, (float)lo);
-    }
-}
-
-// One block per token slot: v[k] = digits(acc_in[b][.][k]) * scale_in[b] * (S ? S[k] : 1), then the
-// same fixed-point split as digitise_kernel into ND_OUT digits.  Optionally writes V x before the
-// S scale (z_out) and clears the next accumulator.
-template <int ND_IN, int ND_OUT, int TOK>
-__global__ void __launch_bounds__(256)
-digitise_acc_kernel(const int* __restrict__ acc_in, int acc_ld, const float* __restrict__ scale_in,
-                    const float* __restrict__ S, int B, int C, int KB, int8_t* __restrict__ D,
-                    float* __restrict__ scale_out, void* __restrict__ z_out, int z_ld, int z_int,
-                    int* __restrict__ zero_buf, int zero_per_token)
-{
-    constexpr int NT = ND_OUT * TOK;
-    const int b = blockIdx.x;
-    const int jt = b / TOK, b_in = b % TOK;
-    const bool live = b < B;
-    const int* a = acc_in + (size_t)b * ND_IN * acc_ld;
-    const float sc_in = live ? scale_in[b] : 0.f;
-    __shared__ float red[8];
-
-    if (zero_buf)
-        for (int i = threadIdx.x; i < zero_per_token; i += 256) zero_buf[(size_t)b * zero_per_token + i] = 0;
-
-    float amax = 0.f;
-    if (live) {
-        for (int c = threadIdx.x; c < C; c += 256) {
-            const float z = combine_digits<ND_IN>(a + c, acc_ld) * sc_in;
-            if (z_out) {
-                if (z_int) reinterpret_cast<int*>(z_out)[(size_t)b * z_ld + c] = a[c];
-                else reinterpret_cast<float*>(z_out)[(size_t)b * z_ld + c] = z;
-            }
-            amax = fmaxf(amax, fabsf(S ? S[c] * z : z));
-        }
-    }
-    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
-    __syncthreads();
-#pragma unroll
-    for (int w = 0; w < 8; ++w) amax = fmaxf(amax, red[w]);
-    int E = -90;
-    if (amax > 0.f) {
-        int e;
-        (void)frexpf(amax, &e);
-        E = max(e, -90);
-    }
-    const float qscale = exp2f((float)(8 * ND_OUT - 2 - E));
-    if (threadIdx.x == 0) scale_out[b] = exp2f((float)(E - (8 * ND_OUT - 2)));
-
-    const int n_chunks = KB * 8;
-    for (int ch = threadIdx.x; ch < n_chunks; ch += 256) {
-        const int kb = ch >> 3, cc = ch & 7;
-        uint32_t dig[ND_OUT][4];
-#pragma unroll
-        for (int d = 0; d < ND_OUT; ++d)
-#pragma unroll
-            for (int w = 0; w < 4; ++w) dig[d][w] = 0;
-        if (live) {
-            int q[16];
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                const int c = ch * 16 + e;
-                float v = 0.f;
-                if (c < C) {
-                    v = combine_digits<ND_IN>(a + c, acc_ld) * sc_in;
-                    if (S) v *= S[c];   // the K multiplications (Table S1, row "diag(s)(.)")
-                }
-                q[e] = __float2int_rn(v * qscale);
-            }
-            digits_of_16<ND_OUT>(q, dig);
-        }
-        int8_t* tile = D + ((size_t)jt * KB + kb) * (size_t)(NT * 128);
-#pragma unroll
-        for (int d = 0; d < ND_OUT; ++d) {
-            const int r = d * TOK + b_in;
-            *reinterpret_cast<uint4*>(tile + r * 128 + ((cc ^ (r & 7)) << 4)) =
-                make_uint4(dig[d][0], dig[d][1], dig[d][2], dig[d][3]);
-        }
-    }
-}
-
-// y[b][m] = digits(acc[b][.][m]) * scale[b], stored as fp32 or (one rounding to nearest even) bf16.
-template <int ND, bool BF16_OUT>
-__global__ void __launch_bounds__(256)
-finish_kernel(const int* __restrict__ acc, int acc_ld, const float* __restrict__ scale, int B, int M,
-              void* __restrict__ y, int ldy)
-{
-    const int b = blockIdx.y;
-    const int m = blockIdx.x * 256 + threadIdx.x;
-    if (b >= B || m >= M) return;
-    const float v = combine_digits<ND>(acc + (size_t)b * ND * acc_ld + m, acc_ld) * scale[b];
-    if constexpr (BF16_OUT) reinterpret_cast<__nv_bfloat16*>(y)[(size_t)b * ldy + m] = __float2bfloat16_rn(v);
-    else reinterpret_cast<float*>(y)[(size_t)b * ldy + m] = v;
-}
-
 template <typename IN_T, int ND, int TOK = tokens_per_tile(ND)>
 cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, const unsigned* amax_bits,
-                            int8_t* D, float* scale, int* zero_buf, int zero_per_token, int* B_pad_out,
+                            int8_t* D, float* scale, int* zero_buf, int zero_total, int* B_pad_out,
                             cudaStream_t stream)
 {
     const int B_pad = (B + TOK - 1) / TOK * TOK;
+    const int zero_per_token = (zero_total + B_pad - 1) / B_pad;   // every token slot clears a share
     if (B_pad * 32 >= 148 * 1024 || KB < 8)   // enough warps to fill the GPU, or short rows
         digitise_kernel<IN_T, ND, 32, TOK><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits,
-                                                                                D, scale, zero_buf, zero_per_token);
+                                                                                D, scale, zero_buf, zero_per_token, zero_total);
     else
         digitise_kernel<IN_T, ND, 256, TOK><<<B_pad, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                                                                       scale, zero_buf, zero_per_token);
+                                                                       scale, zero_buf, zero_per_token, zero_total);
     tsvd_count_launch();
     if (B_pad_out) *B_pad_out = B_pad;
     return cudaGetLastError();
@@ -793,7 +755,8 @@ constexpr int SMALL_TOK = 16;        // tokens per tile on the small-batch path
 constexpr int SMALL_MAX_B = 64;
 
 struct SmallWs {
-    int8_t* Dx; float* scale_x; int* zacc; int8_t* Dt; float* scale_t; int* yacc;
+    int8_t* Dx; float* scale_x; int* zacc; float* t; int8_t* Dt; float* scale_t; int* yacc;
+    int zacc_ints, yacc_ints;     // sums + per-token max + per-tile counters: cleared as one range
     size_t total;
 };
 
@@ -802,19 +765,25 @@ SmallWs carve_small(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, void* base)
     const int ndx = digits_for_x(dt);
     const size_t Bp = align_up(B, SMALL_TOK);
     const size_t KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
+    const size_t j_tiles = Bp / SMALL_TOK;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+    SmallWs w;
+    // [sums Bp*nd*R_pad][max |t| per token Bp][tile counters]
+    w.zacc_ints = (int)(Bp * ndx * (size_t)h->V.R_pad + Bp + (size_t)(h->V.R_pad / BLOCK_R) * j_tiles);
+    w.yacc_ints = (int)(Bp * ND_T * (size_t)h->U.R_pad + (size_t)(h->U.R_pad / BLOCK_R) * j_tiles);
     const size_t o_dx = take(Bp * ndx * KBv * 128);
     const size_t o_sx = take(Bp * sizeof(float));
-    const size_t o_za = take(Bp * ndx * (size_t)h->V.R_pad * sizeof(int));
+    const size_t o_za = take((size_t)w.zacc_ints * sizeof(int));
+    const size_t o_t = take(Bp * (size_t)h->V.R_pad * sizeof(float));
     const size_t o_dt = take(Bp * ND_T * KBu * 128);
     const size_t o_st = take(Bp * sizeof(float));
-    const size_t o_ya = take(Bp * ND_T * (size_t)h->U.R_pad * sizeof(int));
-    SmallWs w;
+    const size_t o_ya = take((size_t)w.yacc_ints * sizeof(int));
     char* b = reinterpret_cast<char*>(base);
     w.Dx = reinterpret_cast<int8_t*>(b + o_dx);
     w.scale_x = reinterpret_cast<float*>(b + o_sx);
     w.zacc = reinterpret_cast<int*>(b + o_za);
+    w.t = reinterpret_cast<float*>(b + o_t);
     w.Dt = reinterpret_cast<int8_t*>(b + o_dt);
     w.scale_t = reinterpret_cast<float*>(b + o_st);
     w.yacc = reinterpret_cast<int*>(b + o_ya);
@@ -833,6 +802,9 @@ int pick_ksplit(int out_tiles, int KB)
     return ks < 1 ? 1 : ks;
 }
 
+// Four launches: x -> digits (clears the V-stage sums) | V-stage parts, the last part of each tile
+// writes t = S*z and the per-token max |t| | t -> digits (clears the U-stage sums) | U-stage
+// parts, the last part of each tile writes y.
 template <typename IN_T, int NDX>
 tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
 {
@@ -843,17 +815,20 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
     cudaStream_t st = a.stream;
     cudaError_t e;
 
-    // activations -> digits; clears the V-stage accumulators
     h->prof.begin(0, st);
     e = launch_digitise<IN_T, NDX, SMALL_TOK>((const IN_T*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                              w.zacc, NDX * h->V.R_pad, nullptr, st);
+                                              w.zacc, w.zacc_ints, nullptr, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
-    // V-stage, contraction split across CTAs
     GemmParams p{};
     p.units = h->V.units; p.KB = KBv; p.R = h->K; p.D = w.Dx; p.B = a.B; p.status = h->dev_status;
+    p.scale = w.scale_x; p.S = h->S; p.t = w.t; p.t_ld = h->V.R_pad;
+    p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
     p.acc = w.zacc; p.acc_ld = h->V.R_pad;
+    p.tmax = reinterpret_cast<unsigned*>(w.zacc + (size_t)Bp * NDX * h->V.R_pad);
+    p.tile_done = w.zacc + (size_t)Bp * NDX * h->V.R_pad + Bp;
+    p.tail = TAIL_T;
     const int v_tiles = h->V.R_pad / BLOCK_R;
     p.ksplit = pick_ksplit(v_tiles * j_tiles, KBv);
     h->prof.begin(1, st);
@@ -861,32 +836,23 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
-    // z = sums * 2^e (optional z_out), t = S*z -> digits; clears the U-stage accumulators
     h->prof.begin(2, st);
-    digitise_acc_kernel<NDX, ND_T, SMALL_TOK><<<Bp, 256, 0, st>>>(
-        w.zacc, h->V.R_pad, w.scale_x, h->S, a.B, h->K, KBu, w.Dt, w.scale_t, a.z_out, h->K,
-        a.dtype == TSVD_I8 ? 1 : 0, w.yacc, ND_T * h->U.R_pad);
-    tsvd_count_launch();
-    e = cudaGetLastError();
+    e = launch_digitise<float, ND_T, SMALL_TOK>(w.t, h->V.R_pad, a.B, h->K, KBu, p.tmax, w.Dt, w.scale_t, w.yacc,
+                                                w.yacc_ints, nullptr, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
-    // U-stage, split likewise, then the final conversion
     GemmParams q{};
     q.units = h->U.units; q.KB = KBu; q.R = h->M; q.D = w.Dt; q.B = a.B; q.status = h->dev_status;
+    q.scale = w.scale_t; q.y = a.y; q.ldy = a.ldy;
+    q.y_bf16 = (a.dtype == TSVD_BF16) && !a.out_f32;
     q.acc = w.yacc; q.acc_ld = h->U.R_pad;
+    q.tile_done = w.yacc + (size_t)Bp * ND_T * h->U.R_pad;
+    q.tail = TAIL_Y;
     const int u_tiles = h->U.R_pad / BLOCK_R;
     q.ksplit = pick_ksplit(u_tiles * j_tiles, KBu);
     h->prof.begin(3, st);
     e = launch_gemm<ND_T, EPI_ACC, SMALL_TOK>(q, u_tiles, st);
-    if (e == cudaSuccess) {
-        const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;
-        dim3 grid((h->M + 255) / 256, a.B);
-        if (bf16_out) finish_kernel<ND_T, true><<<grid, 256, 0, st>>>(w.yacc, h->U.R_pad, w.scale_t, a.B, h->M, a.y, a.ldy);
-        else finish_kernel<ND_T, false><<<grid, 256, 0, st>>>(w.yacc, h->U.R_pad, w.scale_t, a.B, h->M, a.y, a.ldy);
-        tsvd_count_launch();
-        e = cudaGetLastError();
-    }
     h->prof.end(st);
     return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
 }
