@@ -615,28 +615,36 @@ ternary_mma_kernel(const GemmParams p)
                     const int b0 = jt * TOK + half * 8;
                     const bool row_ok = row < p.R;
                     const float s_row = p.tail == TAIL_T ? p.S[row] : 0.f;
+                    // all loads first (they are independent and come from L2), then the arithmetic
+                    int a[8][ND];
+                    float sc[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const bool live = b0 + i < p.B;              // uniform across the warp
+                        sc[i] = live ? __ldg(p.scale + b0 + i) : 0.f;
+#pragma unroll
+                        for (int d = 0; d < ND; ++d)
+                            a[i][d] = live ? __ldcg(p.acc + ((size_t)(b0 + i) * ND + d) * p.acc_ld + row) : 0;
+                    }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const int b = b0 + i;
                         if (b >= p.B) break;                         // uniform across the warp
-                        int a[ND];
-#pragma unroll
-                        for (int d = 0; d < ND; ++d) a[d] = __ldcg(p.acc + ((size_t)b * ND + d) * p.acc_ld + row);
                         float f;
-                        if constexpr (ND == 1) f = (float)a[0];
-                        else if constexpr (ND == 2) f = (float)(a[0] + (a[1] << 8));
+                        if constexpr (ND == 1) f = (float)a[i][0];
+                        else if constexpr (ND == 2) f = (float)(a[i][0] + (a[i][1] << 8));
                         else {
-                            const int lo = a[0] + (a[1] << 8);
-                            int hi = a[2];
-                            if constexpr (ND == 4) hi += a[3] << 8;
+                            const int lo = a[i][0] + (a[i][1] << 8);
+                            int hi = a[i][2];
+                            if constexpr (ND == 4) hi += a[i][3] << 8;
                             f = fmaf((float)hi, 65536.f, (float)lo);
                         }
-                        const float val = f * __ldg(p.scale + b);
+                        const float val = f * sc[i];
                         if (p.tail == TAIL_T) {
                             const float tv = s_row * val;             // the K multiplications (Table S1)
                             p.t[(size_t)b * p.t_ld + row] = tv;
                             if (p.z_out && row_ok) {
-                                if (p.z_int) reinterpret_cast<int*>(p.z_out)[(size_t)b * p.z_ld + row] = a[0];
+                                if (p.z_int) reinterpret_cast<int*>(p.z_out)[(size_t)b * p.z_ld + row] = a[i][0];
                                 else reinterpret_cast<float*>(p.z_out)[(size_t)b * p.z_ld + row] = val;
                             }
                             const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(tv)));
