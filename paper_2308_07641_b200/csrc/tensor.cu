@@ -9,8 +9,12 @@
 // is then an exact integer, the result does not depend on summation order, and the only
 // roundings are the fixed-point step of the operand and the final conversion to fp32.
 //
-//   digitise(x)  ->  V-stage MMA  ->  epilogue: z = int * 2^e, t = S*z (the K multiplications),
-//   per-token max|t|  ->  digitise(t)  ->  U-stage MMA  ->  epilogue: y = int * 2^e
+//   digitise(x)  ->  V-stage MMA  ->  epilogue: z = int * 2^e, t = S*z (the K multiplications)
+//                ->  digitise(t)  ->  U-stage MMA  ->  epilogue: y = int * 2^e
+//
+// Batches above 64 tokens use 192-column tiles, one CTA per tile; smaller batches use 16-token
+// tiles with the contraction split across CTAs (integer atomics, the last part of a tile
+// finishes the stage), so that the packed codes are streamed by about one CTA per SM.
 #include "sm100_ptx.cuh"
 #include "tsvd_internal.cuh"
 

@@ -202,3 +202,16 @@ def test_bounded_wait_gives_up_and_reports_timeout():
         assert binding.tsvd_last_status(layer.handle) == binding.TSVD_OK
     finally:
         layer.close()
+
+
+@pytest.mark.parametrize("B", [63, 64, 65, 128])
+def test_batch_sizes_around_the_small_batch_switch(B):
+    """B <= 64 takes 16-token tiles with a split contraction, B > 64 the 192-column tiles."""
+    spec = gen.scaled(C["cfg2"], name=f"switch_B{B}", M=300, N=520, K=390, B=B, seed=51)
+    _util.run_and_check(spec)
+
+
+def test_small_batch_with_many_row_tiles_runs_unsplit():
+    """More output tiles than SMs: the contraction is not split (every part is the last one)."""
+    spec = gen.scaled(C["cfg5_d20"], name="unsplit", M=128 * 80, N=256, K=128 * 80, B=17, seed=52)
+    _util.run_and_check(spec, sample_tokens=[0, 8, 16])
