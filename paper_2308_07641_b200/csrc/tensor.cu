@@ -29,7 +29,6 @@ constexpr int NT_MAX = 192;    // MMA N extent: digit rows per tile
 constexpr int NP = 8;          // ring depth of the packed codes (shared memory)
 constexpr int NB = 8;          // ring depth of the digit tiles (shared memory) and of the per-block barriers
 constexpr int NA = 4;          // ring depth of the expanded ternary operand (tensor memory)
-constexpr int NBP = NB / 2;    // "MMAs done" is signalled once per pair of contraction blocks
 // tensor memory: two accumulator buffers of 192 columns, then four 32-column slots that hold
 // the expanded ternary operand (128 rows x 128 int8 = 32 columns of 32 bits per row)
 constexpr int TMEM_COLS = 512;
@@ -317,13 +316,11 @@ ternary_mma_kernel(const GemmParams p)
     //   A: expanded int8 operand (tensor memory), lives from expansion to the end of its MMAs;
     //      it never touches shared memory, whose bandwidth the digit tiles need
     //   B: digit tiles (24 KiB, shared memory), live from the copy's issue to the end of their MMAs
-    // Contraction block `it` (counted over all tiles of the CTA) has its "operands ready" barrier
-    // it % NB (the digit copy's byte count plus one arrival per expander warp).  "MMAs done" is
-    // signalled once per PAIR of blocks, barrier (it/2) % NBP: the warp that issues the MMAs is
-    // the critical path of the kernel, an MMA costs it ~48 cycles to issue and a commit ~60, so
-    // per pair it spends 8 MMAs + 1 commit against 768 cycles of execution.  The digit tile sits
-    // in slot it % NB, the expanded operand in tensor-memory slot it % NA; both are free again
-    // once the pair that used them last is done.
+    // Contraction block `it` uses barrier pair it % NB: "operands ready" (the digit copy's byte
+    // count plus one arrival per expander warp) and "MMAs done", so that the warp that issues
+    // the MMAs does one wait and one commit per block; its instruction stream is the critical
+    // path of the kernel.  The digit tile sits in slot it % NB, the expanded operand in tensor-
+    // memory slot it % NA, which is free again once block it - NA is done.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* b_tiles = smem;                                 // NB x 24 KiB, 1024-aligned
@@ -332,7 +329,7 @@ ternary_mma_kernel(const GemmParams p)
     uint64_t* pfull_bar = bars;                      // [NP] packed codes landed
     uint64_t* pempty_bar = pfull_bar + NP;           // [NP] expanders have read them
     uint64_t* ready_bar = pempty_bar + NP;           // [NB] digit tile landed and expanded operand written
-    uint64_t* done_bar = ready_bar + NB;             // [NBP] the MMAs of a pair of blocks have completed
+    uint64_t* done_bar = ready_bar + NB;             // [NB] the MMAs of the block have completed
     uint64_t* accfull_bar = done_bar + NB;           // [2] all MMAs of a tile have completed
     uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
     uint64_t* tail_bar = accempty_bar + 2;           // [2] split contraction: epilogue warps meet, verdict is in
@@ -389,10 +386,7 @@ ternary_mma_kernel(const GemmParams p)
                 const uint8_t* src = is_b ? reinterpret_cast<const uint8_t*>(p.D) + (size_t)tc.jt * KB * B_TILE_BYTES
                                           : reinterpret_cast<const uint8_t*>(p.units) + (size_t)tc.rt * KB * P_TILE_BYTES;
                 for (int kb = tc.kb0; kb < tc.kb1; ++kb, ++issued) {
-                    const uint32_t pr = issued >> 1;   // B slots are released per pair of blocks
-                    const bool free_now = is_b ? mbar_wait(&done_bar[pr % NBP], ((pr / NBP) & 1) ^ 1, abort_flag)
-                                               : mbar_wait(&empty[slot], phase ^ 1, abort_flag);
-                    if (!free_now) { alive = false; break; }
+                    if (!mbar_wait(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
                     if (is_b && p.test_stall) { alive = false; break; }   // nothing will ever land
                     if (elect_one()) {
                         mbar_arrive_expect_tx(&full[slot], bytes);
@@ -417,7 +411,7 @@ ternary_mma_kernel(const GemmParams p)
         //      descriptors stay warp-uniform (the MMA instructions take them from the uniform
         //      register file); one elected lane issues the MMAs and commits. ----
         {
-            uint32_t slot = 0, phase = 0, aslot = 0, local = 0, it = 0;
+            uint32_t slot = 0, phase = 0, aslot = 0, local = 0;
             const uint64_t b_desc0 = umma_desc_k_sw128(smem_u32(b_tiles));
             // readiness of the next slot is tested (without blocking) while the current block's
             // MMAs are being issued, so that the barrier's latency is off the issue path
@@ -430,14 +424,12 @@ ternary_mma_kernel(const GemmParams p)
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
                 int kb0, kb1;
                 tile_kb_range(p, tile, kb0, kb1);
-                const bool last_tile = tile + (int)gridDim.x >= n_tiles;
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!ready && !mbar_wait(&ready_bar[slot], phase, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
                     const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
                     const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_TILE_BYTES_MAX >> 4));
-                    // the pair is complete after its odd block, or at the CTA's very last block
-                    const bool end_of_pair = (it & 1u) || (last_tile && kb == kb1 - 1);
+                    const uint32_t cur = slot;
                     if (++slot == NB) { slot = 0; phase ^= 1; }
                     aslot = (aslot + 1) & (NA - 1);
                     if (elect_one()) {
@@ -448,7 +440,7 @@ ternary_mma_kernel(const GemmParams p)
                         for (int k = 1; k < BLOCK_C / UMMA_K; ++k)
                             umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)),
                                        b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, true);
-                        if (end_of_pair) umma_commit(&done_bar[(it >> 1) % NBP]);   // frees the pair's slots
+                        umma_commit(&done_bar[cur]);   // frees the digit slot and, NA blocks on, the A slot
                     }
                     __syncwarp();
                     ready = mbar_test_wait(&ready_bar[slot], phase);
@@ -485,8 +477,8 @@ ternary_mma_kernel(const GemmParams p)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // codes are in registers: slot reusable
                 if (it >= (uint32_t)NA) {   // the A slot is free once block it - NA is done
-                    const uint32_t pj = (it - NA) >> 1;   // the pair that block it - NA belonged to
-                    if (!mbar_wait(&done_bar[pj % NBP], (pj / NBP) & 1, abort_flag)) { alive = false; break; }
+                    const uint32_t j = it - NA;
+                    if (!mbar_wait(&done_bar[j % NB], (j / NB) & 1, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
                 }
                 tmem_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS), o);
