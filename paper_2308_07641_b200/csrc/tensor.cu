@@ -37,9 +37,10 @@ constexpr int A_COL0 = 2 * ACC_COLS;
 constexpr int A_SLOT_COLS = BLOCK_C / 4;
 // warp 0: digit-tile copies, 1: MMA issue, 2: packed-code copies, 3: idle,
 // 4..11: expand (two groups of four that take alternate contraction blocks), 12..19: epilogue
-constexpr int GEMM_THREADS = 640;
+constexpr int EXP_GROUPS = 3;     // groups of four expander warps; group g takes blocks it % EXP_GROUPS == g
 constexpr int EXP_WARP0 = 4;
-constexpr int EPI_WARP0 = 12;
+constexpr int EPI_WARP0 = EXP_WARP0 + 4 * EXP_GROUPS;
+constexpr int GEMM_THREADS = 32 * (EPI_WARP0 + 8);
 
 // tokens per tile for nd digits: the MMA N extent is nd * tokens = 192 for every nd
 __host__ __device__ constexpr int tokens_per_tile(int nd) { return 192 / nd; }
@@ -449,7 +450,7 @@ ternary_mma_kernel(const GemmParams p)
                 __syncwarp();
             }
         }
-    } else if (warp >= EXP_WARP0 && warp < EXP_WARP0 + 8) {
+    } else if (warp >= EXP_WARP0 && warp < EPI_WARP0) {
         // ---- expanders: thread = row of the tile = tensor-memory lane (warp w may touch lanes
         //      32*(w%4)..+31); the two groups of four warps take alternate contraction blocks, so
         //      that the barrier and memory latencies of one block overlap with work on the next ----
@@ -461,7 +462,7 @@ ternary_mma_kernel(const GemmParams p)
             int kb0, kb1;
             tile_kb_range(p, tile, kb0, kb1);
             for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                if ((it & 1u) != group) continue;
+                if (it % EXP_GROUPS != group) continue;
                 const int sp = it % NP, sa = it % NA, sb = it % NB;
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_TILE_BYTES);
