@@ -268,6 +268,8 @@ struct GemmParams {
                           //   TAIL_Y: y = sums*scale -> p.y (bf16 when p.y_bf16)
     unsigned* tmax;       // TAIL_T: per-token max |t| as float bits
     int y_bf16;
+    int nb;               // depth of the digit-tile ring: NB, or (resident) a whole number of panels of KB
+    int resident;         // the digit tiles of a token tile stay in shared memory across row tiles
     int wait_limit;       // bound of every barrier wait in units of 2^20 clocks (0: default, ~2 s)
     int test_stall;       // test hook: the digit tiles are never copied, so the waits must give up
 };
@@ -290,6 +292,14 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile)
     c.rt = rest % p.row_tiles;
     c.jt = rest / p.row_tiles;
     return c;
+}
+// Each CTA takes a run of consecutive tiles (row tile fastest), so that its tiles share their
+// token tile for as long as possible; the runs differ in length by at most one.
+__device__ __forceinline__ void tile_range(int n_tiles, int& t0, int& t1)
+{
+    const int q = n_tiles / (int)gridDim.x, rem = n_tiles % (int)gridDim.x, c = (int)blockIdx.x;
+    t0 = c * q + min(c, rem);
+    t1 = t0 + q + (c < rem ? 1 : 0);
 }
 // The contraction range alone (no divisions when the contraction is not split).
 __device__ __forceinline__ void tile_kb_range(const GemmParams& p, int tile, int& kb0, int& kb1)
@@ -317,11 +327,16 @@ ternary_mma_kernel(const GemmParams p)
     //   A: expanded int8 operand (tensor memory), lives from expansion to the end of its MMAs;
     //      it never touches shared memory, whose bandwidth the digit tiles need
     //   B: digit tiles (24 KiB, shared memory), live from the copy's issue to the end of their MMAs
-    // Contraction block `it` uses barrier pair it % NB: "operands ready" (the digit copy's byte
+    // Contraction block `it` uses barrier pair it % nb: "operands ready" (the digit copy's byte
     // count plus one arrival per expander warp) and "MMAs done", so that the warp that issues
     // the MMAs does one wait and one commit per block; its instruction stream is the critical
-    // path of the kernel.  The digit tile sits in slot it % NB, the expanded operand in tensor-
+    // path of the kernel.  The digit tile sits in slot it % nb, the expanded operand in tensor-
     // memory slot it % NA, which is free again once block it - NA is done.
+    // An SM takes in about 64 bytes per clock from L2, and a block's 24 KiB digit tile plus
+    // 4 KiB of codes at that rate take longer than its four MMAs.  So when the whole contraction
+    // fits the ring (KB <= NB) the ring depth nb is a whole number of panels of KB blocks, a CTA
+    // walks consecutive row tiles of one token tile, and the digit tiles are copied only when the
+    // token tile changes: per block only the 4 KiB of codes then come from L2.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* b_tiles = smem;                                 // NB x 24 KiB, 1024-aligned
@@ -341,6 +356,9 @@ ternary_mma_kernel(const GemmParams p)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = p.KB;
     const int n_tiles = p.row_tiles * p.j_tiles * p.ksplit;
+    int t0, t1;
+    tile_range(n_tiles, t0, t1);
+    const uint32_t nb = (uint32_t)p.nb;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NP; ++s) { mbar_init(&pfull_bar[s], 1); mbar_init(&pempty_bar[s], 4); }
@@ -374,7 +392,8 @@ ternary_mma_kernel(const GemmParams p)
         //      warp runs the loop (uniform control flow); one elected lane issues the copies ----
         {
             const bool is_b = warp == 0;
-            const uint32_t depth = is_b ? NB : NP;
+            const uint32_t depth = is_b ? nb : (uint32_t)NP;
+            const int panels = p.nb / KB;   // resident: token panels the ring holds
             uint64_t* full = is_b ? ready_bar : pfull_bar;
             uint64_t* empty = is_b ? done_bar : pempty_bar;
             const uint32_t bytes = is_b ? B_TILE_BYTES : (uint32_t)P_TILE_BYTES;
@@ -382,16 +401,28 @@ ternary_mma_kernel(const GemmParams p)
             uint8_t* ring = is_b ? b_tiles : p_tiles;
             uint32_t slot = 0, phase = 0, issued = 0;
             bool alive = true;
-            for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
+            for (int tile = t0; tile < t1 && alive; ++tile) {
                 const TileCoord tc = tile_coord(p, tile);
                 const uint8_t* src = is_b ? reinterpret_cast<const uint8_t*>(p.D) + (size_t)tc.jt * KB * B_TILE_BYTES
                                           : reinterpret_cast<const uint8_t*>(p.units) + (size_t)tc.rt * KB * P_TILE_BYTES;
+                // Resident digit tiles: the ring holds whole panels (all KB blocks of a token tile),
+                // tile L of this CTA uses panel L % panels, and if the tile that used it before had
+                // the same token tile the data are there already: only the barrier is armed.
+                bool copy = true;
+                if (is_b && p.resident) {
+                    const int prev = tile - panels;
+                    copy = prev < t0 || prev / p.row_tiles != tc.jt;
+                }
                 for (int kb = tc.kb0; kb < tc.kb1; ++kb, ++issued) {
                     if (!mbar_wait(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
                     if (is_b && p.test_stall) { alive = false; break; }   // nothing will ever land
                     if (elect_one()) {
-                        mbar_arrive_expect_tx(&full[slot], bytes);
-                        bulk_g2s(ring + slot * slot_bytes, src + (size_t)kb * bytes, bytes, &full[slot]);
+                        if (copy) {
+                            mbar_arrive_expect_tx(&full[slot], bytes);
+                            bulk_g2s(ring + slot * slot_bytes, src + (size_t)kb * bytes, bytes, &full[slot]);
+                        } else {
+                            mbar_arrive(&full[slot]);
+                        }
                     }
                     __syncwarp();
                     if (++slot == depth) { slot = 0; phase ^= 1; }
@@ -418,7 +449,7 @@ ternary_mma_kernel(const GemmParams p)
             // MMAs are being issued, so that the barrier's latency is off the issue path
             bool ready = mbar_test_wait(&ready_bar[0], 0);
             bool alive = true;
-            for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x, ++local) {
+            for (int tile = t0; tile < t1 && alive; ++tile, ++local) {
                 const uint32_t buf = local & 1;
                 if (!mbar_wait(&accempty_bar[buf], ((local >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
@@ -431,7 +462,7 @@ ternary_mma_kernel(const GemmParams p)
                     const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
                     const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_TILE_BYTES_MAX >> 4));
                     const uint32_t cur = slot;
-                    if (++slot == NB) { slot = 0; phase ^= 1; }
+                    if (++slot == nb) { slot = 0; phase ^= 1; }
                     aslot = (aslot + 1) & (NA - 1);
                     if (elect_one()) {
                         // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
@@ -456,14 +487,14 @@ ternary_mma_kernel(const GemmParams p)
         //      that the barrier and memory latencies of one block overlap with work on the next ----
         const int r = (threadIdx.x - EXP_WARP0 * 32) & 127;   // 0..127
         const uint32_t group = (uint32_t)(warp - EXP_WARP0) >> 2;
-        uint32_t it = 0;
+        uint32_t it = 0, sb = 0, phb = 0;   // block counter; its slot and phase in the digit-tile ring
         bool alive = true;
-        for (int tile = blockIdx.x; tile < n_tiles && alive; tile += gridDim.x) {
+        for (int tile = t0; tile < t1 && alive; ++tile) {
             int kb0, kb1;
             tile_kb_range(p, tile, kb0, kb1);
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            for (int kb = kb0; kb < kb1; ++kb, ++it, sb = (sb + 1 == nb ? 0u : sb + 1), phb ^= (sb == 0)) {
                 if (it % EXP_GROUPS != group) continue;
-                const int sp = it % NP, sa = it % NA, sb = it % NB;
+                const int sp = it % NP, sa = it % NA;
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_TILE_BYTES);
                 uint32_t o[32];   // the row's 128 int8 values, four per 32-bit column
@@ -478,8 +509,9 @@ ternary_mma_kernel(const GemmParams p)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // codes are in registers: slot reusable
                 if (it >= (uint32_t)NA) {   // the A slot is free once block it - NA is done
-                    const uint32_t j = it - NA;
-                    if (!mbar_wait(&done_bar[j % NB], (j / NB) & 1, abort_flag)) { alive = false; break; }
+                    uint32_t sd = sb + nb - NA, phd = phb ^ 1;   // its slot, NA back (nb >= NA), and phase
+                    if (sd >= nb) { sd -= nb; phd = phb; }
+                    if (!mbar_wait(&done_bar[sd], phd, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
                 }
                 tmem_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS), o);
@@ -496,7 +528,7 @@ ternary_mma_kernel(const GemmParams p)
         const int half = (warp - EPI_WARP0) >> 2;
         const int row_in = lane_grp * 32 + lane;
         uint32_t local = 0;
-        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++local) {
+        for (int tile = t0; tile < t1; ++tile, ++local) {
             const TileCoord tc = tile_coord(p, tile);
             const int rt = tc.rt, jt = tc.jt;
             const int row = rt * BLOCK_R + row_in;
@@ -711,6 +743,14 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
     q.row_tiles = row_tiles;
     q.j_tiles = (p.B + TOK - 1) / TOK;
     if (q.ksplit < 1) q.ksplit = 1;
+    // A contraction of at most NB blocks leaves room to keep a token tile's digit tiles in shared
+    // memory while the CTA walks the row tiles: the ring then holds whole panels of KB blocks.
+    q.nb = NB;
+    q.resident = 0;
+    if (q.ksplit == 1 && q.KB <= NB) {
+        q.nb = q.KB * (NB / q.KB);
+        q.resident = 1;
+    }
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int n_tiles = q.row_tiles * q.j_tiles * q.ksplit;
