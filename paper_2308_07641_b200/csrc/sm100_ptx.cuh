@@ -75,19 +75,14 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity)
 // up it sets the flag and returns false; the caller carries on to the kernel's normal exit so
 // that tensor memory is released.
 constexpr int kWaitLimitDefault = 4096;  // 2^32 clocks, about two seconds
-// SLEEP_NS > 0: between two tests the warp sleeps about that long instead of spinning, so that
-// a warp with a long wait ahead neither takes issue slots nor keeps the shared-memory pipe busy
-// with barrier reads that the latency-critical warps queue behind.
-template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl)
 {
-    if (mbar_test_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     const long long limit = (long long)ctl[1] << 20;
     unsigned spins = 0;
     while (true) {
-        if constexpr (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
-        if (mbar_test_wait(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
             if (ctl[0]) return false;
             if (clock64() - t0 > limit) {

@@ -414,7 +414,7 @@ ternary_mma_kernel(const GemmParams p)
                     copy = prev < t0 || prev / p.row_tiles != tc.jt;
                 }
                 for (int kb = tc.kb0; kb < tc.kb1; ++kb, ++issued) {
-                    if (!mbar_wait<64>(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
+                    if (!mbar_wait(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
                     if (is_b && p.test_stall) { alive = false; break; }   // nothing will ever land
                     if (elect_one()) {
                         if (copy) {
@@ -495,7 +495,7 @@ ternary_mma_kernel(const GemmParams p)
             for (int kb = kb0; kb < kb1; ++kb, ++it, sb = (sb + 1 == nb ? 0u : sb + 1), phb ^= (sb == 0)) {
                 if (it % EXP_GROUPS != group) continue;
                 const int sp = it % NP, sa = it % NA;
-                if (!mbar_wait<32>(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
+                if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_TILE_BYTES);
                 uint32_t o[32];   // the row's 128 int8 values, four per 32-bit column
 #pragma unroll
@@ -511,7 +511,7 @@ ternary_mma_kernel(const GemmParams p)
                 if (it >= (uint32_t)NA) {   // the A slot is free once block it - NA is done
                     uint32_t sd = sb + nb - NA, phd = phb ^ 1;   // its slot, NA back (nb >= NA), and phase
                     if (sd >= nb) { sd -= nb; phd = phb; }
-                    if (!mbar_wait<32>(&done_bar[sd], phd, abort_flag)) { alive = false; break; }
+                    if (!mbar_wait(&done_bar[sd], phd, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
                 }
                 tmem_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS), o);
@@ -549,7 +549,7 @@ ternary_mma_kernel(const GemmParams p)
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             const bool row_ok = row < p.R;
-            if (!mbar_wait<128>(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
+            if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
             tc_fence_after_sync();
             const uint32_t t_lane = tmem_base + buf * (uint32_t)ACC_COLS + ((uint32_t)(lane_grp * 32) << 16);
 #pragma unroll
