@@ -23,21 +23,24 @@ namespace {
 using namespace ptx;
 
 constexpr int BLOCK_R = 128;   // ternary rows per CTA tile = MMA M
-constexpr int BLOCK_C = 128;   // contraction elements per pipeline stage (one 128-byte swizzle row)
+constexpr int BLOCK_C = 128;   // contraction elements per block (one 128-byte swizzle row)
+constexpr int STEP_BLOCKS = 2; // blocks per pipeline step: one set of barrier handshakes covers this many
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
 constexpr int NT_MAX = 192;    // MMA N extent: digit rows per tile
-constexpr int NP = 8;          // ring depth of the packed codes (shared memory)
-constexpr int NB = 8;          // ring depth of the digit tiles (shared memory) and of the per-block barriers
-constexpr int NA = 4;          // ring depth of the expanded ternary operand (tensor memory)
-// tensor memory: two accumulator buffers of 192 columns, then four 32-column slots that hold
-// the expanded ternary operand (128 rows x 128 int8 = 32 columns of 32 bits per row)
+constexpr int NP = 4;          // ring depth (steps) of the packed codes (shared memory)
+constexpr int NB = 4;          // ring depth (steps) of the digit tiles (shared memory) and of the per-step barriers
+constexpr int NA = 2;          // ring depth (steps) of the expanded ternary operand (tensor memory)
+// tensor memory: two accumulator buffers of 192 columns, then two 64-column slots that hold
+// the expanded ternary operand of a step (per block 128 rows x 128 int8 = 32 columns of 32 bits)
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_COLS = NT_MAX;
 constexpr int A_COL0 = 2 * ACC_COLS;
-constexpr int A_SLOT_COLS = BLOCK_C / 4;
+constexpr int A_BLOCK_COLS = BLOCK_C / 4;
+constexpr int A_SLOT_COLS = STEP_BLOCKS * A_BLOCK_COLS;
+static_assert(A_COL0 + NA * A_SLOT_COLS <= TMEM_COLS, "tensor memory budget");
 // warp 0: digit-tile copies, 1: MMA issue, 2: packed-code copies, 3: idle,
-// 4..11: expand (two groups of four that take alternate contraction blocks), 12..19: epilogue
-constexpr int EXP_GROUPS = 3;     // groups of four expander warps; group g takes blocks it % EXP_GROUPS == g
+// 4..15: expand (three groups of four that take the steps in turn), 16..23: epilogue
+constexpr int EXP_GROUPS = 3;     // groups of four expander warps; group g takes steps it % EXP_GROUPS == g
 constexpr int EXP_WARP0 = 4;
 constexpr int EPI_WARP0 = EXP_WARP0 + 4 * EXP_GROUPS;
 constexpr int GEMM_THREADS = 32 * (EPI_WARP0 + 8);
@@ -47,7 +50,9 @@ __host__ __device__ constexpr int tokens_per_tile(int nd) { return 192 / nd; }
 
 constexpr int P_TILE_BYTES = BLOCK_R * BLOCK_C / 4;      // packed codes of that tile, 4 KiB
 constexpr int B_TILE_BYTES_MAX = NT_MAX * BLOCK_C;       // digit rows, 24 KiB
-constexpr int GEMM_SMEM_BYTES = NB * B_TILE_BYTES_MAX + NP * P_TILE_BYTES +
+constexpr int B_SLOT_BYTES = STEP_BLOCKS * B_TILE_BYTES_MAX;
+constexpr int P_SLOT_BYTES = STEP_BLOCKS * P_TILE_BYTES;
+constexpr int GEMM_SMEM_BYTES = NB * B_SLOT_BYTES + NP * P_SLOT_BYTES +
                                 1024 /*alignment slack*/ + 512 /*barriers*/;
 
 // ---------------------------------------------------------------------------------------
@@ -268,7 +273,7 @@ struct GemmParams {
                           //   TAIL_Y: y = sums*scale -> p.y (bf16 when p.y_bf16)
     unsigned* tmax;       // TAIL_T: per-token max |t| as float bits
     int y_bf16;
-    int nb;               // depth of the digit-tile ring: NB, or (resident) a whole number of panels of KB
+    int nb;               // depth of the digit-tile ring in steps: NB, or (resident) a whole number of panels
     int resident;         // the digit tiles of a token tile stay in shared memory across row tiles
     int wait_limit;       // bound of every barrier wait in units of 2^20 clocks (0: default, ~2 s)
     int test_stall;       // test hook: the digit tiles are never copied, so the waits must give up
@@ -322,26 +327,31 @@ ternary_mma_kernel(const GemmParams p)
     constexpr uint32_t B_TILE_BYTES = NT * BLOCK_C;
     constexpr uint32_t IDESC = umma_idesc_s8(BLOCK_R, NT);
 
+    // The contraction advances in steps of STEP_BLOCKS blocks of 128: the barrier handshakes of a
+    // step cost the issuing warp about as long as four MMAs take to run, so one set of handshakes
+    // has to cover more MMA time than that.
     // Three rings, because their contents live for different times:
-    //   P: packed codes (4 KiB, shared memory), copied far ahead, freed once the expanders read them
+    //   P: packed codes (4 KiB per block, shared memory), copied far ahead, freed once the
+    //      expanders have read them
     //   A: expanded int8 operand (tensor memory), lives from expansion to the end of its MMAs;
     //      it never touches shared memory, whose bandwidth the digit tiles need
-    //   B: digit tiles (24 KiB, shared memory), live from the copy's issue to the end of their MMAs
-    // Contraction block `it` uses barrier pair it % nb: "operands ready" (the digit copy's byte
-    // count plus one arrival per expander warp) and "MMAs done", so that the warp that issues
-    // the MMAs does one wait and one commit per block; its instruction stream is the critical
-    // path of the kernel.  The digit tile sits in slot it % nb, the expanded operand in tensor-
-    // memory slot it % NA, which is free again once block it - NA is done.
+    //   B: digit tiles (24 KiB per block, shared memory), live from the copy's issue to the end
+    //      of their MMAs
+    // Step `it` uses barrier pair it % nb: "operands ready" (the digit copy's byte count plus
+    // one arrival per expander warp) and "MMAs done", so that the warp that issues the MMAs
+    // does one wait and one commit per step; its instruction stream is the critical path of
+    // the kernel.  The digit tiles sit in slot it % nb, the expanded operand in tensor-memory
+    // slot it % NA, which is free again once step it - NA is done.
     // An SM takes in about 64 bytes per clock from L2, and a block's 24 KiB digit tile plus
     // 4 KiB of codes at that rate take longer than its four MMAs.  So when the whole contraction
-    // fits the ring (KB <= NB) the ring depth nb is a whole number of panels of KB blocks, a CTA
+    // fits the ring the ring depth nb is a whole number of panels (all steps of a tile), a CTA
     // walks consecutive row tiles of one token tile, and the digit tiles are copied only when the
     // token tile changes: per block only the 4 KiB of codes then come from L2.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* b_tiles = smem;                                 // NB x 24 KiB, 1024-aligned
-    uint8_t* p_tiles = b_tiles + NB * B_TILE_BYTES_MAX;      // NP x 4 KiB
-    uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + NP * P_TILE_BYTES);
+    uint8_t* b_tiles = smem;                                 // NB x 48 KiB, 1024-aligned
+    uint8_t* p_tiles = b_tiles + NB * B_SLOT_BYTES;          // NP x 8 KiB
+    uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + NP * P_SLOT_BYTES);
     uint64_t* pfull_bar = bars;                      // [NP] packed codes landed
     uint64_t* pempty_bar = pfull_bar + NP;           // [NP] expanders have read them
     uint64_t* ready_bar = pempty_bar + NP;           // [NB] digit tile landed and expanded operand written
@@ -356,8 +366,18 @@ ternary_mma_kernel(const GemmParams p)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = p.KB;
     const int n_tiles = p.row_tiles * p.j_tiles * p.ksplit;
-    int t0, t1;
-    tile_range(n_tiles, t0, t1);
+    // Tile L of this CTA.  Resident digit tiles: a run of consecutive tiles (they share the token
+    // tile).  Otherwise strided, so that the CTAs running at one time read the same digit tiles
+    // and those stay hot in L2.
+    int tile_first = (int)blockIdx.x, tile_step = (int)gridDim.x;
+    int tile_count = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    if (p.resident) {
+        int t0, t1;
+        tile_range(n_tiles, t0, t1);
+        tile_first = t0;
+        tile_step = 1;
+        tile_count = t1 - t0;
+    }
     const uint32_t nb = (uint32_t)p.nb;
 
     if (threadIdx.x == 0) {
@@ -393,33 +413,32 @@ ternary_mma_kernel(const GemmParams p)
         {
             const bool is_b = warp == 0;
             const uint32_t depth = is_b ? nb : (uint32_t)NP;
-            const int panels = p.nb / KB;   // resident: token panels the ring holds
+            const int panels = p.nb / ((KB + STEP_BLOCKS - 1) / STEP_BLOCKS);   // resident: token panels the ring holds
             uint64_t* full = is_b ? ready_bar : pfull_bar;
             uint64_t* empty = is_b ? done_bar : pempty_bar;
-            const uint32_t bytes = is_b ? B_TILE_BYTES : (uint32_t)P_TILE_BYTES;
-            const uint32_t slot_bytes = is_b ? (uint32_t)B_TILE_BYTES_MAX : (uint32_t)P_TILE_BYTES;
+            // the blocks of a step are adjacent both in global memory and in the slot
+            const uint32_t blk_bytes = is_b ? B_TILE_BYTES : (uint32_t)P_TILE_BYTES;
+            const uint32_t slot_bytes = is_b ? (uint32_t)B_SLOT_BYTES : (uint32_t)P_SLOT_BYTES;
             uint8_t* ring = is_b ? b_tiles : p_tiles;
             uint32_t slot = 0, phase = 0, issued = 0;
             bool alive = true;
-            for (int tile = t0; tile < t1 && alive; ++tile) {
+            for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
                 const TileCoord tc = tile_coord(p, tile);
                 const uint8_t* src = is_b ? reinterpret_cast<const uint8_t*>(p.D) + (size_t)tc.jt * KB * B_TILE_BYTES
                                           : reinterpret_cast<const uint8_t*>(p.units) + (size_t)tc.rt * KB * P_TILE_BYTES;
-                // Resident digit tiles: the ring holds whole panels (all KB blocks of a token tile),
+                // Resident digit tiles: the ring holds whole panels (all steps of a token tile),
                 // tile L of this CTA uses panel L % panels, and if the tile that used it before had
                 // the same token tile the data are there already: only the barrier is armed.
                 bool copy = true;
-                if (is_b && p.resident) {
-                    const int prev = tile - panels;
-                    copy = prev < t0 || prev / p.row_tiles != tc.jt;
-                }
-                for (int kb = tc.kb0; kb < tc.kb1; ++kb, ++issued) {
+                if (is_b && p.resident) copy = L < panels || (tile - panels) / p.row_tiles != tc.jt;
+                for (int kb = tc.kb0; kb < tc.kb1; kb += STEP_BLOCKS, ++issued) {
+                    const uint32_t bytes = (uint32_t)min(STEP_BLOCKS, tc.kb1 - kb) * blk_bytes;
                     if (!mbar_wait(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
                     if (is_b && p.test_stall) { alive = false; break; }   // nothing will ever land
                     if (elect_one()) {
                         if (copy) {
                             mbar_arrive_expect_tx(&full[slot], bytes);
-                            bulk_g2s(ring + slot * slot_bytes, src + (size_t)kb * bytes, bytes, &full[slot]);
+                            bulk_g2s(ring + slot * slot_bytes, src + (size_t)kb * blk_bytes, bytes, &full[slot]);
                         } else {
                             mbar_arrive(&full[slot]);
                         }
@@ -443,36 +462,42 @@ ternary_mma_kernel(const GemmParams p)
         //      descriptors stay warp-uniform (the MMA instructions take them from the uniform
         //      register file); one elected lane issues the MMAs and commits. ----
         {
-            uint32_t slot = 0, phase = 0, aslot = 0, local = 0;
+            uint32_t slot = 0, phase = 0, aslot = 0;
             const uint64_t b_desc0 = umma_desc_k_sw128(smem_u32(b_tiles));
-            // readiness of the next slot is tested (without blocking) while the current block's
+            // readiness of the next slot is tested (without blocking) while the current step's
             // MMAs are being issued, so that the barrier's latency is off the issue path
             bool ready = mbar_test_wait(&ready_bar[0], 0);
             bool alive = true;
-            for (int tile = t0; tile < t1 && alive; ++tile, ++local) {
-                const uint32_t buf = local & 1;
-                if (!mbar_wait(&accempty_bar[buf], ((local >> 1) & 1) ^ 1, abort_flag)) break;
+            for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
+                const uint32_t buf = (uint32_t)L & 1u;
+                if (!mbar_wait(&accempty_bar[buf], (((uint32_t)L >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
                 int kb0, kb1;
                 tile_kb_range(p, tile, kb0, kb1);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = kb0; kb < kb1; kb += STEP_BLOCKS) {
+                    const int nblk = min(STEP_BLOCKS, kb1 - kb);
                     if (!ready && !mbar_wait(&ready_bar[slot], phase, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
                     const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
-                    const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_TILE_BYTES_MAX >> 4));
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_SLOT_BYTES >> 4));
                     const uint32_t cur = slot;
                     if (++slot == nb) { slot = 0; phase ^= 1; }
                     aslot = (aslot + 1) & (NA - 1);
                     if (elect_one()) {
                         // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
                         // the swizzled 128-byte rows of B
-                        umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != kb0);
 #pragma unroll
-                        for (int k = 1; k < BLOCK_C / UMMA_K; ++k)
-                            umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)),
-                                       b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, true);
-                        umma_commit(&done_bar[cur]);   // frees the digit slot and, NA blocks on, the A slot
+                        for (int j = 0; j < STEP_BLOCKS; ++j) {
+                            if (j < nblk) {
+#pragma unroll
+                                for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
+                                    umma_s8_ts(d_tmem, a_tmem + (uint32_t)(j * A_BLOCK_COLS + k * (UMMA_K / 4)),
+                                               b_desc + (uint64_t)(j * (B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC,
+                                               kb != kb0 || j != 0 || k != 0);
+                            }
+                        }
+                        umma_commit(&done_bar[cur]);   // frees the digit slot and, NA steps on, the A slot
                     }
                     __syncwarp();
                     ready = mbar_test_wait(&ready_bar[slot], phase);
@@ -483,38 +508,49 @@ ternary_mma_kernel(const GemmParams p)
         }
     } else if (warp >= EXP_WARP0 && warp < EPI_WARP0) {
         // ---- expanders: thread = row of the tile = tensor-memory lane (warp w may touch lanes
-        //      32*(w%4)..+31); the two groups of four warps take alternate contraction blocks, so
-        //      that the barrier and memory latencies of one block overlap with work on the next ----
+        //      32*(w%4)..+31); the groups of four warps take the steps in turn, so that the
+        //      barrier and memory latencies of one step overlap with work on the next ----
         const int r = (threadIdx.x - EXP_WARP0 * 32) & 127;   // 0..127
         const uint32_t group = (uint32_t)(warp - EXP_WARP0) >> 2;
-        uint32_t it = 0, sb = 0, phb = 0;   // block counter; its slot and phase in the digit-tile ring
+        uint32_t it = 0, sb = 0, phb = 0;   // step counter; its slot and phase in the digit-tile ring
         bool alive = true;
-        for (int tile = t0; tile < t1 && alive; ++tile) {
+        for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
             int kb0, kb1;
             tile_kb_range(p, tile, kb0, kb1);
-            for (int kb = kb0; kb < kb1; ++kb, ++it, sb = (sb + 1 == nb ? 0u : sb + 1), phb ^= (sb == 0)) {
+            for (int kb = kb0; kb < kb1; kb += STEP_BLOCKS, ++it, sb = (sb + 1 == nb ? 0u : sb + 1), phb ^= (sb == 0)) {
                 if (it % EXP_GROUPS != group) continue;
+                const int nblk = min(STEP_BLOCKS, kb1 - kb);
                 const int sp = it % NP, sa = it % NA;
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
-                const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_TILE_BYTES);
-                uint32_t o[32];   // the row's 128 int8 values, four per 32-bit column
+                const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_SLOT_BYTES);
+                const uint32_t a_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS);
+                bool ok = true;
 #pragma unroll
-                for (int g = 0; g < 2; ++g) {
-                    const uint4 u = packed[g * 128 + r];
-                    tsvd_expand16(u.x, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 0]));
-                    tsvd_expand16(u.y, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 4]));
-                    tsvd_expand16(u.z, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 8]));
-                    tsvd_expand16(u.w, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 12]));
+                for (int j = 0; j < STEP_BLOCKS; ++j) {
+                    if (j < nblk && ok) {
+                        uint32_t o[32];   // the row's 128 int8 values of block j, four per 32-bit column
+#pragma unroll
+                        for (int g = 0; g < 2; ++g) {
+                            const uint4 u = packed[j * 256 + g * 128 + r];
+                            tsvd_expand16(u.x, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 0]));
+                            tsvd_expand16(u.y, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 4]));
+                            tsvd_expand16(u.z, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 8]));
+                            tsvd_expand16(u.w, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 12]));
+                        }
+                        if (j == nblk - 1) {
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // all codes of the step are in registers
+                        }
+                        if (j == 0 && it >= (uint32_t)NA) {   // the A slot is free once step it - NA is done
+                            uint32_t sd = sb + nb - NA, phd = phb ^ 1;   // its slot, NA back (nb >= NA), and phase
+                            if (sd >= nb) { sd -= nb; phd = phb; }
+                            ok = mbar_wait(&done_bar[sd], phd, abort_flag);
+                            tc_fence_after_sync();
+                        }
+                        if (ok) tmem_st32(a_addr + (uint32_t)(j * A_BLOCK_COLS), o);
+                    }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // codes are in registers: slot reusable
-                if (it >= (uint32_t)NA) {   // the A slot is free once block it - NA is done
-                    uint32_t sd = sb + nb - NA, phd = phb ^ 1;   // its slot, NA back (nb >= NA), and phase
-                    if (sd >= nb) { sd -= nb; phd = phb; }
-                    if (!mbar_wait(&done_bar[sd], phd, abort_flag)) { alive = false; break; }
-                    tc_fence_after_sync();
-                }
-                tmem_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS), o);
+                if (!ok) { alive = false; break; }
                 tmem_st_wait();
                 tc_fence_before_sync();
                 __syncwarp();
@@ -528,7 +564,7 @@ ternary_mma_kernel(const GemmParams p)
         const int half = (warp - EPI_WARP0) >> 2;
         const int row_in = lane_grp * 32 + lane;
         uint32_t local = 0;
-        for (int tile = t0; tile < t1; ++tile, ++local) {
+        for (int tile = tile_first; local < (uint32_t)tile_count; tile += tile_step, ++local) {
             const TileCoord tc = tile_coord(p, tile);
             const int rt = tc.rt, jt = tc.jt;
             const int row = rt * BLOCK_R + row_in;
@@ -743,12 +779,13 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
     q.row_tiles = row_tiles;
     q.j_tiles = (p.B + TOK - 1) / TOK;
     if (q.ksplit < 1) q.ksplit = 1;
-    // A contraction of at most NB blocks leaves room to keep a token tile's digit tiles in shared
-    // memory while the CTA walks the row tiles: the ring then holds whole panels of KB blocks.
+    // A contraction of at most NB steps leaves room to keep a token tile's digit tiles in shared
+    // memory while the CTA walks the row tiles: the ring then holds whole panels (a tile's steps).
     q.nb = NB;
     q.resident = 0;
-    if (q.ksplit == 1 && q.KB <= NB) {
-        q.nb = q.KB * (NB / q.KB);
+    const int steps = (q.KB + STEP_BLOCKS - 1) / STEP_BLOCKS;
+    if (q.ksplit == 1 && steps <= NB) {
+        q.nb = steps * (NB / steps);
         q.resident = 1;
     }
     int sms = 148;
