@@ -460,13 +460,7 @@ ternary_mma_kernel(const GemmParams p)
     } else if (warp == 1) {
         // ---- MMA issue.  The whole warp runs the loop so that slot, phase and the operand
         //      descriptors stay warp-uniform (the MMA instructions take them from the uniform
-        //      register file); one elected lane issues the MMAs and commits.
-        //      A commit holds the issuing thread until the MMAs before it have left the queue,
-        //      so the tensor pipe is nearly out of work when it returns.  The commit that
-        //      signals step s - 1 is therefore issued after the first MMA of step s: when it
-        //      returns the other MMAs of step s are queued at once, and they cover the time
-        //      this warp needs to get to step s + 1.  "Done" (and "accumulator full") of a
-        //      step then fire one MMA late. ----
+        //      register file); one elected lane issues the MMAs and commits. ----
         {
             uint32_t slot = 0, phase = 0, aslot = 0;
             const uint64_t b_desc0 = umma_desc_k_sw128(smem_u32(b_tiles));
@@ -474,10 +468,6 @@ ternary_mma_kernel(const GemmParams p)
             // MMAs are being issued, so that the barrier's latency is off the issue path
             bool ready = mbar_test_wait(&ready_bar[0], 0);
             bool alive = true;
-            // the step whose commit is still owed: its slot, and the accumulator buffer it completed (or -1)
-            bool owed = false;
-            uint32_t owed_slot = 0;
-            int owed_full = -1;
             for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
                 const uint32_t buf = (uint32_t)L & 1u;
                 if (!mbar_wait(&accempty_bar[buf], (((uint32_t)L >> 1) & 1) ^ 1, abort_flag)) break;
@@ -497,33 +487,24 @@ ternary_mma_kernel(const GemmParams p)
                     if (elect_one()) {
                         // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
                         // the swizzled 128-byte rows of B
-                        umma_s8_ts(d_tmem, a_tmem, b_desc, IDESC, kb != kb0);
-                        if (owed) {
-                            umma_commit(&done_bar[owed_slot]);   // frees the digit slot and, NA steps on, the A slot
-                            if (owed_full >= 0) umma_commit(&accfull_bar[owed_full]);
-                        }
 #pragma unroll
                         for (int j = 0; j < STEP_BLOCKS; ++j) {
                             if (j < nblk) {
 #pragma unroll
-                                for (int k = (j == 0 ? 1 : 0); k < BLOCK_C / UMMA_K; ++k)
+                                for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
                                     umma_s8_ts(d_tmem, a_tmem + (uint32_t)(j * A_BLOCK_COLS + k * (UMMA_K / 4)),
-                                               b_desc + (uint64_t)(j * (B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC, true);
+                                               b_desc + (uint64_t)(j * (B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC,
+                                               kb != kb0 || j != 0 || k != 0);
                             }
                         }
+                        umma_commit(&done_bar[cur]);   // frees the digit slot and, NA steps on, the A slot
                     }
-                    owed = true;
-                    owed_slot = cur;
-                    owed_full = kb + STEP_BLOCKS >= kb1 ? (int)buf : -1;
                     __syncwarp();
                     ready = mbar_test_wait(&ready_bar[slot], phase);
                 }
+                if (elect_one()) umma_commit(&accfull_bar[buf]);
+                __syncwarp();
             }
-            if (owed && elect_one()) {
-                umma_commit(&done_bar[owed_slot]);
-                if (owed_full >= 0) umma_commit(&accfull_bar[owed_full]);
-            }
-            __syncwarp();
         }
     } else if (warp >= EXP_WARP0 && warp < EPI_WARP0) {
         // ---- expanders: thread = row of the tile = tensor-memory lane (warp w may touch lanes
