@@ -355,8 +355,8 @@ ternary_mma_kernel(const GemmParams p)
     uint64_t* pfull_bar = bars;                      // [NP] packed codes landed
     uint64_t* pempty_bar = pfull_bar + NP;           // [NP] expanders have read them
     uint64_t* ready_bar = pempty_bar + NP;           // [NB] digit tile landed and expanded operand written
-    uint64_t* done_bar = ready_bar + NB;             // [NB] the MMAs of the block have completed
-    uint64_t* accfull_bar = done_bar + NB;           // [2] all MMAs of a tile have completed
+    uint64_t* done_bar = ready_bar + NB;             // [NB][STEP_BLOCKS] the MMAs of block j of the step have completed
+    uint64_t* accfull_bar = done_bar + NB * STEP_BLOCKS;   // [2] all MMAs of a tile have completed
     uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
     uint64_t* tail_bar = accempty_bar + 2;           // [2] split contraction: epilogue warps meet, verdict is in
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail_bar + 2);
@@ -384,7 +384,7 @@ ternary_mma_kernel(const GemmParams p)
         for (int s = 0; s < NP; ++s) { mbar_init(&pfull_bar[s], 1); mbar_init(&pempty_bar[s], 4); }
         for (int s = 0; s < NB; ++s) {
             mbar_init(&ready_bar[s], 5);   // the copy's expect-tx arrival + one per expander warp of the group
-            mbar_init(&done_bar[s], 1);
+            for (int j = 0; j < STEP_BLOCKS; ++j) mbar_init(&done_bar[s * STEP_BLOCKS + j], 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&accfull_bar[i], 1);
@@ -415,7 +415,9 @@ ternary_mma_kernel(const GemmParams p)
             const uint32_t depth = is_b ? nb : (uint32_t)NP;
             const int panels = p.nb / ((KB + STEP_BLOCKS - 1) / STEP_BLOCKS);   // resident: token panels the ring holds
             uint64_t* full = is_b ? ready_bar : pfull_bar;
-            uint64_t* empty = is_b ? done_bar : pempty_bar;
+            // a digit slot is free when the last block of the step that used it is done
+            uint64_t* empty = is_b ? done_bar + (STEP_BLOCKS - 1) : pempty_bar;
+            const uint32_t empty_stride = is_b ? (uint32_t)STEP_BLOCKS : 1u;
             // the blocks of a step are adjacent both in global memory and in the slot
             const uint32_t blk_bytes = is_b ? B_TILE_BYTES : (uint32_t)P_TILE_BYTES;
             const uint32_t slot_bytes = is_b ? (uint32_t)B_SLOT_BYTES : (uint32_t)P_SLOT_BYTES;
@@ -433,7 +435,7 @@ ternary_mma_kernel(const GemmParams p)
                 if (is_b && p.resident) copy = L < panels || (tile - panels) / p.row_tiles != tc.jt;
                 for (int kb = tc.kb0; kb < tc.kb1; kb += STEP_BLOCKS, ++issued) {
                     const uint32_t bytes = (uint32_t)min(STEP_BLOCKS, tc.kb1 - kb) * blk_bytes;
-                    if (!mbar_wait(&empty[slot], phase ^ 1, abort_flag)) { alive = false; break; }
+                    if (!mbar_wait(&empty[slot * empty_stride], phase ^ 1, abort_flag)) { alive = false; break; }
                     if (is_b && p.test_stall) { alive = false; break; }   // nothing will ever land
                     if (elect_one()) {
                         if (copy) {
@@ -496,8 +498,11 @@ ternary_mma_kernel(const GemmParams p)
                                                b_desc + (uint64_t)(j * (B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC,
                                                kb != kb0 || j != 0 || k != 0);
                             }
+                            // block j of the step is done (a block the step does not have counts as
+                            // done too): its part of the A slot is free NA steps on, and after the
+                            // last block the digit slot
+                            umma_commit(&done_bar[cur * STEP_BLOCKS + j]);
                         }
-                        umma_commit(&done_bar[cur]);   // frees the digit slot and, NA steps on, the A slot
                     }
                     __syncwarp();
                     ready = mbar_test_wait(&ready_bar[slot], phase);
@@ -541,10 +546,10 @@ ternary_mma_kernel(const GemmParams p)
                             __syncwarp();
                             if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // all codes of the step are in registers
                         }
-                        if (j == 0 && it >= (uint32_t)NA) {   // the A slot is free once step it - NA is done
+                        if (it >= (uint32_t)NA) {   // this part of the A slot is free once block j of step it - NA is done
                             uint32_t sd = sb + nb - NA, phd = phb ^ 1;   // its slot, NA back (nb >= NA), and phase
                             if (sd >= nb) { sd -= nb; phd = phb; }
-                            ok = mbar_wait(&done_bar[sd], phd, abort_flag);
+                            ok = mbar_wait(&done_bar[sd * STEP_BLOCKS + j], phd, abort_flag);
                             tc_fence_after_sync();
                         }
                         if (ok) tmem_st32(a_addr + (uint32_t)(j * A_BLOCK_COLS), o);
