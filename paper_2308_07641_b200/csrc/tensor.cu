@@ -530,7 +530,7 @@ ternary_mma_kernel(const GemmParams p)
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_SLOT_BYTES);
                 const uint32_t a_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS);
                 bool ok = true;
-#pragma unroll 1
+#pragma unroll
                 for (int j = 0; j < STEP_BLOCKS; ++j) {
                     if (j < nblk && ok) {
                         uint32_t o[32];   // the row's 128 int8 values of block j, four per 32-bit column
@@ -574,27 +574,33 @@ ternary_mma_kernel(const GemmParams p)
             const int rt = tc.rt, jt = tc.jt;
             const int row = rt * BLOCK_R + row_in;
             const uint32_t buf = local & 1;
-            // this warp takes every second group of 8 tokens
+            // fetch the per-token scales of this warp's groups (8 tokens each; this warp takes
+            // every second group) while the tile is still being contracted: lane i holds the
+            // scale of token 8*g + (i & 7), 0 beyond the batch
             constexpr int N_GROUPS = TOK / 8;
             constexpr int MY_GROUPS = N_GROUPS / 2;
             static_assert(N_GROUPS % 2 == 0, "two epilogue warps per lane group share the token groups");
+            float scales[MY_GROUPS];
+#pragma unroll
+            for (int k = 0; k < MY_GROUPS; ++k) {
+                const int bb = jt * TOK + (half + 2 * k) * 8 + (lane & 7);
+                scales[k] = 0.f;
+                if constexpr (EPI != EPI_ACC) scales[k] = bb < p.B ? __ldg(p.scale + bb) : 0.f;
+            }
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             const bool row_ok = row < p.R;
             if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
             tc_fence_after_sync();
             const uint32_t t_lane = tmem_base + buf * (uint32_t)ACC_COLS + ((uint32_t)(lane_grp * 32) << 16);
-            // (not unrolled: the code of all roles together has to stay within reach of the
-            // instruction caches, or the warp that issues the MMAs stalls on fetches)
-#pragma unroll 1
+#pragma unroll
             for (int k = 0; k < MY_GROUPS; ++k) {
                 const int g = half + 2 * k;
                 uint32_t acc[ND][8];
 #pragma unroll
                 for (int d = 0; d < ND; ++d) tmem_ld8(t_lane + (uint32_t)(d * TOK + g * 8), acc[d]);
                 const int b0 = jt * TOK + g * 8;
-                float my_scale = 0.f;   // lane i: scale of token b0 + (i & 7), 0 beyond the batch
-                if constexpr (EPI != EPI_ACC) my_scale = b0 + (lane & 7) < p.B ? __ldg(p.scale + b0 + (lane & 7)) : 0.f;
+                const float my_scale = scales[k];
                 tmem_ld_wait();
                 const int n_live = min(8, p.B - b0);   // uniform across the warp
                 if constexpr (EPI == EPI_ACC) {
