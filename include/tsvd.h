@@ -45,8 +45,14 @@ typedef enum {
 /* flags of tsvd_forward_ex */
 #define TSVD_FLAG_OUT_F32 0x1u      /* write y as fp32 even for bf16 activations            */
 #define TSVD_FLAG_PATH_SIMPLE 0x10u /* force the CUDA-core reference kernels               */
-#define TSVD_FLAG_PATH_DECODE 0x20u /* force the small-batch streaming kernels             */
+#define TSVD_FLAG_PATH_DECODE 0x20u /* force the decode kernels (B <= TSVD_DECODE_MAX_B)    */
 #define TSVD_FLAG_PATH_TENSOR 0x40u /* force the tcgen05 tensor-core kernels               */
+/* The decode kernels (two launches, one per stage; each CTA streams 16 rows of the packed
+ * codes against fixed-point digits of the stage's input held in shared memory) serve batches
+ * of at most this many tokens, and are what a forward of so few tokens runs by default.
+ * Forcing them for a larger batch, or for a contraction too long for the digits to fit in
+ * shared memory (about 12,000 columns at four tokens), returns TSVD_E_TOOBIG. */
+#define TSVD_DECODE_MAX_B 4
 /* Test hook for the bounded device-side waits: with B > 64 the V-stage kernel's copy
  * producer withholds the activation digits, so every wait on them runs out (after a few
  * milliseconds instead of the usual ~2 s); all CTAs then leave through their normal exit,
@@ -159,8 +165,8 @@ tsvd_status_t tsvd_unpack(tsvd_handle_t h, int8_t* U, float* S, int8_t* V);
 /*
  * tsvd_plan -- which kernels a forward with these arguments would run (no launch).
  *   path  receives TSVD_FLAG_PATH_SIMPLE, _DECODE or _TENSOR
- *   digits_x, digits_t  receive the number of signed 8-bit digits the tensor-core path
- *   uses for the activations and for S*(V x) (0 on the other paths).  Executed tensor
+ *   digits_x, digits_t  receive the number of signed 8-bit digits the tensor-core and
+ *   decode paths use for the activations and for S*(V x) (0 on the CUDA-core path).  Executed tensor
  *   operations per forward = 2*B*(K*N*digits_x + M*K*digits_t) on the padded shapes; the
  *   paper's own count is additions at the nonzeros only (Table S1).
  */

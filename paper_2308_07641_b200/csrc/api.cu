@@ -204,15 +204,17 @@ static tsvd_status_t ensure_ws(tsvd_handle_s* h, size_t bytes)
     return TSVD_OK;
 }
 
-// The dispatch rule shared by tsvd_plan and tsvd_forward_ex.  The tensor-core kernels serve every
-// batch size (a small batch leaves most of a tile's columns empty, yet still streams the packed
-// codes several times faster than the CUDA-core kernels); the CUDA-core kernels remain as the
-// plain reference path, on request.
-static unsigned choose_path(int B, unsigned forced)
+// The dispatch rule shared by tsvd_plan and tsvd_forward_ex.  Up to TSVD_DECODE_MAX_B tokens run
+// the decode kernels when the digits of the stage inputs fit in shared memory; everything else
+// runs the tensor-core kernels (which serve every batch size); the CUDA-core kernels remain as
+// the plain reference path, on request.  Returns 0 when a forced path cannot serve the request.
+static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, unsigned forced)
 {
-    (void)B;
     if (forced == TSVD_FLAG_PATH_SIMPLE) return TSVD_FLAG_PATH_SIMPLE;
-    return TSVD_FLAG_PATH_TENSOR;
+    if (forced == TSVD_FLAG_PATH_TENSOR) return TSVD_FLAG_PATH_TENSOR;
+    const bool fits = tsvd_decode_fits(h, B, dtype);
+    if (forced == TSVD_FLAG_PATH_DECODE) return fits ? TSVD_FLAG_PATH_DECODE : 0u;
+    return fits ? TSVD_FLAG_PATH_DECODE : TSVD_FLAG_PATH_TENSOR;
 }
 
 extern "C" tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, unsigned flags, unsigned* path,
@@ -223,10 +225,11 @@ extern "C" tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, u
     if (dtype_size(dtype) == 0) return TSVD_E_DTYPE;
     const unsigned forced = flags & (TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR);
     if (forced & (forced - 1)) return TSVD_E_DTYPE;
-    const unsigned p = choose_path(B, forced);
+    const unsigned p = choose_path(h, B, dtype, forced);
+    if (p == 0u) return TSVD_E_TOOBIG;
     if (path) *path = p;
-    if (digits_x) *digits_x = (p == TSVD_FLAG_PATH_TENSOR) ? tsvd_tensor_digits_x(dtype) : 0;
-    if (digits_t) *digits_t = (p == TSVD_FLAG_PATH_TENSOR) ? tsvd_tensor_digits_t() : 0;
+    if (digits_x) *digits_x = (p != TSVD_FLAG_PATH_SIMPLE) ? tsvd_tensor_digits_x(dtype) : 0;
+    if (digits_t) *digits_t = (p != TSVD_FLAG_PATH_SIMPLE) ? tsvd_tensor_digits_t() : 0;
     return TSVD_OK;
 }
 
@@ -256,10 +259,17 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     a.test_stall = (flags & TSVD_FLAG_TEST_STALL) != 0;
     a.stream = (cudaStream_t)stream;
 
-    if (choose_path(B, path) == TSVD_FLAG_PATH_TENSOR) {
+    const unsigned chosen = choose_path(h, B, dtype, path);
+    if (chosen == 0u) return TSVD_E_TOOBIG;
+    if (chosen == TSVD_FLAG_PATH_TENSOR) {
         tsvd_status_t st = ensure_ws(h, tsvd_tensor_ws_bytes(h, B, dtype));
         if (st != TSVD_OK) return st;
         return tsvd_forward_tensor(a, h->ws);
+    }
+    if (chosen == TSVD_FLAG_PATH_DECODE) {
+        tsvd_status_t st = ensure_ws(h, tsvd_decode_ws_bytes(h, B));
+        if (st != TSVD_OK) return st;
+        return tsvd_forward_decode(a, h->ws);
     }
     tsvd_status_t st = ensure_ws(h, tsvd_simple_ws_bytes(h, B));
     if (st != TSVD_OK) return st;

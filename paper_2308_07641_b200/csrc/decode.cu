@@ -1,0 +1,307 @@
+// Decode path: y = U(diag(S)(V x)) for one to four tokens, bound by streaming the packed codes.
+//
+// For so few tokens a tensor-core tile is almost empty, and what matters is that every SM
+// streams its share of the 2-bit codes (the whole of U and V is read once per forward) with as
+// little fixed cost as possible.  Two launches, one per stage (Table S1 rows "V(.)" and "U(.)"):
+// each CTA first turns the stage's input (x, or t = S*(V x)) into the same per-token fixed-point
+// digits as the tensor-core path, in shared memory, then walks 16 rows of the packed matrix:
+// a lane owns a row, expands its codes to int8 with two byte permutes per eight entries and adds
+// them to the digits with four-way integer dot products.  All sums are exact integers, so the
+// result does not depend on how the columns are split over the warps.
+#include "tsvd_internal.cuh"
+
+namespace {
+
+constexpr int GEMV_THREADS = 256;
+constexpr int GEMV_WARPS = GEMV_THREADS / 32;
+constexpr int GEMV_ROWS = 16;       // rows per CTA: a warp pass covers 16 rows x 2 column groups
+constexpr int GEMV_MAX_SMEM = 200 * 1024;
+
+enum { STAGE_V = 0, STAGE_U = 1 };
+
+struct GemvParams {
+    const uint4* units;   // packed ternary operand
+    int R, C, C_pad;      // logical rows and columns, padded columns
+    const void* in;       // [B][ld_in]: activations (V-stage) or t (U-stage, fp32)
+    int ld_in;
+    int B;
+    const float* S;       // V-stage: padded to R_pad
+    void* out;            // V-stage: t fp32 [B][ld_out] (all padded rows); U-stage: y [B][ld_out]
+    int ld_out;
+    int out_bf16;
+    void* z_out;          // V-stage, optional: [B][z_ld] int32 (z_int) or fp32
+    int z_ld;
+    int z_int;
+};
+
+template <typename T> __device__ __forceinline__ float as_float(T v);
+template <> __device__ __forceinline__ float as_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ float as_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <> __device__ __forceinline__ float as_float<int8_t>(int8_t v) { return (float)v; }
+
+// Balanced radix-256 digits of four fixed-point integers: word d holds digit d of the four
+// values.  Digit d is byte d of q + 0x80 + 0x8000 + ... (d terms): adding half the radix at the
+// lower positions turns the floor of the shift into rounding, and the top digit is what is left.
+template <int ND>
+__device__ __forceinline__ void digits_of_4(const int (&q)[4], uint32_t (&dig)[ND])
+{
+#pragma unroll
+    for (int d = 0; d < ND; ++d) {
+        const uint32_t off = d == 0 ? 0u : d == 1 ? 0x80u : d == 2 ? 0x8080u : 0x808080u;
+        const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);   // byte d of a, byte d of b
+        const uint32_t lo = __byte_perm((uint32_t)q[0] + off, (uint32_t)q[1] + off, sel);
+        const uint32_t hi = __byte_perm((uint32_t)q[2] + off, (uint32_t)q[3] + off, sel);
+        dig[d] = __byte_perm(lo, hi, 0x5410);
+    }
+}
+
+// grid: R_pad / 16 CTAs of 256 threads.  Dynamic shared memory:
+//   digits [NTOK][ND][C_pad] int8 | partial sums [8 warps][NTOK*ND][16 rows] int32 |
+//   scale [NTOK] | per-warp maxima [8][NTOK]
+template <typename IN_T, int ND, int NTOK, int STAGE>
+__global__ void __launch_bounds__(GEMV_THREADS)
+ternary_gemv_kernel(const GemvParams p)
+{
+    extern __shared__ __align__(16) uint8_t smem[];
+    constexpr bool kInt = sizeof(IN_T) == 1;
+    static_assert(!kInt || ND == 1, "int8 activations are their own digit");
+    int8_t* dig = reinterpret_cast<int8_t*>(smem);
+    int* red = reinterpret_cast<int*>(smem + (size_t)NTOK * ND * p.C_pad);
+    float* scale = reinterpret_cast<float*>(red + GEMV_WARPS * NTOK * ND * GEMV_ROWS);
+    float* wmax = scale + NTOK;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
+
+    // ---- the stage's input as fixed-point digits (every CTA makes its own copy) ----
+    float qscale[NTOK];
+#pragma unroll
+    for (int b = 0; b < NTOK; ++b) qscale[b] = 1.f;
+    if constexpr (!kInt) {
+        float amax[NTOK];
+#pragma unroll
+        for (int b = 0; b < NTOK; ++b) amax[b] = 0.f;
+        for (int c = tid; c < p.C; c += GEMV_THREADS) {
+#pragma unroll
+            for (int b = 0; b < NTOK; ++b)
+                if (b < p.B) amax[b] = fmaxf(amax[b], fabsf(as_float<IN_T>(in[(size_t)b * p.ld_in + c])));
+        }
+#pragma unroll
+        for (int b = 0; b < NTOK; ++b) {
+            for (int o = 16; o > 0; o >>= 1) amax[b] = fmaxf(amax[b], __shfl_xor_sync(0xffffffffu, amax[b], o));
+            if (lane == 0) wmax[warp * NTOK + b] = amax[b];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int b = 0; b < NTOK; ++b) {
+            float m = 0.f;
+#pragma unroll
+            for (int w = 0; w < GEMV_WARPS; ++w) m = fmaxf(m, wmax[w * NTOK + b]);
+            // |v| <= m < 2^E; quantise to q = rint(v * 2^(8ND-2-E)), so |q| <= 2^(8ND-2)
+            int E = -90;
+            if (m > 0.f) {
+                int e;
+                (void)frexpf(m, &e);
+                E = max(e, -90);
+            }
+            qscale[b] = exp2f((float)(8 * ND - 2 - E));
+            if (tid == 0) scale[b] = exp2f((float)(E - (8 * ND - 2)));   // value = q * scale
+        }
+    } else {
+        if (tid < NTOK) scale[tid] = 1.f;
+    }
+    for (int c = tid * 4; c < p.C_pad; c += GEMV_THREADS * 4) {
+#pragma unroll
+        for (int b = 0; b < NTOK; ++b) {
+            int q[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float v = 0.f;
+                if (b < p.B && c + e < p.C) v = as_float<IN_T>(in[(size_t)b * p.ld_in + c + e]);
+                q[e] = __float2int_rn(v * qscale[b]);
+            }
+            uint32_t dw[ND];
+            digits_of_4<ND>(q, dw);
+#pragma unroll
+            for (int d = 0; d < ND; ++d)
+                *reinterpret_cast<uint32_t*>(dig + (size_t)(b * ND + d) * p.C_pad + c) = dw[d];
+        }
+    }
+    __syncthreads();
+
+    // ---- stream the codes: lane = (column-group parity, row), warp w takes groups 2w, 2w+1, +16.. ----
+    const int rsel = lane & 15, csel = lane >> 4;
+    const int row = blockIdx.x * GEMV_ROWS + rsel;
+    const int n_groups = p.C_pad >> 6;
+    int acc[NTOK][ND];
+#pragma unroll
+    for (int b = 0; b < NTOK; ++b)
+#pragma unroll
+        for (int d = 0; d < ND; ++d) acc[b][d] = 0;
+
+    constexpr int AHEAD = 4;   // 16-byte loads in flight per lane
+    for (int cg0 = 2 * warp + csel; cg0 < n_groups; cg0 += 2 * GEMV_WARPS * AHEAD) {
+        uint4 u[AHEAD];
+#pragma unroll
+        for (int a = 0; a < AHEAD; ++a) {
+            const int cg = cg0 + a * 2 * GEMV_WARPS;
+            u[a] = cg < n_groups ? __ldcs(p.units + tsvd_unit_index(row, cg, p.C_pad)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int a = 0; a < AHEAD; ++a) {
+            const int cg = cg0 + a * 2 * GEMV_WARPS;
+            if (cg >= n_groups) break;
+            const uint32_t w[4] = {u[a].x, u[a].y, u[a].z, u[a].w};
+#pragma unroll
+            for (int wi = 0; wi < 4; ++wi) {
+                uint32_t e[4];   // sixteen entries of the row as int8, in column order
+                tsvd_expand16(w[wi], e);
+#pragma unroll
+                for (int b = 0; b < NTOK; ++b) {
+#pragma unroll
+                    for (int d = 0; d < ND; ++d) {
+                        const uint4 xd = *reinterpret_cast<const uint4*>(dig + (size_t)(b * ND + d) * p.C_pad + cg * 64 + wi * 16);
+                        int s = acc[b][d];
+                        s = __dp4a((int)e[0], (int)xd.x, s);
+                        s = __dp4a((int)e[1], (int)xd.y, s);
+                        s = __dp4a((int)e[2], (int)xd.z, s);
+                        s = __dp4a((int)e[3], (int)xd.w, s);
+                        acc[b][d] = s;
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- add the two column-group parities and the eight warps ----
+#pragma unroll
+    for (int b = 0; b < NTOK; ++b)
+#pragma unroll
+        for (int d = 0; d < ND; ++d) {
+            const int v = acc[b][d] + __shfl_xor_sync(0xffffffffu, acc[b][d], 16);
+            if (csel == 0) red[(warp * NTOK * ND + b * ND + d) * GEMV_ROWS + rsel] = v;
+        }
+    __syncthreads();
+
+    // ---- thread (token, row): digits -> fp32 -> the stage's output ----
+    if (tid < NTOK * GEMV_ROWS) {
+        const int b = tid / GEMV_ROWS, r = tid % GEMV_ROWS;
+        const int orow = blockIdx.x * GEMV_ROWS + r;
+        if (b < p.B) {
+            int a[ND];
+#pragma unroll
+            for (int d = 0; d < ND; ++d) {
+                int s = 0;
+#pragma unroll
+                for (int w = 0; w < GEMV_WARPS; ++w) s += red[(w * NTOK * ND + b * ND + d) * GEMV_ROWS + r];
+                a[d] = s;
+            }
+            // lo and hi are exact 32-bit integers; their conversions and the fused multiply-add
+            // round at 2^-24 of |hi|*65536 and |lo|
+            float f;
+            if constexpr (ND == 1) f = (float)a[0];
+            else if constexpr (ND == 2) f = (float)(a[0] + (a[1] << 8));
+            else {
+                const int lo = a[0] + (a[1] << 8);
+                int hi = a[2];
+                if constexpr (ND == 4) hi += a[3] << 8;
+                f = fmaf((float)hi, 65536.f, (float)lo);
+            }
+            const float val = f * scale[b];   // a power of two: exact
+            if constexpr (STAGE == STAGE_V) {
+                // the K multiplications (Table S1); padded rows have S = 0 and no codes
+                reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + orow] = p.S[orow] * val;
+                if (p.z_out && orow < p.R) {
+                    if (p.z_int) reinterpret_cast<int*>(p.z_out)[(size_t)b * p.z_ld + orow] = a[0];
+                    else reinterpret_cast<float*>(p.z_out)[(size_t)b * p.z_ld + orow] = val;
+                }
+            } else if (orow < p.R) {
+                if (p.out_bf16)
+                    reinterpret_cast<__nv_bfloat16*>(p.out)[(size_t)b * p.ld_out + orow] = __float2bfloat16_rn(val);
+                else
+                    reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + orow] = val;
+            }
+        }
+    }
+}
+
+size_t gemv_smem_bytes(int nd, int ntok, int C_pad)
+{
+    return (size_t)ntok * nd * C_pad + (size_t)GEMV_WARPS * ntok * nd * GEMV_ROWS * sizeof(int) +
+           (size_t)ntok * sizeof(float) + (size_t)GEMV_WARPS * ntok * sizeof(float);
+}
+
+template <typename IN_T, int ND, int NTOK, int STAGE>
+cudaError_t launch_gemv(const GemvParams& p, int R_pad, cudaStream_t stream)
+{
+    static bool attr_set[64] = {};   // per instantiation and device
+    const size_t smem = gemv_smem_bytes(ND, NTOK, p.C_pad);
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(ternary_gemv_kernel<IN_T, ND, NTOK, STAGE>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, GEMV_MAX_SMEM);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    ternary_gemv_kernel<IN_T, ND, NTOK, STAGE><<<R_pad / GEMV_ROWS, GEMV_THREADS, smem, stream>>>(p);
+    tsvd_count_launch();
+    return cudaGetLastError();
+}
+
+template <typename IN_T, int ND, int STAGE>
+cudaError_t launch_gemv_tokens(const GemvParams& p, int R_pad, cudaStream_t stream)
+{
+    if (p.B == 1) return launch_gemv<IN_T, ND, 1, STAGE>(p, R_pad, stream);
+    if (p.B == 2) return launch_gemv<IN_T, ND, 2, STAGE>(p, R_pad, stream);
+    return launch_gemv<IN_T, ND, 4, STAGE>(p, R_pad, stream);
+}
+
+constexpr int ND_T = 4;   // digits of the intermediate t (fp32), as on the tensor-core path
+inline int digits_for_x(tsvd_dtype_t dt) { return dt == TSVD_I8 ? 1 : dt == TSVD_BF16 ? 3 : 4; }
+
+}  // namespace
+
+bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt)
+{
+    if (B < 1 || B > TSVD_DECODE_MAX_B) return false;
+    const int ntok = B == 3 ? 4 : B;
+    return gemv_smem_bytes(digits_for_x(dt), ntok, h->V.C_pad) <= (size_t)GEMV_MAX_SMEM &&
+           gemv_smem_bytes(ND_T, ntok, h->U.C_pad) <= (size_t)GEMV_MAX_SMEM;
+}
+
+size_t tsvd_decode_ws_bytes(const tsvd_handle_s* h, int B) { return (size_t)B * h->V.R_pad * sizeof(float); }
+
+tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws)
+{
+    tsvd_handle_s* h = a.h;
+    cudaStream_t st = a.stream;
+    float* t = reinterpret_cast<float*>(ws);
+
+    GemvParams p{};
+    p.units = h->V.units; p.R = h->K; p.C = h->N; p.C_pad = h->V.C_pad;
+    p.in = a.x; p.ld_in = a.ldx; p.B = a.B; p.S = h->S;
+    p.out = t; p.ld_out = h->V.R_pad;
+    p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
+    cudaError_t e;
+    h->prof.begin(1, st);
+    switch (a.dtype) {
+        case TSVD_F32: e = launch_gemv_tokens<float, 4, STAGE_V>(p, h->V.R_pad, st); break;
+        case TSVD_BF16: e = launch_gemv_tokens<__nv_bfloat16, 3, STAGE_V>(p, h->V.R_pad, st); break;
+        case TSVD_I8: e = launch_gemv_tokens<int8_t, 1, STAGE_V>(p, h->V.R_pad, st); break;
+        default: return TSVD_E_DTYPE;
+    }
+    h->prof.end(st);
+    if (e != cudaSuccess) return TSVD_E_CUDA;
+
+    GemvParams q{};
+    q.units = h->U.units; q.R = h->M; q.C = h->K; q.C_pad = h->U.C_pad;
+    q.in = t; q.ld_in = h->V.R_pad; q.B = a.B;
+    q.out = a.y; q.ld_out = a.ldy;
+    q.out_bf16 = (a.dtype == TSVD_BF16) && !a.out_f32;
+    h->prof.begin(3, st);
+    e = launch_gemv_tokens<float, ND_T, STAGE_U>(q, h->U.R_pad, st);
+    h->prof.end(st);
+    return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
+}

@@ -124,6 +124,11 @@ size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt);
 int tsvd_tensor_digits_x(tsvd_dtype_t dt);
 int tsvd_tensor_digits_t();
 
+// decode.cu -- one to four tokens, bound by streaming the packed codes
+bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt);
+size_t tsvd_decode_ws_bytes(const tsvd_handle_s* h, int B);
+tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws);
+
 #define TSVD_CUDA_OK(expr)                            \
     do {                                              \
         cudaError_t _e = (expr);                      \

@@ -99,6 +99,66 @@ def test_small_cases_every_element(spec, path):
     _util.run_and_check(spec, flags=PATHS[path])
 
 
+# ---- decode kernels: one to four tokens ------------------------------------------------------------
+DECODE = [
+    gen.scaled(C["cfg1"], name="dec_tiny_1x1x1", M=1, N=1, K=1, B=1, density=1.0),
+    gen.scaled(C["cfg1"], name="dec_f32_b3", M=300, N=333, K=200, B=3, seed=21),
+    gen.scaled(C["cfg1"], name="dec_f32_b1", M=131, N=1100, K=257, B=1, seed=22),
+    gen.scaled(C["cfg3_b1"], name="dec_bf16_b1", M=512, N=640, K=384),
+    gen.scaled(C["cfg3_b4"], name="dec_bf16_b2", M=520, N=2100, K=390, B=2, seed=23),
+    gen.scaled(C["cfg3_b4"], name="dec_bf16_b4", M=512, N=640, K=384),
+    gen.scaled(C["cfg5_d20"], name="dec_i8_b4", M=256, N=384, K=512, B=4),
+    gen.scaled(C["cfg5_d50"], name="dec_i8_b1_dense", M=129, N=257, K=255, B=1, density=1.0),
+    gen.scaled(C["cfg2"], name="dec_all_zero", M=140, N=130, K=150, B=2, density=0.0),
+    gen.scaled(C["cfg2"], name="dec_row_density_varies", M=260, N=300, K=280, B=4, row_density_spread=0.9),
+]
+
+
+@pytest.mark.parametrize("spec", DECODE, ids=lambda s: s.name)
+def test_decode_cases_every_element(spec):
+    _util.run_and_check(spec, flags=0x20)
+
+
+def test_decode_is_the_default_up_to_four_tokens_and_refuses_more():
+    import torch
+    from paper_2308_07641_b200 import binding
+    rng = np.random.default_rng(5)
+    U = rng.integers(-1, 2, (40, 24)).astype(np.int8); V = rng.integers(-1, 2, (24, 36)).astype(np.int8)
+    S = np.ones(24, np.float32)
+    h = binding.tsvd_pack(U, S, V)
+    try:
+        for B in (1, 2, 3, 4):
+            assert binding.tsvd_plan(h, B, binding.TSVD_BF16)["path"] == "decode"
+            assert binding.tsvd_plan(h, B, binding.TSVD_BF16, 0x40)["path"] == "tensor"
+        assert binding.tsvd_plan(h, 5, binding.TSVD_BF16)["path"] == "tensor"
+        plan = binding.tsvd_plan(h, 4, binding.TSVD_I8, 0x20)
+        assert (plan["path"], plan["digits_x"], plan["digits_t"]) == ("decode", 1, 4)
+        x = torch.zeros(5 * 36, device="cuda"); y = torch.zeros(5 * 40, device="cuda")
+        L = binding.lib()
+        assert L.tsvd_forward_ex(h, x.data_ptr(), 36, y.data_ptr(), 40, 5, 0, 0x20, None, None) == binding.TSVD_E_TOOBIG
+        assert L.tsvd_forward_ex(h, x.data_ptr(), 36, y.data_ptr(), 40, 4, 0, 0x20, None, None) == binding.TSVD_OK
+        torch.cuda.synchronize()
+    finally:
+        binding.tsvd_destroy(h)
+
+
+def test_decode_and_tensor_paths_agree_bit_for_bit():
+    """Both quantise the stage inputs the same way and add exact integers: identical outputs."""
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear
+    spec = gen.scaled(C["cfg3_b4"], name="agree", M=700, N=900, K=520, B=4, seed=31)
+    U, V, S = gen.make_weights(spec)
+    x = _util.torch_x(gen.make_x(spec), spec.x_dtype)
+    layer = TSVDLinear(U, S, V)
+    try:
+        y_dec = layer.forward(x, flags=0x20 | 0x1).clone()
+        y_ten = layer.forward(x, flags=0x40 | 0x1).clone()
+        torch.cuda.synchronize()
+        assert torch.equal(y_dec, y_ten)
+    finally:
+        layer.close()
+
+
 def test_out_f32_flag_and_strides():
     """bf16 activations with fp32 output, and leading dimensions larger than the row length."""
     import torch
