@@ -4,17 +4,23 @@
 // streams its share of the 2-bit codes (the whole of U and V is read once per forward) with as
 // little fixed cost as possible.  Two launches, one per stage (Table S1 rows "V(.)" and "U(.)"):
 // each CTA first turns the stage's input (x, or t = S*(V x)) into the same per-token fixed-point
-// digits as the tensor-core path, in shared memory, then walks 16 rows of the packed matrix:
-// a lane owns a row, expands its codes to int8 with two byte permutes per eight entries and adds
-// them to the digits with four-way integer dot products.  All sums are exact integers, so the
-// result does not depend on how the columns are split over the warps.
+// digits as the tensor-core path, in shared memory, then walks 32 rows of the packed matrix:
+// a lane owns four rows of one 64-column group at a time, expands their codes to int8 with two
+// byte permutes per eight entries and adds them to the digits with four-way integer dot
+// products.  (Four rows per lane because every lane reads the same digits: a shared-memory load
+// that all lanes aim at one address still takes its four passes, so each one has to feed as
+// many dot products as the registers allow.)  All sums are exact integers, so the result does
+// not depend on how the columns are split over the lanes and warps.
 #include "tsvd_internal.cuh"
 
 namespace {
 
 constexpr int GEMV_THREADS = 256;
 constexpr int GEMV_WARPS = GEMV_THREADS / 32;
-constexpr int GEMV_ROWS = 16;       // rows per CTA: a warp pass covers 16 rows x 2 column groups
+constexpr int GEMV_RL = 8;          // lanes of a warp along the rows; the other four take different column groups
+constexpr int GEMV_RPL = 4;         // rows per lane
+constexpr int GEMV_CS = 32 / GEMV_RL;
+constexpr int GEMV_ROWS = GEMV_RL * GEMV_RPL;   // rows per CTA
 constexpr int GEMV_MAX_SMEM = 200 * 1024;
 
 enum { STAGE_V = 0, STAGE_U = 1 };
@@ -55,8 +61,8 @@ __device__ __forceinline__ void digits_of_4(const int (&q)[4], uint32_t (&dig)[N
     }
 }
 
-// grid: R_pad / 16 CTAs of 256 threads.  Dynamic shared memory:
-//   digits [NTOK][ND][C_pad] int8 | partial sums [8 warps][NTOK*ND][16 rows] int32 |
+// grid: R_pad / 32 CTAs of 256 threads.  Dynamic shared memory:
+//   digits [NTOK][ND][C_pad] int8 | partial sums [8 warps][NTOK*ND][32 rows] int32 |
 //   scale [NTOK] | per-warp maxima [8][NTOK]
 template <typename IN_T, int ND, int NTOK, int STAGE>
 __global__ void __launch_bounds__(GEMV_THREADS)
@@ -72,6 +78,22 @@ ternary_gemv_kernel(const GemvParams p)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
+
+    // lane = (column group within the pass, row); rows rsel, rsel + 8, .. of the CTA's 32; warp w
+    // takes column groups 4w + csel, + 32, ..  The first codes are requested before anything
+    // else, so that their trip from HBM overlaps with the digit conversion below.
+    const int rsel = lane & (GEMV_RL - 1), csel = lane / GEMV_RL;
+    const int row_base = blockIdx.x * GEMV_ROWS + rsel;
+    const int n_groups = p.C_pad >> 6;
+    auto load_units = [&](int g, uint4 (&uu)[GEMV_RPL]) {
+#pragma unroll
+        for (int j = 0; j < GEMV_RPL; ++j)
+            uu[j] = g < n_groups ? __ldcs(p.units + tsvd_unit_index(row_base + j * GEMV_RL, g, p.C_pad))
+                                 : make_uint4(0, 0, 0, 0);
+    };
+    int cg = GEMV_CS * warp + csel;
+    uint4 u[GEMV_RPL];
+    load_units(cg, u);
 
     // ---- the stage's input as fixed-point digits (every CTA makes its own copy) ----
     float qscale[NTOK];
@@ -129,58 +151,57 @@ ternary_gemv_kernel(const GemvParams p)
     }
     __syncthreads();
 
-    // ---- stream the codes: lane = (column-group parity, row), warp w takes groups 2w, 2w+1, +16.. ----
-    const int rsel = lane & 15, csel = lane >> 4;
-    const int row = blockIdx.x * GEMV_ROWS + rsel;
-    const int n_groups = p.C_pad >> 6;
-    int acc[NTOK][ND];
+    // ---- stream the codes ----
+    int acc[GEMV_RPL][NTOK][ND];
 #pragma unroll
-    for (int b = 0; b < NTOK; ++b)
+    for (int j = 0; j < GEMV_RPL; ++j)
 #pragma unroll
-        for (int d = 0; d < ND; ++d) acc[b][d] = 0;
+        for (int b = 0; b < NTOK; ++b)
+#pragma unroll
+            for (int d = 0; d < ND; ++d) acc[j][b][d] = 0;
 
-    constexpr int AHEAD = 4;   // 16-byte loads in flight per lane
-    for (int cg0 = 2 * warp + csel; cg0 < n_groups; cg0 += 2 * GEMV_WARPS * AHEAD) {
-        uint4 u[AHEAD];
+    for (; cg < n_groups; cg += GEMV_CS * GEMV_WARPS) {
+        uint4 un[GEMV_RPL];   // the next pass, in flight while this one is summed
+        load_units(cg + GEMV_CS * GEMV_WARPS, un);
 #pragma unroll
-        for (int a = 0; a < AHEAD; ++a) {
-            const int cg = cg0 + a * 2 * GEMV_WARPS;
-            u[a] = cg < n_groups ? __ldcs(p.units + tsvd_unit_index(row, cg, p.C_pad)) : make_uint4(0, 0, 0, 0);
-        }
+        for (int wi = 0; wi < 4; ++wi) {
+            uint32_t e[GEMV_RPL][4];   // sixteen entries of each row as int8, in column order
 #pragma unroll
-        for (int a = 0; a < AHEAD; ++a) {
-            const int cg = cg0 + a * 2 * GEMV_WARPS;
-            if (cg >= n_groups) break;
-            const uint32_t w[4] = {u[a].x, u[a].y, u[a].z, u[a].w};
+            for (int j = 0; j < GEMV_RPL; ++j)
+                tsvd_expand16(wi == 0 ? u[j].x : wi == 1 ? u[j].y : wi == 2 ? u[j].z : u[j].w, e[j]);
 #pragma unroll
-            for (int wi = 0; wi < 4; ++wi) {
-                uint32_t e[4];   // sixteen entries of the row as int8, in column order
-                tsvd_expand16(w[wi], e);
+            for (int b = 0; b < NTOK; ++b) {
 #pragma unroll
-                for (int b = 0; b < NTOK; ++b) {
+                for (int d = 0; d < ND; ++d) {
+                    const uint4 xd = *reinterpret_cast<const uint4*>(dig + (size_t)(b * ND + d) * p.C_pad + cg * 64 + wi * 16);
 #pragma unroll
-                    for (int d = 0; d < ND; ++d) {
-                        const uint4 xd = *reinterpret_cast<const uint4*>(dig + (size_t)(b * ND + d) * p.C_pad + cg * 64 + wi * 16);
-                        int s = acc[b][d];
-                        s = __dp4a((int)e[0], (int)xd.x, s);
-                        s = __dp4a((int)e[1], (int)xd.y, s);
-                        s = __dp4a((int)e[2], (int)xd.z, s);
-                        s = __dp4a((int)e[3], (int)xd.w, s);
-                        acc[b][d] = s;
+                    for (int j = 0; j < GEMV_RPL; ++j) {
+                        int s = acc[j][b][d];
+                        s = __dp4a((int)e[j][0], (int)xd.x, s);
+                        s = __dp4a((int)e[j][1], (int)xd.y, s);
+                        s = __dp4a((int)e[j][2], (int)xd.z, s);
+                        s = __dp4a((int)e[j][3], (int)xd.w, s);
+                        acc[j][b][d] = s;
                     }
                 }
             }
         }
+#pragma unroll
+        for (int j = 0; j < GEMV_RPL; ++j) u[j] = un[j];
     }
 
-    // ---- add the two column-group parities and the eight warps ----
+    // ---- add the lanes that took different column groups, then the eight warps ----
 #pragma unroll
-    for (int b = 0; b < NTOK; ++b)
+    for (int j = 0; j < GEMV_RPL; ++j)
 #pragma unroll
-        for (int d = 0; d < ND; ++d) {
-            const int v = acc[b][d] + __shfl_xor_sync(0xffffffffu, acc[b][d], 16);
-            if (csel == 0) red[(warp * NTOK * ND + b * ND + d) * GEMV_ROWS + rsel] = v;
-        }
+        for (int b = 0; b < NTOK; ++b)
+#pragma unroll
+            for (int d = 0; d < ND; ++d) {
+                int v = acc[j][b][d];
+                v += __shfl_xor_sync(0xffffffffu, v, 8);
+                v += __shfl_xor_sync(0xffffffffu, v, 16);
+                if (csel == 0) red[(warp * NTOK * ND + b * ND + d) * GEMV_ROWS + j * GEMV_RL + rsel] = v;
+            }
     __syncthreads();
 
     // ---- thread (token, row): digits -> fp32 -> the stage's output ----
