@@ -11,6 +11,7 @@
 // that all lanes aim at one address still takes its four passes, so each one has to feed as
 // many dot products as the registers allow.)  All sums are exact integers, so the result does
 // not depend on how the columns are split over the lanes and warps.
+#include "digits.cuh"
 #include "tsvd_internal.cuh"
 
 namespace {
@@ -39,27 +40,6 @@ struct GemvParams {
     int z_ld;
     int z_int;
 };
-
-template <typename T> __device__ __forceinline__ float as_float(T v);
-template <> __device__ __forceinline__ float as_float<float>(float v) { return v; }
-template <> __device__ __forceinline__ float as_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
-template <> __device__ __forceinline__ float as_float<int8_t>(int8_t v) { return (float)v; }
-
-// Balanced radix-256 digits of four fixed-point integers: word d holds digit d of the four
-// values.  Digit d is byte d of q + 0x80 + 0x8000 + ... (d terms): adding half the radix at the
-// lower positions turns the floor of the shift into rounding, and the top digit is what is left.
-template <int ND>
-__device__ __forceinline__ void digits_of_4(const int (&q)[4], uint32_t (&dig)[ND])
-{
-#pragma unroll
-    for (int d = 0; d < ND; ++d) {
-        const uint32_t off = d == 0 ? 0u : d == 1 ? 0x80u : d == 2 ? 0x8080u : 0x808080u;
-        const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);   // byte d of a, byte d of b
-        const uint32_t lo = __byte_perm((uint32_t)q[0] + off, (uint32_t)q[1] + off, sel);
-        const uint32_t hi = __byte_perm((uint32_t)q[2] + off, (uint32_t)q[3] + off, sel);
-        dig[d] = __byte_perm(lo, hi, 0x5410);
-    }
-}
 
 // grid: R_pad / 32 CTAs of 256 threads.  Dynamic shared memory:
 //   digits [NTOK][ND][C_pad] int8 | partial sums [8 warps][NTOK*ND][32 rows] int32 |
@@ -95,18 +75,37 @@ ternary_gemv_kernel(const GemvParams p)
     uint4 u[GEMV_RPL];
     load_units(cg, u);
 
-    // ---- the stage's input as fixed-point digits (every CTA makes its own copy) ----
+    // ---- the stage's input as fixed-point digits (every CTA makes its own copy).  A thread takes
+    //      chunks of 16 consecutive columns; all loads of a pass are independent, so a pass costs
+    //      about one trip to L2, and the first chunk of each token stays in registers between the
+    //      maximum pass and the conversion pass ----
+    const int n_chunks = p.C_pad >> 4;
+    float keep[NTOK][16];
     float qscale[NTOK];
 #pragma unroll
     for (int b = 0; b < NTOK; ++b) qscale[b] = 1.f;
+    bool vec_ok[NTOK];
+#pragma unroll
+    for (int b = 0; b < NTOK; ++b)
+        vec_ok[b] = ((reinterpret_cast<uintptr_t>(in + (size_t)b * p.ld_in)) & 15) == 0;
     if constexpr (!kInt) {
         float amax[NTOK];
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) amax[b] = 0.f;
-        for (int c = tid; c < p.C; c += GEMV_THREADS) {
+        for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
 #pragma unroll
-            for (int b = 0; b < NTOK; ++b)
-                if (b < p.B) amax[b] = fmaxf(amax[b], fabsf(as_float<IN_T>(in[(size_t)b * p.ld_in + c])));
+            for (int b = 0; b < NTOK; ++b) {
+                if (b < p.B) {
+                    float v[16];
+                    load16<IN_T>(in + (size_t)b * p.ld_in, ch * 16, p.C, vec_ok[b], v);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) amax[b] = fmaxf(amax[b], fabsf(v[e]));
+                    if (ch == tid) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) keep[b][e] = v[e];
+                    }
+                }
+            }
         }
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) {
@@ -119,34 +118,38 @@ ternary_gemv_kernel(const GemvParams p)
             float m = 0.f;
 #pragma unroll
             for (int w = 0; w < GEMV_WARPS; ++w) m = fmaxf(m, wmax[w * NTOK + b]);
-            // |v| <= m < 2^E; quantise to q = rint(v * 2^(8ND-2-E)), so |q| <= 2^(8ND-2)
-            int E = -90;
-            if (m > 0.f) {
-                int e;
-                (void)frexpf(m, &e);
-                E = max(e, -90);
-            }
+            const int E = tsvd_quant_exponent(m);
             qscale[b] = exp2f((float)(8 * ND - 2 - E));
             if (tid == 0) scale[b] = exp2f((float)(E - (8 * ND - 2)));   // value = q * scale
         }
     } else {
         if (tid < NTOK) scale[tid] = 1.f;
     }
-    for (int c = tid * 4; c < p.C_pad; c += GEMV_THREADS * 4) {
+    for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) {
-            int q[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float v = 0.f;
-                if (b < p.B && c + e < p.C) v = as_float<IN_T>(in[(size_t)b * p.ld_in + c + e]);
-                q[e] = __float2int_rn(v * qscale[b]);
-            }
-            uint32_t dw[ND];
-            digits_of_4<ND>(q, dw);
+            uint32_t dw[ND][4];
 #pragma unroll
             for (int d = 0; d < ND; ++d)
-                *reinterpret_cast<uint32_t*>(dig + (size_t)(b * ND + d) * p.C_pad + c) = dw[d];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) dw[d][g] = 0u;
+            if (b < p.B) {
+                float v[16];
+                if (!kInt && ch == tid) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] = keep[b][e];
+                } else {
+                    load16<IN_T>(in + (size_t)b * p.ld_in, ch * 16, p.C, vec_ok[b], v);
+                }
+                int q[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) q[e] = __float2int_rn(v[e] * qscale[b]);
+                digits_of_16<ND>(q, dw);
+            }
+#pragma unroll
+            for (int d = 0; d < ND; ++d)
+                *reinterpret_cast<uint4*>(dig + (size_t)(b * ND + d) * p.C_pad + ch * 16) =
+                    make_uint4(dw[d][0], dw[d][1], dw[d][2], dw[d][3]);
         }
     }
     __syncthreads();

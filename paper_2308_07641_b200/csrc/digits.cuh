@@ -1,0 +1,85 @@
+// Fixed-point digits of the real-valued operand, shared by the tensor-core and decode kernels.
+//
+// A token's values v (|v| <= amax < 2^E) are written as integers q = rint(v * 2^(8ND-2-E)),
+// |q| <= 2^(8ND-2), and q as ND balanced radix-256 digits in [-128,127]: every product with a
+// ternary entry and every partial sum is then an exact integer.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+template <typename T> __device__ __forceinline__ float to_float(T v);
+template <> __device__ __forceinline__ float to_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <> __device__ __forceinline__ float to_float<int8_t>(int8_t v) { return (float)v; }
+
+// Balanced radix-256 digits of sixteen fixed-point integers, as ND words of four int8 each per
+// group of four values (dig[d][g] = digit d of values 4g..4g+3).  With q = sum_d digit_d*256^d
+// and digits in [-128,127], digit d is byte d of q + 0x80 + 0x8000 + ... (d terms): adding half
+// the radix at every lower position turns the floor of the arithmetic shift into rounding.
+// The top digit is what is left; it fits because |q| <= 2^(8ND-2).
+template <int ND>
+__device__ __forceinline__ void digits_of_16(const int (&q)[16], uint32_t (&dig)[ND][4])
+{
+#pragma unroll
+    for (int d = 0; d < ND; ++d) {
+        const uint32_t off = d == 0 ? 0u : d == 1 ? 0x80u : d == 2 ? 0x8080u : 0x808080u;
+        const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);   // byte d of a, byte d of b
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const uint32_t lo = __byte_perm((uint32_t)q[4 * g] + off, (uint32_t)q[4 * g + 1] + off, sel);
+            const uint32_t hi = __byte_perm((uint32_t)q[4 * g + 2] + off, (uint32_t)q[4 * g + 3] + off, sel);
+            dig[d][g] = __byte_perm(lo, hi, 0x5410);
+        }
+    }
+}
+
+// Load 16 consecutive values of a row as floats (vector loads when the chunk is whole and
+// 16-byte aligned, guarded scalar loads otherwise).
+template <typename IN_T>
+__device__ __forceinline__ void load16(const IN_T* __restrict__ row, int c0, int C, bool vec_ok, float (&v)[16])
+{
+    if (vec_ok && c0 + 16 <= C) {
+        if constexpr (sizeof(IN_T) == 4) {
+            const float4* p4 = reinterpret_cast<const float4*>(row + c0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 f = __ldg(p4 + i);
+                v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+            }
+        } else if constexpr (sizeof(IN_T) == 2) {
+            const uint4* p4 = reinterpret_cast<const uint4*>(row + c0);
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const uint4 u = __ldg(p4 + i);
+                const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {   // bf16 -> fp32 is a 16-bit shift
+                    v[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+                    v[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+                }
+            }
+        } else {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(row + c0));
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = (float)(int)(int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xFF);
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) v[e] = (c0 + e < C) ? to_float<IN_T>(row[c0 + e]) : 0.f;
+    }
+}
+
+// The exponent E of the rule above for a token whose largest magnitude is amax (0 -> a floor).
+__device__ __forceinline__ int tsvd_quant_exponent(float amax)
+{
+    int E = -90;
+    if (amax > 0.f) {
+        int e;
+        (void)frexpf(amax, &e);
+        E = max(e, -90);
+    }
+    return E;
+}

@@ -15,6 +15,7 @@
 // Batches above 64 tokens use 192-column tiles, one CTA per tile; smaller batches use 16-token
 // tiles with the contraction split across CTAs (integer atomics, the last part of a tile
 // finishes the stage), so that the packed codes are streamed by about one CTA per SM.
+#include "digits.cuh"
 #include "sm100_ptx.cuh"
 #include "tsvd_internal.cuh"
 
@@ -63,68 +64,6 @@ constexpr int GEMM_SMEM_BYTES = NB * B_SLOT_BYTES + NP * P_SLOT_BYTES +
 // K-major 128-byte-swizzle operand layout, so a tile is one contiguous bulk copy.
 // ---------------------------------------------------------------------------------------
 
-template <typename T> __device__ __forceinline__ float to_float(T v);
-template <> __device__ __forceinline__ float to_float<float>(float v) { return v; }
-template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
-template <> __device__ __forceinline__ float to_float<int8_t>(int8_t v) { return (float)v; }
-
-// Balanced radix-256 digits of sixteen fixed-point integers, as ND words of four int8 each per
-// group of four values (dig[d][g] = digit d of values 4g..4g+3).  With q = sum_d digit_d*256^d
-// and digits in [-128,127], digit d is byte d of q + 0x80 + 0x8000 + ... (d terms): adding half
-// the radix at every lower position turns the floor of the arithmetic shift into rounding.
-// The top digit is what is left; it fits because |q| <= 2^(8ND-2).
-template <int ND>
-__device__ __forceinline__ void digits_of_16(const int (&q)[16], uint32_t (&dig)[ND][4])
-{
-#pragma unroll
-    for (int d = 0; d < ND; ++d) {
-        const uint32_t off = d == 0 ? 0u : d == 1 ? 0x80u : d == 2 ? 0x8080u : 0x808080u;
-        const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);   // byte d of a, byte d of b
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const uint32_t lo = __byte_perm((uint32_t)q[4 * g] + off, (uint32_t)q[4 * g + 1] + off, sel);
-            const uint32_t hi = __byte_perm((uint32_t)q[4 * g + 2] + off, (uint32_t)q[4 * g + 3] + off, sel);
-            dig[d][g] = __byte_perm(lo, hi, 0x5410);
-        }
-    }
-}
-
-// Load 16 consecutive values of a row as floats (vector loads when the chunk is whole and
-// 16-byte aligned, guarded scalar loads otherwise).
-template <typename IN_T>
-__device__ __forceinline__ void load16(const IN_T* __restrict__ row, int c0, int C, bool vec_ok, float (&v)[16])
-{
-    if (vec_ok && c0 + 16 <= C) {
-        if constexpr (sizeof(IN_T) == 4) {
-            const float4* p4 = reinterpret_cast<const float4*>(row + c0);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float4 f = __ldg(p4 + i);
-                v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
-            }
-        } else if constexpr (sizeof(IN_T) == 2) {
-            const uint4* p4 = reinterpret_cast<const uint4*>(row + c0);
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const uint4 u = __ldg(p4 + i);
-                const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {   // bf16 -> fp32 is a 16-bit shift
-                    v[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
-                    v[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-                }
-            }
-        } else {
-            const uint4 u = __ldg(reinterpret_cast<const uint4*>(row + c0));
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = (float)(int)(int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xFF);
-        }
-    } else {
-#pragma unroll
-        for (int e = 0; e < 16; ++e) v[e] = (c0 + e < C) ? to_float<IN_T>(row[c0 + e]) : 0.f;
-    }
-}
 
 // TPT threads per token slot b in [0, B_pad): one warp (8 tokens per block) for large batches,
 // a whole block of 256 for small ones, where a row must be spread over more threads to hide
@@ -192,12 +131,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
             for (int w = 0; w < 8; ++w) amax = fmaxf(amax, red[w]);
         }
         // |v| <= amax < 2^E; quantise to q = rint(v * 2^(8ND-2-E)), so |q| <= 2^(8ND-2)
-        int E = -90;
-        if (amax > 0.f) {
-            int e;
-            (void)frexpf(amax, &e);
-            E = max(e, -90);
-        }
+        const int E = tsvd_quant_exponent(amax);
         qscale = exp2f((float)(8 * ND - 2 - E));
         if (lane == 0) scale_out[b] = exp2f((float)(E - (8 * ND - 2)));   // value = q * scale
     } else {
