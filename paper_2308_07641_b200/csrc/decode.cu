@@ -4,7 +4,7 @@
 // streams its share of the 2-bit codes (the whole of U and V is read once per forward) with as
 // little fixed cost as possible.  Two launches, one per stage (Table S1 rows "V(.)" and "U(.)"):
 // each CTA first turns the stage's input (x, or t = S*(V x)) into the same per-token fixed-point
-// digits as the tensor-core path, in shared memory, then walks 32 rows of the packed matrix:
+// digits as the tensor-core path, in shared memory, then walks 16 rows of the packed matrix:
 // a lane owns four rows of one 64-column group at a time, expands their codes to int8 with two
 // byte permutes per eight entries and adds them to the digits with four-way integer dot
 // products.  (Four rows per lane because every lane reads the same digits: a shared-memory load
@@ -18,7 +18,7 @@ namespace {
 
 constexpr int GEMV_THREADS = 256;
 constexpr int GEMV_WARPS = GEMV_THREADS / 32;
-constexpr int GEMV_RL = 8;          // lanes of a warp along the rows; the other four take different column groups
+constexpr int GEMV_RL = 4;          // lanes of a warp along the rows; the other eight take different column groups
 constexpr int GEMV_RPL = 4;         // rows per lane
 constexpr int GEMV_CS = 32 / GEMV_RL;
 constexpr int GEMV_ROWS = GEMV_RL * GEMV_RPL;   // rows per CTA
@@ -41,8 +41,8 @@ struct GemvParams {
     int z_int;
 };
 
-// grid: R_pad / 32 CTAs of 256 threads.  Dynamic shared memory:
-//   digits [NTOK][ND][C_pad] int8 | partial sums [8 warps][NTOK*ND][32 rows] int32 |
+// grid: R_pad / 16 CTAs of 256 threads.  Dynamic shared memory:
+//   digits [NTOK][ND][C_pad] int8 | partial sums [8 warps][NTOK*ND][16 rows] int32 |
 //   scale [NTOK] | per-warp maxima [8][NTOK]
 template <typename IN_T, int ND, int NTOK, int STAGE>
 __global__ void __launch_bounds__(GEMV_THREADS)
@@ -59,8 +59,8 @@ ternary_gemv_kernel(const GemvParams p)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
 
-    // lane = (column group within the pass, row); rows rsel, rsel + 8, .. of the CTA's 32; warp w
-    // takes column groups 4w + csel, + 32, ..  The first codes are requested before anything
+    // lane = (column group within the pass, row); rows rsel, rsel + 4, .. of the CTA's 16; warp w
+    // takes column groups 8w + csel, + 64, ..  The first codes are requested before anything
     // else, so that their trip from HBM overlaps with the digit conversion below.
     const int rsel = lane & (GEMV_RL - 1), csel = lane / GEMV_RL;
     const int row_base = blockIdx.x * GEMV_ROWS + rsel;
@@ -201,8 +201,8 @@ ternary_gemv_kernel(const GemvParams p)
 #pragma unroll
             for (int d = 0; d < ND; ++d) {
                 int v = acc[j][b][d];
-                v += __shfl_xor_sync(0xffffffffu, v, 8);
-                v += __shfl_xor_sync(0xffffffffu, v, 16);
+#pragma unroll
+                for (int o = GEMV_RL; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
                 if (csel == 0) red[(warp * NTOK * ND + b * ND + d) * GEMV_ROWS + j * GEMV_RL + rsel] = v;
             }
     __syncthreads();
