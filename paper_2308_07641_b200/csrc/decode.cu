@@ -16,8 +16,9 @@
 
 namespace {
 
-constexpr int GEMV_THREADS = 256;
-constexpr int GEMV_WARPS = GEMV_THREADS / 32;
+// threads per CTA: with one or two tokens the kernel waits on memory and wants many warps; with
+// four the accumulators need the registers
+__host__ __device__ constexpr int gemv_threads(int ntok) { return ntok <= 2 ? 512 : 256; }
 constexpr int GEMV_RL = 4;          // lanes of a warp along the rows; the other eight take different column groups
 constexpr int GEMV_RPL = 4;         // rows per lane
 constexpr int GEMV_CS = 32 / GEMV_RL;
@@ -42,13 +43,14 @@ struct GemvParams {
 };
 
 // grid: R_pad / 16 CTAs of 256 threads.  Dynamic shared memory:
-//   digits [NTOK][ND][C_pad] int8 | partial sums [8 warps][NTOK*ND][16 rows] int32 |
-//   scale [NTOK] | per-warp maxima [8][NTOK]
+//   digits [NTOK][ND][C_pad] int8 | partial sums [warps][NTOK*ND][16 rows] int32 |
+//   scale [NTOK] | per-warp maxima [warps][NTOK]
 template <typename IN_T, int ND, int NTOK, int STAGE>
-__global__ void __launch_bounds__(GEMV_THREADS)
+__global__ void __launch_bounds__(gemv_threads(NTOK))
 ternary_gemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
+    constexpr int GEMV_THREADS = gemv_threads(NTOK), GEMV_WARPS = GEMV_THREADS / 32;
     constexpr bool kInt = sizeof(IN_T) == 1;
     static_assert(!kInt || ND == 1, "int8 activations are their own digit");
     int8_t* dig = reinterpret_cast<int8_t*>(smem);
@@ -193,7 +195,7 @@ ternary_gemv_kernel(const GemvParams p)
         for (int j = 0; j < GEMV_RPL; ++j) u[j] = un[j];
     }
 
-    // ---- add the lanes that took different column groups, then the eight warps ----
+    // ---- add the lanes that took different column groups, then the warps ----
 #pragma unroll
     for (int j = 0; j < GEMV_RPL; ++j)
 #pragma unroll
@@ -251,8 +253,9 @@ ternary_gemv_kernel(const GemvParams p)
 
 size_t gemv_smem_bytes(int nd, int ntok, int C_pad)
 {
-    return (size_t)ntok * nd * C_pad + (size_t)GEMV_WARPS * ntok * nd * GEMV_ROWS * sizeof(int) +
-           (size_t)ntok * sizeof(float) + (size_t)GEMV_WARPS * ntok * sizeof(float);
+    const size_t warps = gemv_threads(ntok) / 32;
+    return (size_t)ntok * nd * C_pad + warps * ntok * nd * GEMV_ROWS * sizeof(int) +
+           (size_t)ntok * sizeof(float) + warps * ntok * sizeof(float);
 }
 
 template <typename IN_T, int ND, int NTOK, int STAGE>
@@ -269,7 +272,7 @@ cudaError_t launch_gemv(const GemvParams& p, int R_pad, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    ternary_gemv_kernel<IN_T, ND, NTOK, STAGE><<<R_pad / GEMV_ROWS, GEMV_THREADS, smem, stream>>>(p);
+    ternary_gemv_kernel<IN_T, ND, NTOK, STAGE><<<R_pad / GEMV_ROWS, gemv_threads(NTOK), smem, stream>>>(p);
     tsvd_count_launch();
     return cudaGetLastError();
 }
