@@ -4,7 +4,7 @@
 // streams its share of the 2-bit codes (the whole of U and V is read once per forward) with as
 // little fixed cost as possible.  Two launches, one per stage (Table S1 rows "V(.)" and "U(.)"):
 // each CTA first turns the stage's input (x, or t = S*(V x)) into the same per-token fixed-point
-// digits as the tensor-core path, in shared memory, then walks 16 rows of the packed matrix:
+// digits as the tensor-core path, in shared memory, then walks 32 rows of the packed matrix:
 // a lane owns four rows of one 64-column group at a time, expands their codes to int8 with two
 // byte permutes per eight entries and adds them to the digits with four-way integer dot
 // products.  (Four rows per lane because every lane reads the same digits: a shared-memory load
@@ -19,7 +19,7 @@ namespace {
 // threads per CTA: with one or two tokens the kernel waits on memory and wants many warps; with
 // four the accumulators need the registers
 __host__ __device__ constexpr int gemv_threads(int ntok) { return ntok <= 2 ? 512 : 256; }
-constexpr int GEMV_RL = 4;          // lanes of a warp along the rows; the other eight take different column groups
+constexpr int GEMV_RL = 8;          // lanes of a warp along the rows; the other four take different column groups
 constexpr int GEMV_RPL = 4;         // rows per lane
 constexpr int GEMV_CS = 32 / GEMV_RL;
 constexpr int GEMV_ROWS = GEMV_RL * GEMV_RPL;   // rows per CTA
@@ -42,8 +42,8 @@ struct GemvParams {
     int z_int;
 };
 
-// grid: R_pad / 16 CTAs of 256 threads.  Dynamic shared memory:
-//   digits [NTOK][ND][C_pad] int8 | partial sums [warps][NTOK*ND][16 rows] int32 |
+// grid: R_pad / 32 CTAs of 256 threads.  Dynamic shared memory:
+//   digits [NTOK][ND][C_pad] int8 | partial sums [warps][NTOK*ND][32 rows] int32 |
 //   scale [NTOK] | per-warp maxima [warps][NTOK]
 template <typename IN_T, int ND, int NTOK, int STAGE>
 __global__ void __launch_bounds__(gemv_threads(NTOK))
@@ -61,8 +61,8 @@ ternary_gemv_kernel(const GemvParams p)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
 
-    // lane = (column group within the pass, row); rows rsel, rsel + 4, .. of the CTA's 16; warp w
-    // takes column groups 8w + csel, + 64, ..  The first codes are requested before anything
+    // lane = (column group within the pass, row); rows rsel, rsel + 8, .. of the CTA's 32; warp w
+    // takes column groups 4w + csel, + 4 * warps, ..  The first codes are requested before anything
     // else, so that their trip from HBM overlaps with the digit conversion below.
     const int rsel = lane & (GEMV_RL - 1), csel = lane / GEMV_RL;
     const int row_base = blockIdx.x * GEMV_ROWS + rsel;
