@@ -76,6 +76,11 @@ ternary_gemv_kernel(const GemvParams p)
     int cg = GEMV_CS * warp + csel;
     uint4 u[GEMV_RPL];
     load_units(cg, u);
+    // The U-stage is launched as a programmatic dependent of the V-stage: its CTAs may start, and
+    // request their first codes, while the V-stage still runs; t is complete and visible only
+    // after this wait.  (Both instructions do nothing in a launch without that relation.)
+    if constexpr (STAGE == STAGE_V) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    else asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- the stage's input as fixed-point digits (every CTA makes its own copy).  A thread takes
     //      chunks of 16 consecutive columns; all loads of a pass are independent, so a pass costs
@@ -272,9 +277,19 @@ cudaError_t launch_gemv(const GemvParams& p, int R_pad, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    ternary_gemv_kernel<IN_T, ND, NTOK, STAGE><<<R_pad / GEMV_ROWS, gemv_threads(NTOK), smem, stream>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(R_pad / GEMV_ROWS));
+    cfg.blockDim = dim3((unsigned)gemv_threads(NTOK));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = STAGE == STAGE_U ? 1 : 0;   // only the U-stage may overlap its predecessor (the V-stage)
+    cudaError_t e = cudaLaunchKernelEx(&cfg, ternary_gemv_kernel<IN_T, ND, NTOK, STAGE>, p);
     tsvd_count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <typename IN_T, int ND, int STAGE>
