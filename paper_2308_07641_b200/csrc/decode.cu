@@ -76,11 +76,13 @@ ternary_gemv_kernel(const GemvParams p)
     int cg = GEMV_CS * warp + csel;
     uint4 u[GEMV_RPL];
     load_units(cg, u);
-    // The U-stage is launched as a programmatic dependent of the V-stage: its CTAs may start, and
-    // request their first codes, while the V-stage still runs; t is complete and visible only
-    // after this wait.  (Both instructions do nothing in a launch without that relation.)
-    if constexpr (STAGE == STAGE_V) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    else asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Both stages are launched as programmatic dependents of the kernel before them in the
+    // stream: their CTAs may start, and request their first codes (which no kernel writes), while
+    // that kernel still runs.  The stage's input (x, or t from the V-stage) is complete and
+    // visible only after this wait, and the stage's output is written after it, so a kernel that
+    // still reads t or y is never overtaken.  The next kernel in the stream may start likewise.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- the stage's input as fixed-point digits (every CTA makes its own copy).  A thread takes
     //      chunks of 16 consecutive columns; all loads of a pass are independent, so a pass costs
@@ -286,7 +288,7 @@ cudaError_t launch_gemv(const GemvParams& p, int R_pad, cudaStream_t stream)
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = STAGE == STAGE_U ? 1 : 0;   // only the U-stage may overlap its predecessor (the V-stage)
+    cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, ternary_gemv_kernel<IN_T, ND, NTOK, STAGE>, p);
     tsvd_count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
