@@ -81,8 +81,8 @@ ternary_gemv_kernel(const GemvParams p)
     // that kernel still runs.  The stage's input (x, or t from the V-stage) is complete and
     // visible only after this wait, and the stage's output is written after it, so a kernel that
     // still reads t or y is never overtaken.  The next kernel in the stream may start likewise.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_wait();
+    pdl_launch_dependents();
 
     // ---- the stage's input as fixed-point digits (every CTA makes its own copy).  A thread takes
     //      chunks of 16 consecutive columns; all loads of a pass are independent, so a pass costs
@@ -279,17 +279,8 @@ cudaError_t launch_gemv(const GemvParams& p, int R_pad, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(R_pad / GEMV_ROWS));
-    cfg.blockDim = dim3((unsigned)gemv_threads(NTOK));
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, ternary_gemv_kernel<IN_T, ND, NTOK, STAGE>, p);
+    PdlLaunch cfg((unsigned)(R_pad / GEMV_ROWS), (unsigned)gemv_threads(NTOK), smem, stream);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg.cfg, ternary_gemv_kernel<IN_T, ND, NTOK, STAGE>, (const GemvParams)p);
     tsvd_count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

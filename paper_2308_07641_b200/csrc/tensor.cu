@@ -82,6 +82,10 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     const int lane = threadIdx.x % TPT;                       // index among the token's threads
     const int b = blockIdx.x * (256 / TPT) + threadIdx.x / TPT;
     if (b >= B_pad) return;                                   // (whole block when TPT == 256)
+    // launched as a programmatic dependent of the kernel before it in the stream: nothing is
+    // read or written before that kernel has completed; the next kernel may be set up meanwhile
+    pdl_wait();
+    pdl_launch_dependents();
     __shared__ float red[8];
     const int jt = b / TOK, b_in = b % TOK;
     const bool live = b < B;
@@ -338,6 +342,11 @@ ternary_mma_kernel(const GemmParams p)
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Launched as a programmatic dependent of the kernel before it in the stream (the one that
+    // wrote the digits): everything up to here, and the copies of the packed codes (which no
+    // kernel writes), may overlap with that kernel; all other warps wait for it to complete.
+    if (warp != 2) pdl_wait();
+    pdl_launch_dependents();
 
     // Waiting for parity 1 on a barrier that has not completed a phase yet returns at once,
     // which is what a consumer-release barrier needs on its first use.
@@ -690,15 +699,18 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
 {
     const int B_pad = (B + TOK - 1) / TOK * TOK;
     const int zero_per_token = (zero_total + B_pad - 1) / B_pad;   // every token slot clears a share
-    if (B_pad * 32 >= 148 * 1024 || KB < 8)   // enough warps to fill the GPU, or short rows
-        digitise_kernel<IN_T, ND, 32, TOK><<<(B_pad + 7) / 8, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits,
-                                                                                D, scale, zero_buf, zero_per_token, zero_total);
+    // one warp per token when that gives enough warps to fill the GPU, or for short rows
+    PdlLaunch cfg((B_pad * 32 >= 148 * 1024 || KB < 8) ? (unsigned)((B_pad + 7) / 8) : (unsigned)B_pad, 256, 0, stream);
+    cudaError_t e;
+    if (B_pad * 32 >= 148 * 1024 || KB < 8)   // (same rule as above)
+        e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
+                               scale, zero_buf, zero_per_token, zero_total);
     else
-        digitise_kernel<IN_T, ND, 256, TOK><<<B_pad, 256, 0, stream>>>(in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                                                                       scale, zero_buf, zero_per_token, zero_total);
+        e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 256, TOK>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
+                               scale, zero_buf, zero_per_token, zero_total);
     tsvd_count_launch();
     if (B_pad_out) *B_pad_out = B_pad;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <int ND, int EPI, int TOK = tokens_per_tile(ND)>
@@ -731,9 +743,10 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int n_tiles = q.row_tiles * q.j_tiles * q.ksplit;
     const int grid = n_tiles < sms ? n_tiles : sms;
-    ternary_mma_kernel<ND, EPI, TOK><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(q);
+    PdlLaunch cfg((unsigned)grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg.cfg, ternary_mma_kernel<ND, EPI, TOK>, (const GemmParams)q);
     tsvd_count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

@@ -92,6 +92,34 @@ struct tsvd_handle_s {
     StageProfiler prof;
 };
 
+// Programmatic dependent launch: a kernel launched with this configuration may be set up, and
+// run up to its pdl_wait(), while the kernel before it in the stream is still running;
+// pdl_wait() returns once that kernel has completed and its writes are visible.  A kernel calls
+// pdl_launch_dependents() to let the kernel after it start likewise.  Without the launch
+// attribute (or with nothing before or after it) both calls do nothing.
+struct PdlLaunch {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    PdlLaunch(unsigned grid, unsigned block, size_t smem, cudaStream_t stream)
+    {
+        cfg = cudaLaunchConfig_t{};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(block);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    PdlLaunch(const PdlLaunch&) = delete;
+    PdlLaunch& operator=(const PdlLaunch&) = delete;
+};
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
 // launch accounting
 void tsvd_count_launch(unsigned n = 1);
 
