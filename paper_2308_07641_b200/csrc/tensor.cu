@@ -517,19 +517,10 @@ ternary_mma_kernel(const GemmParams p)
             const int rt = tc.rt, jt = tc.jt;
             const int row = rt * BLOCK_R + row_in;
             const uint32_t buf = local & 1;
-            // fetch the per-token scales of this warp's groups (8 tokens each; this warp takes
-            // every second group) while the tile is still being contracted: lane i holds the
-            // scale of token 8*g + (i & 7), 0 beyond the batch
+            // this warp takes every second group of 8 tokens
             constexpr int N_GROUPS = TOK / 8;
             constexpr int MY_GROUPS = N_GROUPS / 2;
             static_assert(N_GROUPS % 2 == 0, "two epilogue warps per lane group share the token groups");
-            float scales[MY_GROUPS];
-#pragma unroll
-            for (int k = 0; k < MY_GROUPS; ++k) {
-                const int bb = jt * TOK + (half + 2 * k) * 8 + (lane & 7);
-                scales[k] = 0.f;
-                if constexpr (EPI != EPI_ACC) scales[k] = bb < p.B ? __ldg(p.scale + bb) : 0.f;
-            }
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             const bool row_ok = row < p.R;
@@ -543,9 +534,19 @@ ternary_mma_kernel(const GemmParams p)
 #pragma unroll
                 for (int d = 0; d < ND; ++d) tmem_ld8(t_lane + (uint32_t)(d * TOK + g * 8), acc[d]);
                 const int b0 = jt * TOK + g * 8;
-                const float my_scale = scales[k];
+                // the group's eight per-token scales: every lane reads the same 32 bytes (the
+                // array is padded to whole tiles), while the tensor-memory loads are in flight
+                float sc[8];
+                if constexpr (EPI != EPI_ACC) {
+                    const float4 s0 = __ldg(reinterpret_cast<const float4*>(p.scale + b0));
+                    const float4 s1 = __ldg(reinterpret_cast<const float4*>(p.scale + b0 + 4));
+                    sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w;
+                    sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
+                }
                 tmem_ld_wait();
                 const int n_live = min(8, p.B - b0);   // uniform across the warp
+                // whole group inside the batch and every row of the warp inside the matrix: no guards
+                const bool full = n_live == 8 && __all_sync(0xffffffffu, row_ok);
                 if constexpr (EPI == EPI_ACC) {
                     // part of a split contraction: add the raw digit sums to the global accumulators
                     // (integer adds commute exactly, so the result does not depend on arrival order)
@@ -575,13 +576,18 @@ ternary_mma_kernel(const GemmParams p)
                         if constexpr (ND == 4) hi += (int)acc[3][i] << 8;
                         f = fmaf((float)hi, 65536.f, (float)lo);
                     }
-                    val[i] = f * __shfl_sync(0xffffffffu, my_scale, i);   // a power of two: exact
+                    val[i] = f * sc[i];   // a power of two: exact
                 }
                 if constexpr (EPI == EPI_V) {
                     float* tp = p.t + (size_t)b0 * p.t_ld + row;
+                    if (n_live == 8) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        if (i < n_live) tp[(size_t)i * p.t_ld] = s_row * val[i];   // the K multiplications (Table S1)
+                        for (int i = 0; i < 8; ++i) tp[(size_t)i * p.t_ld] = s_row * val[i];   // the K multiplications (Table S1)
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (i < n_live) tp[(size_t)i * p.t_ld] = s_row * val[i];
+                    }
                     if (p.z_out && row_ok) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
@@ -594,18 +600,23 @@ ternary_mma_kernel(const GemmParams p)
                     }
                 } else if constexpr (EPI == EPI_U_F32) {
                     float* yp = reinterpret_cast<float*>(p.y) + (size_t)b0 * p.ldy + row;
+                    if (full) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        if (row_ok && i < n_live) yp[(size_t)i * p.ldy] = val[i];
+                        for (int i = 0; i < 8; ++i) yp[(size_t)i * p.ldy] = val[i];
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (row_ok && i < n_live) yp[(size_t)i * p.ldy] = val[i];
+                    }
                 } else {
-                    uint16_t* yp = reinterpret_cast<uint16_t*>(p.y) + (size_t)b0 * p.ldy + row;
+                    __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + (size_t)b0 * p.ldy + row;
+                    if (full) {
 #pragma unroll
-                    for (int i = 0; i < 8; i += 2) {
-                        // one conversion instruction rounds two values (to nearest even)
-                        const __nv_bfloat162 pr = __floats2bfloat162_rn(val[i], val[i + 1]);
-                        const uint32_t u = *reinterpret_cast<const uint32_t*>(&pr);
-                        if (row_ok && i < n_live) yp[(size_t)i * p.ldy] = (uint16_t)(u & 0xFFFFu);
-                        if (row_ok && i + 1 < n_live) yp[(size_t)(i + 1) * p.ldy] = (uint16_t)(u >> 16);
+                        for (int i = 0; i < 8; ++i) yp[(size_t)i * p.ldy] = __float2bfloat16_rn(val[i]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (row_ok && i < n_live) yp[(size_t)i * p.ldy] = __float2bfloat16_rn(val[i]);
                     }
                 }
                 }   // EPI != EPI_ACC
