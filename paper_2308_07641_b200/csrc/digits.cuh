@@ -19,18 +19,24 @@ template <> __device__ __forceinline__ float to_float<int8_t>(int8_t v) { return
 // and digits in [-128,127], digit d is byte d of q + 0x80 + 0x8000 + ... (d terms): adding half
 // the radix at every lower position turns the floor of the arithmetic shift into rounding.
 // The top digit is what is left; it fits because |q| <= 2^(8ND-2).
+// One addition serves all digits: q + (0x80 + 0x8000 + ..., ND-1 terms) has, below the top
+// digit, 0x80 too much in byte d, which an exclusive-or takes out again.  The bytes of four
+// values are then transposed into the four digit words with eight byte permutes.
 template <int ND>
 __device__ __forceinline__ void digits_of_16(const int (&q)[16], uint32_t (&dig)[ND][4])
 {
+    constexpr uint32_t off = ND == 1 ? 0u : ND == 2 ? 0x80u : ND == 3 ? 0x8080u : 0x808080u;
 #pragma unroll
-    for (int d = 0; d < ND; ++d) {
-        const uint32_t off = d == 0 ? 0u : d == 1 ? 0x80u : d == 2 ? 0x8080u : 0x808080u;
-        const uint32_t sel = (uint32_t)d | ((uint32_t)(4 + d) << 4);   // byte d of a, byte d of b
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const uint32_t lo = __byte_perm((uint32_t)q[4 * g] + off, (uint32_t)q[4 * g + 1] + off, sel);
-            const uint32_t hi = __byte_perm((uint32_t)q[4 * g + 2] + off, (uint32_t)q[4 * g + 3] + off, sel);
-            dig[d][g] = __byte_perm(lo, hi, 0x5410);
+    for (int g = 0; g < 4; ++g) {
+        const uint32_t a = (uint32_t)q[4 * g] + off, b = (uint32_t)q[4 * g + 1] + off;
+        const uint32_t c = (uint32_t)q[4 * g + 2] + off, e = (uint32_t)q[4 * g + 3] + off;
+        const uint32_t ab01 = __byte_perm(a, b, 0x5140), cd01 = __byte_perm(c, e, 0x5140);   // bytes 0,1 of each pair
+        dig[0][g] = __byte_perm(ab01, cd01, 0x5410) ^ (ND > 1 ? 0x80808080u : 0u);
+        if constexpr (ND > 1) dig[1][g] = __byte_perm(ab01, cd01, 0x7632) ^ (ND > 2 ? 0x80808080u : 0u);
+        if constexpr (ND > 2) {
+            const uint32_t ab23 = __byte_perm(a, b, 0x7362), cd23 = __byte_perm(c, e, 0x7362);   // bytes 2,3
+            dig[2][g] = __byte_perm(ab23, cd23, 0x5410) ^ (ND > 3 ? 0x80808080u : 0u);
+            if constexpr (ND > 3) dig[3][g] = __byte_perm(ab23, cd23, 0x7632);
         }
     }
 }
