@@ -380,7 +380,16 @@ def main():
     dom = int(np.argmax(stage_ms))
     dom_ms = stage_ms[dom] / max(1, stage_n[dom])
     pad = lambda v: (v + 127) // 128 * 128
-    if dom in (1, 3):
+    if dom in (1, 3) and plan["path"] == "decode":
+        # a decode stage streams its packed matrix once: 2 bits per entry of the padded matrix
+        rows, contr = ((pad(spec.K), pad(spec.N)) if dom == 1 else (pad(spec.M), pad(spec.K)))
+        byts = rows * contr / 4.0
+        achieved = byts / (dom_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved,
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                    "traffic": recorded_traffic(spec.name, binding.STAGE_NAMES[dom]),
+                    "peak_source": f"{peaks_src} (of measured)", "bytes_per_launch": byts}
+    elif dom in (1, 3):
         rows, contr = ((pad(spec.K), pad(spec.N)) if dom == 1 else (pad(spec.M), pad(spec.K)))
         digits = max(1, plan["digits_x"] if dom == 1 else plan["digits_t"])
         # executed dense operations of that launch: 2 * rows * contraction * tokens * digits
@@ -419,7 +428,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": "int32" if plan["path"] == "tensor" else {"f32": "f32", "bf16": "f32", "i8": "int32"}[spec.x_dtype],
+            "dtype": "int32" if plan["path"] in ("tensor", "decode") else {"f32": "f32", "bf16": "f32", "i8": "int32"}[spec.x_dtype],
             "data": "synthetic",
             "config": workload_config(spec, l2_note),
             "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks,
