@@ -44,7 +44,9 @@ static_assert(A_COL0 + NA * A_SLOT_COLS <= TMEM_COLS, "tensor memory budget");
 constexpr int EXP_GROUPS = 3;     // groups of four expander warps; group g takes steps it % EXP_GROUPS == g
 constexpr int EXP_WARP0 = 4;
 constexpr int EPI_WARP0 = EXP_WARP0 + 4 * EXP_GROUPS;
-constexpr int GEMM_THREADS = 32 * (EPI_WARP0 + 8);
+constexpr int EPI_WARPS = 4;      // epilogue warps: one per 32 tensor-memory lanes, times EPI_WARPS / 4 token shares
+constexpr int EPI_SHARES = EPI_WARPS / 4;
+constexpr int GEMM_THREADS = 32 * (EPI_WARP0 + EPI_WARPS);
 
 // tokens per tile for nd digits: the MMA N extent is nd * tokens = 192 for every nd
 __host__ __device__ constexpr int tokens_per_tile(int nd) { return 192 / nd; }
@@ -326,9 +328,9 @@ ternary_mma_kernel(const GemmParams p)
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&accfull_bar[i], 1);
-            mbar_init(&accempty_bar[i], 8);  // one arrival per epilogue warp
+            mbar_init(&accempty_bar[i], EPI_WARPS);  // one arrival per epilogue warp
         }
-        mbar_init(&tail_bar[0], 8);
+        mbar_init(&tail_bar[0], EPI_WARPS);
         mbar_init(&tail_bar[1], 1);
         abort_flag[0] = 0;
         abort_flag[1] = p.wait_limit > 0 ? p.wait_limit : kWaitLimitDefault;
@@ -519,8 +521,8 @@ ternary_mma_kernel(const GemmParams p)
             const uint32_t buf = local & 1;
             // this warp takes every second group of 8 tokens
             constexpr int N_GROUPS = TOK / 8;
-            constexpr int MY_GROUPS = N_GROUPS / 2;
-            static_assert(N_GROUPS % 2 == 0, "two epilogue warps per lane group share the token groups");
+            constexpr int MY_GROUPS = N_GROUPS / EPI_SHARES;
+            static_assert(N_GROUPS % EPI_SHARES == 0, "the epilogue warps of a lane group share the token groups evenly");
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             const bool row_ok = row < p.R;
@@ -529,7 +531,7 @@ ternary_mma_kernel(const GemmParams p)
             const uint32_t t_lane = tmem_base + buf * (uint32_t)ACC_COLS + ((uint32_t)(lane_grp * 32) << 16);
 #pragma unroll
             for (int k = 0; k < MY_GROUPS; ++k) {
-                const int g = half + 2 * k;
+                const int g = half + EPI_SHARES * k;
                 uint32_t acc[ND][8];
 #pragma unroll
                 for (int d = 0; d < ND; ++d) tmem_ld8(t_lane + (uint32_t)(d * TOK + g * 8), acc[d]);
@@ -642,9 +644,10 @@ ternary_mma_kernel(const GemmParams p)
                 }
                 if (!mbar_wait(&tail_bar[1], local & 1, abort_flag)) break;
                 if (*tail_last) {
-                    // this warp: rows 32*(warp%4).. and the 8 tokens of group `half` (TOK == 16)
-                    static_assert(TOK == 16, "the tail assumes two token groups");
-                    const int b0 = jt * TOK + half * 8;
+                  // this warp: rows 32*(warp%4).. and its share of the tile's groups of 8 tokens
+#pragma unroll 1
+                  for (int tg = half; tg < TOK / 8; tg += EPI_SHARES) {
+                    const int b0 = jt * TOK + tg * 8;
                     const bool row_ok = row < p.R;
                     const float s_row = p.tail == TAIL_T ? p.S[row] : 0.f;
                     // all loads first (they are independent and come from L2), then the arithmetic
@@ -688,6 +691,7 @@ ternary_mma_kernel(const GemmParams p)
                                 reinterpret_cast<float*>(p.y)[(size_t)b * p.ldy + row] = val;
                         }
                     }
+                  }
                 }
             }
         }
