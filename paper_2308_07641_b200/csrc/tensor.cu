@@ -40,13 +40,16 @@ constexpr int A_BLOCK_COLS = BLOCK_C / 4;
 constexpr int A_SLOT_COLS = STEP_BLOCKS * A_BLOCK_COLS;
 static_assert(A_COL0 + NA * A_SLOT_COLS <= TMEM_COLS, "tensor memory budget");
 // warp 0: digit-tile copies, 1: MMA issue, 2: packed-code copies, 3: idle,
-// 4..15: expand (three groups of four that take the steps in turn), 16..23: epilogue
+// 4..15: expand (three groups of four that take the steps in turn), 16..: epilogue (four or eight)
 constexpr int EXP_GROUPS = 3;     // groups of four expander warps; group g takes steps it % EXP_GROUPS == g
 constexpr int EXP_WARP0 = 4;
 constexpr int EPI_WARP0 = EXP_WARP0 + 4 * EXP_GROUPS;
-constexpr int EPI_WARPS = 4;      // epilogue warps: one per 32 tensor-memory lanes, times EPI_WARPS / 4 token shares
-constexpr int EPI_SHARES = EPI_WARPS / 4;
-constexpr int GEMM_THREADS = 32 * (EPI_WARP0 + EPI_WARPS);
+// Epilogue warps: one per 32 tensor-memory lanes, times EPIW / 4 shares of a tile's tokens.  Eight
+// keep up with tiles of a few contraction blocks; four are enough for long contractions, and
+// leave the issue slots to the expanders while a tile is drained.
+constexpr int EPI_WARPS_MAX = 8;
+constexpr int EPI_FEWER_FROM_KB = 16;   // contraction blocks per tile from which four epilogue warps are used
+__host__ __device__ constexpr int gemm_threads(int epiw) { return 32 * (EPI_WARP0 + epiw); }
 
 // tokens per tile for nd digits: the MMA N extent is nd * tokens = 192 for every nd
 __host__ __device__ constexpr int tokens_per_tile(int nd) { return 192 / nd; }
@@ -258,10 +261,11 @@ __device__ __forceinline__ void tile_kb_range(const GemmParams& p, int tile, int
     }
 }
 
-template <int ND, int EPI, int TOK>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+template <int ND, int EPI, int TOK, int EPI_WARPS>
+__global__ void __launch_bounds__(gemm_threads(EPI_WARPS), 1)
 ternary_mma_kernel(const GemmParams p)
 {
+    constexpr int EPI_SHARES = EPI_WARPS / 4;
     constexpr int NT = ND * TOK;
     static_assert(NT % 16 == 0 && NT <= NT_MAX && TOK % 16 == 0, "tile shape");
     constexpr uint32_t B_TILE_BYTES = NT * BLOCK_C;
@@ -508,8 +512,8 @@ ternary_mma_kernel(const GemmParams p)
             }
         }
     } else if (warp >= EPI_WARP0) {
-        // ---- epilogue: eight warps; warp w reads tensor-memory lanes 32*(w%4) .. +31 and takes
-        //      every second group of 8 tokens ----
+        // ---- epilogue: warp w reads tensor-memory lanes 32*(w%4) .. +31 and takes its share
+        //      (all, or every second) of the tile's groups of 8 tokens ----
         const int lane_grp = warp & 3;
         const int half = (warp - EPI_WARP0) >> 2;
         const int row_in = lane_grp * 32 + lane;
@@ -519,7 +523,7 @@ ternary_mma_kernel(const GemmParams p)
             const int rt = tc.rt, jt = tc.jt;
             const int row = rt * BLOCK_R + row_in;
             const uint32_t buf = local & 1;
-            // this warp takes every second group of 8 tokens
+            // this warp takes its share of the groups of 8 tokens
             constexpr int N_GROUPS = TOK / 8;
             constexpr int MY_GROUPS = N_GROUPS / EPI_SHARES;
             static_assert(N_GROUPS % EPI_SHARES == 0, "the epilogue warps of a lane group share the token groups evenly");
@@ -728,15 +732,15 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-template <int ND, int EPI, int TOK = tokens_per_tile(ND)>
-cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
+template <int ND, int EPI, int TOK, int EPIW>
+cudaError_t launch_gemm_w(const GemmParams& p, int row_tiles, cudaStream_t stream)
 {
     static bool attr_set[64] = {};   // per instantiation and device
     int dev = 0;
     cudaError_t e0 = cudaGetDevice(&dev);
     if (e0 != cudaSuccess) return e0;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(ternary_mma_kernel<ND, EPI, TOK>,
+        cudaError_t e = cudaFuncSetAttribute(ternary_mma_kernel<ND, EPI, TOK, EPIW>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -758,10 +762,20 @@ cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int n_tiles = q.row_tiles * q.j_tiles * q.ksplit;
     const int grid = n_tiles < sms ? n_tiles : sms;
-    PdlLaunch cfg((unsigned)grid, GEMM_THREADS, GEMM_SMEM_BYTES, stream);
-    const cudaError_t e = cudaLaunchKernelEx(&cfg.cfg, ternary_mma_kernel<ND, EPI, TOK>, (const GemmParams)q);
+    PdlLaunch cfg((unsigned)grid, (unsigned)gemm_threads(EPIW), GEMM_SMEM_BYTES, stream);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg.cfg, ternary_mma_kernel<ND, EPI, TOK, EPIW>, (const GemmParams)q);
     tsvd_count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+template <int ND, int EPI, int TOK = tokens_per_tile(ND)>
+cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
+{
+    // blocks a tile contracts (a split contraction: its longest part)
+    const int ks = p.ksplit < 1 ? 1 : p.ksplit;
+    const int kb_tile = (p.KB + ks - 1) / ks;
+    if (kb_tile >= EPI_FEWER_FROM_KB) return launch_gemm_w<ND, EPI, TOK, 4>(p, row_tiles, stream);
+    return launch_gemm_w<ND, EPI, TOK, EPI_WARPS_MAX>(p, row_tiles, stream);
 }
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
