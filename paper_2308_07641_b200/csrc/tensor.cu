@@ -45,10 +45,11 @@ constexpr int EXP_GROUPS = 3;     // groups of four expander warps; group g take
 constexpr int EXP_WARP0 = 4;
 constexpr int EPI_WARP0 = EXP_WARP0 + 4 * EXP_GROUPS;
 // Epilogue warps: one per 32 tensor-memory lanes, times EPIW / 4 shares of a tile's tokens.  Eight
-// keep up with tiles of a few contraction blocks; four are enough for long contractions, and
-// leave the issue slots to the expanders while a tile is drained.
+// keep up with tiles of a few contraction blocks; four are enough when a tile's MMAs (384 clocks
+// per block) outlast the drain of its TOK tokens per row (about 100 clocks each with four warps),
+// and they leave more issue slots to the expanders meanwhile.
 constexpr int EPI_WARPS_MAX = 8;
-constexpr int EPI_FEWER_FROM_KB = 16;   // contraction blocks per tile from which four epilogue warps are used
+__host__ __device__ constexpr bool four_epilogue_warps(int kb_tile, int tok) { return 3 * kb_tile >= tok; }
 __host__ __device__ constexpr int gemm_threads(int epiw) { return 32 * (EPI_WARP0 + epiw); }
 
 // tokens per tile for nd digits: the MMA N extent is nd * tokens = 192 for every nd
@@ -771,10 +772,9 @@ cudaError_t launch_gemm_w(const GemmParams& p, int row_tiles, cudaStream_t strea
 template <int ND, int EPI, int TOK = tokens_per_tile(ND)>
 cudaError_t launch_gemm(const GemmParams& p, int row_tiles, cudaStream_t stream)
 {
-    // blocks a tile contracts (a split contraction: its longest part)
-    const int ks = p.ksplit < 1 ? 1 : p.ksplit;
-    const int kb_tile = (p.KB + ks - 1) / ks;
-    if (kb_tile >= EPI_FEWER_FROM_KB) return launch_gemm_w<ND, EPI, TOK, 4>(p, row_tiles, stream);
+    if constexpr (EPI != EPI_ACC) {
+        if (four_epilogue_warps(p.KB, TOK)) return launch_gemm_w<ND, EPI, TOK, 4>(p, row_tiles, stream);
+    }
     return launch_gemm_w<ND, EPI, TOK, EPI_WARPS_MAX>(p, row_tiles, stream);
 }
 
