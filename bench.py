@@ -61,7 +61,7 @@ def rank_spec(spec, rank):
 def kernel_source_sha1():
     import hashlib
     h = hashlib.sha1()
-    for name in ("tensor.cu", "sm100_ptx.cuh", "tsvd_internal.cuh"):
+    for name in ("tensor.cu", "decode.cu", "digits.cuh", "sm100_ptx.cuh", "tsvd_internal.cuh"):
         with open(os.path.join(ROOT, "paper_2308_07641_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
