@@ -38,6 +38,18 @@ def test_library_exports_every_declared_symbol(binding):
     assert declared == set(binding.EXPORTS)
 
 
+def test_constants_match_the_header(binding):
+    import re
+    hdr = open(os.path.join(ROOT, "include", "tsvd.h")).read()
+    def define(name):
+        return int(re.search(r"#define\s+" + name + r"\s+(0x[0-9a-fA-F]+|\d+)", hdr).group(1), 0)
+    assert define("TSVD_DECODE_MAX_B") == binding.TSVD_DECODE_MAX_B
+    assert define("TSVD_FLAG_PATH_DECODE") == binding.TSVD_FLAG_PATH_DECODE
+    assert define("TSVD_FLAG_PATH_SIMPLE") == binding.TSVD_FLAG_PATH_SIMPLE
+    assert define("TSVD_FLAG_PATH_TENSOR") == binding.TSVD_FLAG_PATH_TENSOR
+    assert define("TSVD_FLAG_OUT_F32") == binding.TSVD_FLAG_OUT_F32
+
+
 def test_strerror_covers_all_codes(binding):
     seen = {binding.tsvd_strerror(i) for i in range(0, 10)}
     assert len(seen) == 10 and "unknown status" not in seen

@@ -159,6 +159,70 @@ def test_decode_and_tensor_paths_agree_bit_for_bit():
         layer.close()
 
 
+def test_decode_strided_inputs_and_host_entry_point():
+    """Row strides larger than the row, fp32 output of bf16 activations, and the host-buffer call."""
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear, binding
+    spec = gen.scaled(C["cfg3_b4"], name="dec_strided", M=260, N=333, K=200, B=3, seed=41)
+    U, V, S = gen.make_weights(spec)
+    x_np = gen.make_x(spec)
+    ref = oracle.forward(U, S, V, _util.oracle_x(x_np, "bf16"))
+    layer = TSVDLinear(U, S, V)
+    try:
+        x = _util.torch_x(x_np, "bf16")
+        xs = torch.zeros((spec.B, spec.N + 7), dtype=torch.bfloat16, device="cuda")
+        xs[:, :spec.N] = x
+        out = torch.full((spec.B, spec.M + 5), 7.0, dtype=torch.float32, device="cuda")
+        layer.forward(xs[:, :spec.N], out=out[:, :spec.M], flags=0x20 | 0x1)
+        torch.cuda.synchronize()
+        assert float(out[:, spec.M:].min()) == 7.0 and float(out[:, spec.M:].max()) == 7.0
+        _util.check_outputs(out[:, :spec.M].double().cpu().numpy(), None, ref, "bf16", False, "strided decode")
+        # host buffers: the library copies in and out itself (default path for 3 tokens = decode)
+        y_host = np.zeros((spec.B, spec.M), np.float32)
+        binding.tsvd_forward_host(layer.handle, x_np.ctypes.data, y_host.ctypes.data, spec.B, binding.TSVD_BF16, 0x1)
+        _util.check_outputs(y_host.astype(np.float64), None, ref, "bf16", False, "host decode")
+    finally:
+        layer.close()
+
+
+def test_kernels_launched_early_still_see_inputs_written_just_before():
+    """The kernels may start while the kernel before them in the stream still runs; they must not
+    read their input before it has completed.  x is doubled in place between two forwards: every
+    digit stays the same and only the per-token exponent moves, so y doubles exactly."""
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear
+    for B in (2, 40, 200):          # decode, small-batch and large-batch kernels
+        spec = gen.scaled(C["cfg2"], name=f"pdl_B{B}", M=600, N=1500, K=520, B=B, seed=61)
+        U, V, S = gen.make_weights(spec)
+        x = _util.torch_x(gen.make_x(spec), "bf16").float()
+        layer = TSVDLinear(U, S, V)
+        try:
+            y1 = layer.forward(x).clone()
+            for _ in range(5):
+                x.mul_(2.0)
+                y = layer.forward(x)
+                y1.mul_(2.0)
+                assert torch.equal(y, y1)
+            torch.cuda.synchronize()
+        finally:
+            layer.close()
+
+
+def test_decode_falls_back_when_the_digits_do_not_fit_shared_memory():
+    from paper_2308_07641_b200 import binding
+    N = 13000                       # 4 tokens x 4 digits x 13056 columns > 200 KiB
+    U = np.zeros((8, 8), np.int8); V = np.zeros((8, N), np.int8); S = np.ones(8, np.float32)
+    h = binding.tsvd_pack(U, S, V)
+    try:
+        assert binding.tsvd_plan(h, 4, binding.TSVD_F32)["path"] == "tensor"
+        assert binding.tsvd_plan(h, 1, binding.TSVD_F32)["path"] == "decode"
+        with pytest.raises(binding.TSVDError) as ei:
+            binding.tsvd_plan(h, 4, binding.TSVD_F32, 0x20)
+        assert ei.value.status == binding.TSVD_E_TOOBIG
+    finally:
+        binding.tsvd_destroy(h)
+
+
 def test_out_f32_flag_and_strides():
     """bf16 activations with fp32 output, and leading dimensions larger than the row length."""
     import torch
