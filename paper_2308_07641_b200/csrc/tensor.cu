@@ -303,7 +303,7 @@ ternary_mma_kernel(const GemmParams p)
     uint64_t* done_bar = ready_bar + NB;             // [NB][STEP_BLOCKS] the MMAs of block j of the step have completed
     uint64_t* accfull_bar = done_bar + NB * STEP_BLOCKS;   // [2] all MMAs of a tile have completed
     uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
-    uint64_t* tail_bar = accempty_bar + 2;           // [2] split contraction: epilogue warps meet, verdict is in
+    uint64_t* tail_bar = accempty_bar + 2;           // [2] split contraction: epilogue warps meet, outcome is in
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [2]: flag, wait limit
     volatile int* tail_last = abort_flag + 2;        // whether this CTA finished its output tile last
