@@ -40,8 +40,8 @@ constexpr int A_BLOCK_COLS = BLOCK_C / 4;
 constexpr int A_SLOT_COLS = STEP_BLOCKS * A_BLOCK_COLS;
 static_assert(A_COL0 + NA * A_SLOT_COLS <= TMEM_COLS, "tensor memory budget");
 // warp 0: digit-tile copies, 1: MMA issue, 2: packed-code copies, 3: idle,
-// 4..15: expand (three groups of four that take the steps in turn), 16..: epilogue (four or eight)
-constexpr int EXP_GROUPS = 3;     // groups of four expander warps; group g takes steps it % EXP_GROUPS == g
+// 4..11: expand (two groups of four that take alternate steps), 12..: epilogue (four or eight)
+constexpr int EXP_GROUPS = 2;     // groups of four expander warps; group g takes steps it % EXP_GROUPS == g
 constexpr int EXP_WARP0 = 4;
 constexpr int EPI_WARP0 = EXP_WARP0 + 4 * EXP_GROUPS;
 // Epilogue warps: one per 32 tensor-memory lanes, times EPIW / 4 shares of a tile's tokens.  Eight
