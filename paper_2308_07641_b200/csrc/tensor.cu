@@ -479,30 +479,35 @@ ternary_mma_kernel(const GemmParams p)
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_SLOT_BYTES);
                 const uint32_t a_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS);
+                // expand the whole step into registers first, so that only the stores are left to do
+                // once the slot is free
+                uint32_t o[STEP_BLOCKS][32];   // per block: the row's 128 int8 values, four per 32-bit column
+#pragma unroll
+                for (int j = 0; j < STEP_BLOCKS; ++j) {
+                    if (j < nblk) {
+#pragma unroll
+                        for (int g = 0; g < 2; ++g) {
+                            const uint4 u = packed[j * 256 + g * 128 + r];
+                            tsvd_expand16(u.x, *reinterpret_cast<uint32_t(*)[4]>(&o[j][g * 16 + 0]));
+                            tsvd_expand16(u.y, *reinterpret_cast<uint32_t(*)[4]>(&o[j][g * 16 + 4]));
+                            tsvd_expand16(u.z, *reinterpret_cast<uint32_t(*)[4]>(&o[j][g * 16 + 8]));
+                            tsvd_expand16(u.w, *reinterpret_cast<uint32_t(*)[4]>(&o[j][g * 16 + 12]));
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // all codes of the step are in registers
                 bool ok = true;
 #pragma unroll
                 for (int j = 0; j < STEP_BLOCKS; ++j) {
                     if (j < nblk && ok) {
-                        uint32_t o[32];   // the row's 128 int8 values of block j, four per 32-bit column
-#pragma unroll
-                        for (int g = 0; g < 2; ++g) {
-                            const uint4 u = packed[j * 256 + g * 128 + r];
-                            tsvd_expand16(u.x, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 0]));
-                            tsvd_expand16(u.y, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 4]));
-                            tsvd_expand16(u.z, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 8]));
-                            tsvd_expand16(u.w, *reinterpret_cast<uint32_t(*)[4]>(&o[g * 16 + 12]));
-                        }
-                        if (j == nblk - 1) {
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(&pempty_bar[sp]);   // all codes of the step are in registers
-                        }
                         if (it >= (uint32_t)NA) {   // this part of the A slot is free once block j of step it - NA is done
                             uint32_t sd = sb + nb - NA, phd = phb ^ 1;   // its slot, NA back (nb >= NA), and phase
                             if (sd >= nb) { sd -= nb; phd = phb; }
                             ok = mbar_wait(&done_bar[sd * STEP_BLOCKS + j], phd, abort_flag);
                             tc_fence_after_sync();
                         }
-                        if (ok) tmem_st32(a_addr + (uint32_t)(j * A_BLOCK_COLS), o);
+                        if (ok) tmem_st32(a_addr + (uint32_t)(j * A_BLOCK_COLS), o[j]);
                     }
                 }
                 if (!ok) { alive = false; break; }
