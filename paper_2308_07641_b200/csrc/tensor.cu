@@ -15,7 +15,6 @@
 // Batches above 64 tokens use 192-column tiles, one CTA per tile; smaller batches use 16-token
 // tiles with the contraction split across CTAs (integer atomics, the last part of a tile
 // finishes the stage), so that the packed codes are streamed by about one CTA per SM.
-#include <cstdlib>
 #include "digits.cuh"
 #include "sm100_ptx.cuh"
 #include "tsvd_internal.cuh"
@@ -221,7 +220,6 @@ struct GemmParams {
     int y_bf16;
     int nb;               // depth of the digit-tile ring in steps: NB, or (resident) a whole number of panels
     int resident;         // the digit tiles of a token tile stay in shared memory across row tiles
-    int resident_a;       // the expanded operand of a row tile stays in tensor memory across token tiles
     int wait_limit;       // bound of every barrier wait in units of 2^20 clocks (0: default, ~2 s)
     int test_stall;       // test hook: the digit tiles are never copied, so the waits must give up
 };
@@ -241,13 +239,8 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile)
         c.kb0 = ks * p.KB / p.ksplit;          // ksplit <= 16 and KB < 2^20: no overflow
         c.kb1 = (ks + 1) * p.KB / p.ksplit;
     }
-    if (p.resident_a) {   // token tile fastest: consecutive tiles share the row tile
-        c.rt = rest / p.j_tiles;
-        c.jt = rest % p.j_tiles;
-    } else {
-        c.rt = rest % p.row_tiles;
-        c.jt = rest / p.row_tiles;
-    }
+    c.rt = rest % p.row_tiles;
+    c.jt = rest / p.row_tiles;
     return c;
 }
 // Each CTA takes a run of consecutive tiles (row tile fastest), so that its tiles share their
@@ -324,7 +317,7 @@ ternary_mma_kernel(const GemmParams p)
     // and those stay hot in L2.
     int tile_first = (int)blockIdx.x, tile_step = (int)gridDim.x;
     int tile_count = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    if (p.resident || p.resident_a) {
+    if (p.resident) {
         int t0, t1;
         tile_range(n_tiles, t0, t1);
         tile_first = t0;
@@ -391,8 +384,6 @@ ternary_mma_kernel(const GemmParams p)
                 // the same token tile the data are there already: only the barrier is armed.
                 bool copy = true;
                 if (is_b && p.resident) copy = L < panels || (tile - panels) / p.row_tiles != tc.jt;
-                // resident expanded operand: a tile with the row tile of the one before needs no codes
-                if (!is_b && p.resident_a && L > 0 && tile % p.j_tiles != 0) continue;
                 for (int kb = tc.kb0; kb < tc.kb1; kb += STEP_BLOCKS, ++issued) {
                     const uint32_t bytes = (uint32_t)min(STEP_BLOCKS, tc.kb1 - kb) * blk_bytes;
                     if (!mbar_wait(&empty[slot * empty_stride], phase ^ 1, abort_flag)) { alive = false; break; }
@@ -478,32 +469,15 @@ ternary_mma_kernel(const GemmParams p)
         const int r = (threadIdx.x - EXP_WARP0 * 32) & 127;   // 0..127
         const uint32_t group = (uint32_t)(warp - EXP_WARP0) >> 2;
         uint32_t it = 0, sb = 0, phb = 0;   // step counter; its slot and phase in the digit-tile ring
-        uint32_t pit = 0;                   // steps whose codes were copied (position in the code ring)
         bool alive = true;
         for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
             int kb0, kb1;
             tile_kb_range(p, tile, kb0, kb1);
-            // Resident expanded operand (a tile has exactly NA steps, so step s of every tile uses
-            // slot s): a tile with the row tile of the one before finds its operand in place.
-            const bool reuse_a = p.resident_a && L > 0 && tile % p.j_tiles != 0;
             for (int kb = kb0; kb < kb1; kb += STEP_BLOCKS, ++it, sb = (sb + 1 == nb ? 0u : sb + 1), phb ^= (sb == 0)) {
-                if (reuse_a) {
-                    if (it % EXP_GROUPS == group) {
-                        // only the barrier is armed, after the wait a store would need, so that the
-                        // arrival falls into this step's phase of the barrier
-                        uint32_t sd = sb + nb - NA, phd = phb ^ 1;
-                        if (sd >= nb) { sd -= nb; phd = phb; }
-                        if (!mbar_wait(&done_bar[sd * STEP_BLOCKS + STEP_BLOCKS - 1], phd, abort_flag)) { alive = false; break; }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&ready_bar[sb]);
-                    }
-                    continue;
-                }
-                const uint32_t my_p = pit++;
                 if (it % EXP_GROUPS != group) continue;
                 const int nblk = min(STEP_BLOCKS, kb1 - kb);
-                const int sp = my_p % NP, sa = it % NA;
-                if (!mbar_wait(&pfull_bar[sp], (my_p / NP) & 1, abort_flag)) { alive = false; break; }
+                const int sp = it % NP, sa = it % NA;
+                if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_SLOT_BYTES);
                 const uint32_t a_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS);
                 // expand the whole step into registers first, so that only the stores are left to do
@@ -785,16 +759,10 @@ cudaError_t launch_gemm_w(const GemmParams& p, int row_tiles, cudaStream_t strea
     // memory while the CTA walks the row tiles: the ring then holds whole panels (a tile's steps).
     q.nb = NB;
     q.resident = 0;
-    q.resident_a = 0;
     const int steps = (q.KB + STEP_BLOCKS - 1) / STEP_BLOCKS;
     if (q.ksplit == 1 && steps <= NB) {
         q.nb = steps * (NB / steps);
         q.resident = 1;
-    }
-    if (q.ksplit == 1 && steps == NA && EPI != EPI_ACC && getenv("TSVD_RESIDENT_A")) {
-        q.nb = NB;
-        q.resident = 0;
-        q.resident_a = 1;
     }
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
