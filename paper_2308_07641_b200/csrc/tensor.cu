@@ -27,11 +27,11 @@ constexpr int BLOCK_R = 128;   // ternary rows per CTA tile = MMA M
 constexpr int BLOCK_C = 128;   // contraction elements per block (one 128-byte swizzle row)
 constexpr int STEP_BLOCKS = 2; // blocks per pipeline step: one set of barrier handshakes covers this many
 constexpr int UMMA_K = 32;     // contraction elements per kind::i8 instruction
-constexpr int NT_MAX = 160;    // largest MMA N extent: digit rows per tile
+constexpr int NT_MAX = 192;    // MMA N extent: digit rows per tile
 constexpr int NP = 4;          // ring depth (steps) of the packed codes (shared memory)
 constexpr int NB = 4;          // ring depth (steps) of the digit tiles (shared memory) and of the per-step barriers
-constexpr int NA = 3;          // ring depth (steps) of the expanded ternary operand (tensor memory)
-// tensor memory: two accumulator buffers of 160 columns, then three 64-column slots that hold
+constexpr int NA = 2;          // ring depth (steps) of the expanded ternary operand (tensor memory)
+// tensor memory: two accumulator buffers of 192 columns, then two 64-column slots that hold
 // the expanded ternary operand of a step (per block 128 rows x 128 int8 = 32 columns of 32 bits)
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_COLS = NT_MAX;
@@ -52,9 +52,8 @@ constexpr int EPI_WARPS_MAX = 8;
 __host__ __device__ constexpr bool four_epilogue_warps(int kb_tile, int tok) { return 3 * kb_tile >= tok; }
 __host__ __device__ constexpr int gemm_threads(int epiw) { return 32 * (EPI_WARP0 + epiw); }
 
-// tokens per tile for nd digits: a multiple of 8 with an MMA N extent nd * tokens <= 160 that is
-// a multiple of 16 (160, 144, 160, 160 columns for 1..4 digits)
-__host__ __device__ constexpr int tokens_per_tile(int nd) { return nd == 3 ? 48 : 160 / nd; }
+// tokens per tile for nd digits: the MMA N extent is nd * tokens = 192 for every nd
+__host__ __device__ constexpr int tokens_per_tile(int nd) { return 192 / nd; }
 
 constexpr int P_TILE_BYTES = BLOCK_R * BLOCK_C / 4;      // packed codes of that tile, 4 KiB
 constexpr int B_TILE_BYTES_MAX = NT_MAX * BLOCK_C;       // digit rows, 24 KiB
@@ -269,7 +268,7 @@ ternary_mma_kernel(const GemmParams p)
 {
     constexpr int EPI_SHARES = EPI_WARPS / 4;
     constexpr int NT = ND * TOK;
-    static_assert(NT % 16 == 0 && NT <= NT_MAX && TOK % 8 == 0, "tile shape");
+    static_assert(NT % 16 == 0 && NT <= NT_MAX && TOK % 16 == 0, "tile shape");
     constexpr uint32_t B_TILE_BYTES = NT * BLOCK_C;
     constexpr uint32_t IDESC = umma_idesc_s8(BLOCK_R, NT);
 
@@ -436,7 +435,7 @@ ternary_mma_kernel(const GemmParams p)
                     const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_SLOT_BYTES >> 4));
                     const uint32_t cur = slot;
                     if (++slot == nb) { slot = 0; phase ^= 1; }
-                    if (++aslot == NA) aslot = 0;
+                    aslot = (aslot + 1) & (NA - 1);
                     if (elect_one()) {
                         // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
                         // the swizzled 128-byte rows of B
@@ -532,6 +531,8 @@ ternary_mma_kernel(const GemmParams p)
             const uint32_t buf = local & 1;
             // this warp takes its share of the groups of 8 tokens
             constexpr int N_GROUPS = TOK / 8;
+            constexpr int MY_GROUPS = N_GROUPS / EPI_SHARES;
+            static_assert(N_GROUPS % EPI_SHARES == 0, "the epilogue warps of a lane group share the token groups evenly");
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             const bool row_ok = row < p.R;
@@ -539,9 +540,8 @@ ternary_mma_kernel(const GemmParams p)
             tc_fence_after_sync();
             const uint32_t t_lane = tmem_base + buf * (uint32_t)ACC_COLS + ((uint32_t)(lane_grp * 32) << 16);
 #pragma unroll
-            for (int g0 = 0; g0 < N_GROUPS; g0 += EPI_SHARES) {
-                const int g = g0 + half;
-                if (g >= N_GROUPS) break;   // (an odd number of groups: the second share has one fewer)
+            for (int k = 0; k < MY_GROUPS; ++k) {
+                const int g = half + EPI_SHARES * k;
                 uint32_t acc[ND][8];
 #pragma unroll
                 for (int d = 0; d < ND; ++d) tmem_ld8(t_lane + (uint32_t)(d * TOK + g * 8), acc[d]);
