@@ -419,11 +419,10 @@ ternary_mma_kernel(const GemmParams p)
             // readiness of the next slot is tested (without blocking) while the current step's
             // MMAs are being issued, so that the barrier's latency is off the issue path
             bool ready = mbar_test_wait(&ready_bar[0], 0);
-            bool acc_free = true;   // both accumulators are free at the start; later tested early, as `ready` is
             bool alive = true;
             for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
                 const uint32_t buf = (uint32_t)L & 1u;
-                if (!acc_free && !mbar_wait(&accempty_bar[buf], (((uint32_t)L >> 1) & 1) ^ 1, abort_flag)) break;
+                if (!mbar_wait(&accempty_bar[buf], (((uint32_t)L >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
                 int kb0, kb1;
@@ -460,9 +459,6 @@ ternary_mma_kernel(const GemmParams p)
                 }
                 if (elect_one()) umma_commit(&accfull_bar[buf]);
                 __syncwarp();
-                // has the epilogue drained the other accumulator (tile L + 1 uses it for the
-                // ((L + 1) >> 1)-th time)?  Tested here, behind the commits, off the next tile's path.
-                acc_free = mbar_test_wait(&accempty_bar[buf ^ 1u], ((((uint32_t)L + 1u) >> 1) & 1) ^ 1);
             }
         }
     } else if (warp >= EXP_WARP0 && warp < EPI_WARP0) {
