@@ -412,102 +412,53 @@ ternary_mma_kernel(const GemmParams p)
     } else if (warp == 1) {
         // ---- MMA issue.  The whole warp runs the loop so that slot, phase and the operand
         //      descriptors stay warp-uniform (the MMA instructions take them from the uniform
-        //      register file); one elected lane issues the MMAs and commits.
-        //      A commit holds the issuing thread until the MMAs before it have started, so when
-        //      it returns the tensor pipe has about one MMA of work left.  Everything this warp
-        //      has to do for the NEXT step (loop control, the accumulator switch at a tile
-        //      boundary, the test of the next step's barrier, the descriptors) is therefore done
-        //      between queueing the current step's last MMAs and its last commit, while those
-        //      MMAs are still queued; after the commit only the next MMAs remain to be issued. ----
+        //      register file); one elected lane issues the MMAs and commits. ----
         {
-            struct Step {
-                uint32_t d_tmem, a_tmem, slot, phase, buf;
-                uint64_t b_desc;
-                int nblk;
-                bool first, last;   // first / last step of its tile
-            };
             uint32_t slot = 0, phase = 0, aslot = 0;
-            int L = 0, tile = tile_first, kb = 0, kb0 = 0, kb1 = 0;
             const uint64_t b_desc0 = umma_desc_k_sw128(smem_u32(b_tiles));
-            if (tile_count > 0) tile_kb_range(p, tile, kb0, kb1);
-            kb = kb0;
-            // the step at (L, kb), and the ring positions it takes
-            auto make_step = [&](Step& st) {
-                st.buf = (uint32_t)L & 1u;
-                st.d_tmem = tmem_base + st.buf * (uint32_t)ACC_COLS;
-                st.a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
-                st.b_desc = b_desc0 + (uint64_t)(slot * (B_SLOT_BYTES >> 4));
-                st.slot = slot;
-                st.phase = phase;
-                st.nblk = min(STEP_BLOCKS, kb1 - kb);
-                st.first = kb == kb0;
-                st.last = kb + STEP_BLOCKS >= kb1;
-                if (++slot == nb) { slot = 0; phase ^= 1; }
-                aslot = (aslot + 1) & (NA - 1);
-            };
-            // move (L, tile, kb) to the next step; false when this CTA has no more
-            auto advance = [&]() -> bool {
-                kb += STEP_BLOCKS;
-                if (kb < kb1) return true;
-                ++L;
-                tile += tile_step;
-                if (L >= tile_count) return false;
-                tile_kb_range(p, tile, kb0, kb1);
-                kb = kb0;
-                return true;
-            };
-            bool have = tile_count > 0;
-            Step cur{};
-            if (have) {
-                make_step(cur);
-                // (the first use of an accumulator buffer never waits)
-                have = mbar_wait(&ready_bar[cur.slot], cur.phase, abort_flag);
+            // readiness of the next slot is tested (without blocking) while the current step's
+            // MMAs are being issued, so that the barrier's latency is off the issue path
+            bool ready = mbar_test_wait(&ready_bar[0], 0);
+            bool alive = true;
+            for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
+                const uint32_t buf = (uint32_t)L & 1u;
+                if (!mbar_wait(&accempty_bar[buf], (((uint32_t)L >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
-            }
-            while (have) {
-                if (elect_one()) {
-                    // 32 contraction elements per instruction: 8 columns of A, 32 bytes of the
-                    // swizzled 128-byte rows of B
-#pragma unroll
-                    for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
-                        umma_s8_ts(cur.d_tmem, cur.a_tmem + (uint32_t)(k * (UMMA_K / 4)),
-                                   cur.b_desc + (uint64_t)(k * (UMMA_K >> 4)), IDESC, !cur.first || k != 0);
-                    // block 0 of the step is done: its half of the A slot is free NA steps on
-                    umma_commit(&done_bar[cur.slot * STEP_BLOCKS]);
-                    if (cur.nblk > 1) {
-#pragma unroll
-                        for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
-                            umma_s8_ts(cur.d_tmem, cur.a_tmem + (uint32_t)(A_BLOCK_COLS + k * (UMMA_K / 4)),
-                                       cur.b_desc + (uint64_t)((B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC, true);
-                    }
-                }
-                __syncwarp();
-                // ---- everything for the next step, while the MMAs above are queued ----
-                Step nxt{};
-                const bool have_n = advance();
-                bool rdy = false, acc_ok = true;
-                if (have_n) {
-                    make_step(nxt);
-                    if (nxt.first)   // a new tile: has the epilogue drained its accumulator buffer?
-                        acc_ok = mbar_test_wait(&accempty_bar[nxt.buf], (((uint32_t)L >> 1) & 1) ^ 1);
-                    rdy = mbar_test_wait(&ready_bar[nxt.slot], nxt.phase);
-                }
-                if (elect_one()) {
-                    // the step's last block is done (a block the step does not have counts as done
-                    // too): the digit slot is free, and the tile's accumulator is complete after its last step
-                    umma_commit(&done_bar[cur.slot * STEP_BLOCKS + 1]);
-                    if (cur.last) umma_commit(&accfull_bar[cur.buf]);
-                }
-                __syncwarp();
-                if (have_n) {
-                    bool ok = true;
-                    if (!acc_ok) ok = mbar_wait(&accempty_bar[nxt.buf], (((uint32_t)L >> 1) & 1) ^ 1, abort_flag);
-                    if (ok && !rdy) ok = mbar_wait(&ready_bar[nxt.slot], nxt.phase, abort_flag);
+                const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
+                int kb0, kb1;
+                tile_kb_range(p, tile, kb0, kb1);
+                for (int kb = kb0; kb < kb1; kb += STEP_BLOCKS) {
+                    const int nblk = min(STEP_BLOCKS, kb1 - kb);
+                    if (!ready && !mbar_wait(&ready_bar[slot], phase, abort_flag)) { alive = false; break; }
                     tc_fence_after_sync();
-                    if (!ok) break;
+                    const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_SLOT_BYTES >> 4));
+                    const uint32_t cur = slot;
+                    if (++slot == nb) { slot = 0; phase ^= 1; }
+                    aslot = (aslot + 1) & (NA - 1);
+                    if (elect_one()) {
+                        // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
+                        // the swizzled 128-byte rows of B
+#pragma unroll
+                        for (int j = 0; j < STEP_BLOCKS; ++j) {
+                            if (j < nblk) {
+#pragma unroll
+                                for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
+                                    umma_s8_ts(d_tmem, a_tmem + (uint32_t)(j * A_BLOCK_COLS + k * (UMMA_K / 4)),
+                                               b_desc + (uint64_t)(j * (B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC,
+                                               kb != kb0 || j != 0 || k != 0);
+                            }
+                            // block j of the step is done (a block the step does not have counts as
+                            // done too): its part of the A slot is free NA steps on, and after the
+                            // last block the digit slot
+                            umma_commit(&done_bar[cur * STEP_BLOCKS + j]);
+                        }
+                    }
+                    __syncwarp();
+                    ready = mbar_test_wait(&ready_bar[slot], phase);
                 }
-                cur = nxt;
-                have = have_n;
+                if (elect_one()) umma_commit(&accfull_bar[buf]);
+                __syncwarp();
             }
         }
     } else if (warp >= EXP_WARP0 && warp < EPI_WARP0) {
