@@ -22,12 +22,12 @@ template <> __device__ __forceinline__ float to_float<int8_t>(int8_t v) { return
 // One addition serves all digits: q + (0x80 + 0x8000 + ..., ND-1 terms) has, below the top
 // digit, 0x80 too much in byte d, which an exclusive-or takes out again.  The bytes of four
 // values are then transposed into the four digit words with eight byte permutes.
-template <int ND>
-__device__ __forceinline__ void digits_of_16(const int (&q)[16], uint32_t (&dig)[ND][4])
+template <int ND, int G>
+__device__ __forceinline__ void digits_of(const int (&q)[4 * G], uint32_t (&dig)[ND][G])
 {
     constexpr uint32_t off = ND == 1 ? 0u : ND == 2 ? 0x80u : ND == 3 ? 0x8080u : 0x808080u;
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {
+    for (int g = 0; g < G; ++g) {
         const uint32_t a = (uint32_t)q[4 * g] + off, b = (uint32_t)q[4 * g + 1] + off;
         const uint32_t c = (uint32_t)q[4 * g + 2] + off, e = (uint32_t)q[4 * g + 3] + off;
         const uint32_t ab01 = __byte_perm(a, b, 0x5140), cd01 = __byte_perm(c, e, 0x5140);   // bytes 0,1 of each pair
@@ -38,6 +38,40 @@ __device__ __forceinline__ void digits_of_16(const int (&q)[16], uint32_t (&dig)
             dig[2][g] = __byte_perm(ab23, cd23, 0x5410) ^ (ND > 3 ? 0x80808080u : 0u);
             if constexpr (ND > 3) dig[3][g] = __byte_perm(ab23, cd23, 0x7632);
         }
+    }
+}
+
+template <int ND>
+__device__ __forceinline__ void digits_of_16(const int (&q)[16], uint32_t (&dig)[ND][4]) { digits_of<ND, 4>(q, dig); }
+
+// Load 8 consecutive values of a row as floats (one or two vector loads when the chunk is whole
+// and the row 16-byte aligned, guarded scalar loads otherwise).
+template <typename IN_T>
+__device__ __forceinline__ void load8(const IN_T* __restrict__ row, int c0, int C, bool vec_ok, float (&v)[8])
+{
+    if (vec_ok && c0 + 8 <= C) {
+        if constexpr (sizeof(IN_T) == 4) {
+            const float4 f0 = __ldg(reinterpret_cast<const float4*>(row + c0));
+            const float4 f1 = __ldg(reinterpret_cast<const float4*>(row + c0) + 1);
+            v[0] = f0.x; v[1] = f0.y; v[2] = f0.z; v[3] = f0.w;
+            v[4] = f1.x; v[5] = f1.y; v[6] = f1.z; v[7] = f1.w;
+        } else if constexpr (sizeof(IN_T) == 2) {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(row + c0));
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {   // bf16 -> fp32 is a 16-bit shift
+                v[2 * j] = __uint_as_float(w[j] << 16);
+                v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+            }
+        } else {
+            const uint2 u = __ldg(reinterpret_cast<const uint2*>(row + c0));
+            const uint32_t w[2] = {u.x, u.y};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = (float)(int)(int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xFF);
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = (c0 + e < C) ? to_float<IN_T>(row[c0 + e]) : 0.f;
     }
 }
 

@@ -73,10 +73,12 @@ constexpr int GEMM_SMEM_BYTES = NB * B_SLOT_BYTES + NP * P_SLOT_BYTES +
 
 // TPT threads per token slot b in [0, B_pad): one warp (8 tokens per block) for large batches,
 // a whole block of 256 for small ones, where a row must be spread over more threads to hide
-// latency.  ND digits.  `amax_bits` (optional) holds the precomputed max |value| of each token
+// latency.  ND digits.  A thread converts chunks of CH = 16 or 8 consecutive values; 8 when that
+// spreads a row evenly over the warp (768 values = 3 x 32 chunks of 8, against 48 chunks of 16
+// for 32 lanes).  `amax_bits` (optional) holds the precomputed max |value| of each token
 // as float bits; otherwise the token's threads reduce it.  For int8 input (ND == 1) the
 // values are their own single digit and the scale is 1.
-template <typename IN_T, int ND, int TPT, int TOK>
+template <typename IN_T, int ND, int TPT, int TOK, int CH>
 __global__ void __launch_bounds__(256, 4)   // <= 64 registers: a batch of 4096 tokens is then one wave
 digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
@@ -84,7 +86,11 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
 {
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
+    constexpr int G = CH / 4;                   // groups of four values per chunk
+    constexpr int KEEP = CH == 16 ? 2 : 3;      // chunks per thread that stay in registers between the passes
+    constexpr int PER_BLOCK = BLOCK_C / CH;     // chunks per 128-deep contraction block
     static_assert(TPT == 32 || TPT == 256, "one warp or one block per token");
+    static_assert(CH == 16 || CH == 8, "chunk size");
     const int lane = threadIdx.x % TPT;                       // index among the token's threads
     const int b = blockIdx.x * (256 / TPT) + threadIdx.x / TPT;
     if (b >= B_pad) return;                                   // (whole block when TPT == 256)
@@ -97,16 +103,19 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     const bool live = b < B;
     const IN_T* row = in + (size_t)b * ld_in;
     const bool vec_ok = ((((uintptr_t)in) | ((size_t)ld_in * sizeof(IN_T))) & 15) == 0;
-    const int n_chunks = KB * 8;
+    const int n_chunks = KB * PER_BLOCK;
+    auto load_chunk = [&](int ch, float (&v)[CH]) {
+        if constexpr (CH == 16) load16<IN_T>(row, ch * CH, C, vec_ok, v);
+        else load8<IN_T>(row, ch * CH, C, vec_ok, v);
+    };
 
     if (zero_buf)   // clear this token's slice of the accumulators a later kernel adds into
         for (int i = lane; i < zero_per_token; i += TPT)
             if ((size_t)b * zero_per_token + i < (size_t)zero_total) zero_buf[(size_t)b * zero_per_token + i] = 0;
 
-    // Rows of up to two chunks per thread (C <= 1024 with one warp per token, <= 8192 with a
-    // block) are loaded once and kept in registers for both passes.
-    const bool cached = n_chunks <= 2 * TPT;
-    float keep[2][16];
+    // Rows of up to KEEP chunks per thread are loaded once and kept in registers for both passes.
+    const bool cached = n_chunks <= KEEP * TPT;
+    float keep[KEEP][CH];
     float qscale = 1.f;
     if constexpr (!kInt) {
         float amax = 0.f;
@@ -115,20 +124,20 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
                 amax = __uint_as_float(amax_bits[b]);
             } else if (cached) {
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
+                for (int j = 0; j < KEEP; ++j) {
                     const int ch = lane + j * TPT;
                     if (ch < n_chunks) {
-                        load16<IN_T>(row, ch * 16, C, vec_ok, keep[j]);
+                        load_chunk(ch, keep[j]);
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) amax = fmaxf(amax, fabsf(keep[j][e]));
+                        for (int e = 0; e < CH; ++e) amax = fmaxf(amax, fabsf(keep[j][e]));
                     }
                 }
             } else {
                 for (int ch = lane; ch < n_chunks; ch += TPT) {
-                    float v[16];
-                    load16<IN_T>(row, ch * 16, C, vec_ok, v);
+                    float v[CH];
+                    load_chunk(ch, v);
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) amax = fmaxf(amax, fabsf(v[e]));
+                    for (int e = 0; e < CH; ++e) amax = fmaxf(amax, fabsf(v[e]));
                 }
             }
             // warp-wide maximum (live is uniform across the warp)
@@ -148,34 +157,53 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
         if (lane == 0) scale_out[b] = 1.f;
     }
 
-    // each lane converts chunks of 16 consecutive contraction elements
-    for (int ch = lane; ch < n_chunks; ch += TPT) {
-        const int kb = ch >> 3, cc = ch & 7;
-        uint32_t dig[ND][4];
+    // one chunk: values -> digits -> the chunk's place in the swizzled tile (zeros for a dead token)
+    auto convert = [&](int ch, const float (&v)[CH]) {
+        uint32_t dig[ND][G];
 #pragma unroll
         for (int d = 0; d < ND; ++d)
 #pragma unroll
-            for (int w = 0; w < 4; ++w) dig[d][w] = 0;
+            for (int w = 0; w < G; ++w) dig[d][w] = 0;
         if (live) {
-            float v[16];
-            const int j = ch >= TPT ? 1 : 0;          // ch = lane + j * TPT
-            if (!kInt && cached && !amax_bits) {
+            int q[CH];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = j ? keep[1][e] : keep[0][e];
-            } else {
-                load16<IN_T>(row, ch * 16, C, vec_ok, v);
-            }
-            int q[16];
-#pragma unroll
-            for (int e = 0; e < 16; ++e) q[e] = __float2int_rn(v[e] * qscale);
-            digits_of_16<ND>(q, dig);
+            for (int e = 0; e < CH; ++e) q[e] = __float2int_rn(v[e] * qscale);
+            digits_of<ND, G>(q, dig);
         }
+        const int kb = ch / PER_BLOCK, in_block = ch % PER_BLOCK;
+        const int cc = in_block * CH / 16, sub = (in_block * CH) % 16;   // 16-byte chunk of the row, offset inside it
         int8_t* tile = D + ((size_t)jt * KB + kb) * (size_t)(NT * 128);
 #pragma unroll
         for (int d = 0; d < ND; ++d) {
             const int r = d * TOK + b_in;
-            uint4 v4 = make_uint4(dig[d][0], dig[d][1], dig[d][2], dig[d][3]);
-            *reinterpret_cast<uint4*>(tile + r * 128 + ((cc ^ (r & 7)) << 4)) = v4;
+            int8_t* dst = tile + r * 128 + ((cc ^ (r & 7)) << 4) + sub;
+            if constexpr (CH == 16) *reinterpret_cast<uint4*>(dst) = make_uint4(dig[d][0], dig[d][1], dig[d][2], dig[d][3]);
+            else *reinterpret_cast<uint2*>(dst) = make_uint2(dig[d][0], dig[d][1]);
+        }
+    };
+    if (cached) {
+#pragma unroll
+        for (int j = 0; j < KEEP; ++j) {
+            const int ch = lane + j * TPT;
+            if (ch < n_chunks) {
+                if (!kInt && live && !amax_bits) {
+                    convert(ch, keep[j]);
+                } else {
+                    float v[CH];
+#pragma unroll
+                    for (int e = 0; e < CH; ++e) v[e] = 0.f;
+                    if (live) load_chunk(ch, v);
+                    convert(ch, v);
+                }
+            }
+        }
+    } else {
+        for (int ch = lane; ch < n_chunks; ch += TPT) {
+            float v[CH];
+#pragma unroll
+            for (int e = 0; e < CH; ++e) v[e] = 0.f;
+            if (live) load_chunk(ch, v);
+            convert(ch, v);
         }
     }
 }
@@ -727,12 +755,19 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
     // one warp per token when that gives enough warps to fill the GPU, or for short rows
     PdlLaunch cfg((B_pad * 32 >= 148 * 1024 || KB < 8) ? (unsigned)((B_pad + 7) / 8) : (unsigned)B_pad, 256, 0, stream);
     cudaError_t e;
-    if (B_pad * 32 >= 148 * 1024 || KB < 8)   // (same rule as above)
-        e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
+    if (B_pad * 32 >= 148 * 1024 || KB < 8) {   // (same rule as above)
+        // chunks of 8 values when chunks of 16 would leave part of the warp without work in the last
+        // round and the row still fits the registers (three chunks of 8 per lane)
+        if ((KB * 8) % 32 != 0 && KB * 16 <= 3 * 32)
+            e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK, 8>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
+                                   scale, zero_buf, zero_per_token, zero_total);
+        else
+            e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK, 16>, in, ld_in, B, B_pad, C, KB, amax_bits,
+                                   D, scale, zero_buf, zero_per_token, zero_total);
+    } else {
+        e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 256, TOK, 16>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
                                scale, zero_buf, zero_per_token, zero_total);
-    else
-        e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 256, TOK>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                               scale, zero_buf, zero_per_token, zero_total);
+    }
     tsvd_count_launch();
     if (B_pad_out) *B_pad_out = B_pad;
     return e != cudaSuccess ? e : cudaGetLastError();
