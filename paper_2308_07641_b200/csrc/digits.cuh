@@ -22,10 +22,12 @@ template <> __device__ __forceinline__ float to_float<int8_t>(int8_t v) { return
 // One addition serves all digits: q + (0x80 + 0x8000 + ..., ND-1 terms) has, below the top
 // digit, 0x80 too much in byte d, which an exclusive-or takes out again.  The bytes of four
 // values are then transposed into the four digit words with eight byte permutes.
+// `bias` is subtracted from every q first (0, or the integer image of the rounding constant when
+// q comes from tsvd_round_bits below); it folds into the one addition.
 template <int ND, int G>
-__device__ __forceinline__ void digits_of(const int (&q)[4 * G], uint32_t (&dig)[ND][G])
+__device__ __forceinline__ void digits_of(const int (&q)[4 * G], uint32_t (&dig)[ND][G], uint32_t bias = 0u)
 {
-    constexpr uint32_t off = ND == 1 ? 0u : ND == 2 ? 0x80u : ND == 3 ? 0x8080u : 0x808080u;
+    const uint32_t off = (ND == 1 ? 0u : ND == 2 ? 0x80u : ND == 3 ? 0x8080u : 0x808080u) - bias;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
         const uint32_t a = (uint32_t)q[4 * g] + off, b = (uint32_t)q[4 * g + 1] + off;
@@ -39,6 +41,16 @@ __device__ __forceinline__ void digits_of(const int (&q)[4 * G], uint32_t (&dig)
             if constexpr (ND > 3) dig[3][g] = __byte_perm(ab23, cd23, 0x7632);
         }
     }
+}
+
+// rint(v * qscale) for |v * qscale| <= 2^22 without a conversion instruction: adding 1.5 * 2^23
+// rounds the product to an integer (to nearest, ties to even, as cvt.rni does; the product itself is
+// exact because qscale is a power of two), and the sum's bit pattern is that integer plus
+// TSVD_ROUND_BIAS.
+constexpr uint32_t TSVD_ROUND_BIAS = 0x4B400000u;
+__device__ __forceinline__ int tsvd_round_bits(float v, float qscale)
+{
+    return __float_as_int(fmaf(v, qscale, 12582912.f));
 }
 
 template <int ND>

@@ -157,6 +157,9 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
         if (lane == 0) scale_out[b] = 1.f;
     }
 
+    static_assert(TOK % 8 == 0, "digit rows of one token must share their swizzle term");
+    const int sw = b_in & 7;
+    int8_t* tok_base = D + (size_t)jt * KB * (size_t)(NT * 128) + b_in * 128;
     // one chunk: values -> digits -> the chunk's place in the swizzled tile (zeros for a dead token)
     auto convert = [&](int ch, const float (&v)[CH]) {
         uint32_t dig[ND][G];
@@ -166,17 +169,23 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
             for (int w = 0; w < G; ++w) dig[d][w] = 0;
         if (live) {
             int q[CH];
+            if constexpr (ND <= 3) {   // |q| <= 2^22: round by adding a constant, whose image the digit offset absorbs
 #pragma unroll
-            for (int e = 0; e < CH; ++e) q[e] = __float2int_rn(v[e] * qscale);
-            digits_of<ND, G>(q, dig);
+                for (int e = 0; e < CH; ++e) q[e] = tsvd_round_bits(v[e], qscale);
+                digits_of<ND, G>(q, dig, TSVD_ROUND_BIAS);
+            } else {
+#pragma unroll
+                for (int e = 0; e < CH; ++e) q[e] = __float2int_rn(v[e] * qscale);
+                digits_of<ND, G>(q, dig);
+            }
         }
         const int kb = ch / PER_BLOCK, in_block = ch % PER_BLOCK;
         const int cc = in_block * CH / 16, sub = (in_block * CH) % 16;   // 16-byte chunk of the row, offset inside it
-        int8_t* tile = D + ((size_t)jt * KB + kb) * (size_t)(NT * 128);
+        // (TOK is a multiple of 8, so all digit rows of a token share the swizzle term b_in & 7)
+        int8_t* dst0 = tok_base + (size_t)kb * (size_t)(NT * 128) + ((cc ^ sw) << 4) + sub;
 #pragma unroll
         for (int d = 0; d < ND; ++d) {
-            const int r = d * TOK + b_in;
-            int8_t* dst = tile + r * 128 + ((cc ^ (r & 7)) << 4) + sub;
+            int8_t* dst = dst0 + d * (TOK * 128);
             if constexpr (CH == 16) *reinterpret_cast<uint4*>(dst) = make_uint4(dig[d][0], dig[d][1], dig[d][2], dig[d][3]);
             else *reinterpret_cast<uint2*>(dst) = make_uint2(dig[d][0], dig[d][1]);
         }
