@@ -128,8 +128,8 @@ ternary_gemv_kernel(const GemvParams p)
 #pragma unroll
             for (int w = 0; w < GEMV_WARPS; ++w) m = fmaxf(m, wmax[w * NTOK + b]);
             const int E = tsvd_quant_exponent(m);
-            qscale[b] = exp2f((float)(8 * ND - 2 - E));
-            if (tid == 0) scale[b] = exp2f((float)(E - (8 * ND - 2)));   // value = q * scale
+            qscale[b] = tsvd_pow2(8 * ND - 2 - E);
+            if (tid == 0) scale[b] = tsvd_pow2(E - (8 * ND - 2));   // value = q * scale
         }
     } else {
         if (tid < NTOK) scale[tid] = 1.f;

@@ -124,14 +124,12 @@ __device__ __forceinline__ void load16(const IN_T* __restrict__ row, int c0, int
     }
 }
 
-// The exponent E of the rule above for a token whose largest magnitude is amax (0 -> a floor).
+// The exponent E of the rule above for a token whose largest magnitude is amax: amax = m * 2^E with
+// m in [0.5, 1), read from the exponent field (zero and subnormal maxima take the floor of -90).
 __device__ __forceinline__ int tsvd_quant_exponent(float amax)
 {
-    int E = -90;
-    if (amax > 0.f) {
-        int e;
-        (void)frexpf(amax, &e);
-        E = max(e, -90);
-    }
-    return E;
+    const int e = (int)((__float_as_uint(amax) >> 23) & 0xFFu) - 126;
+    return max(e, -90);
 }
+// 2^e for -126 <= e <= 127, exactly.
+__device__ __forceinline__ float tsvd_pow2(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }

@@ -151,8 +151,8 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
         }
         // |v| <= amax < 2^E; quantise to q = rint(v * 2^(8ND-2-E)), so |q| <= 2^(8ND-2)
         const int E = tsvd_quant_exponent(amax);
-        qscale = exp2f((float)(8 * ND - 2 - E));
-        if (lane == 0) scale_out[b] = exp2f((float)(E - (8 * ND - 2)));   // value = q * scale
+        qscale = tsvd_pow2(8 * ND - 2 - E);
+        if (lane == 0) scale_out[b] = tsvd_pow2(E - (8 * ND - 2));   // value = q * scale
     } else {
         if (lane == 0) scale_out[b] = 1.f;
     }
