@@ -75,20 +75,40 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity)
 // up it sets the flag and returns false; the caller carries on to the kernel's normal exit so
 // that tensor memory is released.
 constexpr int kWaitLimitDefault = 4096;  // 2^32 clocks, about two seconds
+// Up to 64 tries in one tight loop (two tries per trip: the polling warps share their schedulers'
+// issue slots with the warps that do the work, so a try has to cost as few instructions as possible).
+__device__ __forceinline__ bool mbar_try_wait_64(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+        "mov.u32 n, 32;\n"
+        "TRY:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra DONE;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra DONE;\n\t"
+        "sub.u32 n, n, 1;\n\t"
+        "setp.ne.u32 q, n, 0;\n\t"
+        "@q bra TRY;\n"
+        "DONE:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     const long long limit = (long long)ctl[1] << 20;
-    unsigned spins = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 63u) == 0) {
-            if (ctl[0]) return false;
-            if (clock64() - t0 > limit) {
-                ctl[0] = 1;
-                return false;
-            }
+        if (mbar_try_wait_64(bar, parity)) return true;
+        if (ctl[0]) return false;
+        if (clock64() - t0 > limit) {
+            ctl[0] = 1;
+            return false;
         }
     }
 }
