@@ -77,55 +77,34 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity)
 constexpr int kWaitLimitDefault = 4096;  // 2^32 clocks, about two seconds
 // Up to 64 tries in one tight loop (two tries per trip: the polling warps share their schedulers'
 // issue slots with the warps that do the work, so a try has to cost as few instructions as possible).
-// HINT_NS > 0: each try may stay suspended for up to that long before it reports "not yet" (it
-// still returns as soon as the phase completes), for warps whose wait is long and not urgent.
-template <int HINT_NS>
 __device__ __forceinline__ bool mbar_try_wait_64(uint64_t* bar, uint32_t parity)
 {
     uint32_t ok;
-    if constexpr (HINT_NS > 0) {
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
-            "mov.u32 n, 64;\n"
-            "TRY:\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "@p bra DONE;\n\t"
-            "sub.u32 n, n, 1;\n\t"
-            "setp.ne.u32 q, n, 0;\n\t"
-            "@q bra TRY;\n"
-            "DONE:\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity), "r"((uint32_t)HINT_NS)
-            : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
-            "mov.u32 n, 32;\n"
-            "TRY:\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "@p bra DONE;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "@p bra DONE;\n\t"
-            "sub.u32 n, n, 1;\n\t"
-            "setp.ne.u32 q, n, 0;\n\t"
-            "@q bra TRY;\n"
-            "DONE:\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity)
-            : "memory");
-    }
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+        "mov.u32 n, 32;\n"
+        "TRY:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra DONE;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra DONE;\n\t"
+        "sub.u32 n, n, 1;\n\t"
+        "setp.ne.u32 q, n, 0;\n\t"
+        "@q bra TRY;\n"
+        "DONE:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
     return ok != 0;
 }
-template <int HINT_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     const long long limit = (long long)ctl[1] << 20;
     while (true) {
-        if (mbar_try_wait_64<HINT_NS>(bar, parity)) return true;
+        if (mbar_try_wait_64(bar, parity)) return true;
         if (ctl[0]) return false;
         if (clock64() - t0 > limit) {
             ctl[0] = 1;

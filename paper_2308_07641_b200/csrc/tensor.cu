@@ -573,7 +573,7 @@ ternary_mma_kernel(const GemmParams p)
             float s_row = 0.f;
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             const bool row_ok = row < p.R;
-            if (!mbar_wait<1000>(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;   // long, and not urgent
+            if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
             tc_fence_after_sync();
             const uint32_t t_lane = tmem_base + buf * (uint32_t)ACC_COLS + ((uint32_t)(lane_grp * 32) << 16);
 #pragma unroll
