@@ -341,8 +341,7 @@ ternary_mma_kernel(const GemmParams p)
     uint64_t* accfull_bar = done_bar + NB * STEP_BLOCKS;   // [2] all MMAs of a tile have completed
     uint64_t* accempty_bar = accfull_bar + 2;        // [2] the epilogue has drained the accumulator
     uint64_t* tail_bar = accempty_bar + 2;           // [2] split contraction: epilogue warps meet, outcome is in
-    uint64_t* ready2_bar = tail_bar + 2;             // [NB] the second block of the step's expanded operand is written
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ready2_bar + NB);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [2]: flag, wait limit
     volatile int* tail_last = abort_flag + 2;        // whether this CTA finished its output tile last
 
@@ -366,8 +365,7 @@ ternary_mma_kernel(const GemmParams p)
     if (threadIdx.x == 0) {
         for (int s = 0; s < NP; ++s) { mbar_init(&pfull_bar[s], 1); mbar_init(&pempty_bar[s], 4); }
         for (int s = 0; s < NB; ++s) {
-            mbar_init(&ready_bar[s], 5);   // the copy's expect-tx arrival + one per expander warp of the group (block 0 written)
-            mbar_init(&ready2_bar[s], 4);  // one per expander warp of the group (block 1 written)
+            mbar_init(&ready_bar[s], 5);   // the copy's expect-tx arrival + one per expander warp of the group
             for (int j = 0; j < STEP_BLOCKS; ++j) mbar_init(&done_bar[s * STEP_BLOCKS + j], 1);
         }
         for (int i = 0; i < 2; ++i) {
@@ -472,35 +470,26 @@ ternary_mma_kernel(const GemmParams p)
                     tc_fence_after_sync();
                     const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
                     const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_SLOT_BYTES >> 4));
-                    const uint32_t cur = slot, cur_phase = phase;
+                    const uint32_t cur = slot;
                     if (++slot == nb) { slot = 0; phase ^= 1; }
                     aslot = (aslot + 1) & (NA - 1);
-                    static_assert(STEP_BLOCKS == 2, "the two blocks of a step are issued separately");
-                    // 32 contraction elements per instruction: 8 columns of A, 32 bytes of the
-                    // swizzled 128-byte rows of B.  Block j of the step is done (a block the step
-                    // does not have counts as done too): its part of the A slot is free NA steps
-                    // on, and after the last block the digit slot.
                     if (elect_one()) {
+                        // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
+                        // the swizzled 128-byte rows of B
 #pragma unroll
-                        for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
-                            umma_s8_ts(d_tmem, a_tmem + (uint32_t)(k * (UMMA_K / 4)), b_desc + (uint64_t)(k * (UMMA_K >> 4)),
-                                       IDESC, kb != kb0 || k != 0);
-                        umma_commit(&done_bar[cur * STEP_BLOCKS]);
-                    }
-                    __syncwarp();
-                    // the second block's operand has a barrier of its own (usually complete by now; it is
-                    // waited for even when the step has no second block, so that its phases stay in step)
-                    if (!mbar_test_wait(&ready2_bar[cur], cur_phase) &&
-                        !mbar_wait(&ready2_bar[cur], cur_phase, abort_flag)) { alive = false; break; }
-                    tc_fence_after_sync();
-                    if (elect_one()) {
-                        if (nblk > 1) {
+                        for (int j = 0; j < STEP_BLOCKS; ++j) {
+                            if (j < nblk) {
 #pragma unroll
-                            for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
-                                umma_s8_ts(d_tmem, a_tmem + (uint32_t)(A_BLOCK_COLS + k * (UMMA_K / 4)),
-                                           b_desc + (uint64_t)((B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC, true);
+                                for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
+                                    umma_s8_ts(d_tmem, a_tmem + (uint32_t)(j * A_BLOCK_COLS + k * (UMMA_K / 4)),
+                                               b_desc + (uint64_t)(j * (B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC,
+                                               kb != kb0 || j != 0 || k != 0);
+                            }
+                            // block j of the step is done (a block the step does not have counts as
+                            // done too): its part of the A slot is free NA steps on, and after the
+                            // last block the digit slot
+                            umma_commit(&done_bar[cur * STEP_BLOCKS + j]);
                         }
-                        umma_commit(&done_bar[cur * STEP_BLOCKS + 1]);
                     }
                     __syncwarp();
                     ready = mbar_test_wait(&ready_bar[slot], phase);
@@ -555,21 +544,14 @@ ternary_mma_kernel(const GemmParams p)
                             ok = mbar_wait(&done_bar[sd * STEP_BLOCKS + j], phd, abort_flag);
                             tc_fence_after_sync();
                         }
-                        if (ok) {
-                            // each block is handed over as soon as it is written
-                            tmem_st32(a_addr + (uint32_t)(j * A_BLOCK_COLS), o[j]);
-                            tmem_st_wait();
-                            tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(j == 0 ? &ready_bar[sb] : &ready2_bar[sb]);
-                        }
+                        if (ok) tmem_st32(a_addr + (uint32_t)(j * A_BLOCK_COLS), o[j]);
                     }
                 }
                 if (!ok) { alive = false; break; }
-                if (nblk == 1) {   // no second block: its barrier still completes its phase
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ready2_bar[sb]);
-                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ready_bar[sb]);
             }
         }
     } else if (warp >= EPI_WARP0) {
