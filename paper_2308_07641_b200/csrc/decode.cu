@@ -18,7 +18,7 @@ namespace {
 
 // threads per CTA: with one or two tokens the kernel waits on memory and wants many warps; with
 // four the accumulators need the registers
-__host__ __device__ constexpr int gemv_threads(int ntok) { return ntok <= 4 ? 512 : 256; }
+__host__ __device__ constexpr int gemv_threads(int ntok) { return ntok <= 2 ? 512 : 256; }
 constexpr int GEMV_RL = 8;          // lanes of a warp along the rows; the other four take different column groups
 constexpr int GEMV_RPL = 4;         // rows per lane
 constexpr int GEMV_CS = 32 / GEMV_RL;
