@@ -803,15 +803,14 @@ cudaError_t launch_gemm_w(const GemmParams& p, int row_tiles, cudaStream_t strea
     // memory while the CTA walks the row tiles: the ring then holds whole panels (a tile's steps).
     q.nb = NB;
     q.resident = 0;
-    int sms = 148;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int n_tiles = q.row_tiles * q.j_tiles * q.ksplit;
     const int steps = (q.KB + STEP_BLOCKS - 1) / STEP_BLOCKS;
-    // (it pays only when a CTA's run of tiles is long enough to stay within a token tile for a while)
-    if (q.ksplit == 1 && steps <= NB && n_tiles >= 4 * sms) {
+    if (q.ksplit == 1 && steps <= NB) {
         q.nb = steps * (NB / steps);
         q.resident = 1;
     }
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int n_tiles = q.row_tiles * q.j_tiles * q.ksplit;
     const int grid = n_tiles < sms ? n_tiles : sms;
     PdlLaunch cfg((unsigned)grid, (unsigned)gemm_threads(EPIW), GEMM_SMEM_BYTES, stream);
     const cudaError_t e = cudaLaunchKernelEx(&cfg.cfg, ternary_mma_kernel<ND, EPI, TOK, EPIW>, (const GemmParams)q);
