@@ -234,28 +234,6 @@ __device__ __forceinline__ void umma_s8_ts(uint32_t d_tmem, uint32_t a_tmem, uin
         "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
         : "memory");
 }
-// The same, executed under a per-thread predicate instead of inside a branch: every lane of the
-// (converged) warp runs the instruction stream, one lane's predicate is set.
-__device__ __forceinline__ void umma_s8_ts_if(uint32_t leader, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
-                                              uint32_t idesc, bool accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p, pl;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "setp.ne.b32 pl, %5, 0;\n\t"
-        "@pl tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(leader)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit_if(uint32_t leader, uint64_t* bar)
-{
-    asm volatile(
-        "{\n\t.reg .pred pl;\n\t"
-        "setp.ne.b32 pl, %1, 0;\n\t"
-        "@pl tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(smem_u32(bar)),
-        "r"(leader)
-        : "memory");
-}
 // Arrive on an mbarrier when all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint64_t* bar)
 {

@@ -457,7 +457,6 @@ ternary_mma_kernel(const GemmParams p)
             // MMAs are being issued, so that the barrier's latency is off the issue path
             bool ready = mbar_test_wait(&ready_bar[0], 0);
             bool alive = true;
-            const uint32_t leader = elect_one() ? 1u : 0u;   // the lane that issues; no branch around the MMAs
             for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
                 const uint32_t buf = (uint32_t)L & 1u;
                 if (!mbar_wait(&accempty_bar[buf], (((uint32_t)L >> 1) & 1) ^ 1, abort_flag)) break;
@@ -474,7 +473,7 @@ ternary_mma_kernel(const GemmParams p)
                     const uint32_t cur = slot;
                     if (++slot == nb) { slot = 0; phase ^= 1; }
                     aslot = (aslot + 1) & (NA - 1);
-                    {
+                    if (elect_one()) {
                         // 32 contraction elements per instruction: 8 columns of A, 32 bytes of
                         // the swizzled 128-byte rows of B
 #pragma unroll
@@ -482,19 +481,21 @@ ternary_mma_kernel(const GemmParams p)
                             if (j < nblk) {
 #pragma unroll
                                 for (int k = 0; k < BLOCK_C / UMMA_K; ++k)
-                                    umma_s8_ts_if(leader, d_tmem, a_tmem + (uint32_t)(j * A_BLOCK_COLS + k * (UMMA_K / 4)),
-                                                  b_desc + (uint64_t)(j * (B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC,
-                                                  kb != kb0 || j != 0 || k != 0);
+                                    umma_s8_ts(d_tmem, a_tmem + (uint32_t)(j * A_BLOCK_COLS + k * (UMMA_K / 4)),
+                                               b_desc + (uint64_t)(j * (B_TILE_BYTES >> 4) + k * (UMMA_K >> 4)), IDESC,
+                                               kb != kb0 || j != 0 || k != 0);
                             }
                             // block j of the step is done (a block the step does not have counts as
                             // done too): its part of the A slot is free NA steps on, and after the
                             // last block the digit slot
-                            umma_commit_if(leader, &done_bar[cur * STEP_BLOCKS + j]);
+                            umma_commit(&done_bar[cur * STEP_BLOCKS + j]);
                         }
                     }
+                    __syncwarp();
                     ready = mbar_test_wait(&ready_bar[slot], phase);
                 }
-                umma_commit_if(leader, &accfull_bar[buf]);
+                if (elect_one()) umma_commit(&accfull_bar[buf]);
+                __syncwarp();
             }
         }
     } else if (warp >= EXP_WARP0 && warp < EPI_WARP0) {
