@@ -47,11 +47,11 @@ typedef enum {
 #define TSVD_FLAG_PATH_SIMPLE 0x10u /* force the CUDA-core reference kernels               */
 #define TSVD_FLAG_PATH_DECODE 0x20u /* force the decode kernels (B <= TSVD_DECODE_MAX_B)    */
 #define TSVD_FLAG_PATH_TENSOR 0x40u /* force the tcgen05 tensor-core kernels               */
-/* The decode kernels (two launches, one per stage; each CTA streams 16 rows of the packed
+/* The decode kernels (two launches, one per stage; each CTA streams 32 rows of the packed
  * codes against fixed-point digits of the stage's input held in shared memory) serve batches
  * of at most this many tokens, and are what a forward of so few tokens runs by default.
  * Forcing them for a larger batch, or for a contraction too long for the digits to fit in
- * shared memory (about 12,000 columns at four tokens), returns TSVD_E_TOOBIG. */
+ * shared memory (about 10,000 columns at four tokens), returns TSVD_E_TOOBIG. */
 #define TSVD_DECODE_MAX_B 4
 /* Test hook for the bounded device-side waits: with B > 64 the V-stage kernel's copy
  * producer withholds the activation digits, so every wait on them runs out (after a few

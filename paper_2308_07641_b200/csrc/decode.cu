@@ -1,28 +1,33 @@
 // Decode path: y = U(diag(S)(V x)) for one to four tokens, bound by streaming the packed codes.
 //
-// For so few tokens a tensor-core tile is almost empty, and what matters is that every SM
+// For so few tokens a 128-row tcgen05 tile is almost empty, and what matters is that every SM
 // streams its share of the 2-bit codes (the whole of U and V is read once per forward) with as
-// little fixed cost as possible.  Two launches, one per stage (Table S1 rows "V(.)" and "U(.)"):
-// each CTA first turns the stage's input (x, or t = S*(V x)) into the same per-token fixed-point
-// digits as the tensor-core path, in shared memory, then walks 32 rows of the packed matrix:
-// a lane owns four rows of one 64-column group at a time, expands their codes to int8 with two
-// byte permutes per eight entries and adds them to the digits with four-way integer dot
-// products.  (Four rows per lane because every lane reads the same digits: a shared-memory load
-// that all lanes aim at one address still takes its four passes, so each one has to feed as
-// many dot products as the registers allow.)  All sums are exact integers, so the result does
-// not depend on how the columns are split over the lanes and warps.
+// little fixed cost and as few instructions per code as possible.  Two launches, one per stage
+// (Table S1 rows "V(.)" and "U(.)"): each CTA first turns the stage's input (x, or t = S*(V x))
+// into the same per-token fixed-point digits as the tensor-core path, in shared memory, then
+// takes 32 rows of the packed matrix.  The additions run on the warp-level integer MMA
+// (m16n8k32, int8 x int8 -> int32, operands in registers): the A operand is 16 rows x 32 columns
+// of codes expanded to int8 in registers (two byte permutes per eight entries), the B operand 32
+// columns x 8 (token, digit) pairs read from shared memory, so one instruction does the work of
+// 128 four-way dot products and the instruction count per code is set by the expansion alone
+// (9 per 16 entries).  A per-lane dot-product kernel was bound by exactly that arithmetic:
+// 1.8 us per token and stage on a 4096 x 4096 matrix against 0.65 us to stream it.  All sums are
+// exact integers, so the result does not depend on how the columns are split over the warps.
+//
+// Column order inside an MMA: a thread (row group g = lane / 4, quarter q = lane % 4) loads word q
+// of the 16-byte unit of rows g and g + 8, i.e. columns 16q .. 16q+15 of a 64-column group, and
+// one 16-byte slice of digits for the same columns.  The instruction's contraction index is
+// only a label, so the first MMA of a group takes columns 16q .. 16q+7 of every quarter and the
+// second 16q+8 .. 16q+15; each loaded word and digit slice is used whole and nothing is shuffled.
 #include "digits.cuh"
 #include "tsvd_internal.cuh"
 
 namespace {
 
-// threads per CTA: with one or two tokens the kernel waits on memory and wants many warps; with
-// four the accumulators need the registers
-__host__ __device__ constexpr int gemv_threads(int ntok) { return ntok <= 2 ? 512 : 256; }
-constexpr int GEMV_RL = 8;          // lanes of a warp along the rows; the other four take different column groups
-constexpr int GEMV_RPL = 4;         // rows per lane
-constexpr int GEMV_CS = 32 / GEMV_RL;
-constexpr int GEMV_ROWS = GEMV_RL * GEMV_RPL;   // rows per CTA
+constexpr int GEMV_THREADS = 512, GEMV_WARPS = GEMV_THREADS / 32;
+constexpr int GEMV_ROWS = 32;       // rows per CTA: two MMA row tiles
+constexpr int GEMV_PRE = 4;         // column groups a warp has in flight at a time
+constexpr int GEMV_DIG_PAD = 64;    // bytes between digit rows beyond C_pad: eight rows x four quarters hit all banks
 constexpr int GEMV_MAX_SMEM = 200 * 1024;
 
 enum { STAGE_V = 0, STAGE_U = 1 };
@@ -42,40 +47,70 @@ struct GemvParams {
     int z_int;
 };
 
-// grid: R_pad / 32 CTAs of 256 threads.  Dynamic shared memory:
-//   digits [NTOK][ND][C_pad] int8 | partial sums [warps][NTOK*ND][32 rows] int32 |
+// D (16 x 8, int32) += A (16 x 32, int8, rows) * B (32 x 8, int8, columns).  Lane (g, q):
+// a0/a2 = row g, contraction bytes 4q..4q+3 and 16+4q..; a1/a3 = row g + 8, the same bytes;
+// b0/b1 = column g, the same bytes; c0,c1 = row g, columns 2q, 2q+1; c2,c3 = row g + 8.
+__device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// A streaming 32-bit load that stays where it is written: the compiler moves an ordinary load
+// down to its first use, which for the codes is after the digit conversion, and their trip from
+// HBM (the longest wait of the kernel) would then start only there.
+__device__ __forceinline__ uint32_t ld_stream_now(const uint32_t* ptr)
+{
+    uint32_t v;
+    asm volatile("ld.global.cs.b32 %0, [%1];" : "=r"(v) : "l"(ptr));
+    return v;
+}
+
+// grid: R_pad / 32 CTAs of 512 threads.  Dynamic shared memory:
+//   digits [NTOK*ND][C_pad + 64] int8 | partial sums [warps][NTOK*ND][32 rows] int32 |
 //   scale [NTOK] | per-warp maxima [warps][NTOK]
 template <typename IN_T, int ND, int NTOK, int STAGE>
-__global__ void __launch_bounds__(gemv_threads(NTOK))
+__global__ void __launch_bounds__(GEMV_THREADS)
 ternary_gemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
-    constexpr int GEMV_THREADS = gemv_threads(NTOK), GEMV_WARPS = GEMV_THREADS / 32;
     constexpr bool kInt = sizeof(IN_T) == 1;
     static_assert(!kInt || ND == 1, "int8 activations are their own digit");
+    constexpr int NCOL = NTOK * ND;            // (token, digit) pairs = columns of the B operand
+    constexpr int NT = (NCOL + 7) / 8;         // MMA column tiles
+    const int dstride = p.C_pad + GEMV_DIG_PAD;
     int8_t* dig = reinterpret_cast<int8_t*>(smem);
-    int* red = reinterpret_cast<int*>(smem + (size_t)NTOK * ND * p.C_pad);
-    float* scale = reinterpret_cast<float*>(red + GEMV_WARPS * NTOK * ND * GEMV_ROWS);
+    int* red = reinterpret_cast<int*>(smem + (size_t)NCOL * dstride);
+    float* scale = reinterpret_cast<float*>(red + GEMV_WARPS * NCOL * GEMV_ROWS);
     float* wmax = scale + NTOK;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, q = lane & 3;
     const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
 
-    // lane = (column group within the pass, row); rows rsel, rsel + 8, .. of the CTA's 32; warp w
-    // takes column groups 4w + csel, + 4 * warps, ..  The first codes are requested before anything
-    // else, so that their trip from HBM overlaps with the digit conversion below.
-    const int rsel = lane & (GEMV_RL - 1), csel = lane / GEMV_RL;
-    const int row_base = blockIdx.x * GEMV_ROWS + rsel;
+    // Warp w takes column groups w, w + 16, ..; a lane's word of rows 16h + g and 16h + g + 8
+    // (h = 0, 1) of each.  One warp-wide load is 8 rows x 16 bytes = 128 contiguous bytes.  The
+    // first GEMV_PRE groups are requested before anything else, so that their trip from HBM
+    // overlaps with the digit conversion below.  All addresses are one pointer plus constants:
+    // the 32 rows lie in one 128-row block, and 16 column groups on is 16 blocks of 2 KiB on.
+    // (The kernel is bound by the number of instructions it issues, not by any one wait: address
+    // arithmetic repeated per load was a third of them.)
     const int n_groups = p.C_pad >> 6;
-    auto load_units = [&](int g, uint4 (&uu)[GEMV_RPL]) {
+    constexpr int GROUP_STEP = GEMV_WARPS * 128 * 4;   // words between a warp's consecutive column groups
+    const uint32_t* wp = reinterpret_cast<const uint32_t*>(p.units) +
+                         (tsvd_unit_index(blockIdx.x * GEMV_ROWS, warp, p.C_pad) + g) * 4 + q;
+    uint32_t w[GEMV_PRE][2][2];
 #pragma unroll
-        for (int j = 0; j < GEMV_RPL; ++j)
-            uu[j] = g < n_groups ? __ldcs(p.units + tsvd_unit_index(row_base + j * GEMV_RL, g, p.C_pad))
-                                 : make_uint4(0, 0, 0, 0);
-    };
-    int cg = GEMV_CS * warp + csel;
-    uint4 u[GEMV_RPL];
-    load_units(cg, u);
+    for (int i = 0; i < GEMV_PRE; ++i) {
+        const bool there = warp + i * GEMV_WARPS < n_groups;
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int r = 0; r < 2; ++r)
+                w[i][h][r] = there ? ld_stream_now(wp + i * GROUP_STEP + (16 * h + 8 * r) * 4) : 0u;
+    }
     // Both stages are launched as programmatic dependents of the kernel before them in the
     // stream: their CTAs may start, and request their first codes (which no kernel writes), while
     // that kernel still runs.  The stage's input (x, or t from the V-stage) is complete and
@@ -85,48 +120,52 @@ ternary_gemv_kernel(const GemvParams p)
     pdl_launch_dependents();
 
     // ---- the stage's input as fixed-point digits (every CTA makes its own copy).  A thread takes
-    //      chunks of 16 consecutive columns; all loads of a pass are independent, so a pass costs
+    //      chunks of 8 consecutive columns; all loads of a pass are independent, so a pass costs
     //      about one trip to L2, and the first chunk of each token stays in registers between the
     //      maximum pass and the conversion pass ----
-    const int n_chunks = p.C_pad >> 4;
-    float keep[NTOK][16];
+    const int n_chunks = p.C_pad >> 3;
+    float keep[NTOK][8];
     float qscale[NTOK];
 #pragma unroll
     for (int b = 0; b < NTOK; ++b) qscale[b] = 1.f;
+    // tokens beyond the batch re-read token 0 (the loads of all tokens are then unconditional and go
+    // out together); what they read is never used
+    const IN_T* rows[NTOK];
     bool vec_ok[NTOK];
 #pragma unroll
-    for (int b = 0; b < NTOK; ++b)
-        vec_ok[b] = ((reinterpret_cast<uintptr_t>(in + (size_t)b * p.ld_in)) & 15) == 0;
+    for (int b = 0; b < NTOK; ++b) {
+        rows[b] = in + (size_t)(b < p.B ? b : 0) * p.ld_in;
+        vec_ok[b] = ((reinterpret_cast<uintptr_t>(rows[b])) & 15) == 0;
+    }
     if constexpr (!kInt) {
         float amax[NTOK];
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) amax[b] = 0.f;
         for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
+            float v[NTOK][8];
+#pragma unroll
+            for (int b = 0; b < NTOK; ++b) load8<IN_T>(rows[b], ch * 8, p.C, vec_ok[b], v[b]);
 #pragma unroll
             for (int b = 0; b < NTOK; ++b) {
-                if (b < p.B) {
-                    float v[16];
-                    load16<IN_T>(in + (size_t)b * p.ld_in, ch * 16, p.C, vec_ok[b], v);
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) amax[b] = fmaxf(amax[b], fabsf(v[e]));
-                    if (ch == tid) {
+                for (int e = 0; e < 8; ++e) amax[b] = fmaxf(amax[b], fabsf(v[b][e]));
+                if (ch == tid) {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) keep[b][e] = v[e];
-                    }
+                    for (int e = 0; e < 8; ++e) keep[b][e] = v[b][e];
                 }
             }
         }
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) {
             for (int o = 16; o > 0; o >>= 1) amax[b] = fmaxf(amax[b], __shfl_xor_sync(0xffffffffu, amax[b], o));
-            if (lane == 0) wmax[warp * NTOK + b] = amax[b];
+            if (lane == 0) wmax[b * GEMV_WARPS + warp] = amax[b];
         }
         __syncthreads();
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) {
-            float m = 0.f;
-#pragma unroll
-            for (int w = 0; w < GEMV_WARPS; ++w) m = fmaxf(m, wmax[w * NTOK + b]);
+            // the sixteen warps' maxima: one per lane of each half-warp, then across its lanes
+            float m = wmax[b * GEMV_WARPS + (lane & (GEMV_WARPS - 1))];
+            for (int o = GEMV_WARPS / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
             const int E = tsvd_quant_exponent(m);
             qscale[b] = tsvd_pow2(8 * ND - 2 - E);
             if (tid == 0) scale[b] = tsvd_pow2(E - (8 * ND - 2));   // value = q * scale
@@ -135,84 +174,103 @@ ternary_gemv_kernel(const GemvParams p)
         if (tid < NTOK) scale[tid] = 1.f;
     }
     for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
+        float v[NTOK][8];
+        if (!kInt && ch == tid) {
+#pragma unroll
+            for (int b = 0; b < NTOK; ++b)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[b][e] = keep[b][e];
+        } else {
+#pragma unroll
+            for (int b = 0; b < NTOK; ++b) load8<IN_T>(rows[b], ch * 8, p.C, vec_ok[b], v[b]);
+        }
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) {
-            uint32_t dw[ND][4];
+            uint32_t dw[ND][2];
 #pragma unroll
-            for (int d = 0; d < ND; ++d)
-#pragma unroll
-                for (int g = 0; g < 4; ++g) dw[d][g] = 0u;
+            for (int d = 0; d < ND; ++d) dw[d][0] = dw[d][1] = 0u;
             if (b < p.B) {
-                float v[16];
-                if (!kInt && ch == tid) {
+                int qv[8];
+                if constexpr (ND <= 3) {   // |q| <= 2^22: round by adding a constant, whose image the digit offset absorbs
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) v[e] = keep[b][e];
+                    for (int e = 0; e < 8; ++e) qv[e] = tsvd_round_bits(v[b][e], qscale[b]);
+                    digits_of<ND, 2>(qv, dw, TSVD_ROUND_BIAS);
                 } else {
-                    load16<IN_T>(in + (size_t)b * p.ld_in, ch * 16, p.C, vec_ok[b], v);
-                }
-                int q[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) q[e] = __float2int_rn(v[e] * qscale[b]);
-                digits_of_16<ND>(q, dw);
+                    for (int e = 0; e < 8; ++e) qv[e] = __float2int_rn(v[b][e] * qscale[b]);
+                    digits_of<ND, 2>(qv, dw);
+                }
             }
 #pragma unroll
             for (int d = 0; d < ND; ++d)
-                *reinterpret_cast<uint4*>(dig + (size_t)(b * ND + d) * p.C_pad + ch * 16) =
-                    make_uint4(dw[d][0], dw[d][1], dw[d][2], dw[d][3]);
+                *reinterpret_cast<uint2*>(dig + (size_t)(b * ND + d) * dstride + ch * 8) = make_uint2(dw[d][0], dw[d][1]);
         }
     }
     __syncthreads();
 
     // ---- stream the codes ----
-    int acc[GEMV_RPL][NTOK][ND];
+    int acc[2][NT][4];
 #pragma unroll
-    for (int j = 0; j < GEMV_RPL; ++j)
+    for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int b = 0; b < NTOK; ++b)
+        for (int j = 0; j < NT; ++j)
 #pragma unroll
-            for (int d = 0; d < ND; ++d) acc[j][b][d] = 0;
+            for (int c = 0; c < 4; ++c) acc[h][j][c] = 0;
 
-    for (; cg < n_groups; cg += GEMV_CS * GEMV_WARPS) {
-        uint4 un[GEMV_RPL];   // the next pass, in flight while this one is summed
-        load_units(cg + GEMV_CS * GEMV_WARPS, un);
+    const int8_t* dp = dig + (size_t)g * dstride + warp * 64 + q * 16;   // this lane's digit slice of group `warp`
+    bool col_there[NT];
 #pragma unroll
-        for (int wi = 0; wi < 4; ++wi) {
-            uint32_t e[GEMV_RPL][4];   // sixteen entries of each row as int8, in column order
+    for (int j = 0; j < NT; ++j) col_there[j] = 8 * j + g < NCOL;
+#pragma unroll 1
+    for (int first = warp; first < n_groups; first += GEMV_PRE * GEMV_WARPS) {
+        wp += GEMV_PRE * GROUP_STEP;
+        uint32_t wn[GEMV_PRE][2][2];   // the next groups, in flight while these are summed
 #pragma unroll
-            for (int j = 0; j < GEMV_RPL; ++j)
-                tsvd_expand16(wi == 0 ? u[j].x : wi == 1 ? u[j].y : wi == 2 ? u[j].z : u[j].w, e[j]);
+        for (int i = 0; i < GEMV_PRE; ++i) {
+            const bool there = first + (GEMV_PRE + i) * GEMV_WARPS < n_groups;
 #pragma unroll
-            for (int b = 0; b < NTOK; ++b) {
+            for (int h = 0; h < 2; ++h)
 #pragma unroll
-                for (int d = 0; d < ND; ++d) {
-                    const uint4 xd = *reinterpret_cast<const uint4*>(dig + (size_t)(b * ND + d) * p.C_pad + cg * 64 + wi * 16);
+                for (int r = 0; r < 2; ++r)
+                    wn[i][h][r] = there ? ld_stream_now(wp + i * GROUP_STEP + (16 * h + 8 * r) * 4) : 0u;
+        }
 #pragma unroll
-                    for (int j = 0; j < GEMV_RPL; ++j) {
-                        int s = acc[j][b][d];
-                        s = __dp4a((int)e[j][0], (int)xd.x, s);
-                        s = __dp4a((int)e[j][1], (int)xd.y, s);
-                        s = __dp4a((int)e[j][2], (int)xd.z, s);
-                        s = __dp4a((int)e[j][3], (int)xd.w, s);
-                        acc[j][b][d] = s;
+        for (int i = 0; i < GEMV_PRE; ++i) {
+            if (first + i * GEMV_WARPS < n_groups) {   // the same for the whole warp
+                uint4 xd[NT];      // digits of columns 16q .. 16q+15 of this group, (token, digit) pair 8j + g
+#pragma unroll
+                for (int j = 0; j < NT; ++j)
+                    xd[j] = col_there[j] ? *reinterpret_cast<const uint4*>(dp + (size_t)(8 * j) * dstride + i * GEMV_WARPS * 64)
+                                         : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t e0[4], e1[4];   // sixteen entries of rows 16h + g and 16h + g + 8 as int8
+                    tsvd_expand16(w[i][h][0], e0);
+                    tsvd_expand16(w[i][h][1], e1);
+#pragma unroll
+                    for (int j = 0; j < NT; ++j) {
+                        mma_s8(acc[h][j], e0[0], e1[0], e0[1], e1[1], xd[j].x, xd[j].y);
+                        mma_s8(acc[h][j], e0[2], e1[2], e0[3], e1[3], xd[j].z, xd[j].w);
                     }
                 }
             }
         }
+        dp += GEMV_PRE * GEMV_WARPS * 64;
 #pragma unroll
-        for (int j = 0; j < GEMV_RPL; ++j) u[j] = un[j];
+        for (int i = 0; i < GEMV_PRE; ++i)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) { w[i][h][0] = wn[i][h][0]; w[i][h][1] = wn[i][h][1]; }
     }
 
-    // ---- add the lanes that took different column groups, then the warps ----
+    // ---- the warps took different column groups: leave the partial sums for the adders ----
 #pragma unroll
-    for (int j = 0; j < GEMV_RPL; ++j)
+    for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int b = 0; b < NTOK; ++b)
+        for (int j = 0; j < NT; ++j)
 #pragma unroll
-            for (int d = 0; d < ND; ++d) {
-                int v = acc[j][b][d];
-#pragma unroll
-                for (int o = GEMV_RL; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (csel == 0) red[(warp * NTOK * ND + b * ND + d) * GEMV_ROWS + j * GEMV_RL + rsel] = v;
+            for (int c = 0; c < 4; ++c) {
+                const int n = 8 * j + 2 * q + (c & 1), r = 16 * h + g + 8 * (c >> 1);
+                if (n < NCOL) red[(warp * NCOL + n) * GEMV_ROWS + r] = acc[h][j][c];
             }
     __syncthreads();
 
@@ -226,7 +284,7 @@ ternary_gemv_kernel(const GemvParams p)
             for (int d = 0; d < ND; ++d) {
                 int s = 0;
 #pragma unroll
-                for (int w = 0; w < GEMV_WARPS; ++w) s += red[(w * NTOK * ND + b * ND + d) * GEMV_ROWS + r];
+                for (int wi = 0; wi < GEMV_WARPS; ++wi) s += red[(wi * NCOL + b * ND + d) * GEMV_ROWS + r];
                 a[d] = s;
             }
             // lo and hi are exact 32-bit integers; their conversions and the fused multiply-add
@@ -260,9 +318,8 @@ ternary_gemv_kernel(const GemvParams p)
 
 size_t gemv_smem_bytes(int nd, int ntok, int C_pad)
 {
-    const size_t warps = gemv_threads(ntok) / 32;
-    return (size_t)ntok * nd * C_pad + warps * ntok * nd * GEMV_ROWS * sizeof(int) +
-           (size_t)ntok * sizeof(float) + warps * ntok * sizeof(float);
+    return (size_t)ntok * nd * (C_pad + GEMV_DIG_PAD) + (size_t)GEMV_WARPS * ntok * nd * GEMV_ROWS * sizeof(int) +
+           (size_t)ntok * sizeof(float) + (size_t)GEMV_WARPS * ntok * sizeof(float);
 }
 
 template <typename IN_T, int ND, int NTOK, int STAGE>
@@ -279,7 +336,7 @@ cudaError_t launch_gemv(const GemvParams& p, int R_pad, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    PdlLaunch cfg((unsigned)(R_pad / GEMV_ROWS), (unsigned)gemv_threads(NTOK), smem, stream);
+    PdlLaunch cfg((unsigned)(R_pad / GEMV_ROWS), (unsigned)GEMV_THREADS, smem, stream);
     const cudaError_t e = cudaLaunchKernelEx(&cfg.cfg, ternary_gemv_kernel<IN_T, ND, NTOK, STAGE>, (const GemvParams)p);
     tsvd_count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
