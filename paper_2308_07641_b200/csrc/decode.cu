@@ -69,8 +69,8 @@ __device__ __forceinline__ uint32_t ld_stream_now(const uint32_t* ptr)
 }
 
 // grid: R_pad / 32 CTAs of 512 threads.  Dynamic shared memory:
-//   digits [NTOK*ND][C_pad + 64] int8 | partial sums [warps][NTOK*ND][32 rows] int32 |
-//   scale [NTOK] | per-warp maxima [warps][NTOK]
+//   digits [NTOK*ND][C_pad + 64] int8 | sums [NTOK*ND][32 rows] int32 |
+//   scale [NTOK] | per-warp maxima [NTOK][warps]
 template <typename IN_T, int ND, int NTOK, int STAGE>
 __global__ void __launch_bounds__(GEMV_THREADS)
 ternary_gemv_kernel(const GemvParams p)
@@ -83,12 +83,13 @@ ternary_gemv_kernel(const GemvParams p)
     const int dstride = p.C_pad + GEMV_DIG_PAD;
     int8_t* dig = reinterpret_cast<int8_t*>(smem);
     int* red = reinterpret_cast<int*>(smem + (size_t)NCOL * dstride);
-    float* scale = reinterpret_cast<float*>(red + GEMV_WARPS * NCOL * GEMV_ROWS);
+    float* scale = reinterpret_cast<float*>(red + NCOL * GEMV_ROWS);
     float* wmax = scale + NTOK;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, q = lane & 3;
     const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
+    for (int i = tid; i < NCOL * GEMV_ROWS; i += GEMV_THREADS) red[i] = 0;   // the warps add into these after two barriers
 
     // Warp w takes column groups w, w + 16, ..; a lane's word of rows 16h + g and 16h + g + 8
     // (h = 0, 1) of each.  One warp-wide load is 8 rows x 16 bytes = 128 contiguous bytes.  The
@@ -226,13 +227,20 @@ ternary_gemv_kernel(const GemvParams p)
         wp += GEMV_PRE * GROUP_STEP;
         uint32_t wn[GEMV_PRE][2][2];   // the next groups, in flight while these are summed
 #pragma unroll
-        for (int i = 0; i < GEMV_PRE; ++i) {
-            const bool there = first + (GEMV_PRE + i) * GEMV_WARPS < n_groups;
+        for (int i = 0; i < GEMV_PRE; ++i)
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
+            for (int h = 0; h < 2; ++h) wn[i][h][0] = wn[i][h][1] = 0u;
+        if (first + GEMV_PRE * GEMV_WARPS < n_groups) {   // one test when nothing is left (the usual case at 4096 columns)
 #pragma unroll
-                for (int r = 0; r < 2; ++r)
-                    wn[i][h][r] = there ? ld_stream_now(wp + i * GROUP_STEP + (16 * h + 8 * r) * 4) : 0u;
+            for (int i = 0; i < GEMV_PRE; ++i) {
+                if (first + (GEMV_PRE + i) * GEMV_WARPS < n_groups) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int r = 0; r < 2; ++r)
+                            wn[i][h][r] = ld_stream_now(wp + i * GROUP_STEP + (16 * h + 8 * r) * 4);
+                }
+            }
         }
 #pragma unroll
         for (int i = 0; i < GEMV_PRE; ++i) {
@@ -262,7 +270,8 @@ ternary_gemv_kernel(const GemvParams p)
             for (int h = 0; h < 2; ++h) { w[i][h][0] = wn[i][h][0]; w[i][h][1] = wn[i][h][1]; }
     }
 
-    // ---- the warps took different column groups: leave the partial sums for the adders ----
+    // ---- the warps took different column groups: their sums meet in shared memory (integer
+    //      additions: exact in any order) ----
 #pragma unroll
     for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -270,7 +279,7 @@ ternary_gemv_kernel(const GemvParams p)
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int n = 8 * j + 2 * q + (c & 1), r = 16 * h + g + 8 * (c >> 1);
-                if (n < NCOL) red[(warp * NCOL + n) * GEMV_ROWS + r] = acc[h][j][c];
+                if (n < NCOL) atomicAdd(&red[n * GEMV_ROWS + r], acc[h][j][c]);
             }
     __syncthreads();
 
@@ -281,12 +290,7 @@ ternary_gemv_kernel(const GemvParams p)
         if (b < p.B) {
             int a[ND];
 #pragma unroll
-            for (int d = 0; d < ND; ++d) {
-                int s = 0;
-#pragma unroll
-                for (int wi = 0; wi < GEMV_WARPS; ++wi) s += red[(wi * NCOL + b * ND + d) * GEMV_ROWS + r];
-                a[d] = s;
-            }
+            for (int d = 0; d < ND; ++d) a[d] = red[(b * ND + d) * GEMV_ROWS + r];
             // lo and hi are exact 32-bit integers; their conversions and the fused multiply-add
             // round at 2^-24 of |hi|*65536 and |lo|
             float f;
@@ -318,7 +322,7 @@ ternary_gemv_kernel(const GemvParams p)
 
 size_t gemv_smem_bytes(int nd, int ntok, int C_pad)
 {
-    return (size_t)ntok * nd * (C_pad + GEMV_DIG_PAD) + (size_t)GEMV_WARPS * ntok * nd * GEMV_ROWS * sizeof(int) +
+    return (size_t)ntok * nd * (C_pad + GEMV_DIG_PAD) + (size_t)ntok * nd * GEMV_ROWS * sizeof(int) +
            (size_t)ntok * sizeof(float) + (size_t)GEMV_WARPS * ntok * sizeof(float);
 }
 
