@@ -138,14 +138,25 @@ ternary_gemv_kernel(const GemvParams p)
         rows[b] = in + (size_t)(b < p.B ? b : 0) * p.ld_in;
         vec_ok[b] = ((reinterpret_cast<uintptr_t>(rows[b])) & 15) == 0;
     }
+    bool all_vec = true;   // every token's row allows vector loads: one test per chunk, and the loads in a row
+#pragma unroll
+    for (int b = 0; b < NTOK; ++b) all_vec = all_vec && vec_ok[b];
+    auto load_tokens = [&](int ch, float (&v)[NTOK][8]) {
+        if (all_vec && ch * 8 + 8 <= p.C) {
+#pragma unroll
+            for (int b = 0; b < NTOK; ++b) load8<IN_T>(rows[b], ch * 8, 0x7fffffff, true, v[b]);
+        } else {
+#pragma unroll
+            for (int b = 0; b < NTOK; ++b) load8<IN_T>(rows[b], ch * 8, p.C, vec_ok[b], v[b]);
+        }
+    };
     if constexpr (!kInt) {
         float amax[NTOK];
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) amax[b] = 0.f;
         for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
             float v[NTOK][8];
-#pragma unroll
-            for (int b = 0; b < NTOK; ++b) load8<IN_T>(rows[b], ch * 8, p.C, vec_ok[b], v[b]);
+            load_tokens(ch, v);
 #pragma unroll
             for (int b = 0; b < NTOK; ++b) {
 #pragma unroll
@@ -182,8 +193,7 @@ ternary_gemv_kernel(const GemvParams p)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) v[b][e] = keep[b][e];
         } else {
-#pragma unroll
-            for (int b = 0; b < NTOK; ++b) load8<IN_T>(rows[b], ch * 8, p.C, vec_ok[b], v[b]);
+            load_tokens(ch, v);
         }
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) {
