@@ -58,24 +58,25 @@ def rank_spec(spec, rank):
     return gen.scaled(spec, seed=spec.seed + 1000 * rank) if rank else spec
 
 
-def kernel_source_sha1():
+def kernel_source_sha1(names):
     import hashlib
     h = hashlib.sha1()
-    for name in ("tensor.cu", "decode.cu", "digits.cuh", "sm100_ptx.cuh", "tsvd_internal.cuh"):
+    for name in names:
         with open(os.path.join(ROOT, "paper_2308_07641_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
 
 
 def recorded_traffic(workload, stage):
-    """DRAM bytes per launch from the committed ncu capture, or None when the kernel sources have
-    changed since that capture was taken (profiles/dram_traffic.txt holds JSON)."""
+    """DRAM bytes per launch from the committed ncu capture, or None when the sources of the kernels
+    that workload runs have changed since that capture was taken (profiles/dram_traffic.txt holds
+    JSON: per workload the source files hashed, their hash, and the bytes per launch of each stage)."""
     try:
         with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
-            d = json.load(f)
-        if d.get("kernel_source_sha1") != kernel_source_sha1():
+            d = json.load(f)["workloads"][workload]
+        if d["sha1"] != kernel_source_sha1(d["sources"]):
             return None
-        return d["bytes_per_launch"][workload][stage]
+        return d["bytes_per_launch"][stage]
     except Exception:
         return None
 
@@ -421,6 +422,10 @@ def main():
                           f"{sum(prof_step_ms) / args.steps:.4f}")
     roofline["plan"] = plan
     # whole-step tensor figure: all executed tensor operations over the whole step time
+    if plan["path"] == "decode":
+        # whole-step figure: all packed bytes over the graph-timed step (both launches, no event pairs)
+        roofline["step_hbm_gbs"] = info["packed_bytes"] / (ms_per_step * 1e-3) / 1e9
+        roofline["step_hbm_frac"] = roofline["step_hbm_gbs"] / peaks["hbm_gbs"]
     if plan["path"] == "tensor":
         all_ops = 2.0 * spec.B * (pad(spec.K) * pad(spec.N) * plan["digits_x"] + pad(spec.M) * pad(spec.K) * plan["digits_t"])
         roofline["step_tensor_frac"] = all_ops / (ms_per_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * INT8_OVER_BF16)
