@@ -224,12 +224,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg2", choices=sorted(gen.CONFIGS))
-    ap.add_argument("--path", default="auto", choices=["auto", "simple", "decode", "tensor"])
+    ap.add_argument("--path", default="auto", choices=["auto", "simple", "decode", "tensor", "index"],
+                    help="index = the index-list form (one to four tokens; meant for nonzero rates below 1/8)")
+    ap.add_argument("--density", type=float, default=None,
+                    help="override the workload's nonzero rate of U and V (the sparse sweep of the index-list form)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eager", action="store_true", help="time eager launches with an L2 flush per step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     spec = gen.CONFIGS[args.config]
+    if args.density is not None:
+        spec = gen.scaled(spec, name=f"{spec.name}_density{args.density:g}", density=args.density)
 
     if args.impl == "reference":
         run_reference(args, spec)
@@ -255,10 +260,11 @@ def main():
         dist.barrier()
 
     flags = {"auto": 0, "simple": TSVD_FLAG_PATH_SIMPLE, "decode": TSVD_FLAG_PATH_DECODE,
-             "tensor": TSVD_FLAG_PATH_TENSOR}[args.path]
+             "tensor": TSVD_FLAG_PATH_TENSOR, "index": binding.TSVD_FLAG_PATH_INDEX}[args.path]
+    pack_flags = binding.TSVD_PACK_INDEX_LISTS if args.path == "index" else 0
     U, V, S = gen.make_weights(spec)
     x_np = gen.make_x(rank_spec(spec, rank))
-    layer = TSVDLinear(U, S, V)
+    layer = TSVDLinear(U, S, V, pack_flags)
     info = layer.info
     from tests._util import torch_x
     x = torch_x(x_np, spec.x_dtype)
@@ -284,7 +290,7 @@ def main():
     n_layers = 1
     if info["packed_bytes"] > pair_bytes:
         n_layers = int(min(64, max(2, -(-2 * l2_bytes // info["packed_bytes"]))))
-    layers = [layer] + [TSVDLinear(U, S, V) for _ in range(1, n_layers)]
+    layers = [layer] + [TSVDLinear(U, S, V, pack_flags) for _ in range(1, n_layers)]
     for i, extra in enumerate(layers[1:]):       # size their scratch outside any timed region
         extra.forward(xs[0], out=ys[0], flags=flags)
 
@@ -381,7 +387,17 @@ def main():
     dom = int(np.argmax(stage_ms))
     dom_ms = stage_ms[dom] / max(1, stage_n[dom])
     pad = lambda v: (v + 127) // 128 * 128
-    if dom in (1, 3) and plan["path"] == "decode":
+    if dom in (1, 3) and plan["path"] == "index":
+        # an index-list stage streams its row pointers and 16-bit entries once
+        v_bytes, u_bytes = binding.tsvd_index_bytes(layer.handle)
+        byts = float(v_bytes if dom == 1 else u_bytes)
+        achieved = byts / (dom_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": binding.STAGE_NAMES[dom] + "_index", "achieved": achieved,
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                    "traffic": None, "peak_source": f"{peaks_src} (of measured)", "bytes_per_launch": byts,
+                    "step_hbm_gbs": (v_bytes + u_bytes) / (ms_per_step * 1e-3) / 1e9}
+        roofline["step_hbm_frac"] = roofline["step_hbm_gbs"] / peaks["hbm_gbs"]
+    elif dom in (1, 3) and plan["path"] == "decode":
         # a decode stage streams its packed matrix once: 2 bits per entry of the padded matrix
         rows, contr = ((pad(spec.K), pad(spec.N)) if dom == 1 else (pad(spec.M), pad(spec.K)))
         byts = rows * contr / 4.0
@@ -433,7 +449,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": "int32" if plan["path"] in ("tensor", "decode") else {"f32": "f32", "bf16": "f32", "i8": "int32"}[spec.x_dtype],
+            "dtype": "int64" if plan["path"] == "index" else "int32" if plan["path"] in ("tensor", "decode") else {"f32": "f32", "bf16": "f32", "i8": "int32"}[spec.x_dtype],
             "data": "synthetic",
             "config": workload_config(spec, l2_note),
             "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks,

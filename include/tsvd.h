@@ -47,6 +47,8 @@ typedef enum {
 #define TSVD_FLAG_PATH_SIMPLE 0x10u /* force the CUDA-core reference kernels               */
 #define TSVD_FLAG_PATH_DECODE 0x20u /* force the decode kernels (B <= TSVD_DECODE_MAX_B)    */
 #define TSVD_FLAG_PATH_TENSOR 0x40u /* force the tcgen05 tensor-core kernels               */
+#define TSVD_FLAG_PATH_INDEX 0x80u  /* run the index-list kernels (see TSVD_PACK_INDEX_LISTS) */
+#define TSVD_FLAG_PATH_MASK 0xF0u   /* at most one of the four may be set                     */
 /* The decode kernels (two launches, one per stage; each CTA streams 32 rows of the packed
  * codes against fixed-point digits of the stage's input held in shared memory) serve batches
  * of at most this many tokens, and are what a forward of so few tokens runs by default.
@@ -60,6 +62,16 @@ typedef enum {
  * context and the handle stay usable. */
 #define TSVD_FLAG_TEST_STALL 0x100u
 
+/* tsvd_pack flag: also keep U and V as index lists -- per row the list of its nonzeros, 16
+ * bits each, (column << 1) | (1 for -1) -- for forwards of up to TSVD_DECODE_MAX_B tokens with
+ * TSVD_FLAG_PATH_INDEX.  The paper calls 2 bits per element a redundant code for sparse U
+ * and V (Section "Connection with BNN and What Next"); this form is the smaller one below a
+ * nonzero rate of 1/8 and its forward does exactly the additions of Table S1, one per nonzero.
+ * It is run on request only (never chosen by default); a forward that asks for it on a handle
+ * packed without it, or for more tokens, returns TSVD_E_TOOBIG. */
+#define TSVD_PACK_INDEX_LISTS 0x1u
+#define TSVD_INDEX_MAX_COLUMNS 32768 /* a column index has 15 bits */
+
 /*
  * tsvd_pack -- store U and V in the 2-bit sign/nonzero form (the paper: "we only
  * need 2 bits to store each element of a ternary matrix", Section "Connection with
@@ -68,12 +80,14 @@ typedef enum {
  *
  *   U  host, int8 [M,K] row-major        V  host, int8 [K,N] row-major
  *   S  host, float [K] (any finite values: negative, zero, unsorted are all fine)
- *   flags  must be 0
+ *   flags  0, or TSVD_PACK_INDEX_LISTS
  *   out    receives the handle; device memory lives on the current CUDA device
  *
  * The inputs are copied; the caller keeps ownership of U, S, V.  Any M,K,N >= 1:
  * ragged sizes are padded with zero entries, which contribute nothing.
- * Synchronous.  Errors: E_NULL, E_SHAPE, E_VALUE (nothing is kept), E_NOMEM, E_CUDA.
+ * Synchronous.  Errors: E_NULL, E_SHAPE, E_VALUE (nothing is kept), E_NOMEM, E_CUDA,
+ * E_DTYPE (unknown flag), E_TOOBIG (index lists asked for with N or K above
+ * TSVD_INDEX_MAX_COLUMNS).
  */
 tsvd_status_t tsvd_pack(const int8_t* U, const float* S, const int8_t* V, int M, int K, int N,
                         unsigned flags, tsvd_handle_t* out);
@@ -158,13 +172,17 @@ tsvd_status_t tsvd_last_status(tsvd_handle_t h);
 tsvd_status_t tsvd_info(tsvd_handle_t h, int* M, int* K, int* N, size_t* packed_bytes,
                         double* density_u, double* density_v);
 
+/* Bytes of the index-list form of V and of U (row pointers + 16-bit entries: what an
+ * index-list forward streams); 0 for a handle packed without TSVD_PACK_INDEX_LISTS. */
+tsvd_status_t tsvd_index_bytes(tsvd_handle_t h, size_t* v_bytes, size_t* u_bytes);
+
 /* Inverse of tsvd_pack, for tests: writes the stored U [M,K], V [K,N] (int8) and
  * S [K] back to HOST buffers (any of them may be NULL). */
 tsvd_status_t tsvd_unpack(tsvd_handle_t h, int8_t* U, float* S, int8_t* V);
 
 /*
  * tsvd_plan -- which kernels a forward with these arguments would run (no launch).
- *   path  receives TSVD_FLAG_PATH_SIMPLE, _DECODE or _TENSOR
+ *   path  receives TSVD_FLAG_PATH_SIMPLE, _DECODE, _TENSOR or _INDEX
  *   digits_x, digits_t  receive the number of signed 8-bit digits the tensor-core and
  *   decode paths use for the activations and for S*(V x) (0 on the CUDA-core path).  Executed tensor
  *   operations per forward = 2*B*(K*N*digits_x + M*K*digits_t) on the padded shapes; the

@@ -15,8 +15,8 @@ from .binding import (DTYPES, TSVD_BF16, TSVD_F32, TSVD_I8, TSVD_FLAG_OUT_F32,  
 class TSVDLinear:
     """A packed TSVD layer living on the current CUDA device."""
 
-    def __init__(self, U, S, V):
-        self.handle = binding.tsvd_pack(U, S, V)
+    def __init__(self, U, S, V, pack_flags: int = 0):
+        self.handle = binding.tsvd_pack(U, S, V, pack_flags)
         self.info = binding.tsvd_info(self.handle)
 
     @staticmethod

@@ -25,13 +25,16 @@ TSVD_FLAG_PATH_SIMPLE = 0x10
 TSVD_FLAG_PATH_DECODE = 0x20
 TSVD_DECODE_MAX_B = 4        # largest batch the decode kernels serve (tsvd.h)
 TSVD_FLAG_PATH_TENSOR = 0x40
+TSVD_FLAG_PATH_INDEX = 0x80      # index-list kernels, for handles packed with TSVD_PACK_INDEX_LISTS
+TSVD_PACK_INDEX_LISTS = 0x1      # tsvd_pack flag
+TSVD_INDEX_MAX_COLUMNS = 32768
 TSVD_FLAG_TEST_STALL = 0x100
 
 DTYPES = {"f32": TSVD_F32, "bf16": TSVD_BF16, "i8": TSVD_I8}
 
 # every symbol include/tsvd.h declares
 EXPORTS = ("tsvd_pack", "tsvd_forward", "tsvd_forward_ex", "tsvd_forward_host", "tsvd_forward_static",
-           "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
+           "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_index_bytes", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
            "tsvd_launch_count", "tsvd_destroy", "tsvd_strerror")
 
 _lib: Optional[ctypes.CDLL] = None
@@ -68,6 +71,8 @@ def lib() -> ctypes.CDLL:
                                 ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_double),
                                 ctypes.POINTER(ctypes.c_double)]
         L.tsvd_info.restype = ci
+        L.tsvd_index_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+        L.tsvd_index_bytes.restype = ci
         L.tsvd_unpack.argtypes = [vp, vp, vp, vp]
         L.tsvd_unpack.restype = ci
         L.tsvd_plan.argtypes = [vp, ci, ci, cu, ctypes.POINTER(cu), ctypes.POINTER(ci), ctypes.POINTER(ci)]
@@ -161,13 +166,20 @@ def tsvd_unpack(h: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     return U, S, V
 
 
+def tsvd_index_bytes(h: int):
+    """(bytes of V's index lists, bytes of U's); zeros when the handle has none."""
+    v, u = ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib().tsvd_index_bytes(h, ctypes.byref(v), ctypes.byref(u)), "tsvd_index_bytes")
+    return v.value, u.value
+
+
 def tsvd_plan(h: int, B: int, dtype: int, flags: int = 0) -> dict:
     """The dispatch decision for a forward with these arguments (nothing is launched)."""
     path, dx, dt = ctypes.c_uint(), ctypes.c_int(), ctypes.c_int()
     _check(lib().tsvd_plan(h, B, dtype, flags, ctypes.byref(path), ctypes.byref(dx), ctypes.byref(dt)),
            "tsvd_plan")
     name = {TSVD_FLAG_PATH_SIMPLE: "simple", TSVD_FLAG_PATH_DECODE: "decode",
-            TSVD_FLAG_PATH_TENSOR: "tensor"}[path.value]
+            TSVD_FLAG_PATH_TENSOR: "tensor", TSVD_FLAG_PATH_INDEX: "index"}[path.value]
     return {"path": name, "digits_x": dx.value, "digits_t": dt.value}
 
 

@@ -88,6 +88,10 @@ static void free_handle(tsvd_handle_s* h)
     if (h->V.units) cudaFree(h->V.units);
     if (h->U.units) cudaFree(h->U.units);
     if (h->S) cudaFree(h->S);
+    for (IndexMat* im : {&h->Vi, &h->Ui}) {
+        if (im->row_ptr) cudaFree(im->row_ptr);
+        if (im->entries) cudaFree(im->entries);
+    }
     if (h->ws) cudaFree(h->ws);
     if (h->io) cudaFree(h->io);
     if (h->dev_status) cudaFree(h->dev_status);
@@ -113,7 +117,8 @@ extern "C" tsvd_status_t tsvd_pack(const int8_t* U, const float* S, const int8_t
     *out = nullptr;
     if (!U || !S || !V) return TSVD_E_NULL;
     if (M < 1 || K < 1 || N < 1) return TSVD_E_SHAPE;
-    if (flags != 0) return TSVD_E_DTYPE;
+    if (flags & ~TSVD_PACK_INDEX_LISTS) return TSVD_E_DTYPE;
+    if ((flags & TSVD_PACK_INDEX_LISTS) && (N > TSVD_INDEX_MAX_COLUMNS || K > TSVD_INDEX_MAX_COLUMNS)) return TSVD_E_TOOBIG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return TSVD_E_CUDA; }
 
@@ -133,6 +138,10 @@ extern "C" tsvd_status_t tsvd_pack(const int8_t* U, const float* S, const int8_t
             st = TSVD_E_CUDA; break;
         }
         if (flag) { st = TSVD_E_VALUE; break; }
+        if (flags & TSVD_PACK_INDEX_LISTS) {
+            if ((st = tsvd_build_index_lists(V, K, N, &h->Vi)) != TSVD_OK) break;
+            if ((st = tsvd_build_index_lists(U, M, K, &h->Ui)) != TSVD_OK) break;
+        }
         const size_t s_len = (size_t)h->V.R_pad;
         if (cudaMalloc(&h->S, s_len * sizeof(float)) != cudaSuccess) { st = TSVD_E_NOMEM; break; }
         if (cudaMemset(h->S, 0, s_len * sizeof(float)) != cudaSuccess) { st = TSVD_E_CUDA; break; }
@@ -160,6 +169,14 @@ extern "C" tsvd_status_t tsvd_info(tsvd_handle_t h, int* M, int* K, int* N, size
     if (packed_bytes) *packed_bytes = h->U.bytes() + h->V.bytes() + (size_t)h->K * sizeof(float);
     if (density_u) *density_u = (double)h->U.nnz / ((double)h->M * (double)h->K);
     if (density_v) *density_v = (double)h->V.nnz / ((double)h->K * (double)h->N);
+    return TSVD_OK;
+}
+
+extern "C" tsvd_status_t tsvd_index_bytes(tsvd_handle_t h, size_t* v_bytes, size_t* u_bytes)
+{
+    if (!h) return TSVD_E_NULL;
+    if (v_bytes) *v_bytes = h->Vi.bytes();
+    if (u_bytes) *u_bytes = h->Ui.bytes();
     return TSVD_OK;
 }
 
@@ -207,11 +224,13 @@ static tsvd_status_t ensure_ws(tsvd_handle_s* h, size_t bytes)
 // The dispatch rule shared by tsvd_plan and tsvd_forward_ex.  Up to TSVD_DECODE_MAX_B tokens run
 // the decode kernels when the digits of the stage inputs fit in shared memory; everything else
 // runs the tensor-core kernels (which serve every batch size); the CUDA-core kernels remain as
-// the plain reference path, on request.  Returns 0 when a forced path cannot serve the request.
+// the plain reference path, and the index-list kernels (handles packed with index lists, up to
+// TSVD_DECODE_MAX_B tokens) are run on request.  Returns 0 when a forced path cannot serve the request.
 static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, unsigned forced)
 {
     if (forced == TSVD_FLAG_PATH_SIMPLE) return TSVD_FLAG_PATH_SIMPLE;
     if (forced == TSVD_FLAG_PATH_TENSOR) return TSVD_FLAG_PATH_TENSOR;
+    if (forced == TSVD_FLAG_PATH_INDEX) return tsvd_index_fits(h, B) ? TSVD_FLAG_PATH_INDEX : 0u;
     const bool fits = tsvd_decode_fits(h, B, dtype);
     if (forced == TSVD_FLAG_PATH_DECODE) return fits ? TSVD_FLAG_PATH_DECODE : 0u;
     return fits ? TSVD_FLAG_PATH_DECODE : TSVD_FLAG_PATH_TENSOR;
@@ -223,11 +242,12 @@ extern "C" tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, u
     if (!h) return TSVD_E_NULL;
     if (B < 1) return TSVD_E_SHAPE;
     if (dtype_size(dtype) == 0) return TSVD_E_DTYPE;
-    const unsigned forced = flags & (TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR);
+    const unsigned forced = flags & TSVD_FLAG_PATH_MASK;
     if (forced & (forced - 1)) return TSVD_E_DTYPE;
     const unsigned p = choose_path(h, B, dtype, forced);
     if (p == 0u) return TSVD_E_TOOBIG;
     if (path) *path = p;
+    // the index-list kernels quantise by the same rule (as many bytes, not split into digits)
     if (digits_x) *digits_x = (p != TSVD_FLAG_PATH_SIMPLE) ? tsvd_tensor_digits_x(dtype) : 0;
     if (digits_t) *digits_t = (p != TSVD_FLAG_PATH_SIMPLE) ? tsvd_tensor_digits_t() : 0;
     return TSVD_OK;
@@ -240,10 +260,9 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     if (B < 1) return TSVD_E_SHAPE;
     const size_t xs = dtype_size(dtype);
     if (xs == 0) return TSVD_E_DTYPE;
-    const unsigned known = TSVD_FLAG_OUT_F32 | TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR |
-                           TSVD_FLAG_TEST_STALL;
+    const unsigned known = TSVD_FLAG_OUT_F32 | TSVD_FLAG_PATH_MASK | TSVD_FLAG_TEST_STALL;
     if (flags & ~known) return TSVD_E_DTYPE;
-    const unsigned path = flags & (TSVD_FLAG_PATH_SIMPLE | TSVD_FLAG_PATH_DECODE | TSVD_FLAG_PATH_TENSOR);
+    const unsigned path = flags & TSVD_FLAG_PATH_MASK;
     if (path & (path - 1)) return TSVD_E_DTYPE;  // at most one forced path
     if (ldx < h->N || ldy < h->M) return TSVD_E_SHAPE;
     if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)z_out & 3)) return TSVD_E_ALIGN;
@@ -270,6 +289,11 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
         tsvd_status_t st = ensure_ws(h, tsvd_decode_ws_bytes(h, B));
         if (st != TSVD_OK) return st;
         return tsvd_forward_decode(a, h->ws);
+    }
+    if (chosen == TSVD_FLAG_PATH_INDEX) {
+        tsvd_status_t st = ensure_ws(h, tsvd_decode_ws_bytes(h, B));   // the same t [B][K padded]
+        if (st != TSVD_OK) return st;
+        return tsvd_forward_index(a, h->ws);
     }
     tsvd_status_t st = ensure_ws(h, tsvd_simple_ws_bytes(h, B));
     if (st != TSVD_OK) return st;

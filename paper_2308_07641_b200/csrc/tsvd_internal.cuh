@@ -40,6 +40,15 @@ struct PackedMat {
     size_t bytes() const { return n_units * sizeof(uint4); }
 };
 
+// Index-list form of a ternary matrix (index.cu): per row the list of its nonzeros.
+struct IndexMat {
+    int* row_ptr = nullptr;        // device, [R + 1]
+    uint16_t* entries = nullptr;   // device, [nnz]: (column << 1) | (1 if the entry is -1)
+    int R = 0, C = 0, C_pad = 0;
+    size_t nnz = 0;
+    size_t bytes() const { return row_ptr ? ((size_t)R + 1) * sizeof(int) + nnz * sizeof(uint16_t) : 0; }
+};
+
 __host__ __device__ inline size_t tsvd_unit_index(int row, int col_group, int C_pad)
 {
     return ((size_t)(row >> 7) * (size_t)(C_pad >> 6) + (size_t)col_group) * 128 + (size_t)(row & 127);
@@ -83,6 +92,7 @@ struct tsvd_handle_s {
     PackedMat V;          // rows K, contraction N
     PackedMat U;          // rows M, contraction K
     float* S = nullptr;   // device, length V.R_pad (zero padded)
+    IndexMat Vi, Ui;      // only with TSVD_PACK_INDEX_LISTS
     // scratch shared by all forwards on this handle
     void* ws = nullptr;
     size_t ws_bytes = 0;
@@ -156,6 +166,11 @@ int tsvd_tensor_digits_t();
 bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt);
 size_t tsvd_decode_ws_bytes(const tsvd_handle_s* h, int B);
 tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws);
+
+// index.cu -- index-list form for very sparse rows, one to four tokens
+tsvd_status_t tsvd_build_index_lists(const int8_t* host, int R, int C, IndexMat* out);
+bool tsvd_index_fits(const tsvd_handle_s* h, int B);
+tsvd_status_t tsvd_forward_index(const ForwardArgs& a, void* ws);
 
 #define TSVD_CUDA_OK(expr)                            \
     do {                                              \

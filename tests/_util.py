@@ -74,12 +74,12 @@ def check_outputs(y64: np.ndarray, z, ref: "oracle.OracleResult", x_dtype: str, 
     return out
 
 
-def run_and_check(spec: "gen.CaseSpec", flags: int = 0, sample_tokens=None):
+def run_and_check(spec: "gen.CaseSpec", flags: int = 0, sample_tokens=None, pack_flags: int = 0):
     """Build the case, run it on the GPU at full batch, compare (all tokens, or a sample)."""
     from paper_2308_07641_b200 import TSVDLinear
     U, V, S = gen.make_weights(spec)
     x = gen.make_x(spec)
-    layer = TSVDLinear(U, S, V)
+    layer = TSVDLinear(U, S, V, pack_flags)
     try:
         y64, z, y_bf16 = run_gpu(layer, x, spec.x_dtype, flags)
     finally:

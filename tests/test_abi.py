@@ -48,6 +48,11 @@ def test_constants_match_the_header(binding):
     assert define("TSVD_FLAG_PATH_SIMPLE") == binding.TSVD_FLAG_PATH_SIMPLE
     assert define("TSVD_FLAG_PATH_TENSOR") == binding.TSVD_FLAG_PATH_TENSOR
     assert define("TSVD_FLAG_OUT_F32") == binding.TSVD_FLAG_OUT_F32
+    assert define("TSVD_FLAG_PATH_INDEX") == binding.TSVD_FLAG_PATH_INDEX
+    assert define("TSVD_PACK_INDEX_LISTS") == binding.TSVD_PACK_INDEX_LISTS
+    assert define("TSVD_INDEX_MAX_COLUMNS") == binding.TSVD_INDEX_MAX_COLUMNS
+    assert define("TSVD_FLAG_PATH_MASK") == (binding.TSVD_FLAG_PATH_SIMPLE | binding.TSVD_FLAG_PATH_DECODE |
+                                            binding.TSVD_FLAG_PATH_TENSOR | binding.TSVD_FLAG_PATH_INDEX)
 
 
 def test_strerror_covers_all_codes(binding):
