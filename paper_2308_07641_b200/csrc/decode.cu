@@ -10,8 +10,9 @@
 // of codes expanded to int8 in registers (two byte permutes per eight entries), the B operand 32
 // columns x 8 (token, digit) pairs read from shared memory, so one instruction does the work of
 // 128 four-way dot products and the instruction count per code is set by the expansion alone
-// (9 per 16 entries).  A per-lane dot-product kernel was bound by exactly that arithmetic:
-// 1.8 us per token and stage on a 4096 x 4096 matrix against 0.65 us to stream it.  All sums are
+// (9 per 16 entries).  A per-lane dot-product kernel issued four dot products per 16 entries,
+// token and digit on top of that: 1.8 us per token and stage on a 4096 x 4096 matrix against
+// 0.65 us to stream it.  All sums are
 // exact integers, so the result does not depend on how the columns are split over the warps.
 //
 // Column order inside an MMA: a thread (row group g = lane / 4, quarter q = lane % 4) loads word q
@@ -71,8 +72,13 @@ __device__ __forceinline__ uint32_t ld_stream_now(const uint32_t* ptr)
 // grid: R_pad / 32 CTAs of 512 threads.  Dynamic shared memory:
 //   digits [NTOK*ND][C_pad + 64] int8 | sums [NTOK*ND][32 rows] int32 |
 //   scale [NTOK] | per-warp maxima [NTOK][warps]
+// Registers: at one token the kernel stays within 64 per thread, so that two CTAs fit an SM: that
+// is what lets the next kernel's CTAs start, and request their codes, while this kernel still runs
+// (a variant that needed 67 took 7.9 instead of 6.2 us per forward).  With more tokens the
+// conversion's working set does not fit 64 registers (capped, it spilled: 16.6 and 22 us at four
+// tokens against 9.6), so those run one CTA per SM.
 template <typename IN_T, int ND, int NTOK, int STAGE>
-__global__ void __launch_bounds__(GEMV_THREADS)
+__global__ void __launch_bounds__(GEMV_THREADS, NTOK == 1 ? 2 : 1)
 ternary_gemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
