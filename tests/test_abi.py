@@ -92,3 +92,25 @@ def test_product_does_not_import_the_checker():
             if fn.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, fn)).read()
                 assert "oracle" not in text, f"{fn} mentions the checker"
+
+
+def test_recorded_dram_traffic_is_well_formed():
+    """profiles/dram_traffic.txt: per workload the hashed source files exist, and the lookup bench.py
+    uses returns either the recorded bytes (sources unchanged since the capture) or None."""
+    import importlib.util
+    import json
+    spec = importlib.util.spec_from_file_location("bench_for_test", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+        rec = json.load(f)["workloads"]
+    assert rec
+    for workload, w in rec.items():
+        for name in w["sources"]:
+            assert os.path.exists(os.path.join(ROOT, "paper_2308_07641_b200", "csrc", name))
+        fresh = w["sha1"] == bench.kernel_source_sha1(w["sources"])
+        for stage, byts in w["bytes_per_launch"].items():
+            assert isinstance(byts, int) and byts > 0
+            assert bench.recorded_traffic(workload, stage) == (byts if fresh else None)
+    assert bench.recorded_traffic("no_such_workload", "v_stage") is None
+

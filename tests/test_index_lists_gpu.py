@@ -93,3 +93,11 @@ def test_index_and_decode_paths_give_the_same_integers():
         assert float((y_idx - y_dec).abs().max()) <= 1e-6 * scale
     finally:
         layer.close()
+
+
+def test_index_lists_at_full_size():
+    """The sparsest workload's layer (4096 x 4096, rank 8192, nonzero rate 0.05) at four int8 tokens:
+    z bit-exact and y within the fp32 tolerance, every element."""
+    spec = gen.scaled(C["cfg5_d05"], name="idx_full_size", B=4)
+    _util.run_and_check(spec, flags=INDEX, pack_flags=LISTS)
+
