@@ -45,10 +45,10 @@ def _load() -> ctypes.CDLL:
         f64p = ctypes.POINTER(ctypes.c_double)
         i64p = ctypes.POINTER(ctypes.c_longlong)
         lib.tsvd_oracle_forward_f64.argtypes = [i8p, f32p, i8p, ctypes.c_int, ctypes.c_int,
-                                                ctypes.c_int, f64p, ctypes.c_int, f64p, f64p, i64p]
+                                                ctypes.c_int, f64p, ctypes.c_int, f32p, f64p, f64p, i64p]
         lib.tsvd_oracle_forward_f64.restype = ctypes.c_int
         lib.tsvd_oracle_forward_i8.argtypes = [i8p, f32p, i8p, ctypes.c_int, ctypes.c_int,
-                                               ctypes.c_int, i8p, ctypes.c_int, f64p, i64p, i64p]
+                                               ctypes.c_int, i8p, ctypes.c_int, f32p, f64p, i64p, i64p]
         lib.tsvd_oracle_forward_i8.restype = ctypes.c_int
         lib.tsvd_oracle_threads.restype = ctypes.c_int
         _lib = lib
@@ -72,11 +72,14 @@ def _ptr(a: np.ndarray, ctype):
     return a.ctypes.data_as(ctypes.POINTER(ctype))
 
 
-def forward(U: np.ndarray, S: np.ndarray, V: np.ndarray, x: np.ndarray) -> OracleResult:
-    """y = U (diag(S) (V x)) for a token-major batch x [B,N].
+def forward(U: np.ndarray, S: np.ndarray, V: np.ndarray, x: np.ndarray,
+            bias: Optional[np.ndarray] = None) -> OracleResult:
+    """y = U (diag(S) (V x)) (+ bias) for a token-major batch x [B,N].
 
     U int8 [M,K], V int8 [K,N], S float32 [K].  x is float64 (already widened
-    exactly from its storage type) or int8 (integer V-stage).
+    exactly from its storage type) or int8 (integer V-stage).  bias: None, or
+    float32 [M] (the converted layer keeps the original layer's bias: the
+    supplement's architecture listing has bias=True on every layer).
     """
     lib = _load()
     U = np.ascontiguousarray(U, dtype=np.int8)
@@ -89,6 +92,12 @@ def forward(U: np.ndarray, S: np.ndarray, V: np.ndarray, x: np.ndarray) -> Oracl
     if x.ndim != 2 or x.shape[1] != N:
         raise ValueError("x must be [B,N]")
     B = x.shape[0]
+    bp = None
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+        if bias.shape != (M,):
+            raise ValueError("bias must be [M]")
+        bp = _ptr(bias, ctypes.c_float)
     y = np.zeros((B, M), dtype=np.float64)
     counts = np.zeros(2, dtype=np.int64)
     if x.dtype == np.int8:
@@ -96,7 +105,7 @@ def forward(U: np.ndarray, S: np.ndarray, V: np.ndarray, x: np.ndarray) -> Oracl
         zraw = np.zeros((B, K), dtype=np.int64)
         rc = lib.tsvd_oracle_forward_i8(_ptr(U, ctypes.c_int8), _ptr(S, ctypes.c_float),
                                         _ptr(V, ctypes.c_int8), M, K, N,
-                                        _ptr(xx, ctypes.c_int8), B, _ptr(y, ctypes.c_double),
+                                        _ptr(xx, ctypes.c_int8), B, bp, _ptr(y, ctypes.c_double),
                                         _ptr(zraw, ctypes.c_longlong),
                                         _ptr(counts, ctypes.c_longlong))
     elif x.dtype == np.float64:
@@ -104,7 +113,7 @@ def forward(U: np.ndarray, S: np.ndarray, V: np.ndarray, x: np.ndarray) -> Oracl
         zraw = np.zeros((B, K), dtype=np.float64)
         rc = lib.tsvd_oracle_forward_f64(_ptr(U, ctypes.c_int8), _ptr(S, ctypes.c_float),
                                          _ptr(V, ctypes.c_int8), M, K, N,
-                                         _ptr(xx, ctypes.c_double), B, _ptr(y, ctypes.c_double),
+                                         _ptr(xx, ctypes.c_double), B, bp, _ptr(y, ctypes.c_double),
                                          _ptr(zraw, ctypes.c_double),
                                          _ptr(counts, ctypes.c_longlong))
     else:

@@ -14,6 +14,11 @@
  *                                             one per nonzero of V      (row "V(.)")
  *   S-stage   z[k]    = S[k] * zraw[k]        K multiplications         (row "diag(s)(.)")
  *   U-stage   y[m]    = sum_k U[m,k] z[k]     one add/sub per nonzero   (row "U(.)")
+ *   bias      y[m]   += b[m]                  optional.  Eq. 1 is written "without any
+ *                                             bias", yet every layer of the supplement's
+ *                                             architecture listing has bias=True: the
+ *                                             converted layer keeps the original layer's
+ *                                             bias, one addition per output.
  *
  * Floating-point activations are accumulated in IEEE double in index order.
  * int8 activations take the V-stage in 64-bit integers (exact), then the
@@ -52,12 +57,13 @@ static int check_ternary(const int8_t* A, long long n)
 }
 
 /*
- * counts (optional, length 2): counts[0] = additions+subtractions performed,
- * counts[1] = multiplications performed, summed over all B columns.
+ * counts (optional, length 2): counts[0] = additions+subtractions performed
+ * (the bias additions included when there is a bias), counts[1] = multiplications
+ * performed, summed over all B columns.  bias: NULL, or M single-precision values.
  */
 int tsvd_oracle_forward_f64(const int8_t* U, const float* S, const int8_t* V,
                             int M, int K, int N,
-                            const double* x, int B,
+                            const double* x, int B, const float* bias,
                             double* y, double* zraw_out, long long* counts)
 {
     if (check_ternary(U, (long long)M * K) || check_ternary(V, (long long)K * N)) return 1;
@@ -93,6 +99,7 @@ int tsvd_oracle_forward_f64(const int8_t* U, const float* S, const int8_t* V,
                 if (urow[k] == 1) { acc += zb[k]; ++adds; }
                 else if (urow[k] == -1) { acc -= zb[k]; ++adds; }
             }
+            if (bias) { acc += (double)bias[m]; ++adds; }
             y[(size_t)b * M + m] = acc;
         }
     }
@@ -104,7 +111,7 @@ int tsvd_oracle_forward_f64(const int8_t* U, const float* S, const int8_t* V,
 /* int8 activations: zraw_out (optional) receives the exact integer V x as int64. */
 int tsvd_oracle_forward_i8(const int8_t* U, const float* S, const int8_t* V,
                            int M, int K, int N,
-                           const int8_t* x, int B,
+                           const int8_t* x, int B, const float* bias,
                            double* y, long long* zraw_out, long long* counts)
 {
     if (check_ternary(U, (long long)M * K) || check_ternary(V, (long long)K * N)) return 1;
@@ -138,6 +145,7 @@ int tsvd_oracle_forward_i8(const int8_t* U, const float* S, const int8_t* V,
                 if (urow[k] == 1) { acc += zb[k]; ++adds; }
                 else if (urow[k] == -1) { acc -= zb[k]; ++adds; }
             }
+            if (bias) { acc += (double)bias[m]; ++adds; }
             y[(size_t)b * M + m] = acc;
         }
     }

@@ -93,15 +93,47 @@ def test_exact_rational(seed):
 def test_handworked_golden():
     with open(os.path.join(GOLDEN, "handworked_forward.json")) as f:
         data = json.load(f)
-    assert len(data["cases"]) >= 3
+    assert len(data["cases"]) >= 4
     for c in data["cases"]:
         U = np.array(c["U"], dtype=np.int8)
         V = np.array(c["V"], dtype=np.int8)
         S = np.array(c["S"], dtype=np.float32)
         x = np.array(c["x"], dtype=np.float64)
-        res = oracle.forward(U, S, V, x)
+        bias = np.array(c["bias"], dtype=np.float32) if "bias" in c else None
+        res = oracle.forward(U, S, V, x, bias)
         assert np.array_equal(res.zraw, np.array(c["zraw"])), c["name"]
         assert np.array_equal(res.y, np.array(c["y"])), c["name"]
+
+
+# bias (the supplement's architecture listing keeps bias=True on every converted layer): one
+# addition per output after the U-stage, pinned by the dense form W' x + b, exact rationals, the
+# hand-worked case above, the int8 entry point and the operation count
+@pytest.mark.parametrize("seed", range(6))
+def test_bias_dense_and_exact(seed):
+    g = np.random.default_rng(50 + seed)
+    M, K, N, B = (int(g.integers(1, 9)) for _ in range(4))
+    U, S, V, x = _rand_case(2000 + seed, M, K, N, B)
+    bias = g.integers(-40, 41, size=M).astype(np.float32) / 8.0
+    res = oracle.forward(U, S, V, x, bias)
+    ref = _dense(U, S, V, x) + bias.astype(np.float64)[None, :]
+    assert np.abs(res.y - ref).max() <= 1e-12 * max(1.0, np.abs(ref).max())
+    # the bias enters after everything else: exactly the no-bias result plus b, and nowhere else
+    plain = oracle.forward(U, S, V, x)
+    assert np.array_equal(res.y, plain.y + bias.astype(np.float64)[None, :])
+    assert np.array_equal(res.zraw, plain.zraw)
+    assert res.adds == plain.adds + B * M and res.muls == plain.muls
+    # integer activations, dyadic S and bias: exact rational evaluation
+    xi = g.integers(-100, 101, size=(B, N)).astype(np.int8)
+    Sf = [Fraction(int(g.integers(-64, 65)), 32) for _ in range(K)]
+    S2 = np.array([float(f) for f in Sf], dtype=np.float32)
+    r8 = oracle.forward(U, S2, V, xi, bias)
+    for b in range(B):
+        for m in range(M):
+            yv = sum(int(U[m, k]) * Sf[k] * sum(int(V[k, n]) * int(xi[b, n]) for n in range(N))
+                     for k in range(K)) + Fraction(float(bias[m]))
+            assert Fraction(r8.y[b, m]) == yv
+    with pytest.raises(ValueError):
+        oracle.forward(U, S, V, x, np.zeros(M + 1, np.float32))
 
 
 # P4 -- Winograd minimal filtering is a lossless TSVD (Section "Connection with Winograd",
