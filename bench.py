@@ -151,16 +151,15 @@ class ClockSampler:
 def cpu_baseline(spec, U, S, V, x_np, target_s=8.0, y_gpu=None):
     """Time the CPU checker, as it stands, on a bounded sample of the workload's tokens."""
     import oracle
-    from tests import _util
     cores = oracle.threads()
     n0 = min(spec.B, max(cores, 8))
-    xs = _util.oracle_x(x_np[:n0], spec.x_dtype)
+    xs = gen.widen_x(x_np[:n0], spec.x_dtype)
     oracle.forward(U, S, V, xs[:1])                      # warm-up (page in, thread pool)
     t0 = time.perf_counter(); oracle.forward(U, S, V, xs); t1 = time.perf_counter()
     per_tok = (t1 - t0) / n0
     n = int(min(spec.B, max(n0, target_s / max(per_tok, 1e-9))))
     n = max(cores, n - n % cores) if n >= cores else n
-    xs = _util.oracle_x(x_np[:n], spec.x_dtype)
+    xs = gen.widen_x(x_np[:n], spec.x_dtype)
     t0 = time.perf_counter(); ref = oracle.forward(U, S, V, xs); t1 = time.perf_counter()
     out = {"value": n / (t1 - t0), "unit": UNIT, "cores": cores, "kind": "oracle",
            "sample": f"first {n} of {spec.B} tokens of {spec.name}, one call, {t1 - t0:.2f} s wall"}
@@ -181,18 +180,17 @@ def run_reference(args, spec):
     if rank != 0:
         return
     import oracle
-    from tests import _util
     U, V, S = gen.make_weights(spec)
     cores = oracle.threads()
     # size the per-step sample so that warmup+steps stay within about two minutes
     x_probe = gen.make_x(spec, 0, min(spec.B, cores))
-    xp = _util.oracle_x(x_probe, spec.x_dtype)
+    xp = gen.widen_x(x_probe, spec.x_dtype)
     oracle.forward(U, S, V, xp[:1])
     t0 = time.perf_counter(); oracle.forward(U, S, V, xp); per_tok = (time.perf_counter() - t0) / len(xp)
     budget = 100.0 / max(1, args.steps + args.warmup)
     n = int(min(spec.B, max(cores, budget / max(per_tok, 1e-9))))
     n = max(1, n - n % cores) if n >= cores else n
-    x = _util.oracle_x(gen.make_x(spec, 0, n), spec.x_dtype)
+    x = gen.widen_x(gen.make_x(spec, 0, n), spec.x_dtype)
     for _ in range(args.warmup):
         oracle.forward(U, S, V, x)
     t0 = time.perf_counter()
@@ -266,8 +264,8 @@ def main():
     x_np = gen.make_x(rank_spec(spec, rank))
     layer = TSVDLinear(U, S, V, pack_flags)
     info = layer.info
-    from tests._util import torch_x
-    x = torch_x(x_np, spec.x_dtype)
+    from paper_2308_07641_b200 import device_activations
+    x = device_activations(x_np, spec.x_dtype)
     y = layer.forward(x, flags=flags)
     torch.cuda.synchronize()
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")

@@ -128,6 +128,32 @@ def make_x(spec: CaseSpec, b_start: int = 0, b_count: int | None = None) -> np.n
     raise ValueError(spec.x_dtype)
 
 
+def widen_x(x: np.ndarray, x_dtype: str) -> np.ndarray:
+    """The stored activations as the array a double-precision consumer takes: bf16 bit patterns
+    and fp32 widened exactly to float64, int8 left as it is."""
+    if x_dtype == "bf16":
+        return rng.bf16_bits_to_f32(x).astype(np.float64)
+    if x_dtype == "i8":
+        return x
+    return x.astype(np.float64)
+
+
+def set_entries(x: np.ndarray, x_dtype: str, tokens, cols, value: float) -> np.ndarray:
+    """A copy of the stored activations x [B,N] with x[tokens, cols] = value (outliers, zeros,
+    extreme int8 codes); `value` must be representable in the storage type."""
+    out = x.copy()
+    tokens = np.atleast_1d(np.asarray(tokens))
+    cols = np.atleast_1d(np.asarray(cols))
+    if x_dtype == "bf16":
+        bits = rng.f32_to_bf16_bits(np.array([value], dtype=np.float32))[0]
+        if float(rng.bf16_bits_to_f32(np.array([bits], dtype=np.uint16))[0]) != float(value):
+            raise ValueError("value is not a bf16 number")
+        out[np.ix_(tokens, cols)] = bits
+    else:
+        out[np.ix_(tokens, cols)] = np.asarray(value).astype(out.dtype)
+    return out
+
+
 def make_case(spec: CaseSpec) -> Case:
     U, V, S = make_weights(spec)
     return Case(spec=spec, U=U, V=V, S=S, x=make_x(spec))

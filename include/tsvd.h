@@ -13,6 +13,26 @@
  * thrown across the boundary; arguments are validated on the host before any
  * kernel is launched.  There is no CPU implementation behind these calls: without
  * a CUDA device they return TSVD_E_CUDA.
+ *
+ * Arithmetic of the fast kernels (tensor-core, decode and index-list paths), which is
+ * what bounds their accuracy.  Per token, the activations are rounded once to a
+ * multiple of 2^(E-22) (bf16 activations; 2^(E-30) with TSVD_FLAG_WIDE_X) or 2^(E-30)
+ * (fp32 activations), where 2^E is the power of two just above the token's largest
+ * magnitude; int8 activations are used as they are.  From there the V-stage is exact
+ * integer arithmetic (z = V x is bit-exact for int8 activations), t = S * z is one fp32
+ * product per rank component, t is rounded likewise to a multiple of 2^(E_t-30), the
+ * U-stage is exact again, and y is rounded once to its output type.  Consequences:
+ *   - activations must be finite (NaN and Inf are not detected; y is then unspecified);
+ *   - entries far below a token's largest magnitude lose bits: an entry 2^-s of the
+ *     largest keeps 22-s (30-s) bits.  With the bulk of a bf16 token within 2^8 of its
+ *     largest entry (2^16 with TSVD_FLAG_WIDE_X and for fp32), every output meets
+ *     |y - y_exact| <= 1e-2 |y_exact| + 1e-3 at the value scales of transformer
+ *     activations; a forward that meets a token outside that range reports
+ *     TSVD_E_RANGE through tsvd_last_status (see there), and the CUDA-core path
+ *     (TSVD_FLAG_PATH_SIMPLE: fp32 partial sums per 64 columns, fp64 across) has no
+ *     such limit;
+ *   - a token whose largest magnitude is below 2^-90 is scaled as if it were 2^-90,
+ *     so it loses bits, and below about 2^-120 it is treated as zero.
  */
 #ifndef TSVD_H
 #define TSVD_H
@@ -39,8 +59,14 @@ typedef enum {
     TSVD_E_CUDA = 6,    /* a CUDA runtime call failed (or there is no device)      */
     TSVD_E_TIMEOUT = 7, /* a bounded device-side wait gave up                      */
     TSVD_E_NOMEM = 8,   /* host or device allocation failed                        */
-    TSVD_E_TOOBIG = 9   /* request exceeds a fixed capacity (see tsvd_forward_static) */
+    TSVD_E_TOOBIG = 9,  /* request exceeds a fixed capacity (tsvd_forward_static, TSVD_MAX_CONTRACTION) */
+    TSVD_E_RANGE = 10   /* tsvd_last_status only: a token's dynamic range exceeded what the
+                           fixed-point digits resolve (see the note on arithmetic above)   */
 } tsvd_status_t;
+
+/* Longest contraction (N and K) a handle may have: the digit sums of a row are combined in
+ * 32-bit integers, |sum| <= 128 * 257 * columns, which stays below 2^31 up to here. */
+#define TSVD_MAX_CONTRACTION 65280
 
 /* flags of tsvd_forward_ex */
 #define TSVD_FLAG_OUT_F32 0x1u      /* write y as fp32 even for bf16 activations            */
@@ -49,6 +75,10 @@ typedef enum {
 #define TSVD_FLAG_PATH_TENSOR 0x40u /* force the tcgen05 tensor-core kernels               */
 #define TSVD_FLAG_PATH_INDEX 0x80u  /* run the index-list kernels (see TSVD_PACK_INDEX_LISTS) */
 #define TSVD_FLAG_PATH_MASK 0xF0u   /* at most one of the four may be set                     */
+/* bf16 activations as four signed 8-bit digits (30 bits of the token's range) instead of
+ * three (22 bits): for tokens with outliers up to 2^16 times their bulk.  The V-stage of the
+ * tensor-core path then executes 4/3 of the operations; no effect on fp32 and int8. */
+#define TSVD_FLAG_WIDE_X 0x200u
 /* The decode kernels (two launches, one per stage; each CTA streams 32 rows of the packed
  * codes against fixed-point digits of the stage's input held in shared memory) serve batches
  * of at most this many tokens, and are what a forward of so few tokens runs by default.
@@ -73,10 +103,9 @@ typedef enum {
 #define TSVD_INDEX_MAX_COLUMNS 32768 /* a column index has 15 bits */
 
 /*
- * tsvd_pack -- store U and V in the 2-bit sign/nonzero form (the paper: "we only
- * need 2 bits to store each element of a ternary matrix", Section "Connection with
- * BNN and What Next"; the split U = U+ - U-, V = V+ - V- of the same section) and
- * copy S.
+ * tsvd_pack -- store U and V in a 2-bit sign/nonzero form (two bits per entry are what
+ * the paper says a ternary matrix needs, Section "Connection with BNN and What Next";
+ * the split U = U+ - U-, V = V+ - V- of the same section) and copy S.
  *
  *   U  host, int8 [M,K] row-major        V  host, int8 [K,N] row-major
  *   S  host, float [K] (any finite values: negative, zero, unsorted are all fine)
@@ -105,7 +134,8 @@ tsvd_status_t tsvd_pack(const int8_t* U, const float* S, const int8_t* V, int M,
  * x and y stay owned by the caller and must be 16-byte aligned.  The handle's
  * scratch memory is shared by all calls on it: calls on one handle must be
  * ordered on one stream (or otherwise serialised).  Scratch grows on the first call
- * with a larger B (that call synchronises the device once).
+ * with a larger B (that call synchronises the device once) unless tsvd_reserve has
+ * sized it beforehand.  x must be finite (see the note on arithmetic at the top).
  * Errors: E_NULL, E_SHAPE (B < 1), E_DTYPE, E_ALIGN, E_NOMEM, E_CUDA.
  */
 tsvd_status_t tsvd_forward(tsvd_handle_t h, const void* x, void* y, int B, tsvd_dtype_t dtype,
@@ -162,9 +192,40 @@ tsvd_status_t tsvd_forward_host(tsvd_handle_t h, const void* x, void* y, int B,
 tsvd_status_t tsvd_forward_static(tsvd_handle_t h, const void* x, void* y, int B,
                                   tsvd_dtype_t dtype, void* stream);
 
-/* Device-side error word of the last forward on this handle (read after the
- * stream has been synchronised): TSVD_OK, or TSVD_E_TIMEOUT if a bounded wait
- * inside a kernel gave up.  Resets the word. */
+/*
+ * tsvd_reserve -- size the handle's scratch once, so that no later tsvd_forward /
+ * tsvd_forward_ex with at most B_max tokens of this dtype (any flags, any path)
+ * allocates, frees or synchronises: such forwards can then be captured in a CUDA graph
+ * from the first call on.  Synchronises the device if the scratch has to grow.
+ * (Measurement and deployment support; the paper has no counterpart.)
+ * Errors: E_NULL, E_SHAPE, E_DTYPE, E_NOMEM, E_CUDA.
+ */
+tsvd_status_t tsvd_reserve(tsvd_handle_t h, int B_max, tsvd_dtype_t dtype);
+
+/*
+ * tsvd_set_bias -- y = U(diag(S)(V x)) + b.  Eq. 1 of the paper is written without a bias,
+ * but every layer of its architecture listing (supplement) carries one (`bias=True`); it is
+ * added in fp32 to the U-stage result before the single rounding to the output type.
+ *   bias  host, float [M]; copied.  NULL removes the bias again.
+ * Synchronous; must not be called while a forward on this handle is in flight.
+ * Errors: E_NULL (h), E_NOMEM, E_CUDA.
+ */
+tsvd_status_t tsvd_set_bias(tsvd_handle_t h, const float* bias);
+
+/* Device-side status word of the forwards on this handle since the last read (read after
+ * the stream has been synchronised).  Resets the word.  Returns
+ *   TSVD_E_TIMEOUT if a bounded wait inside a kernel gave up (y is then unspecified), else
+ *   TSVD_E_RANGE   if some token's dynamic range was wider than the fixed-point digits
+ *                  resolve: while converting a stage's input the kernels sample one value
+ *                  in eight, and raise this when, among at least 32 nonzero samples of a
+ *                  token that one warp converted, fewer than a quarter reach 2^12
+ *                  quantisation steps (most entries then keep fewer than 12 bits; for a
+ *                  normally distributed bulk this happens from an outlier of about 2^10
+ *                  times the bulk's scale with three digits, 2^18 with four).  y is still
+ *                  the result of the arithmetic described at the top of this file; rerun
+ *                  with TSVD_FLAG_WIDE_X or TSVD_FLAG_PATH_SIMPLE if it must meet the
+ *                  tolerance;
+ *   TSVD_OK        otherwise. */
 tsvd_status_t tsvd_last_status(tsvd_handle_t h);
 
 /* Shapes, packed size in bytes (U and V codes plus S: the bytes a forward must

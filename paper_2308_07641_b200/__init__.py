@@ -9,7 +9,17 @@ from __future__ import annotations
 from . import binding
 from .binding import (DTYPES, TSVD_BF16, TSVD_F32, TSVD_I8, TSVD_FLAG_OUT_F32,  # noqa: F401
                       TSVD_FLAG_PATH_DECODE, TSVD_FLAG_PATH_SIMPLE, TSVD_FLAG_PATH_TENSOR,
-                      TSVDError)
+                      TSVD_FLAG_WIDE_X, TSVDError)
+
+
+def device_activations(x_np, x_dtype: str):
+    """A host array of stored activations ([B,N] float32, int8, or uint16 holding bf16 bit
+    patterns) as a CUDA tensor of the matching torch dtype.  Marshalling only."""
+    import numpy as np
+    import torch
+    if x_dtype == "bf16":
+        return torch.from_numpy(np.ascontiguousarray(x_np).view(np.int16).copy()).cuda().view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(x_np)).cuda()
 
 
 class TSVDLinear:
@@ -18,6 +28,12 @@ class TSVDLinear:
     def __init__(self, U, S, V, pack_flags: int = 0):
         self.handle = binding.tsvd_pack(U, S, V, pack_flags)
         self.info = binding.tsvd_info(self.handle)
+
+    def set_bias(self, bias) -> None:
+        binding.tsvd_set_bias(self.handle, bias)
+
+    def reserve(self, B_max: int, x_dtype: str) -> None:
+        binding.tsvd_reserve(self.handle, B_max, DTYPES[x_dtype])
 
     @staticmethod
     def _dtype_of(x) -> int:

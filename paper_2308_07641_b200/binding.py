@@ -18,7 +18,8 @@ LIB_PATH = os.path.join(_HERE, "libtsvd.so")
 TSVD_F32, TSVD_BF16, TSVD_I8 = 0, 1, 2
 TSVD_OK = 0
 (TSVD_E_NULL, TSVD_E_SHAPE, TSVD_E_VALUE, TSVD_E_DTYPE, TSVD_E_ALIGN, TSVD_E_CUDA,
- TSVD_E_TIMEOUT, TSVD_E_NOMEM, TSVD_E_TOOBIG) = range(1, 10)
+ TSVD_E_TIMEOUT, TSVD_E_NOMEM, TSVD_E_TOOBIG, TSVD_E_RANGE) = range(1, 11)
+TSVD_MAX_CONTRACTION = 65280
 TSVD_STATIC_SCRATCH_BYTES = 4 << 20
 TSVD_FLAG_OUT_F32 = 0x1
 TSVD_FLAG_PATH_SIMPLE = 0x10
@@ -29,12 +30,13 @@ TSVD_FLAG_PATH_INDEX = 0x80      # index-list kernels, for handles packed with T
 TSVD_PACK_INDEX_LISTS = 0x1      # tsvd_pack flag
 TSVD_INDEX_MAX_COLUMNS = 32768
 TSVD_FLAG_TEST_STALL = 0x100
+TSVD_FLAG_WIDE_X = 0x200         # bf16 activations as four digits (outliers up to 2^16 of the bulk)
 
 DTYPES = {"f32": TSVD_F32, "bf16": TSVD_BF16, "i8": TSVD_I8}
 
 # every symbol include/tsvd.h declares
 EXPORTS = ("tsvd_pack", "tsvd_forward", "tsvd_forward_ex", "tsvd_forward_host", "tsvd_forward_static",
-           "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_index_bytes", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
+           "tsvd_reserve", "tsvd_set_bias", "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_index_bytes", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
            "tsvd_launch_count", "tsvd_destroy", "tsvd_strerror")
 
 _lib: Optional[ctypes.CDLL] = None
@@ -65,6 +67,10 @@ def lib() -> ctypes.CDLL:
         L.tsvd_forward_host.restype = ci
         L.tsvd_forward_static.argtypes = [vp, vp, vp, ci, ci, vp]
         L.tsvd_forward_static.restype = ci
+        L.tsvd_reserve.argtypes = [vp, ci, ci]
+        L.tsvd_reserve.restype = ci
+        L.tsvd_set_bias.argtypes = [vp, vp]
+        L.tsvd_set_bias.restype = ci
         L.tsvd_last_status.argtypes = [vp]
         L.tsvd_last_status.restype = ci
         L.tsvd_info.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci),
@@ -141,6 +147,20 @@ def tsvd_forward_static(h: int, x_ptr: int, y_ptr: int, B: int, dtype: int, stre
     """tsvd_forward without any allocation: the intermediate lives in a fixed array inside the
     library (TSVD_STATIC_SCRATCH_BYTES); larger requests raise with status TSVD_E_TOOBIG."""
     _check(lib().tsvd_forward_static(h, x_ptr, y_ptr, B, dtype, stream or None), "tsvd_forward_static")
+
+
+def tsvd_reserve(h: int, B_max: int, dtype: int) -> None:
+    """Size the handle's scratch for forwards of up to B_max tokens (no allocation afterwards)."""
+    _check(lib().tsvd_reserve(h, B_max, dtype), "tsvd_reserve")
+
+
+def tsvd_set_bias(h: int, bias: Optional[np.ndarray]) -> None:
+    """Attach (or with None remove) a float32 bias [M], added after the U-stage."""
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+        if bias.shape != (tsvd_info(h)["M"],):
+            raise TSVDError(TSVD_E_SHAPE, "tsvd_set_bias")
+    _check(lib().tsvd_set_bias(h, _np_ptr(bias)), "tsvd_set_bias")
 
 
 def tsvd_last_status(h: int) -> int:

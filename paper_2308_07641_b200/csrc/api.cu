@@ -22,7 +22,8 @@ extern "C" const char* tsvd_strerror(tsvd_status_t s)
         case TSVD_E_CUDA: return "CUDA runtime error (or no CUDA device)";
         case TSVD_E_TIMEOUT: return "a bounded device-side wait gave up";
         case TSVD_E_NOMEM: return "out of memory";
-        case TSVD_E_TOOBIG: return "request exceeds the fixed scratch capacity of this entry point";
+        case TSVD_E_TOOBIG: return "request exceeds a fixed capacity (static scratch, contraction length or index width)";
+        case TSVD_E_RANGE: return "a token's dynamic range exceeded what the fixed-point digits resolve";
     }
     return "unknown status";
 }
@@ -88,6 +89,7 @@ static void free_handle(tsvd_handle_s* h)
     if (h->V.units) cudaFree(h->V.units);
     if (h->U.units) cudaFree(h->U.units);
     if (h->S) cudaFree(h->S);
+    if (h->bias) cudaFree(h->bias);
     for (IndexMat* im : {&h->Vi, &h->Ui}) {
         if (im->row_ptr) cudaFree(im->row_ptr);
         if (im->entries) cudaFree(im->entries);
@@ -118,6 +120,8 @@ extern "C" tsvd_status_t tsvd_pack(const int8_t* U, const float* S, const int8_t
     if (!U || !S || !V) return TSVD_E_NULL;
     if (M < 1 || K < 1 || N < 1) return TSVD_E_SHAPE;
     if (flags & ~TSVD_PACK_INDEX_LISTS) return TSVD_E_DTYPE;
+    // the digit sums of a row are combined in 32-bit integers: bound the contraction length
+    if (N > TSVD_MAX_CONTRACTION || K > TSVD_MAX_CONTRACTION) return TSVD_E_TOOBIG;
     if ((flags & TSVD_PACK_INDEX_LISTS) && (N > TSVD_INDEX_MAX_COLUMNS || K > TSVD_INDEX_MAX_COLUMNS)) return TSVD_E_TOOBIG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return TSVD_E_CUDA; }
@@ -196,7 +200,27 @@ extern "C" tsvd_status_t tsvd_last_status(tsvd_handle_t h)
     int word = 0;
     TSVD_CUDA_OK(cudaMemcpy(&word, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost));
     if (word) TSVD_CUDA_OK(cudaMemset(h->dev_status, 0, sizeof(int)));
-    return word ? TSVD_E_TIMEOUT : TSVD_OK;
+    if (word & TSVD_DEV_TIMEOUT) return TSVD_E_TIMEOUT;
+    return (word & TSVD_DEV_RANGE) ? TSVD_E_RANGE : TSVD_OK;
+}
+
+extern "C" tsvd_status_t tsvd_set_bias(tsvd_handle_t h, const float* bias)
+{
+    if (!h) return TSVD_E_NULL;
+    TSVD_CUDA_OK(cudaDeviceSynchronize());
+    if (!bias) {
+        if (h->bias) { cudaFree(h->bias); h->bias = nullptr; }
+        return TSVD_OK;
+    }
+    const size_t len = (size_t)h->U.R_pad;
+    if (!h->bias && cudaMalloc(&h->bias, len * sizeof(float)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        h->bias = nullptr;
+        return TSVD_E_NOMEM;
+    }
+    TSVD_CUDA_OK(cudaMemset(h->bias, 0, len * sizeof(float)));
+    TSVD_CUDA_OK(cudaMemcpy(h->bias, bias, (size_t)h->M * sizeof(float), cudaMemcpyHostToDevice));
+    return TSVD_OK;
 }
 
 static size_t dtype_size(tsvd_dtype_t d)
@@ -226,12 +250,12 @@ static tsvd_status_t ensure_ws(tsvd_handle_s* h, size_t bytes)
 // runs the tensor-core kernels (which serve every batch size); the CUDA-core kernels remain as
 // the plain reference path, and the index-list kernels (handles packed with index lists, up to
 // TSVD_DECODE_MAX_B tokens) are run on request.  Returns 0 when a forced path cannot serve the request.
-static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, unsigned forced)
+static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, unsigned forced, bool wide_x)
 {
     if (forced == TSVD_FLAG_PATH_SIMPLE) return TSVD_FLAG_PATH_SIMPLE;
     if (forced == TSVD_FLAG_PATH_TENSOR) return TSVD_FLAG_PATH_TENSOR;
     if (forced == TSVD_FLAG_PATH_INDEX) return tsvd_index_fits(h, B) ? TSVD_FLAG_PATH_INDEX : 0u;
-    const bool fits = tsvd_decode_fits(h, B, dtype);
+    const bool fits = tsvd_decode_fits(h, B, dtype, wide_x);
     if (forced == TSVD_FLAG_PATH_DECODE) return fits ? TSVD_FLAG_PATH_DECODE : 0u;
     return fits ? TSVD_FLAG_PATH_DECODE : TSVD_FLAG_PATH_TENSOR;
 }
@@ -244,11 +268,12 @@ extern "C" tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, u
     if (dtype_size(dtype) == 0) return TSVD_E_DTYPE;
     const unsigned forced = flags & TSVD_FLAG_PATH_MASK;
     if (forced & (forced - 1)) return TSVD_E_DTYPE;
-    const unsigned p = choose_path(h, B, dtype, forced);
+    const bool wide_x = (flags & TSVD_FLAG_WIDE_X) != 0;
+    const unsigned p = choose_path(h, B, dtype, forced, wide_x);
     if (p == 0u) return TSVD_E_TOOBIG;
     if (path) *path = p;
     // the index-list kernels quantise by the same rule (as many bytes, not split into digits)
-    if (digits_x) *digits_x = (p != TSVD_FLAG_PATH_SIMPLE) ? tsvd_tensor_digits_x(dtype) : 0;
+    if (digits_x) *digits_x = (p != TSVD_FLAG_PATH_SIMPLE) ? tsvd_tensor_digits_x(dtype, wide_x) : 0;
     if (digits_t) *digits_t = (p != TSVD_FLAG_PATH_SIMPLE) ? tsvd_tensor_digits_t() : 0;
     return TSVD_OK;
 }
@@ -260,7 +285,7 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     if (B < 1) return TSVD_E_SHAPE;
     const size_t xs = dtype_size(dtype);
     if (xs == 0) return TSVD_E_DTYPE;
-    const unsigned known = TSVD_FLAG_OUT_F32 | TSVD_FLAG_PATH_MASK | TSVD_FLAG_TEST_STALL;
+    const unsigned known = TSVD_FLAG_OUT_F32 | TSVD_FLAG_PATH_MASK | TSVD_FLAG_TEST_STALL | TSVD_FLAG_WIDE_X;
     if (flags & ~known) return TSVD_E_DTYPE;
     const unsigned path = flags & TSVD_FLAG_PATH_MASK;
     if (path & (path - 1)) return TSVD_E_DTYPE;  // at most one forced path
@@ -276,12 +301,13 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     a.out_f32 = (flags & TSVD_FLAG_OUT_F32) != 0;
     a.z_out = z_out;
     a.test_stall = (flags & TSVD_FLAG_TEST_STALL) != 0;
+    a.wide_x = (flags & TSVD_FLAG_WIDE_X) != 0;
     a.stream = (cudaStream_t)stream;
 
-    const unsigned chosen = choose_path(h, B, dtype, path);
+    const unsigned chosen = choose_path(h, B, dtype, path, a.wide_x);
     if (chosen == 0u) return TSVD_E_TOOBIG;
     if (chosen == TSVD_FLAG_PATH_TENSOR) {
-        tsvd_status_t st = ensure_ws(h, tsvd_tensor_ws_bytes(h, B, dtype));
+        tsvd_status_t st = ensure_ws(h, tsvd_tensor_ws_bytes(h, B, dtype, a.wide_x));
         if (st != TSVD_OK) return st;
         return tsvd_forward_tensor(a, h->ws);
     }
@@ -300,6 +326,31 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     a.t = reinterpret_cast<float*>(h->ws);
     a.t_ld = h->V.R_pad;
     return tsvd_forward_simple(a);
+}
+
+// The largest scratch any path asks for with up to B_max tokens of this dtype: every path's need
+// grows with the batch inside its own regime, so the regime boundaries and B_max cover it.
+extern "C" tsvd_status_t tsvd_reserve(tsvd_handle_t h, int B_max, tsvd_dtype_t dtype)
+{
+    if (!h) return TSVD_E_NULL;
+    if (B_max < 1) return TSVD_E_SHAPE;
+    if (dtype_size(dtype) == 0) return TSVD_E_DTYPE;
+    int dev = 0;
+    TSVD_CUDA_OK(cudaGetDevice(&dev));
+    if (dev != h->device) return TSVD_E_CUDA;
+    size_t need = 0;
+    const int marks[] = {B_max, 64, TSVD_DECODE_MAX_B};
+    for (int B : marks) {
+        if (B > B_max) continue;
+        for (int wide = 0; wide < 2; ++wide) {
+            const size_t t = tsvd_tensor_ws_bytes(h, B, dtype, wide != 0);
+            if (t > need) need = t;
+        }
+        const size_t d = tsvd_decode_ws_bytes(h, B), s = tsvd_simple_ws_bytes(h, B);
+        if (d > need) need = d;
+        if (s > need) need = s;
+    }
+    return ensure_ws(h, need);
 }
 
 extern "C" tsvd_status_t tsvd_forward(tsvd_handle_t h, const void* x, void* y, int B, tsvd_dtype_t dtype,

@@ -46,6 +46,8 @@ struct GemvParams {
     void* z_out;          // V-stage, optional: [B][z_ld] int32 (z_int) or fp32
     int z_ld;
     int z_int;
+    const float* bias;    // U-stage, optional (padded to R_pad): added before the output rounding
+    int* status;          // device status word (range diagnostic)
 };
 
 // D (16 x 8, int32) += A (16 x 32, int8, rows) * B (32 x 8, int8, columns).  Lane (g, q):
@@ -191,6 +193,9 @@ ternary_gemv_kernel(const GemvParams p)
     } else {
         if (tid < NTOK) scale[tid] = 1.f;
     }
+    unsigned range_cnt[NTOK];   // range diagnostic: the first value of every chunk is sampled
+#pragma unroll
+    for (int b = 0; b < NTOK; ++b) range_cnt[b] = 0;
     for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
         float v[NTOK][8];
         if (!kInt && ch == tid) {
@@ -208,6 +213,7 @@ ternary_gemv_kernel(const GemvParams p)
             for (int d = 0; d < ND; ++d) dw[d][0] = dw[d][1] = 0u;
             if (b < p.B) {
                 int qv[8];
+                if constexpr (!kInt) tsvd_range_sample(range_cnt[b], v[b][0], qscale[b]);
                 if constexpr (ND <= 3) {   // |q| <= 2^22: round by adding a constant, whose image the digit offset absorbs
 #pragma unroll
                     for (int e = 0; e < 8; ++e) qv[e] = tsvd_round_bits(v[b][e], qscale[b]);
@@ -222,6 +228,11 @@ ternary_gemv_kernel(const GemvParams p)
             for (int d = 0; d < ND; ++d)
                 *reinterpret_cast<uint2*>(dig + (size_t)(b * ND + d) * dstride + ch * 8) = make_uint2(dw[d][0], dw[d][1]);
         }
+    }
+    if constexpr (!kInt) {
+#pragma unroll
+        for (int b = 0; b < NTOK; ++b)
+            if (tsvd_range_flagged(range_cnt[b]) && lane == 0) atomicOr(p.status, TSVD_DEV_RANGE);
     }
     __syncthreads();
 
@@ -327,10 +338,11 @@ ternary_gemv_kernel(const GemvParams p)
                     else reinterpret_cast<float*>(p.z_out)[(size_t)b * p.z_ld + orow] = val;
                 }
             } else if (orow < p.R) {
+                const float yv = p.bias ? val + __ldg(p.bias + orow) : val;
                 if (p.out_bf16)
-                    reinterpret_cast<__nv_bfloat16*>(p.out)[(size_t)b * p.ld_out + orow] = __float2bfloat16_rn(val);
+                    reinterpret_cast<__nv_bfloat16*>(p.out)[(size_t)b * p.ld_out + orow] = __float2bfloat16_rn(yv);
                 else
-                    reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + orow] = val;
+                    reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + orow] = yv;
             }
         }
     }
@@ -371,15 +383,15 @@ cudaError_t launch_gemv_tokens(const GemvParams& p, int R_pad, cudaStream_t stre
 }
 
 constexpr int ND_T = 4;   // digits of the intermediate t (fp32), as on the tensor-core path
-inline int digits_for_x(tsvd_dtype_t dt) { return dt == TSVD_I8 ? 1 : dt == TSVD_BF16 ? 3 : 4; }
+inline int digits_for_x(tsvd_dtype_t dt, bool wide) { return dt == TSVD_I8 ? 1 : (dt == TSVD_BF16 && !wide) ? 3 : 4; }
 
 }  // namespace
 
-bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt)
+bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x)
 {
     if (B < 1 || B > TSVD_DECODE_MAX_B) return false;
     const int ntok = B == 3 ? 4 : B;
-    return gemv_smem_bytes(digits_for_x(dt), ntok, h->V.C_pad) <= (size_t)GEMV_MAX_SMEM &&
+    return gemv_smem_bytes(digits_for_x(dt, wide_x), ntok, h->V.C_pad) <= (size_t)GEMV_MAX_SMEM &&
            gemv_smem_bytes(ND_T, ntok, h->U.C_pad) <= (size_t)GEMV_MAX_SMEM;
 }
 
@@ -396,11 +408,15 @@ tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws)
     p.in = a.x; p.ld_in = a.ldx; p.B = a.B; p.S = h->S;
     p.out = t; p.ld_out = h->V.R_pad;
     p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
+    p.status = h->dev_status;
     cudaError_t e;
     h->prof.begin(1, st);
     switch (a.dtype) {
         case TSVD_F32: e = launch_gemv_tokens<float, 4, STAGE_V>(p, h->V.R_pad, st); break;
-        case TSVD_BF16: e = launch_gemv_tokens<__nv_bfloat16, 3, STAGE_V>(p, h->V.R_pad, st); break;
+        case TSVD_BF16:
+            e = a.wide_x ? launch_gemv_tokens<__nv_bfloat16, 4, STAGE_V>(p, h->V.R_pad, st)
+                         : launch_gemv_tokens<__nv_bfloat16, 3, STAGE_V>(p, h->V.R_pad, st);
+            break;
         case TSVD_I8: e = launch_gemv_tokens<int8_t, 1, STAGE_V>(p, h->V.R_pad, st); break;
         default: return TSVD_E_DTYPE;
     }
@@ -412,6 +428,7 @@ tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws)
     q.in = t; q.ld_in = h->V.R_pad; q.B = a.B;
     q.out = a.y; q.ld_out = a.ldy;
     q.out_bf16 = (a.dtype == TSVD_BF16) && !a.out_f32;
+    q.bias = h->bias; q.status = h->dev_status;
     h->prof.begin(3, st);
     e = launch_gemv_tokens<float, ND_T, STAGE_U>(q, h->U.R_pad, st);
     h->prof.end(st);

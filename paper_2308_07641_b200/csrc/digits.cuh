@@ -124,6 +124,26 @@ __device__ __forceinline__ void load16(const IN_T* __restrict__ row, int c0, int
     }
 }
 
+// Range diagnostic (TSVD_E_RANGE): while a stage's input is converted, one value in eight is
+// sampled; a sample counts when it is nonzero, and as resolved when it reaches 2^12 quantisation
+// steps.  The two counts travel in one word (low half: nonzero, high half: resolved; a warp sees at
+// most 65280 / 8 samples of a token).  A warp raises the flag when, among at least 32 nonzero
+// samples of a token, fewer than a quarter are resolved.  For a bulk of normally distributed
+// entries under an outlier 2^p times their scale the resolved share is 0.62 at p = 8 (p = 16 with
+// four digits of a bf16 token, or for fp32), 0.32 one binade further and 0.05 two binades further,
+// which is where outputs that do not see the outlier begin to leave the bf16 tolerance.
+__device__ __forceinline__ void tsvd_range_sample(unsigned& cnt, float v, float qscale)
+{
+    const float a = fabsf(v) * qscale;
+    cnt += (a != 0.f ? 1u : 0u) + (a >= 4096.f ? 0x10000u : 0u);
+}
+__device__ __forceinline__ bool tsvd_range_flagged(unsigned cnt)   // whole warp; the same answer in every lane
+{
+    const unsigned tot = __reduce_add_sync(0xffffffffu, cnt);
+    const unsigned nz = tot & 0xffffu, big = tot >> 16;
+    return nz >= 32u && 4u * big < nz;
+}
+
 // The exponent E of the rule above for a token whose largest magnitude is amax: amax = m * 2^E with
 // m in [0.5, 1), read from the exponent field (zero and subnormal maxima take the floor of -90).
 __device__ __forceinline__ int tsvd_quant_exponent(float amax)

@@ -39,6 +39,8 @@ struct IndexParams {
     void* z_out;               // V-stage, optional: [B][z_ld] int32 (z_int) or fp32
     int z_ld;
     int z_int;
+    const float* bias;         // U-stage, optional: added before the output rounding
+    int* status;               // device status word (range diagnostic)
 };
 
 // grid: ceil(R / 16) CTAs of 512 threads.  Dynamic shared memory:
@@ -105,6 +107,9 @@ ternary_index_kernel(const IndexParams p)
     } else {
         if (tid < NTOK) scale[tid] = 1.f;
     }
+    unsigned range_cnt[NTOK];   // range diagnostic: the first value of every chunk is sampled
+#pragma unroll
+    for (int b = 0; b < NTOK; ++b) range_cnt[b] = 0;
     for (int ch = tid; ch < n_chunks; ch += IDX_THREADS) {
         float v[NTOK][8];
 #pragma unroll
@@ -112,12 +117,18 @@ ternary_index_kernel(const IndexParams p)
 #pragma unroll
         for (int b = 0; b < NTOK; ++b) {
             int qv[8];
+            if constexpr (!kInt) { if (b < p.B) tsvd_range_sample(range_cnt[b], v[b][0], qscale[b]); }
 #pragma unroll
             for (int e = 0; e < 8; ++e) qv[e] = b < p.B ? __float2int_rn(v[b][e] * qscale[b]) : 0;
             int4* dst = reinterpret_cast<int4*>(q + (size_t)b * p.C_pad + ch * 8);
             dst[0] = make_int4(qv[0], qv[1], qv[2], qv[3]);
             dst[1] = make_int4(qv[4], qv[5], qv[6], qv[7]);
         }
+    }
+    if constexpr (!kInt) {
+#pragma unroll
+        for (int b = 0; b < NTOK; ++b)
+            if (tsvd_range_flagged(range_cnt[b]) && lane == 0) atomicOr(p.status, TSVD_DEV_RANGE);
     }
     __syncthreads();
 
@@ -153,10 +164,11 @@ ternary_index_kernel(const IndexParams p)
                 else reinterpret_cast<float*>(p.z_out)[(size_t)b * p.z_ld + row] = val;
             }
         } else {
+            const float yv = p.bias ? val + __ldg(p.bias + row) : val;
             if (p.out_bf16)
-                reinterpret_cast<__nv_bfloat16*>(p.out)[(size_t)b * p.ld_out + row] = __float2bfloat16_rn(val);
+                reinterpret_cast<__nv_bfloat16*>(p.out)[(size_t)b * p.ld_out + row] = __float2bfloat16_rn(yv);
             else
-                reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + row] = val;
+                reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + row] = yv;
         }
     }
 }
@@ -246,11 +258,14 @@ tsvd_status_t tsvd_forward_index(const ForwardArgs& a, void* ws)
     p.in = a.x; p.ld_in = a.ldx; p.B = a.B; p.S = h->S;
     p.out = t; p.ld_out = h->V.R_pad;
     p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
+    p.status = h->dev_status;
     cudaError_t e;
     h->prof.begin(1, st);
     switch (a.dtype) {
         case TSVD_F32: e = launch_index_tokens<float, 4, STAGE_V>(p, st); break;
-        case TSVD_BF16: e = launch_index_tokens<__nv_bfloat16, 3, STAGE_V>(p, st); break;
+        case TSVD_BF16:
+            e = a.wide_x ? launch_index_tokens<__nv_bfloat16, 4, STAGE_V>(p, st) : launch_index_tokens<__nv_bfloat16, 3, STAGE_V>(p, st);
+            break;
         case TSVD_I8: e = launch_index_tokens<int8_t, 1, STAGE_V>(p, st); break;
         default: return TSVD_E_DTYPE;
     }
@@ -262,6 +277,7 @@ tsvd_status_t tsvd_forward_index(const ForwardArgs& a, void* ws)
     u.in = t; u.ld_in = h->V.R_pad; u.B = a.B;
     u.out = a.y; u.ld_out = a.ldy;
     u.out_bf16 = (a.dtype == TSVD_BF16) && !a.out_f32;
+    u.bias = h->bias; u.status = h->dev_status;
     h->prof.begin(3, st);
     e = launch_index_tokens<float, ND_T, STAGE_U>(u, st);
     h->prof.end(st);

@@ -1,6 +1,6 @@
 // Packer: int8 ternary matrices -> 2-bit codes in the tiled layout of tsvd_internal.cuh,
-// and its inverse for tests.  The paper states only the storage cost ("2 bits to store
-// each element of a ternary matrix", Section "Connection with BNN and What Next").
+// and its inverse for tests.  The paper states only the storage cost, two bits per entry
+// of a ternary matrix (Section "Connection with BNN and What Next").
 #include "tsvd_internal.cuh"
 
 namespace {

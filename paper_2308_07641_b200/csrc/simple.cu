@@ -28,7 +28,7 @@ __global__ void __launch_bounds__(128)
 ternary_rows_kernel(const uint4* __restrict__ units, int R, int C, int C_pad,
                     const IN_T* __restrict__ in, int ld_in, int B,
                     const float* __restrict__ S, void* __restrict__ out, int ld_out,
-                    void* __restrict__ z_out, int z_ld)
+                    void* __restrict__ z_out, int z_ld)   // S: the scales (V-stage) or the optional bias (U-stage)
 {
     constexpr bool kInt = sizeof(IN_T) == 1;
     using acc_t = typename Acc<IN_T>::type;
@@ -96,11 +96,13 @@ ternary_rows_kernel(const uint4* __restrict__ units, int R, int C, int C_pad,
                 if (z_out) reinterpret_cast<float*>(z_out)[(size_t)b * z_ld + row] = z;
             }
             reinterpret_cast<float*>(out)[(size_t)b * ld_out + row] = S[row] * z;
-        } else if constexpr (EPI == EPI_Y_F32) {
-            reinterpret_cast<float*>(out)[(size_t)b * ld_out + row] = (float)acc[t];
         } else {
-            reinterpret_cast<__nv_bfloat16*>(out)[(size_t)b * ld_out + row] =
-                __float2bfloat16_rn((float)acc[t]);
+            // the optional bias is added in fp32 before the one rounding to the output type
+            const float yv = S ? (float)acc[t] + S[row] : (float)acc[t];
+            if constexpr (EPI == EPI_Y_F32)
+                reinterpret_cast<float*>(out)[(size_t)b * ld_out + row] = yv;
+            else
+                reinterpret_cast<__nv_bfloat16*>(out)[(size_t)b * ld_out + row] = __float2bfloat16_rn(yv);
         }
     }
 }
@@ -151,9 +153,9 @@ tsvd_status_t tsvd_forward_simple(const ForwardArgs& a)
     // U-stage: y[b,m] = sum_k U[m,k] t[b,k]
     const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;
     if (bf16_out)
-        e = launch<float, EPI_Y_BF16>(h->U, a.t, a.t_ld, a.B, nullptr, a.y, a.ldy, nullptr, 0, a.stream);
+        e = launch<float, EPI_Y_BF16>(h->U, a.t, a.t_ld, a.B, h->bias, a.y, a.ldy, nullptr, 0, a.stream);
     else
-        e = launch<float, EPI_Y_F32>(h->U, a.t, a.t_ld, a.B, nullptr, a.y, a.ldy, nullptr, 0, a.stream);
+        e = launch<float, EPI_Y_F32>(h->U, a.t, a.t_ld, a.B, h->bias, a.y, a.ldy, nullptr, 0, a.stream);
     h->prof.end(a.stream);
     return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
 }
@@ -218,8 +220,8 @@ extern "C" tsvd_status_t tsvd_forward_static(tsvd_handle_t h, const void* x, voi
         e = launch<int8_t, EPI_SCALE_TO_T>(h->V, (const int8_t*)x, h->N, B, h->S, t, t_ld, nullptr, 0, s);
     if (e != cudaSuccess) return TSVD_E_CUDA;
     if (dtype == TSVD_BF16)
-        e = launch<float, EPI_Y_BF16>(h->U, t, t_ld, B, nullptr, y, h->M, nullptr, 0, s);
+        e = launch<float, EPI_Y_BF16>(h->U, t, t_ld, B, h->bias, y, h->M, nullptr, 0, s);
     else
-        e = launch<float, EPI_Y_F32>(h->U, t, t_ld, B, nullptr, y, h->M, nullptr, 0, s);
+        e = launch<float, EPI_Y_F32>(h->U, t, t_ld, B, h->bias, y, h->M, nullptr, 0, s);
     return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
 }

@@ -82,7 +82,7 @@ template <typename IN_T, int ND, int TPT, int TOK, int CH>
 __global__ void __launch_bounds__(256, 4)   // <= 64 registers: a batch of 4096 tokens is then one wave
 digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
-                int* __restrict__ zero_buf, int zero_per_token, int zero_total)
+                int* __restrict__ zero_buf, int zero_per_token, int zero_total, int* __restrict__ status)
 {
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
@@ -159,6 +159,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
 
     static_assert(TOK % 8 == 0, "digit rows of one token must share their swizzle term");
     const int sw = b_in & 7;
+    unsigned range_cnt = 0;   // range diagnostic: the first value of every chunk is sampled
     int8_t* tok_base = D + (size_t)jt * KB * (size_t)(NT * 128) + b_in * 128;
     // one chunk: values -> digits -> the chunk's place in the swizzled tile (zeros for a dead token)
     auto convert = [&](int ch, const float (&v)[CH]) {
@@ -169,6 +170,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
             for (int w = 0; w < G; ++w) dig[d][w] = 0;
         if (live) {
             int q[CH];
+            if constexpr (!kInt) tsvd_range_sample(range_cnt, v[0], qscale);
             if constexpr (ND <= 3) {   // |q| <= 2^22: round by adding a constant, whose image the digit offset absorbs
 #pragma unroll
                 for (int e = 0; e < CH; ++e) q[e] = tsvd_round_bits(v[e], qscale);
@@ -215,6 +217,9 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
             convert(ch, v);
         }
     }
+    if constexpr (!kInt) {
+        if (tsvd_range_flagged(range_cnt) && (threadIdx.x & 31) == 0) atomicOr(status, TSVD_DEV_RANGE);
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -242,6 +247,7 @@ struct GemmParams {
     int z_int;
     void* y;              // EPI_U_*: out [B][ldy]
     int ldy;
+    const float* bias;    // EPI_U_* / TAIL_Y: optional, padded to R_pad: added before the output rounding
     int* status;          // device error word
     int row_tiles;        // tiles of 128 rows
     int j_tiles;          // tiles of TOK tokens
@@ -570,8 +576,9 @@ ternary_mma_kernel(const GemmParams p)
             constexpr int N_GROUPS = TOK / 8;
             constexpr int MY_GROUPS = N_GROUPS / EPI_SHARES;
             static_assert(N_GROUPS % EPI_SHARES == 0, "the epilogue warps of a lane group share the token groups evenly");
-            float s_row = 0.f;
+            float s_row = 0.f;   // EPI_V: S of the row; EPI_U_*: the row's bias
             if constexpr (EPI == EPI_V) s_row = p.S[row];
+            if constexpr (EPI == EPI_U_F32 || EPI == EPI_U_BF16) s_row = p.bias ? __ldg(p.bias + row) : 0.f;
             const bool row_ok = row < p.R;
             if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
             tc_fence_after_sync();
@@ -626,6 +633,7 @@ ternary_mma_kernel(const GemmParams p)
                         f = fmaf((float)hi, 65536.f, (float)lo);
                     }
                     val[i] = f * sc[i];   // a power of two: exact
+                    if constexpr (EPI == EPI_U_F32 || EPI == EPI_U_BF16) val[i] += s_row;   // bias (0 without one)
                 }
                 if constexpr (EPI == EPI_V) {
                     float* tp = p.t + (size_t)b0 * p.t_ld + row;
@@ -696,7 +704,7 @@ ternary_mma_kernel(const GemmParams p)
                   for (int tg = half; tg < TOK / 8; tg += EPI_SHARES) {
                     const int b0 = jt * TOK + tg * 8;
                     const bool row_ok = row < p.R;
-                    const float s_row = p.tail == TAIL_T ? p.S[row] : 0.f;
+                    const float s_row = p.tail == TAIL_T ? p.S[row] : (p.bias ? __ldg(p.bias + row) : 0.f);
                     // all loads first (they are independent and come from L2), then the arithmetic
                     int a[8][ND];
                     float sc[8];
@@ -732,10 +740,11 @@ ternary_mma_kernel(const GemmParams p)
                             const unsigned m = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(tv)));
                             if (lane == 0) atomicMax(p.tmax + b, m);
                         } else if (row_ok) {
+                            const float yv = val + s_row;   // bias (0 without one)
                             if (p.y_bf16)
-                                reinterpret_cast<__nv_bfloat16*>(p.y)[(size_t)b * p.ldy + row] = __float2bfloat16_rn(val);
+                                reinterpret_cast<__nv_bfloat16*>(p.y)[(size_t)b * p.ldy + row] = __float2bfloat16_rn(yv);
                             else
-                                reinterpret_cast<float*>(p.y)[(size_t)b * p.ldy + row] = val;
+                                reinterpret_cast<float*>(p.y)[(size_t)b * p.ldy + row] = yv;
                         }
                     }
                   }
@@ -747,7 +756,7 @@ ternary_mma_kernel(const GemmParams p)
     // ---- teardown ----
     tc_fence_before_sync();
     __syncthreads();
-    if (*abort_flag && threadIdx.x == 0) atomicExch(p.status, 1);
+    if (*abort_flag && threadIdx.x == 0) atomicOr(p.status, TSVD_DEV_TIMEOUT);
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, TMEM_COLS);
@@ -756,7 +765,7 @@ ternary_mma_kernel(const GemmParams p)
 
 template <typename IN_T, int ND, int TOK = tokens_per_tile(ND)>
 cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, const unsigned* amax_bits,
-                            int8_t* D, float* scale, int* zero_buf, int zero_total, int* B_pad_out,
+                            int8_t* D, float* scale, int* zero_buf, int zero_total, int* status,
                             cudaStream_t stream)
 {
     const int B_pad = (B + TOK - 1) / TOK * TOK;
@@ -769,16 +778,15 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
         // round and the row still fits the registers (three chunks of 8 per lane)
         if ((KB * 8) % 32 != 0 && KB * 16 <= 3 * 32)
             e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK, 8>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                                   scale, zero_buf, zero_per_token, zero_total);
+                                   scale, zero_buf, zero_per_token, zero_total, status);
         else
             e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK, 16>, in, ld_in, B, B_pad, C, KB, amax_bits,
-                                   D, scale, zero_buf, zero_per_token, zero_total);
+                                   D, scale, zero_buf, zero_per_token, zero_total, status);
     } else {
         e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 256, TOK, 16>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                               scale, zero_buf, zero_per_token, zero_total);
+                               scale, zero_buf, zero_per_token, zero_total, status);
     }
     tsvd_count_launch();
-    if (B_pad_out) *B_pad_out = B_pad;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -832,7 +840,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // digit counts: int8 activations are their own single digit; bf16 needs 3 (22-bit fixed
 // point holds every bf16 value within 2^-12 of the token's largest exactly); fp32 and the
 // intermediate t use 4 (30 bits).
-inline int digits_for_x(tsvd_dtype_t dt) { return dt == TSVD_I8 ? 1 : dt == TSVD_BF16 ? 3 : 4; }
+inline int digits_for_x(tsvd_dtype_t dt, bool wide) { return dt == TSVD_I8 ? 1 : (dt == TSVD_BF16 && !wide) ? 3 : 4; }
 constexpr int ND_T = 4;
 
 struct TensorWs {
@@ -840,9 +848,9 @@ struct TensorWs {
     size_t total;
 };
 
-TensorWs carve(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, void* base)
+TensorWs carve(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide, void* base)
 {
-    const int ndx = digits_for_x(dt);
+    const int ndx = digits_for_x(dt, wide);
     const int tokx = tokens_per_tile(ndx), tokt = tokens_per_tile(ND_T);
     const size_t Bx = align_up(B, tokx), Bt = align_up(B, tokt);
     const size_t Bmax = Bx > Bt ? Bx : Bt;
@@ -880,9 +888,9 @@ struct SmallWs {
     size_t total;
 };
 
-SmallWs carve_small(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, void* base)
+SmallWs carve_small(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide, void* base)
 {
-    const int ndx = digits_for_x(dt);
+    const int ndx = digits_for_x(dt, wide);
     const size_t Bp = align_up(B, SMALL_TOK);
     const size_t KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
     const size_t j_tiles = Bp / SMALL_TOK;
@@ -937,7 +945,7 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
 
     h->prof.begin(0, st);
     e = launch_digitise<IN_T, NDX, SMALL_TOK>((const IN_T*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                              w.zacc, w.zacc_ints, nullptr, st);
+                                              w.zacc, w.zacc_ints, h->dev_status, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
@@ -958,13 +966,13 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
 
     h->prof.begin(2, st);
     e = launch_digitise<float, ND_T, SMALL_TOK>(w.t, h->V.R_pad, a.B, h->K, KBu, p.tmax, w.Dt, w.scale_t, w.yacc,
-                                                w.yacc_ints, nullptr, st);
+                                                w.yacc_ints, h->dev_status, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
     GemmParams q{};
     q.units = h->U.units; q.KB = KBu; q.R = h->M; q.D = w.Dt; q.B = a.B; q.status = h->dev_status;
-    q.scale = w.scale_t; q.y = a.y; q.ldy = a.ldy;
+    q.scale = w.scale_t; q.y = a.y; q.ldy = a.ldy; q.bias = h->bias;
     q.y_bf16 = (a.dtype == TSVD_BF16) && !a.out_f32;
     q.acc = w.yacc; q.acc_ld = h->U.R_pad;
     q.tile_done = w.yacc + (size_t)Bp * ND_T * h->U.R_pad;
@@ -979,13 +987,13 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
 
 }  // namespace
 
-int tsvd_tensor_digits_x(tsvd_dtype_t dt) { return digits_for_x(dt); }
+int tsvd_tensor_digits_x(tsvd_dtype_t dt, bool wide_x) { return digits_for_x(dt, wide_x); }
 int tsvd_tensor_digits_t() { return ND_T; }
 
-size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt)
+size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x)
 {
-    if (B <= SMALL_MAX_B) return carve_small(h, B, dt, nullptr).total;
-    return carve(h, B, dt, nullptr).total;
+    if (B <= SMALL_MAX_B) return carve_small(h, B, dt, wide_x, nullptr).total;
+    return carve(h, B, dt, wide_x, nullptr).total;
 }
 
 tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
@@ -993,15 +1001,16 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     tsvd_handle_s* h = a.h;
     if (a.B <= SMALL_MAX_B) {
         // small batches: 16-token tiles, the contraction split across CTAs
-        const SmallWs sw = carve_small(h, a.B, a.dtype, ws);
+        const SmallWs sw = carve_small(h, a.B, a.dtype, a.wide_x, ws);
         switch (a.dtype) {
             case TSVD_F32: return forward_small<float, 4>(a, sw);
-            case TSVD_BF16: return forward_small<__nv_bfloat16, 3>(a, sw);
+            case TSVD_BF16: return a.wide_x ? forward_small<__nv_bfloat16, 4>(a, sw) : forward_small<__nv_bfloat16, 3>(a, sw);
             case TSVD_I8: return forward_small<int8_t, 1>(a, sw);
             default: return TSVD_E_DTYPE;
         }
     }
-    const TensorWs w = carve(h, a.B, a.dtype, ws);
+    const TensorWs w = carve(h, a.B, a.dtype, a.wide_x, ws);
+    const bool wide_bf16 = a.dtype == TSVD_BF16 && a.wide_x;
     const int KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
     cudaStream_t st = a.stream;
     cudaError_t e;
@@ -1011,15 +1020,19 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     switch (a.dtype) {
         case TSVD_F32:
             e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, nullptr, 0,
-                                          nullptr, st);
+                                          h->dev_status, st);
             break;
         case TSVD_BF16:
-            e = launch_digitise<__nv_bfloat16, 3>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
-                                                  w.scale_x, nullptr, 0, nullptr, st);
+            if (wide_bf16)
+                e = launch_digitise<__nv_bfloat16, 4>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
+                                                      w.scale_x, nullptr, 0, h->dev_status, st);
+            else
+                e = launch_digitise<__nv_bfloat16, 3>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
+                                                      w.scale_x, nullptr, 0, h->dev_status, st);
             break;
         case TSVD_I8:
             e = launch_digitise<int8_t, 1>((const int8_t*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                           nullptr, 0, nullptr, st);
+                                           nullptr, 0, h->dev_status, st);
             break;
         default:
             return TSVD_E_DTYPE;
@@ -1035,7 +1048,7 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     if (a.test_stall) { p.test_stall = 1; p.wait_limit = 16; }   // ~8 ms instead of ~2 s
     const int v_tiles = h->V.R_pad / BLOCK_R;
     h->prof.begin(1, st);
-    if (a.dtype == TSVD_F32) e = launch_gemm<4, EPI_V>(p, v_tiles, st);
+    if (a.dtype == TSVD_F32 || wide_bf16) e = launch_gemm<4, EPI_V>(p, v_tiles, st);
     else if (a.dtype == TSVD_BF16) e = launch_gemm<3, EPI_V>(p, v_tiles, st);
     else e = launch_gemm<1, EPI_V>(p, v_tiles, st);
     h->prof.end(st);
@@ -1043,14 +1056,15 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
 
     // stage 2: t -> digits (each token's scale comes from its own max |t|)
     h->prof.begin(2, st);
-    e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, 0, nullptr, st);
+    e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, 0,
+                                     h->dev_status, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
     // stage 3: U-stage
     GemmParams q{};
     q.units = h->U.units; q.KB = KBu; q.R = h->M; q.D = w.Dt; q.scale = w.scale_t; q.B = a.B;
-    q.y = a.y; q.ldy = a.ldy; q.status = h->dev_status;
+    q.y = a.y; q.ldy = a.ldy; q.status = h->dev_status; q.bias = h->bias;
     const int u_tiles = h->U.R_pad / BLOCK_R;
     const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;
     h->prof.begin(3, st);

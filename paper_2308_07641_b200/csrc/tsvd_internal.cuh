@@ -92,15 +92,20 @@ struct tsvd_handle_s {
     PackedMat V;          // rows K, contraction N
     PackedMat U;          // rows M, contraction K
     float* S = nullptr;   // device, length V.R_pad (zero padded)
+    float* bias = nullptr;  // device, length U.R_pad (zero padded), or null: no bias
     IndexMat Vi, Ui;      // only with TSVD_PACK_INDEX_LISTS
     // scratch shared by all forwards on this handle
     void* ws = nullptr;
     size_t ws_bytes = 0;
     void* io = nullptr;   // device staging for the host-buffer entry point
     size_t io_bytes = 0;
-    int* dev_status = nullptr;  // device error word
+    int* dev_status = nullptr;  // device status word: TSVD_DEV_* bits
     StageProfiler prof;
 };
+
+// bits of the device status word
+constexpr int TSVD_DEV_TIMEOUT = 1;   // a bounded wait gave up
+constexpr int TSVD_DEV_RANGE = 2;     // a token's dynamic range exceeded what the digits resolve
 
 // Programmatic dependent launch: a kernel launched with this configuration may be set up, and
 // run up to its pdl_wait(), while the kernel before it in the stream is still running;
@@ -149,6 +154,7 @@ struct ForwardArgs {
     bool out_f32;
     void* z_out;
     bool test_stall = false;   // TSVD_FLAG_TEST_STALL
+    bool wide_x = false;       // TSVD_FLAG_WIDE_X: bf16 activations as four digits
     float* t;        // scratch [B][t_ld] fp32: S * (V x)
     int t_ld;
     cudaStream_t stream;
@@ -158,12 +164,12 @@ size_t tsvd_simple_ws_bytes(const tsvd_handle_s* h, int B);
 
 // tensor.cu -- tcgen05 path
 tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws);
-size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt);
-int tsvd_tensor_digits_x(tsvd_dtype_t dt);
+size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x);
+int tsvd_tensor_digits_x(tsvd_dtype_t dt, bool wide_x);
 int tsvd_tensor_digits_t();
 
 // decode.cu -- one to four tokens, bound by streaming the packed codes
-bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt);
+bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x);
 size_t tsvd_decode_ws_bytes(const tsvd_handle_s* h, int B);
 tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws);
 

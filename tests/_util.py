@@ -16,10 +16,8 @@ BF16_RTOL, BF16_ATOL = 1e-2, 1e-3
 
 
 def torch_x(case_x: np.ndarray, x_dtype: str):
-    import torch
-    if x_dtype == "bf16":
-        return torch.from_numpy(case_x.view(np.int16).copy()).cuda().view(torch.bfloat16)
-    return torch.from_numpy(np.ascontiguousarray(case_x)).cuda()
+    from paper_2308_07641_b200 import device_activations
+    return device_activations(case_x, x_dtype)
 
 
 def run_gpu(layer, x_np: np.ndarray, x_dtype: str, flags: int = 0, want_z: bool = True):
@@ -41,11 +39,7 @@ def run_gpu(layer, x_np: np.ndarray, x_dtype: str, flags: int = 0, want_z: bool 
 
 
 def oracle_x(x_np: np.ndarray, x_dtype: str) -> np.ndarray:
-    if x_dtype == "bf16":
-        return rng.bf16_bits_to_f32(x_np).astype(np.float64)
-    if x_dtype == "i8":
-        return x_np
-    return x_np.astype(np.float64)
+    return gen.widen_x(x_np, x_dtype)
 
 
 def check_outputs(y64: np.ndarray, z, ref: "oracle.OracleResult", x_dtype: str, y_bf16: bool, what=""):
@@ -74,19 +68,31 @@ def check_outputs(y64: np.ndarray, z, ref: "oracle.OracleResult", x_dtype: str, 
     return out
 
 
-def run_and_check(spec: "gen.CaseSpec", flags: int = 0, sample_tokens=None, pack_flags: int = 0):
-    """Build the case, run it on the GPU at full batch, compare (all tokens, or a sample)."""
-    from paper_2308_07641_b200 import TSVDLinear
-    U, V, S = gen.make_weights(spec)
-    x = gen.make_x(spec)
+def run_and_check(spec: "gen.CaseSpec", flags: int = 0, sample_tokens=None, pack_flags: int = 0,
+                  weights=None, x=None, bias=None, expect_status=0):
+    """Build the case (or take the given weights (U, V, S) / activations / bias), run it on the GPU at
+    full batch, compare with the checker (all tokens, or a sample), and check the device status word
+    (expect_status: a status, a collection of allowed statuses, or None for no check)."""
+    from paper_2308_07641_b200 import TSVDLinear, binding
+    U, V, S = weights if weights is not None else gen.make_weights(spec)
+    if x is None:
+        x = gen.make_x(spec)
     layer = TSVDLinear(U, S, V, pack_flags)
     try:
+        if bias is not None:
+            layer.set_bias(bias)
         y64, z, y_bf16 = run_gpu(layer, x, spec.x_dtype, flags)
+        status = binding.tsvd_last_status(layer.handle)
     finally:
         layer.close()
+    if expect_status is not None:
+        allowed = (expect_status,) if isinstance(expect_status, int) else tuple(expect_status)
+        assert status in allowed, f"{spec.name}: device status {status}, expected one of {allowed}"
     if sample_tokens is None:
-        idx = np.arange(spec.B)
+        idx = np.arange(x.shape[0])
     else:
         idx = np.asarray(sample_tokens)
-    ref = oracle.forward(U, S, V, oracle_x(x[idx], spec.x_dtype))
-    return check_outputs(y64[idx], None if z is None else z[idx], ref, spec.x_dtype, y_bf16, spec.name)
+    ref = oracle.forward(U, S, V, oracle_x(x[idx], spec.x_dtype), bias)
+    out = check_outputs(y64[idx], None if z is None else z[idx], ref, spec.x_dtype, y_bf16, spec.name)
+    out["status"] = status
+    return out

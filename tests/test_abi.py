@@ -51,13 +51,16 @@ def test_constants_match_the_header(binding):
     assert define("TSVD_FLAG_PATH_INDEX") == binding.TSVD_FLAG_PATH_INDEX
     assert define("TSVD_PACK_INDEX_LISTS") == binding.TSVD_PACK_INDEX_LISTS
     assert define("TSVD_INDEX_MAX_COLUMNS") == binding.TSVD_INDEX_MAX_COLUMNS
+    assert define("TSVD_MAX_CONTRACTION") == binding.TSVD_MAX_CONTRACTION
+    assert define("TSVD_FLAG_WIDE_X") == binding.TSVD_FLAG_WIDE_X
+    assert int(re.search(r"TSVD_E_RANGE\s*=\s*(\d+)", hdr).group(1)) == binding.TSVD_E_RANGE
     assert define("TSVD_FLAG_PATH_MASK") == (binding.TSVD_FLAG_PATH_SIMPLE | binding.TSVD_FLAG_PATH_DECODE |
                                             binding.TSVD_FLAG_PATH_TENSOR | binding.TSVD_FLAG_PATH_INDEX)
 
 
 def test_strerror_covers_all_codes(binding):
-    seen = {binding.tsvd_strerror(i) for i in range(0, 10)}
-    assert len(seen) == 10 and "unknown status" not in seen
+    seen = {binding.tsvd_strerror(i) for i in range(0, 11)}
+    assert len(seen) == 11 and "unknown status" not in seen
     assert binding.tsvd_strerror(99) == "unknown status"
 
 
@@ -70,6 +73,15 @@ def test_host_side_validation(binding):
     assert lib.tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, 0, 2, 2, 0, ctypes.byref(h)) == binding.TSVD_E_SHAPE
     assert lib.tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, 2, 2, 2, 7, ctypes.byref(h)) == binding.TSVD_E_DTYPE
     assert h.value is None
+    # The digit sums of a row are combined in 32-bit integers, |sum| <= 128 * 257 * columns: the
+    # contraction length is bounded where that would leave 31 bits (checked before any device call).
+    big = binding.TSVD_MAX_CONTRACTION + 1
+    assert 128 * 257 * binding.TSVD_MAX_CONTRACTION < 2 ** 31 <= 128 * 257 * (binding.TSVD_MAX_CONTRACTION + 128)
+    assert lib.tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, 2, 2, big, 0, ctypes.byref(h)) == binding.TSVD_E_TOOBIG
+    assert lib.tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, 2, big, 2, 0, ctypes.byref(h)) == binding.TSVD_E_TOOBIG
+    assert h.value is None
+    assert lib.tsvd_reserve(None, 1, 0) == binding.TSVD_E_NULL
+    assert lib.tsvd_set_bias(None, None) == binding.TSVD_E_NULL
     assert lib.tsvd_forward(None, None, None, 1, 0, None) == binding.TSVD_E_NULL
     assert lib.tsvd_info(None, None, None, None, None, None, None) == binding.TSVD_E_NULL
     assert lib.tsvd_last_status(None) == binding.TSVD_E_NULL

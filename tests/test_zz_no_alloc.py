@@ -6,14 +6,16 @@ allocator, or a latency-critical section that cannot afford the device synchroni
 allocation implies.  For them the library keeps the intermediate S*(V x) in a fixed array
 inside its own image.  This test calls that entry point through the C ABI twice in a row
 (different inputs and batch sizes, so stale contents of the shared array would show) and
-compares each result with the ordinary tsvd_forward on the same inputs, with the tolerances
-the other parity tests use.  It is collected last so that a stop-at-first-failure run has
+compares each result with the ordinary tsvd_forward on the same inputs and with the CPU
+checker, with the tolerances the other parity tests use, and checks that the device memory in
+use is the same before and after the calls.  It is collected last so that a stop-at-first-failure run has
 already covered everything else; it also passes when run alone in a fresh process.
 """
 import numpy as np
 import pytest
 
 import gen
+import oracle
 from tests import _util
 
 pytestmark = pytest.mark.gpu
@@ -28,8 +30,12 @@ def _forward_pair(binding, h, x_np, x_dtype, M):
     y_sta = torch.full((B, M), 3.0, dtype=out_dtype, device="cuda")
     dt = binding.DTYPES[x_dtype]
     binding.tsvd_forward(h, x.data_ptr(), y_ref.data_ptr(), B, dt)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
     binding.tsvd_forward_static(h, x.data_ptr(), y_sta.data_ptr(), B, dt)
     torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "tsvd_forward_static changed the device memory in use"
     return y_ref.double().cpu().numpy(), y_sta.double().cpu().numpy()
 
 
@@ -42,6 +48,7 @@ def test_static_matches_forward_on_two_calls_in_a_row(x_dtype, base):
     x = gen.make_x(spec)
     h = binding.tsvd_pack(U, S, V)
     try:
+        _forward_pair(binding, h, x[:1], x_dtype, spec.M)      # first call on the device: address look-up
         for xs in (x, x[5:24]):              # second call: other inputs, smaller batch
             y_ref, y_sta = _forward_pair(binding, h, xs, x_dtype, spec.M)
             err = np.abs(y_sta - y_ref)
@@ -49,6 +56,8 @@ def test_static_matches_forward_on_two_calls_in_a_row(x_dtype, base):
                 assert np.all(err <= _util.BF16_RTOL * np.abs(y_ref) + _util.BF16_ATOL)
             else:
                 assert err.max() <= _util.F32_REL_MAX * np.abs(y_ref).max()
+            chk = oracle.forward(U, S, V, _util.oracle_x(xs, x_dtype))
+            _util.check_outputs(y_sta, None, chk, x_dtype, x_dtype == "bf16", "tsvd_forward_static")
     finally:
         binding.tsvd_destroy(h)
 
