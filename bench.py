@@ -1,18 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the TSVD linear map y = U(diag(S)(V x)) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config cfg2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config cfg4]
 
-One step = one full forward (V-stage, S scale, U-stage) over one batch of B synthetic
-tokens.  Prints ONE JSON line: tokens/s with inputs resident in HBM (`value`), the same
-through the host-buffer entry point with copies inside the timed region (`e2e`), the
-roofline figures of the dominant kernel, and the CPU checker timed on the host cores.
-With N > 1 (torchrun) every rank runs its own replica on its own tokens (weak scaling,
-no data-path collective); the time is the max over ranks.
+One step = one full forward (V-stage, S scale, U-stage) over one batch of B synthetic tokens.
+Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM: the K steps are captured
+in one CUDA graph, the graph is replayed `--repeats` times between CUDA events, and the median
+replay is reported (with the fastest and slowest).  `e2e` is the same through the host-buffer
+entry point with the copies inside the timed region.  `roofline` describes the dominant kernel,
+whose duration is taken inside the graph from time stamps the kernels write themselves.
+`sustained` repeats the replays back to back for more than a second with the SM clock sampled.
+`per_config` carries the same figures, and a parity check against the CPU checker on a bounded
+token sample, for every workload of gen.CONFIGS.  `cpu_baseline` is the CPU checker timed on
+the host cores.  With N > 1 (torchrun) every rank runs its own replica on its own tokens (weak
+scaling, no data-path collective); the time is the max over ranks.
 """
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import statistics
@@ -31,11 +37,14 @@ import gen  # noqa: E402
 
 METRIC = "tsvd_linear_tokens_per_s"
 UNIT = "tokens/s"
-L2_FLUSH_BYTES = 256 << 20
 # measured on this machine's B200s (copy bandwidth, cuBLAS bf16 burst / sustained); used when
 # MEASURED_PEAKS.json is not next to this file
-PEAKS_COPY = {"hbm_gbs": 6524.9, "bf16_tflops": 1681.0, "bf16_tflops_sustained": 1398.7}
-INT8_OVER_BF16 = 2.0  # nominal dense tensor ratio (4.5 / 2.25 PFLOP/s)
+PEAKS_COPY = {"hbm_gbs": 6471.4, "bf16_tflops": 1711.9, "bf16_tflops_sustained": 1428.0}
+INT8_OVER_BF16 = 2.0          # nominal dense tensor ratio (4.5 / 2.25 PFLOP/s)
+INT8_MAC_PER_CLK_PER_SM = 8192  # tcgen05 kind::i8: the hardware rate the clock-derived peak uses
+HEADLINE = "cfg4"             # the largest single-GPU workload
+ALL_CONFIGS = ("cfg1", "cfg2", "cfg3_b1", "cfg3_b4", "cfg3_b16", "cfg4", "cfg5_d05", "cfg5_d20", "cfg5_d50")
+SUSTAINED = ("cfg2", "cfg4")
 
 
 def max_over_ranks(dist, value, device):
@@ -92,8 +101,9 @@ def load_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason sampler running during the timed region."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """nvidia-smi clock / throttle-reason sampler; `window(t0, t1)` summarises the samples whose
+    own time stamp lies inside a wall-clock interval (the timed region)."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -101,6 +111,7 @@ class ClockSampler:
         self.gpu = gpu_index
         self.proc = None
         self.path = None
+        self.rows = []
 
     def start(self):
         try:
@@ -108,47 +119,76 @@ class ClockSampler:
             os.close(fd)
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
-            return out
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
         self.f.close()
-        sm, mx, reasons = [], [], set()
         try:
             for line in open(self.path):
                 parts = [p.strip() for p in line.split(",")]
                 if len(parts) < 9:
                     continue
                 try:
-                    sm.append(float(parts[1])); mx.append(float(parts[2]))
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    row = (ts, float(parts[1]), float(parts[2]), float(parts[3]),
+                           [n for n, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                               "sw_power_cap"), parts[5:9]) if v.lower().startswith("active")])
                 except ValueError:
                     continue
-                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
-                                    "sw_power_cap"), parts[5:9]):
-                    if v.lower().startswith("active"):
-                        reasons.add(name)
+                self.rows.append(row)
         finally:
             try:
                 os.unlink(self.path)
             except OSError:
                 pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
-        out["reasons"] = sorted(reasons)
+        self.proc = None
+
+    def window(self, t0, t1):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w_max": None}
+        rows = [r for r in self.rows if t0 <= r[0] <= t1]
+        if not rows and self.rows:      # a region shorter than the sampling period: the nearest sample
+            rows = sorted(self.rows, key=lambda r: abs(r[0] - 0.5 * (t0 + t1)))[:1]
+            out["note"] = "no sample fell inside the region; nearest sample reported"
+        if rows:
+            out.update(sm_mhz=statistics.median(r[1] for r in rows), sm_max_mhz=max(r[2] for r in rows),
+                       samples=len(rows), power_w_max=max(r[3] for r in rows),
+                       reasons=sorted({n for r in rows for n in r[4]}))
         return out
 
 
-def cpu_baseline(spec, U, S, V, x_np, target_s=8.0, y_gpu=None):
+def parity_against_checker(spec, U, S, V, x_np, y_gpu64, tokens):
+    """The GPU output of the listed tokens against the CPU checker, at the stated tolerances."""
+    import oracle
+    idx = np.asarray(tokens)
+    ref = oracle.forward(U, S, V, gen.widen_x(x_np[idx], spec.x_dtype))
+    err = np.abs(y_gpu64[idx] - ref.y)
+    if spec.x_dtype == "bf16":
+        tol = 1e-2 * np.abs(ref.y) + 1e-3
+        return {"tokens": int(idx.size), "violations": int((err > tol).sum()),
+                "worst_err_over_tol": float((err / tol).max()), "rule": "|y-ref| <= 1e-2|ref| + 1e-3 per element"}
+    scale = float(np.abs(ref.y).max())
+    return {"tokens": int(idx.size), "max_err_over_max_ref": float(err.max() / scale) if scale else float(err.max()),
+            "violations": int(err.max() > 1e-5 * scale), "rule": "max|y-ref| <= 1e-5 max|ref|"}
+
+
+def sample_tokens(B):
+    """All tokens of a small batch; else the first and last ones and the tile edges at 48 and 64."""
+    if B <= 16:
+        return list(range(B))
+    return sorted({0, 1, B // 2, B - 2, B - 1, 47, 48, 63, 64} & set(range(B)))
+
+
+def cpu_baseline(spec, U, S, V, x_np, target_s=10.0):
     """Time the CPU checker, as it stands, on a bounded sample of the workload's tokens."""
     import oracle
     cores = oracle.threads()
@@ -160,18 +200,9 @@ def cpu_baseline(spec, U, S, V, x_np, target_s=8.0, y_gpu=None):
     n = int(min(spec.B, max(n0, target_s / max(per_tok, 1e-9))))
     n = max(cores, n - n % cores) if n >= cores else n
     xs = gen.widen_x(x_np[:n], spec.x_dtype)
-    t0 = time.perf_counter(); ref = oracle.forward(U, S, V, xs); t1 = time.perf_counter()
-    out = {"value": n / (t1 - t0), "unit": UNIT, "cores": cores, "kind": "oracle",
-           "sample": f"first {n} of {spec.B} tokens of {spec.name}, one call, {t1 - t0:.2f} s wall"}
-    parity = None
-    if y_gpu is not None:
-        err = np.abs(y_gpu[:n] - ref.y)
-        if spec.x_dtype == "bf16":
-            tol = 1e-2 * np.abs(ref.y) + 1e-3
-            parity = {"tokens": n, "violations": int((err > tol).sum()), "worst_err_over_tol": float((err / tol).max())}
-        else:
-            parity = {"tokens": n, "max_err_over_max_ref": float(err.max() / np.abs(ref.y).max())}
-    return out, parity
+    t0 = time.perf_counter(); oracle.forward(U, S, V, xs); t1 = time.perf_counter()
+    return {"value": n / (t1 - t0), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n} of {spec.B} tokens of {spec.name}, one call, {t1 - t0:.2f} s wall"}
 
 
 def run_reference(args, spec):
@@ -202,32 +233,223 @@ def run_reference(args, spec):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": workload_config(spec, "host cores; no GPU"),
+            "data": "synthetic", "config": workload_config(spec),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
-def workload_config(spec, l2_note):
+def workload_config(spec):
     return {"workload": spec.name, "M": spec.M, "N": spec.N, "K": spec.K, "B": spec.B,
-            "density": spec.density, "x_dtype": spec.x_dtype, "s_dist": spec.s_dist, "seed": spec.seed,
-            "l2": l2_note}
+            "density": spec.density, "x_dtype": spec.x_dtype, "s_dist": spec.s_dist, "seed": spec.seed}
+
+
+def pad128(v):
+    return (v + 127) // 128 * 128
+
+
+class Workload:
+    """One packed layer (plus rotating copies and buffers larger than the L2) ready to be timed."""
+
+    def __init__(self, spec, rank, pack_flags, flags, local_rank):
+        import torch
+        from paper_2308_07641_b200 import TSVDLinear, binding, device_activations
+        self.spec, self.flags, self.binding = spec, flags, binding
+        self.U, self.V, self.S = gen.make_weights(spec)
+        self.x_np = gen.make_x(rank_spec(spec, rank))
+        self.layer = TSVDLinear(self.U, self.S, self.V, pack_flags)
+        self.info = self.layer.info
+        self.layer.reserve(spec.B, spec.x_dtype)
+        self.x = device_activations(self.x_np, spec.x_dtype)
+        self.y = self.layer.forward(self.x, flags=flags)
+        torch.cuda.synchronize()
+        # Rotating input/output buffers: together larger than twice the L2, so that every step
+        # streams its activations from HBM and writes its results there.
+        self.l2_bytes = int(torch.cuda.get_device_properties(local_rank).L2_cache_size)
+        self.pair_bytes = self.x.numel() * self.x.element_size() + self.y.numel() * self.y.element_size()
+        self.n_sets = int(min(64, max(2, -(-2 * self.l2_bytes // self.pair_bytes))))
+        self.xs = [self.x] + [torch.roll(self.x, i, dims=0).contiguous() for i in range(1, self.n_sets)]
+        self.ys = [self.y] + [torch.empty_like(self.y) for _ in range(1, self.n_sets)]
+        # When the packed weights outweigh the activations (small batches) the weights are what must
+        # come from HBM: pack the same layer several times and rotate over the copies as well.
+        self.n_layers = 1
+        if self.info["packed_bytes"] > self.pair_bytes:
+            self.n_layers = int(min(64, max(2, -(-2 * self.l2_bytes // self.info["packed_bytes"]))))
+        self.layers = [self.layer] + [TSVDLinear(self.U, self.S, self.V, pack_flags) for _ in range(1, self.n_layers)]
+        for extra in self.layers[1:]:
+            extra.reserve(spec.B, spec.x_dtype)
+        self.plan = binding.tsvd_plan(self.layer.handle, spec.B, binding.DTYPES[spec.x_dtype], flags)
+        self.l2_note = (f"inputs larger than L2: {self.n_sets} rotating x/y buffer pairs "
+                        f"({self.n_sets * self.pair_bytes / 1e6:.0f} MB) and {self.n_layers} packed copies of the layer "
+                        f"({self.n_layers * self.info['packed_bytes'] / 1e6:.0f} MB) against {self.l2_bytes / 1e6:.0f} MB of L2")
+
+    def step(self, i):
+        self.layers[i % self.n_layers].forward(self.xs[i % self.n_sets], out=self.ys[i % self.n_sets], flags=self.flags)
+
+    def capture(self, steps, stamps=False):
+        """`steps` forwards in one CUDA graph (no host launch latency between kernels).  With
+        `stamps` every kernel also writes its own begin/end time; returns (graph, launches)."""
+        import torch
+        b = self.binding
+        for L in self.layers:
+            b.tsvd_profile_enable(L.handle, 2 if stamps else 0)
+        side = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        n0 = b.tsvd_launch_count()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(steps):
+                    self.step(i)
+        return g, b.tsvd_launch_count() - n0
+
+    def stage_times(self):
+        """Summed in-graph kernel time (ms) and launches per stage over all rotating copies."""
+        b = self.binding
+        ms = [0.0] * b.N_STAGES
+        n = [0] * b.N_STAGES
+        for L in self.layers:
+            m, c = b.tsvd_profile_read(L.handle)
+            ms = [a + v for a, v in zip(ms, m)]
+            n = [a + v for a, v in zip(n, c)]
+            b.tsvd_profile_enable(L.handle, 0)
+        return ms, n
+
+    def close(self):
+        for L in self.layers:
+            L.close()
+
+
+def replay_times(g, repeats, barrier):
+    """`repeats` replays of a captured graph, each between its own pair of CUDA events, queued back to
+    back; returns the per-replay times in ms and the wall-clock interval of the region."""
+    import torch
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+    g.replay()                         # one untimed replay (graph upload)
+    barrier()
+    t0 = time.time()
+    ev[0].record()
+    for i in range(repeats):
+        g.replay()
+        ev[i + 1].record()
+    barrier()
+    t1 = time.time()
+    return [ev[i].elapsed_time(ev[i + 1]) for i in range(repeats)], (t0, t1)
+
+
+def roofline_of(w, peaks, peaks_src, ms_per_step, stage_ms, stage_n, sm_mhz):
+    """The dominant kernel of one workload against the roofline that bounds it."""
+    b, spec, plan, info = w.binding, w.spec, w.plan, w.info
+    per_launch = [m / c if c else 0.0 for m, c in zip(stage_ms, stage_n)]
+    dom = int(np.argmax(per_launch))
+    dom_ms = per_launch[dom]
+    name = b.STAGE_NAMES[dom]
+    rows, contr = (pad128(spec.K), pad128(spec.N)) if dom in (0, 1) else (pad128(spec.M), pad128(spec.K))
+    out = {"kernel": name, "ms_per_launch": dom_ms, "plan": plan,
+           "stage_us_per_launch": {n: 1e3 * v for n, v in zip(b.STAGE_NAMES, per_launch)},
+           "timing": "time stamps written by the kernels inside a captured graph of the same steps "
+                     "(begin: the first CTA once its wait for the previous kernel has ended; end: the last warp)"}
+    if dom_ms <= 0:
+        out.update(bound="hbm", achieved=None, peak=peaks["hbm_gbs"], unit="GB/s", frac=None, traffic=None)
+        return out
+    if dom in (1, 3) and plan["path"] in ("decode", "index"):
+        if plan["path"] == "index":
+            v_bytes, u_bytes = b.tsvd_index_bytes(w.layer.handle)
+            byts, all_bytes = float(v_bytes if dom == 1 else u_bytes), float(v_bytes + u_bytes)
+        else:
+            byts, all_bytes = rows * contr / 4.0, float(info["packed_bytes"])   # 2 bits per padded entry
+        achieved = byts / (dom_ms * 1e-3) / 1e9
+        out.update(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
+                   traffic=recorded_traffic(spec.name, name), bytes_per_launch=byts,
+                   peak_source=f"{peaks_src} (of measured)",
+                   step_hbm_gbs=all_bytes / (ms_per_step * 1e-3) / 1e9)
+        out["step_hbm_frac"] = out["step_hbm_gbs"] / peaks["hbm_gbs"]
+    elif dom in (1, 3):
+        digits = max(1, plan["digits_x"] if dom == 1 else plan["digits_t"])
+        ops = 2.0 * rows * contr * spec.B * digits        # executed dense operations of that launch
+        useful = 2.0 * rows * contr * spec.B              # the same contraction without the digit split
+        if plan["path"] == "tensor":
+            peak, note = peaks["bf16_tflops"] * INT8_OVER_BF16, "int8 = measured bf16 burst x 2 (nominal ratio)"
+        else:
+            peak, note = peaks["bf16_tflops"], "measured bf16 burst"
+        achieved = ops / (dom_ms * 1e-3) / 1e12
+        out.update(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
+                   traffic=recorded_traffic(spec.name, name), ops_per_launch=ops, digits=digits,
+                   peak_source=f"{note}; {peaks_src} (of measured)", useful_frac=useful / (dom_ms * 1e-3) / 1e12 / peak)
+        if plan["path"] == "tensor" and sm_mhz:
+            clock_peak = 148 * INT8_MAC_PER_CLK_PER_SM * 2 * sm_mhz * 1e6 / 1e12
+            out["clock_peak"] = {"tops": clock_peak, "frac": achieved / clock_peak,
+                                 "useful_frac": out["useful_frac"] * peak / clock_peak,
+                                 "how": f"148 SMs x {INT8_MAC_PER_CLK_PER_SM} int8 MAC/clk x 2 x {sm_mhz:.0f} MHz "
+                                        "(median sampled SM clock of the timed region)"}
+    else:
+        in_bytes = {"f32": 4, "bf16": 2, "i8": 1}[spec.x_dtype] if dom == 0 else 4
+        nd = plan["digits_x"] if dom == 0 else plan["digits_t"]
+        byts = float(spec.B * contr) * (in_bytes + nd)     # values read, digits written
+        achieved = byts / (dom_ms * 1e-3) / 1e9
+        out.update(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
+                   traffic=None, bytes_per_launch=byts, peak_source=f"{peaks_src} (of measured)")
+    if plan["path"] == "tensor":
+        all_ops = 2.0 * spec.B * (pad128(spec.K) * pad128(spec.N) * plan["digits_x"] + pad128(spec.M) * pad128(spec.K) * plan["digits_t"])
+        single = 2.0 * spec.B * (pad128(spec.K) * pad128(spec.N) + pad128(spec.M) * pad128(spec.K))
+        int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
+        out["step_tensor_frac"] = all_ops / (ms_per_step * 1e-3) / 1e12 / int8_peak
+        out["step_useful_frac_of_bf16_peak"] = single / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"]
+    return out
+
+
+def measure(w, steps, repeats, barrier, dist, world, sustained_s=0.0):
+    """Median-of-replays step time of one workload and its in-graph kernel times."""
+    import torch
+    spec = w.spec
+    g, launches = w.capture(steps)
+    times, (t0, t1) = replay_times(g, repeats, barrier)
+    med = max_over_ranks(dist, statistics.median(times), "cuda")
+    ms_per_step = med / steps
+    res = {"ms_per_step": ms_per_step, "ms_per_step_min": min(times) / steps, "ms_per_step_max": max(times) / steps,
+           "tokens_per_s": aggregate_tokens_per_s(world, spec.B, ms_per_step), "launches_per_step": launches / steps,
+           "launches": launches * repeats, "window": (t0, t1), "path": w.plan["path"]}
+    if sustained_s > 0:
+        n = max(2, int(sustained_s * 1e3 / max(med, 1e-3)) + 1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        s0 = time.time()
+        a.record()
+        for _ in range(n):
+            g.replay()
+        b.record()
+        barrier()
+        s1 = time.time()
+        tot = max_over_ranks(dist, a.elapsed_time(b), "cuda")
+        res["sustained"] = {"ms_per_step": tot / (n * steps), "seconds": tot * 1e-3, "steps": n * steps,
+                            "tokens_per_s": aggregate_tokens_per_s(world, spec.B, tot / (n * steps)), "window": (s0, s1)}
+    del g
+    # the same steps once more with the kernels stamping their own begin and end
+    g2, _ = w.capture(steps, stamps=True)
+    stamp_times, _ = replay_times(g2, 2, barrier)
+    stage_ms, stage_n = w.stage_times()
+    del g2
+    res["stage_ms"], res["stage_n"] = stage_ms, stage_n
+    res["ms_per_step_with_stamps"] = statistics.median(stamp_times) / steps
+    return res
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=100, help="forwards per captured graph = steps of one timed region")
     ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--repeats", type=int, default=10, help="timed replays of the graph; the median is reported")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg2", choices=sorted(gen.CONFIGS))
+    ap.add_argument("--config", default=HEADLINE, choices=sorted(gen.CONFIGS))
     ap.add_argument("--path", default="auto", choices=["auto", "simple", "decode", "tensor", "index"],
                     help="index = the index-list form (one to four tokens; meant for nonzero rates below 1/8)")
     ap.add_argument("--density", type=float, default=None,
                     help="override the workload's nonzero rate of U and V (the sparse sweep of the index-list form)")
+    ap.add_argument("--wide-x", action="store_true", help="bf16 activations as four digits (TSVD_FLAG_WIDE_X)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--eager", action="store_true", help="time eager launches with an L2 flush per step")
+    ap.add_argument("--no-per-config", action="store_true", help="only the headline workload")
+    ap.add_argument("--no-sustained", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     spec = gen.CONFIGS[args.config]
@@ -239,7 +461,7 @@ def main():
         return
 
     import torch
-    from paper_2308_07641_b200 import TSVDLinear, binding, build as lib_build
+    from paper_2308_07641_b200 import binding, build as lib_build
     from paper_2308_07641_b200 import TSVD_FLAG_PATH_DECODE, TSVD_FLAG_PATH_SIMPLE, TSVD_FLAG_PATH_TENSOR
 
     rank = int(os.environ.get("RANK", "0"))
@@ -257,211 +479,152 @@ def main():
     if dist:
         dist.barrier()
 
-    flags = {"auto": 0, "simple": TSVD_FLAG_PATH_SIMPLE, "decode": TSVD_FLAG_PATH_DECODE,
-             "tensor": TSVD_FLAG_PATH_TENSOR, "index": binding.TSVD_FLAG_PATH_INDEX}[args.path]
-    pack_flags = binding.TSVD_PACK_INDEX_LISTS if args.path == "index" else 0
-    U, V, S = gen.make_weights(spec)
-    x_np = gen.make_x(rank_spec(spec, rank))
-    layer = TSVDLinear(U, S, V, pack_flags)
-    info = layer.info
-    from paper_2308_07641_b200 import device_activations
-    x = device_activations(x_np, spec.x_dtype)
-    y = layer.forward(x, flags=flags)
-    torch.cuda.synchronize()
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
-
     def barrier():
         torch.cuda.synchronize()
         if dist:
             dist.barrier()
             torch.cuda.synchronize()
 
-    # Rotating input/output buffers: together larger than twice the L2, so that every step
-    # streams its activations from HBM and writes its results there.
-    l2_bytes = int(torch.cuda.get_device_properties(local_rank).L2_cache_size)
-    pair_bytes = x.numel() * x.element_size() + y.numel() * y.element_size()
-    n_sets = int(min(64, max(2, -(-2 * l2_bytes // pair_bytes))))
-    xs = [x] + [torch.roll(x, i, dims=0).contiguous() for i in range(1, n_sets)]
-    ys = [y] + [torch.empty_like(y) for _ in range(1, n_sets)]
-    # When the packed weights outweigh the activations (small batches) the weights are what must
-    # come from HBM: pack the same layer several times and rotate over the copies as well.
-    n_layers = 1
-    if info["packed_bytes"] > pair_bytes:
-        n_layers = int(min(64, max(2, -(-2 * l2_bytes // info["packed_bytes"]))))
-    layers = [layer] + [TSVDLinear(U, S, V, pack_flags) for _ in range(1, n_layers)]
-    for i, extra in enumerate(layers[1:]):       # size their scratch outside any timed region
-        extra.forward(xs[0], out=ys[0], flags=flags)
-
-    for i in range(args.warmup):
-        flush.zero_()
-        layer.forward(xs[i % n_sets], out=ys[i % n_sets], flags=flags)
-    barrier()
-
-    def timed_pass(steps):
-        """`steps` eager forwards, L2 flushed before each, one CUDA-event pair per step."""
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        barrier()
-        for a, b in ev:
-            flush.zero_()                 # evict inputs, outputs and weights from L2 between steps
-            a.record()
-            layer.forward(x, out=y, flags=flags)
-            b.record()
-        barrier()
-        return [a.elapsed_time(b) for a, b in ev]
-
-    def graph_pass(steps):
-        """`steps` forwards captured in one CUDA graph (no host launch latency between kernels),
-        replayed once between two events; returns (total ms, launches in the graph)."""
-        side = torch.cuda.Stream()
-        g = torch.cuda.CUDAGraph()
-        n0 = binding.tsvd_launch_count()
-        with torch.cuda.stream(side):
-            with torch.cuda.graph(g, stream=side):
-                for i in range(steps):
-                    layers[i % n_layers].forward(xs[i % n_sets], out=ys[i % n_sets], flags=flags)
-        n_launch = binding.tsvd_launch_count() - n0
-        g.replay()                         # one untimed replay (graph upload)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        a.record()
-        g.replay()
-        b.record()
-        barrier()
-        return a.elapsed_time(b), n_launch
-
+    flags = {"auto": 0, "simple": TSVD_FLAG_PATH_SIMPLE, "decode": TSVD_FLAG_PATH_DECODE,
+             "tensor": TSVD_FLAG_PATH_TENSOR, "index": binding.TSVD_FLAG_PATH_INDEX}[args.path]
+    if args.wide_x:
+        flags |= binding.TSVD_FLAG_WIDE_X
+    pack_flags = binding.TSVD_PACK_INDEX_LISTS if args.path == "index" else 0
+    peaks, peaks_src = load_peaks()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
-    # pass 1: the timed region proper (no per-kernel events: they cost ~5 us per kernel)
-    if args.eager:
-        launches0 = binding.tsvd_launch_count()
-        step_ms = timed_pass(args.steps)
-        launches = binding.tsvd_launch_count() - launches0
-        total_ms = float(sum(step_ms))
-        l2_note = "flushed between steps (256 MiB memset); eager launches"
-    else:
-        total_ms, launches = graph_pass(args.steps)
-        l2_note = (f"inputs larger than L2: {n_sets} rotating x/y buffer pairs ({n_sets * pair_bytes / 1e6:.0f} MB) and "
-                   f"{n_layers} packed copies of the layer ({n_layers * info['packed_bytes'] / 1e6:.0f} MB) against "
-                   f"{l2_bytes / 1e6:.0f} MB of L2; the {args.steps} steps are one CUDA graph")
-    # pass 2: the same steps again with an event pair around every kernel, for the roofline
-    binding.tsvd_profile_enable(layer.handle, True)
-    prof_step_ms = timed_pass(args.steps)
-    stage_ms, stage_n = binding.tsvd_profile_read(layer.handle)
-    binding.tsvd_profile_enable(layer.handle, False)
-    clocks = sampler.stop() if rank == 0 else None
-    total_ms = max_over_ranks(dist, total_ms, "cuda")
-    ms_per_step = total_ms / args.steps
-    value = aggregate_tokens_per_s(world, spec.B, ms_per_step)
+        time.sleep(0.5)
+
+    # ---- the headline workload ----
+    w = Workload(spec, rank, pack_flags, flags, local_rank)
+    for i in range(args.warmup):
+        w.step(i)
+    barrier()
+    want_sustained = (not args.no_sustained) and spec.name in SUSTAINED
+    head = measure(w, args.steps, args.repeats, barrier, dist, world, sustained_s=1.5 if want_sustained else 0.0)
 
     # end to end: host buffers, copies inside the timed region
-    x_host = torch.from_numpy(x_np.view(np.int16) if spec.x_dtype == "bf16" else x_np).pin_memory()
-    y_bf16 = y.dtype == torch.bfloat16
+    x_host = torch.from_numpy(w.x_np.view(np.int16) if spec.x_dtype == "bf16" else w.x_np).pin_memory()
+    y_bf16 = w.y.dtype == torch.bfloat16
     y_host = torch.empty((spec.B, spec.M), dtype=torch.int16 if y_bf16 else torch.float32).pin_memory()
     dt_code = binding.DTYPES[spec.x_dtype]
     e2e_steps = max(3, min(args.steps, 20))
     for _ in range(2):
-        binding.tsvd_forward_host(layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
+        binding.tsvd_forward_host(w.layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        binding.tsvd_forward_host(layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
+        binding.tsvd_forward_host(w.layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
     e2e_s = max_over_ranks(dist, e2e_s, "cuda")
     e2e = {"value": aggregate_tokens_per_s(world, spec.B, e2e_s * 1e3), "unit": UNIT,
            "h2d_bytes_per_step": int(x_host.numel() * x_host.element_size()),
-           "d2h_bytes_per_step": int(y_host.numel() * y_host.element_size()), "steps": e2e_steps}
+           "d2h_bytes_per_step": int(y_host.numel() * y_host.element_size()), "steps": e2e_steps,
+           "ms_per_step": e2e_s * 1e3}
+    y_e2e = (y_host.view(torch.bfloat16).float() if y_bf16 else y_host).double().numpy()
+    w.layer.forward(w.x, out=w.y, flags=flags)
+    torch.cuda.synchronize()
+    y_gpu = w.y.float().double().cpu().numpy()
+    e2e["matches_device_path"] = bool(np.array_equal(y_e2e, y_gpu))
 
     if rank != 0:
+        w.close()
         if dist:
             dist.destroy_process_group()
         return
 
-    # roofline of the dominant kernel
-    peaks, peaks_src = load_peaks()
-    plan = binding.tsvd_plan(layer.handle, spec.B, binding.DTYPES[spec.x_dtype], flags)
-    dom = int(np.argmax(stage_ms))
-    dom_ms = stage_ms[dom] / max(1, stage_n[dom])
-    pad = lambda v: (v + 127) // 128 * 128
-    if dom in (1, 3) and plan["path"] == "index":
-        # an index-list stage streams its row pointers and 16-bit entries once
-        v_bytes, u_bytes = binding.tsvd_index_bytes(layer.handle)
-        byts = float(v_bytes if dom == 1 else u_bytes)
-        achieved = byts / (dom_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": binding.STAGE_NAMES[dom] + "_index", "achieved": achieved,
-                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                    "traffic": None, "peak_source": f"{peaks_src} (of measured)", "bytes_per_launch": byts,
-                    "step_hbm_gbs": (v_bytes + u_bytes) / (ms_per_step * 1e-3) / 1e9}
-        roofline["step_hbm_frac"] = roofline["step_hbm_gbs"] / peaks["hbm_gbs"]
-    elif dom in (1, 3) and plan["path"] == "decode":
-        # a decode stage streams its packed matrix once: 2 bits per entry of the padded matrix
-        rows, contr = ((pad(spec.K), pad(spec.N)) if dom == 1 else (pad(spec.M), pad(spec.K)))
-        byts = rows * contr / 4.0
-        achieved = byts / (dom_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved,
-                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                    "traffic": recorded_traffic(spec.name, binding.STAGE_NAMES[dom]),
-                    "peak_source": f"{peaks_src} (of measured)", "bytes_per_launch": byts}
-    elif dom in (1, 3):
-        rows, contr = ((pad(spec.K), pad(spec.N)) if dom == 1 else (pad(spec.M), pad(spec.K)))
-        digits = max(1, plan["digits_x"] if dom == 1 else plan["digits_t"])
-        # executed dense operations of that launch: 2 * rows * contraction * tokens * digits
-        ops = 2.0 * rows * contr * spec.B * digits
-        if plan["path"] == "tensor":
-            peak, peak_note = peaks["bf16_tflops"] * INT8_OVER_BF16, "int8 = measured bf16 burst x 2 (nominal ratio)"
-        else:
-            peak, peak_note = peaks["bf16_tflops"], "measured bf16 burst"
-        achieved = ops / (dom_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved, "peak": peak,
-                    "unit": "TFLOP/s", "frac": achieved / peak,
-                    "traffic": recorded_traffic(spec.name, binding.STAGE_NAMES[dom]),
-                    "peak_source": f"{peak_note}; {peaks_src} (of measured)", "ops_per_launch": ops,
-                    "digits": digits}
-    else:
-        # a digit-conversion pass dominates: it is bound by HBM traffic (read values, write digits)
-        elems = spec.B * (pad(spec.N) if dom == 0 else pad(spec.K))
-        in_bytes = {"f32": 4, "bf16": 2, "i8": 1}[spec.x_dtype] if dom == 0 else 4
-        nd = plan["digits_x"] if dom == 0 else plan["digits_t"]
-        byts = float(elems) * (in_bytes + nd)
-        achieved = byts / (dom_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": binding.STAGE_NAMES[dom], "achieved": achieved,
-                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                    "traffic": None, "peak_source": f"{peaks_src} (of measured)", "bytes_per_launch": byts}
-    roofline["ms_per_launch"] = dom_ms
-    roofline["stage_ms_per_step"] = {n: m / args.steps for n, m in zip(binding.STAGE_NAMES, stage_ms)}
-    roofline["timing"] = ("second pass of the same steps with a CUDA-event pair around each kernel on its stream; "
-                          "a pair includes the launch latency, so achieved is a lower bound; ms_per_step of that pass: "
-                          f"{sum(prof_step_ms) / args.steps:.4f}")
-    roofline["plan"] = plan
-    # whole-step tensor figure: all executed tensor operations over the whole step time
-    if plan["path"] == "decode":
-        # whole-step figure: all packed bytes over the graph-timed step (both launches, no event pairs)
-        roofline["step_hbm_gbs"] = info["packed_bytes"] / (ms_per_step * 1e-3) / 1e9
-        roofline["step_hbm_frac"] = roofline["step_hbm_gbs"] / peaks["hbm_gbs"]
-    if plan["path"] == "tensor":
-        all_ops = 2.0 * spec.B * (pad(spec.K) * pad(spec.N) * plan["digits_x"] + pad(spec.M) * pad(spec.K) * plan["digits_t"])
-        roofline["step_tensor_frac"] = all_ops / (ms_per_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * INT8_OVER_BF16)
+    # ---- every workload in the same line (one GPU only) ----
+    per_config = None
+    extra = {}
+    if world == 1 and not args.no_per_config:
+        per_config = {}
+        for name in ALL_CONFIGS:
+            if name == spec.name and args.path == "auto" and not args.wide_x:
+                continue                  # the headline is filled in below
+            s2 = gen.CONFIGS[name]
+            w2 = Workload(s2, 0, 0, 0, local_rank)
+            for i in range(3):
+                w2.step(i)
+            barrier()
+            r2 = measure(w2, args.steps, args.repeats, barrier, None, 1,
+                         sustained_s=1.5 if (not args.no_sustained and name in SUSTAINED) else 0.0)
+            w2.layer.forward(w2.x, out=w2.y)
+            torch.cuda.synchronize()
+            y2 = w2.y.float().double().cpu().numpy()
+            r2["parity"] = parity_against_checker(s2, w2.U, w2.S, w2.V, w2.x_np, y2, sample_tokens(s2.B))
+            r2["status_word"] = binding.tsvd_last_status(w2.layer.handle)
+            extra[name] = (w2, r2)
+            # keep only what the summary needs; free the device memory before the next workload
+            w2.xs, w2.ys, w2.x, w2.y = None, None, None, None
+            for L in w2.layers[1:]:
+                L.close()
+            w2.layers = w2.layers[:1]
+            torch.cuda.empty_cache()
+    sampler.stop()
 
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+    def summarise(wk, r):
+        clocks = sampler.window(*r["window"])
+        roof = roofline_of(wk, peaks, peaks_src, r["ms_per_step"], r["stage_ms"], r["stage_n"], clocks["sm_mhz"])
+        out = {"us_per_step": 1e3 * r["ms_per_step"], "us_per_step_min": 1e3 * r["ms_per_step_min"],
+               "us_per_step_max": 1e3 * r["ms_per_step_max"], "tokens_per_s": r["tokens_per_s"], "path": r["path"],
+               "launches_per_step": r["launches_per_step"], "roofline": roof, "clocks": clocks,
+               "us_per_step_with_stamps": 1e3 * r["ms_per_step_with_stamps"],
+               "ms_x_mhz": r["ms_per_step"] * (clocks["sm_mhz"] or 0.0)}
+        if "sustained" in r:
+            s = dict(r["sustained"])
+            sc = sampler.window(*s.pop("window"))
+            s["clocks"] = sc
+            s["ms_x_mhz"] = s["ms_per_step"] * (sc["sm_mhz"] or 0.0)
+            if wk.plan["path"] == "tensor":
+                all_ops = 2.0 * wk.spec.B * (pad128(wk.spec.K) * pad128(wk.spec.N) * wk.plan["digits_x"] +
+                                             pad128(wk.spec.M) * pad128(wk.spec.K) * wk.plan["digits_t"])
+                s["step_tensor_frac_of_sustained_peak"] = (all_ops / (s["ms_per_step"] * 1e-3) / 1e12 /
+                                                           (peaks["bf16_tflops_sustained"] * INT8_OVER_BF16))
+            out["sustained"] = s
+        if "parity" in r:
+            out["parity"] = r["parity"]
+            out["status_word"] = r["status_word"]
+        return out
+
+    head_sum = summarise(w, head)
+    head_sum["parity"] = parity_against_checker(spec, w.U, w.S, w.V, w.x_np, y_gpu, sample_tokens(spec.B))
+    head_sum["status_word"] = binding.tsvd_last_status(w.layer.handle)
+    if per_config is not None:
+        for name in ALL_CONFIGS:
+            if name in extra:
+                w2, r2 = extra[name]
+                per_config[name] = summarise(w2, r2)
+                per_config[name]["roofline"].pop("timing", None)
+                w2.close()
+            else:
+                per_config[name] = "the headline of this line"
+
+    plan = w.plan
+    line = {"metric": METRIC, "value": head["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
             "dtype": "int64" if plan["path"] == "index" else "int32" if plan["path"] in ("tensor", "decode") else {"f32": "f32", "bf16": "f32", "i8": "int32"}[spec.x_dtype],
             "data": "synthetic",
-            "config": workload_config(spec, l2_note),
-            "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks,
-            "packed_bytes": info["packed_bytes"],
-            "algorithmic_adds_per_token": info["density_u"] * spec.M * spec.K + info["density_v"] * spec.K * spec.N,
-            "path": args.path}
+            "config": dict(workload_config(spec), l2=w.l2_note + f"; the {args.steps} steps are one CUDA graph"),
+            "timing": {"repeats": args.repeats, "statistic": "median over the replays of the graph",
+                       "ms_per_step_min": head["ms_per_step_min"], "ms_per_step_max": head["ms_per_step_max"],
+                       "ms_per_step_with_stamps": head["ms_per_step_with_stamps"],
+                       "ms_x_mhz": head_sum["ms_x_mhz"],
+                       "kind": "burst: one replay lasts milliseconds; `sustained` holds the same replays back to back for seconds"},
+            "e2e": e2e, "gpu_launches": int(head["launches"]), "roofline": head_sum["roofline"], "clocks": head_sum["clocks"],
+            "packed_bytes": w.info["packed_bytes"],
+            "algorithmic_adds_per_token": w.info["density_u"] * spec.M * spec.K + w.info["density_v"] * spec.K * spec.N,
+            "path": args.path, "parity_on_cpu_sample": head_sum["parity"], "status_word": head_sum["status_word"]}
+    if "sustained" in head_sum:
+        line["sustained"] = head_sum["sustained"]
+    if per_config is not None:
+        line["per_config"] = per_config
     if world == 1 and not args.no_cpu_baseline:
-        y_gpu = y.float().double().cpu().numpy()
-        cb, parity = cpu_baseline(spec, U, S, V, x_np, y_gpu=y_gpu)
-        line["cpu_baseline"] = cb
-        line["parity_on_cpu_sample"] = parity
+        line["cpu_baseline"] = cpu_baseline(spec, w.U, w.S, w.V, w.x_np)
     print(json.dumps(line), flush=True)
-    for extra in layers:
-        extra.close()
+    w.close()
     if dist:
         dist.destroy_process_group()
 

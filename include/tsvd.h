@@ -254,16 +254,25 @@ tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, unsigned fla
 
 /*
  * Per-stage device timing (measurement support; the paper reports operation counts
- * per stage in Table S1 and no timings).  While enabled, every forward on the handle
- * records CUDA events on its own stream around each kernel it launches.
- * tsvd_profile_read waits for those events, then returns, per stage, the summed
- * device time in milliseconds and the number of launches since the last read (both
- * arrays have TSVD_N_STAGES entries), and resets the sums.
+ * per stage in Table S1 and no timings).
+ *   mode 0  off
+ *   mode 1  every forward on the handle records a CUDA-event pair on its stream around
+ *           each kernel it launches (eager streams only; a pair includes the launch
+ *           latency of a short kernel)
+ *   mode 2  every kernel launched for the handle writes the device's nanosecond timer
+ *           itself: its first CTA once its wait for the kernel before it has ended, and
+ *           every warp when it finishes (the maximum is kept).  This works inside a
+ *           captured CUDA graph: each captured launch owns a pair of words, which every
+ *           replay overwrites.  Up to 32768 launches are recorded after the call.
+ * tsvd_profile_read synchronises, then returns, per stage, the summed device time in
+ * milliseconds and the number of launches (both arrays have TSVD_N_STAGES entries).  In
+ * mode 1 it covers the launches since the last read and resets the sums; in mode 2 it
+ * covers every launch recorded since tsvd_profile_enable, as last executed.
  *   stage 0: activations -> integer digits     stage 1: V-stage (+ S scale)
  *   stage 2: S*(V x)     -> integer digits     stage 3: U-stage
  */
 #define TSVD_N_STAGES 4
-tsvd_status_t tsvd_profile_enable(tsvd_handle_t h, int on);
+tsvd_status_t tsvd_profile_enable(tsvd_handle_t h, int mode);
 tsvd_status_t tsvd_profile_read(tsvd_handle_t h, float* ms_sum, unsigned* launches);
 
 /* Number of kernels this library has launched in this process (all handles). */

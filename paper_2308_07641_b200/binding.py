@@ -207,8 +207,10 @@ N_STAGES = 4
 STAGE_NAMES = ("x_digits", "v_stage", "t_digits", "u_stage")
 
 
-def tsvd_profile_enable(h: int, on: bool) -> None:
-    _check(lib().tsvd_profile_enable(h, 1 if on else 0), "tsvd_profile_enable")
+def tsvd_profile_enable(h: int, mode) -> None:
+    """mode 0/False: off; 1/True: CUDA-event pairs around every kernel; 2: time stamps written by
+    the kernels themselves (works inside a captured graph)."""
+    _check(lib().tsvd_profile_enable(h, int(mode)), "tsvd_profile_enable")
 
 
 def tsvd_profile_read(h: int):

@@ -45,6 +45,13 @@ void StageProfiler::end(cudaStream_t s)
     cudaEventRecord(pending.back().b, s);
 }
 
+unsigned long long* StageProfiler::slot(int stage)
+{
+    if (mode != 2 || !stamps || slot_stage.size() >= (size_t)TSVD_STAMP_SLOTS) return nullptr;
+    slot_stage.push_back(stage);
+    return stamps + 2 * (slot_stage.size() - 1);
+}
+
 void StageProfiler::drain()
 {
     for (auto& p : pending) {
@@ -60,18 +67,48 @@ void StageProfiler::drain()
     pending.clear();
 }
 
-extern "C" tsvd_status_t tsvd_profile_enable(tsvd_handle_t h, int on)
+extern "C" tsvd_status_t tsvd_profile_enable(tsvd_handle_t h, int mode)
 {
     if (!h) return TSVD_E_NULL;
+    if (mode < 0 || mode > 2) return TSVD_E_DTYPE;
     h->prof.drain();
     for (int i = 0; i < TSVD_N_STAGES; ++i) { h->prof.ms[i] = 0.f; h->prof.launches[i] = 0; }
-    h->prof.on = on != 0;
+    h->prof.slot_stage.clear();
+    h->prof.mode = mode;
+    h->prof.on = mode == 1;
+    if (mode == 2) {
+        const size_t bytes = (size_t)TSVD_STAMP_SLOTS * 2 * sizeof(unsigned long long);
+        if (!h->prof.stamps && cudaMalloc(&h->prof.stamps, bytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            h->prof.stamps = nullptr;
+            h->prof.mode = 0;
+            return TSVD_E_NOMEM;
+        }
+        TSVD_CUDA_OK(cudaMemset(h->prof.stamps, 0, bytes));
+    }
     return TSVD_OK;
 }
 
 extern "C" tsvd_status_t tsvd_profile_read(tsvd_handle_t h, float* ms_sum, unsigned* launches)
 {
     if (!h || !ms_sum || !launches) return TSVD_E_NULL;
+    if (h->prof.mode == 2) {
+        // the pairs of every launch recorded since tsvd_profile_enable, as the kernels last wrote them
+        const size_t n = h->prof.slot_stage.size();
+        std::vector<unsigned long long> host(2 * n + 2);
+        TSVD_CUDA_OK(cudaDeviceSynchronize());
+        if (n) TSVD_CUDA_OK(cudaMemcpy(host.data(), h->prof.stamps, 2 * n * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+        for (int i = 0; i < TSVD_N_STAGES; ++i) { ms_sum[i] = 0.f; launches[i] = 0; }
+        double ns[TSVD_N_STAGES] = {0, 0, 0, 0};
+        for (size_t i = 0; i < n; ++i) {
+            const unsigned long long b = host[2 * i], e = host[2 * i + 1];
+            if (b == 0 || e <= b) continue;     // never ran
+            ns[h->prof.slot_stage[i]] += (double)(e - b);
+            launches[h->prof.slot_stage[i]] += 1;
+        }
+        for (int i = 0; i < TSVD_N_STAGES; ++i) ms_sum[i] = (float)(ns[i] * 1e-6);
+        return TSVD_OK;
+    }
     h->prof.drain();
     for (int i = 0; i < TSVD_N_STAGES; ++i) {
         ms_sum[i] = h->prof.ms[i];
@@ -97,6 +134,7 @@ static void free_handle(tsvd_handle_s* h)
     if (h->ws) cudaFree(h->ws);
     if (h->io) cudaFree(h->io);
     if (h->dev_status) cudaFree(h->dev_status);
+    if (h->prof.stamps) cudaFree(h->prof.stamps);
     (void)cudaGetLastError();
     delete h;
 }

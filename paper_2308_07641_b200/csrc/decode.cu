@@ -48,6 +48,7 @@ struct GemvParams {
     int z_int;
     const float* bias;    // U-stage, optional (padded to R_pad): added before the output rounding
     int* status;          // device status word (range diagnostic)
+    unsigned long long* stamp;   // time stamps of this launch, or null
 };
 
 // D (16 x 8, int32) += A (16 x 32, int8, rows) * B (32 x 8, int8, columns).  Lane (g, q):
@@ -127,6 +128,7 @@ ternary_gemv_kernel(const GemvParams p)
     // still reads t or y is never overtaken.  The next kernel in the stream may start likewise.
     pdl_wait();
     pdl_launch_dependents();
+    tsvd_stamp_begin(p.stamp);
 
     // ---- the stage's input as fixed-point digits (every CTA makes its own copy).  A thread takes
     //      chunks of 8 consecutive columns; all loads of a pass are independent, so a pass costs
@@ -346,6 +348,7 @@ ternary_gemv_kernel(const GemvParams p)
             }
         }
     }
+    tsvd_stamp_end(p.stamp);
 }
 
 size_t gemv_smem_bytes(int nd, int ntok, int C_pad)
@@ -408,7 +411,7 @@ tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws)
     p.in = a.x; p.ld_in = a.ldx; p.B = a.B; p.S = h->S;
     p.out = t; p.ld_out = h->V.R_pad;
     p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
-    p.status = h->dev_status;
+    p.status = h->dev_status; p.stamp = h->prof.slot(1);
     cudaError_t e;
     h->prof.begin(1, st);
     switch (a.dtype) {
@@ -428,7 +431,7 @@ tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws)
     q.in = t; q.ld_in = h->V.R_pad; q.B = a.B;
     q.out = a.y; q.ld_out = a.ldy;
     q.out_bf16 = (a.dtype == TSVD_BF16) && !a.out_f32;
-    q.bias = h->bias; q.status = h->dev_status;
+    q.bias = h->bias; q.status = h->dev_status; q.stamp = h->prof.slot(3);
     h->prof.begin(3, st);
     e = launch_gemv_tokens<float, ND_T, STAGE_U>(q, h->U.R_pad, st);
     h->prof.end(st);

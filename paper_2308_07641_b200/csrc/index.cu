@@ -41,6 +41,7 @@ struct IndexParams {
     int z_int;
     const float* bias;         // U-stage, optional: added before the output rounding
     int* status;               // device status word (range diagnostic)
+    unsigned long long* stamp; // time stamps of this launch, or null
 };
 
 // grid: ceil(R / 16) CTAs of 512 threads.  Dynamic shared memory:
@@ -65,6 +66,7 @@ ternary_index_kernel(const IndexParams p)
     // and its output written, only after this wait
     pdl_wait();
     pdl_launch_dependents();
+    tsvd_stamp_begin(p.stamp);
 
     // ---- the stage's input as fixed-point integers ----
     const int n_chunks = p.C_pad >> 3;
@@ -171,6 +173,7 @@ ternary_index_kernel(const IndexParams p)
                 reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + row] = yv;
         }
     }
+    tsvd_stamp_end(p.stamp);
 }
 
 size_t index_smem_bytes(int ntok, int C_pad)
@@ -258,7 +261,7 @@ tsvd_status_t tsvd_forward_index(const ForwardArgs& a, void* ws)
     p.in = a.x; p.ld_in = a.ldx; p.B = a.B; p.S = h->S;
     p.out = t; p.ld_out = h->V.R_pad;
     p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
-    p.status = h->dev_status;
+    p.status = h->dev_status; p.stamp = h->prof.slot(1);
     cudaError_t e;
     h->prof.begin(1, st);
     switch (a.dtype) {
@@ -277,7 +280,7 @@ tsvd_status_t tsvd_forward_index(const ForwardArgs& a, void* ws)
     u.in = t; u.ld_in = h->V.R_pad; u.B = a.B;
     u.out = a.y; u.ld_out = a.ldy;
     u.out_bf16 = (a.dtype == TSVD_BF16) && !a.out_f32;
-    u.bias = h->bias; u.status = h->dev_status;
+    u.bias = h->bias; u.status = h->dev_status; u.stamp = h->prof.slot(3);
     h->prof.begin(3, st);
     e = launch_index_tokens<float, ND_T, STAGE_U>(u, st);
     h->prof.end(st);

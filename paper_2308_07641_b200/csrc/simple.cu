@@ -28,8 +28,10 @@ __global__ void __launch_bounds__(128)
 ternary_rows_kernel(const uint4* __restrict__ units, int R, int C, int C_pad,
                     const IN_T* __restrict__ in, int ld_in, int B,
                     const float* __restrict__ S, void* __restrict__ out, int ld_out,
-                    void* __restrict__ z_out, int z_ld)   // S: the scales (V-stage) or the optional bias (U-stage)
+                    void* __restrict__ z_out, int z_ld,   // S: the scales (V-stage) or the optional bias (U-stage)
+                    unsigned long long* __restrict__ stamp)
 {
+    tsvd_stamp_begin(stamp);
     constexpr bool kInt = sizeof(IN_T) == 1;
     using acc_t = typename Acc<IN_T>::type;
     using part_t = typename std::conditional<kInt, int, float>::type;
@@ -81,7 +83,7 @@ ternary_rows_kernel(const uint4* __restrict__ units, int R, int C, int C_pad,
         for (int t = 0; t < TB; ++t) acc[t] += (acc_t)part[t];
     }
 
-    if (row >= R) return;
+    if (row >= R) { tsvd_stamp_end(stamp); return; }
 #pragma unroll
     for (int t = 0; t < TB; ++t) {
         const int b = b0 + t;
@@ -105,15 +107,16 @@ ternary_rows_kernel(const uint4* __restrict__ units, int R, int C, int C_pad,
                 reinterpret_cast<__nv_bfloat16*>(out)[(size_t)b * ld_out + row] = __float2bfloat16_rn(yv);
         }
     }
+    tsvd_stamp_end(stamp);
 }
 
 template <typename IN_T, int EPI>
 cudaError_t launch(const PackedMat& pm, const IN_T* in, int ld_in, int B, const float* S, void* out,
-                   int ld_out, void* z_out, int z_ld, cudaStream_t stream)
+                   int ld_out, void* z_out, int z_ld, cudaStream_t stream, unsigned long long* stamp = nullptr)
 {
     dim3 grid(pm.R_pad / TSVD_ROW_TILE, (B + TB - 1) / TB);
     ternary_rows_kernel<IN_T, EPI><<<grid, 128, 0, stream>>>(pm.units, pm.R, pm.C, pm.C_pad, in, ld_in,
-                                                             B, S, out, ld_out, z_out, z_ld);
+                                                             B, S, out, ld_out, z_out, z_ld, stamp);
     tsvd_count_launch();
     return cudaGetLastError();
 }
@@ -129,20 +132,21 @@ tsvd_status_t tsvd_forward_simple(const ForwardArgs& a)
 {
     tsvd_handle_s* h = a.h;
     cudaError_t e;
+    unsigned long long* const stamp_v = h->prof.slot(1);
     h->prof.begin(1, a.stream);
     // V-stage + S-stage: t[b,k] = S[k] * sum_n V[k,n] x[b,n]
     switch (a.dtype) {
         case TSVD_F32:
             e = launch<float, EPI_SCALE_TO_T>(h->V, (const float*)a.x, a.ldx, a.B, h->S, a.t, a.t_ld,
-                                              a.z_out, h->K, a.stream);
+                                              a.z_out, h->K, a.stream, stamp_v);
             break;
         case TSVD_BF16:
             e = launch<__nv_bfloat16, EPI_SCALE_TO_T>(h->V, (const __nv_bfloat16*)a.x, a.ldx, a.B, h->S,
-                                                      a.t, a.t_ld, a.z_out, h->K, a.stream);
+                                                      a.t, a.t_ld, a.z_out, h->K, a.stream, stamp_v);
             break;
         case TSVD_I8:
             e = launch<int8_t, EPI_SCALE_TO_T>(h->V, (const int8_t*)a.x, a.ldx, a.B, h->S, a.t, a.t_ld,
-                                               a.z_out, h->K, a.stream);
+                                               a.z_out, h->K, a.stream, stamp_v);
             break;
         default:
             return TSVD_E_DTYPE;
@@ -152,10 +156,11 @@ tsvd_status_t tsvd_forward_simple(const ForwardArgs& a)
     h->prof.begin(3, a.stream);
     // U-stage: y[b,m] = sum_k U[m,k] t[b,k]
     const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;
+    unsigned long long* const stamp_u = h->prof.slot(3);
     if (bf16_out)
-        e = launch<float, EPI_Y_BF16>(h->U, a.t, a.t_ld, a.B, h->bias, a.y, a.ldy, nullptr, 0, a.stream);
+        e = launch<float, EPI_Y_BF16>(h->U, a.t, a.t_ld, a.B, h->bias, a.y, a.ldy, nullptr, 0, a.stream, stamp_u);
     else
-        e = launch<float, EPI_Y_F32>(h->U, a.t, a.t_ld, a.B, h->bias, a.y, a.ldy, nullptr, 0, a.stream);
+        e = launch<float, EPI_Y_F32>(h->U, a.t, a.t_ld, a.B, h->bias, a.y, a.ldy, nullptr, 0, a.stream, stamp_u);
     h->prof.end(a.stream);
     return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
 }

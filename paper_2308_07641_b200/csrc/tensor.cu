@@ -82,7 +82,8 @@ template <typename IN_T, int ND, int TPT, int TOK, int CH>
 __global__ void __launch_bounds__(256, 4)   // <= 64 registers: a batch of 4096 tokens is then one wave
 digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
-                int* __restrict__ zero_buf, int zero_per_token, int zero_total, int* __restrict__ status)
+                int* __restrict__ zero_buf, int zero_per_token, int zero_total, int* __restrict__ status,
+                unsigned long long* __restrict__ stamp)
 {
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
@@ -98,6 +99,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     // read or written before that kernel has completed; the next kernel may be set up meanwhile
     pdl_wait();
     pdl_launch_dependents();
+    tsvd_stamp_begin(stamp);
     __shared__ float red[8];
     const int jt = b / TOK, b_in = b % TOK;
     const bool live = b < B;
@@ -220,6 +222,7 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     if constexpr (!kInt) {
         if (tsvd_range_flagged(range_cnt) && (threadIdx.x & 31) == 0) atomicOr(status, TSVD_DEV_RANGE);
     }
+    tsvd_stamp_end(stamp);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -262,6 +265,7 @@ struct GemmParams {
     int y_bf16;
     int nb;               // depth of the digit-tile ring in steps: NB, or (resident) a whole number of panels
     int resident;         // the digit tiles of a token tile stay in shared memory across row tiles
+    unsigned long long* stamp;   // time stamps of this launch, or null
     int wait_limit;       // bound of every barrier wait in units of 2^20 clocks (0: default, ~2 s)
     int test_stall;       // test hook: the digit tiles are never copied, so the waits must give up
 };
@@ -397,6 +401,7 @@ ternary_mma_kernel(const GemmParams p)
     // kernel writes), may overlap with that kernel; all other warps wait for it to complete.
     if (warp != 2) pdl_wait();
     pdl_launch_dependents();
+    tsvd_stamp_begin(p.stamp);
 
     // Waiting for parity 1 on a barrier that has not completed a phase yet returns at once,
     // which is what a consumer-release barrier needs on its first use.
@@ -757,6 +762,7 @@ ternary_mma_kernel(const GemmParams p)
     tc_fence_before_sync();
     __syncthreads();
     if (*abort_flag && threadIdx.x == 0) atomicOr(p.status, TSVD_DEV_TIMEOUT);
+    if (threadIdx.x == 0) tsvd_stamp_end(p.stamp);
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, TMEM_COLS);
@@ -766,7 +772,7 @@ ternary_mma_kernel(const GemmParams p)
 template <typename IN_T, int ND, int TOK = tokens_per_tile(ND)>
 cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, const unsigned* amax_bits,
                             int8_t* D, float* scale, int* zero_buf, int zero_total, int* status,
-                            cudaStream_t stream)
+                            unsigned long long* stamp, cudaStream_t stream)
 {
     const int B_pad = (B + TOK - 1) / TOK * TOK;
     const int zero_per_token = (zero_total + B_pad - 1) / B_pad;   // every token slot clears a share
@@ -778,13 +784,13 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
         // round and the row still fits the registers (three chunks of 8 per lane)
         if ((KB * 8) % 32 != 0 && KB * 16 <= 3 * 32)
             e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK, 8>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                                   scale, zero_buf, zero_per_token, zero_total, status);
+                                   scale, zero_buf, zero_per_token, zero_total, status, stamp);
         else
             e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK, 16>, in, ld_in, B, B_pad, C, KB, amax_bits,
-                                   D, scale, zero_buf, zero_per_token, zero_total, status);
+                                   D, scale, zero_buf, zero_per_token, zero_total, status, stamp);
     } else {
         e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 256, TOK, 16>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                               scale, zero_buf, zero_per_token, zero_total, status);
+                               scale, zero_buf, zero_per_token, zero_total, status, stamp);
     }
     tsvd_count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
@@ -945,7 +951,7 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
 
     h->prof.begin(0, st);
     e = launch_digitise<IN_T, NDX, SMALL_TOK>((const IN_T*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                              w.zacc, w.zacc_ints, h->dev_status, st);
+                                              w.zacc, w.zacc_ints, h->dev_status, h->prof.slot(0), st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
@@ -956,7 +962,7 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
     p.acc = w.zacc; p.acc_ld = h->V.R_pad;
     p.tmax = reinterpret_cast<unsigned*>(w.zacc + (size_t)Bp * NDX * h->V.R_pad);
     p.tile_done = w.zacc + (size_t)Bp * NDX * h->V.R_pad + Bp;
-    p.tail = TAIL_T;
+    p.tail = TAIL_T; p.stamp = h->prof.slot(1);
     const int v_tiles = h->V.R_pad / BLOCK_R;
     p.ksplit = pick_ksplit(v_tiles * j_tiles, KBv);
     h->prof.begin(1, st);
@@ -966,7 +972,7 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
 
     h->prof.begin(2, st);
     e = launch_digitise<float, ND_T, SMALL_TOK>(w.t, h->V.R_pad, a.B, h->K, KBu, p.tmax, w.Dt, w.scale_t, w.yacc,
-                                                w.yacc_ints, h->dev_status, st);
+                                                w.yacc_ints, h->dev_status, h->prof.slot(2), st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
@@ -976,7 +982,7 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
     q.y_bf16 = (a.dtype == TSVD_BF16) && !a.out_f32;
     q.acc = w.yacc; q.acc_ld = h->U.R_pad;
     q.tile_done = w.yacc + (size_t)Bp * ND_T * h->U.R_pad;
-    q.tail = TAIL_Y;
+    q.tail = TAIL_Y; q.stamp = h->prof.slot(3);
     const int u_tiles = h->U.R_pad / BLOCK_R;
     q.ksplit = pick_ksplit(u_tiles * j_tiles, KBu);
     h->prof.begin(3, st);
@@ -1016,23 +1022,24 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     cudaError_t e;
 
     // stage 0: activations -> digits
+    unsigned long long* const stamp0 = h->prof.slot(0);
     h->prof.begin(0, st);
     switch (a.dtype) {
         case TSVD_F32:
             e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, nullptr, 0,
-                                          h->dev_status, st);
+                                          h->dev_status, stamp0, st);
             break;
         case TSVD_BF16:
             if (wide_bf16)
                 e = launch_digitise<__nv_bfloat16, 4>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
-                                                      w.scale_x, nullptr, 0, h->dev_status, st);
+                                                      w.scale_x, nullptr, 0, h->dev_status, stamp0, st);
             else
                 e = launch_digitise<__nv_bfloat16, 3>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
-                                                      w.scale_x, nullptr, 0, h->dev_status, st);
+                                                      w.scale_x, nullptr, 0, h->dev_status, stamp0, st);
             break;
         case TSVD_I8:
             e = launch_digitise<int8_t, 1>((const int8_t*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                           nullptr, 0, h->dev_status, st);
+                                           nullptr, 0, h->dev_status, stamp0, st);
             break;
         default:
             return TSVD_E_DTYPE;
@@ -1044,7 +1051,7 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     p.units = h->V.units; p.KB = KBv; p.R = h->K; p.D = w.Dx; p.scale = w.scale_x; p.B = a.B;
     p.S = h->S; p.t = w.t; p.t_ld = h->V.R_pad;
     p.z_out = a.z_out; p.z_ld = h->K; p.z_int = (a.dtype == TSVD_I8);
-    p.status = h->dev_status;
+    p.status = h->dev_status; p.stamp = h->prof.slot(1);
     if (a.test_stall) { p.test_stall = 1; p.wait_limit = 16; }   // ~8 ms instead of ~2 s
     const int v_tiles = h->V.R_pad / BLOCK_R;
     h->prof.begin(1, st);
@@ -1057,14 +1064,14 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     // stage 2: t -> digits (each token's scale comes from its own max |t|)
     h->prof.begin(2, st);
     e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, 0,
-                                     h->dev_status, st);
+                                     h->dev_status, h->prof.slot(2), st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
     // stage 3: U-stage
     GemmParams q{};
     q.units = h->U.units; q.KB = KBu; q.R = h->M; q.D = w.Dt; q.scale = w.scale_t; q.B = a.B;
-    q.y = a.y; q.ldy = a.ldy; q.status = h->dev_status; q.bias = h->bias;
+    q.y = a.y; q.ldy = a.ldy; q.status = h->dev_status; q.bias = h->bias; q.stamp = h->prof.slot(3);
     const int u_tiles = h->U.R_pad / BLOCK_R;
     const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;
     h->prof.begin(3, st);

@@ -74,17 +74,27 @@ __device__ __forceinline__ void tsvd_expand16(uint32_t w, uint32_t out[4])
     tsvd_expand8((w >> 2) & 0x33333333u, out[2], out[3]);
 }
 
-// Event-pair recorder behind tsvd_profile_enable / tsvd_profile_read.
+// Per-kernel timing behind tsvd_profile_enable / tsvd_profile_read.  Mode 1: a CUDA-event pair
+// around every launch (eager streams only; a pair carries the launch latency).  Mode 2: the kernels
+// themselves write the global nanosecond timer into a pair of words per launch -- the first CTA when
+// its wait for the previous kernel ends, every warp when it finishes (maximum) -- which also works
+// inside a captured graph: each captured launch keeps its own pair and every replay overwrites it
+// (the timer only grows, so the maximum needs no reset).
 struct StageProfiler {
-    bool on = false;
+    int mode = 0;
+    bool on = false;            // mode 1
     struct Pair { cudaEvent_t a, b; int stage; };
     std::vector<Pair> pending;
     float ms[TSVD_N_STAGES] = {0, 0, 0, 0};
     unsigned launches[TSVD_N_STAGES] = {0, 0, 0, 0};
+    unsigned long long* stamps = nullptr;   // mode 2: device, [TSVD_STAMP_SLOTS][2] = {begin, end}
+    std::vector<int> slot_stage;            // stage of every slot handed out
     void begin(int stage, cudaStream_t s);
     void end(cudaStream_t s);
     void drain();
+    unsigned long long* slot(int stage);    // mode 2: this launch's pair (null when off or full)
 };
+constexpr int TSVD_STAMP_SLOTS = 1 << 15;
 
 struct tsvd_handle_s {
     int device = 0;
@@ -131,6 +141,21 @@ struct PdlLaunch {
     PdlLaunch& operator=(const PdlLaunch&) = delete;
 };
 #ifdef __CUDACC__
+__device__ __forceinline__ unsigned long long tsvd_globaltimer()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Time stamps of one launch (see StageProfiler, mode 2); `s` is null unless profiling is on.
+__device__ __forceinline__ void tsvd_stamp_begin(unsigned long long* s)
+{
+    if (s && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) s[0] = tsvd_globaltimer();
+}
+__device__ __forceinline__ void tsvd_stamp_end(unsigned long long* s)   // every warp, at its end
+{
+    if (s && (threadIdx.x & 31) == 0) atomicMax(s + 1, tsvd_globaltimer());
+}
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
