@@ -83,8 +83,10 @@ typedef enum {
  * codes against fixed-point digits of the stage's input held in shared memory) serve batches
  * of at most this many tokens, and are what a forward of so few tokens runs by default.
  * Forcing them for a larger batch, or for a contraction too long for the digits to fit in
- * shared memory (about 10,000 columns at four tokens), returns TSVD_E_TOOBIG. */
-#define TSVD_DECODE_MAX_B 4
+ * shared memory (about 10,000 columns at four tokens, 6,000 at eight), returns TSVD_E_TOOBIG. */
+#define TSVD_DECODE_MAX_B 8
+/* the index-list kernels serve at most this many tokens */
+#define TSVD_INDEX_MAX_B 4
 /* Test hook for the bounded device-side waits: with B > 64 the V-stage kernel's copy
  * producer withholds the activation digits, so every wait on them runs out (after a few
  * milliseconds instead of the usual ~2 s); all CTAs then leave through their normal exit,
@@ -93,7 +95,7 @@ typedef enum {
 #define TSVD_FLAG_TEST_STALL 0x100u
 
 /* tsvd_pack flag: also keep U and V as index lists -- per row the list of its nonzeros, 16
- * bits each, (column << 1) | (1 for -1) -- for forwards of up to TSVD_DECODE_MAX_B tokens with
+ * bits each, (column << 1) | (1 for -1) -- for forwards of up to TSVD_INDEX_MAX_B tokens with
  * TSVD_FLAG_PATH_INDEX.  The paper calls 2 bits per element a redundant code for sparse U
  * and V (Section "Connection with BNN and What Next"); this form is the smaller one below a
  * nonzero rate of 1/8 and its forward does exactly the additions of Table S1, one per nonzero.

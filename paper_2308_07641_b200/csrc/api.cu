@@ -49,7 +49,7 @@ unsigned long long* StageProfiler::slot(int stage)
 {
     if (mode != 2 || !stamps || slot_stage.size() >= (size_t)TSVD_STAMP_SLOTS) return nullptr;
     slot_stage.push_back(stage);
-    return stamps + 2 * (slot_stage.size() - 1);
+    return stamps + TSVD_STAMP_WORDS * (slot_stage.size() - 1);
 }
 
 void StageProfiler::drain()
@@ -77,7 +77,7 @@ extern "C" tsvd_status_t tsvd_profile_enable(tsvd_handle_t h, int mode)
     h->prof.mode = mode;
     h->prof.on = mode == 1;
     if (mode == 2) {
-        const size_t bytes = (size_t)TSVD_STAMP_SLOTS * 2 * sizeof(unsigned long long);
+        const size_t bytes = (size_t)TSVD_STAMP_SLOTS * TSVD_STAMP_WORDS * sizeof(unsigned long long);
         if (!h->prof.stamps && cudaMalloc(&h->prof.stamps, bytes) != cudaSuccess) {
             (void)cudaGetLastError();
             h->prof.stamps = nullptr;
@@ -89,19 +89,32 @@ extern "C" tsvd_status_t tsvd_profile_enable(tsvd_handle_t h, int mode)
     return TSVD_OK;
 }
 
+#ifdef TSVD_PHASES
+// development builds only: the raw words of the first `n` recorded launches and their stages
+extern "C" int tsvd_debug_phases(tsvd_handle_t h, unsigned long long* out, int* stages, int n)
+{
+    cudaDeviceSynchronize();
+    const int have = (int)h->prof.slot_stage.size();
+    if (n > have) n = have;
+    cudaMemcpy(out, h->prof.stamps, (size_t)n * TSVD_STAMP_WORDS * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+    for (int i = 0; i < n; ++i) stages[i] = h->prof.slot_stage[i];
+    return n;
+}
+#endif
+
 extern "C" tsvd_status_t tsvd_profile_read(tsvd_handle_t h, float* ms_sum, unsigned* launches)
 {
     if (!h || !ms_sum || !launches) return TSVD_E_NULL;
     if (h->prof.mode == 2) {
         // the pairs of every launch recorded since tsvd_profile_enable, as the kernels last wrote them
         const size_t n = h->prof.slot_stage.size();
-        std::vector<unsigned long long> host(2 * n + 2);
+        std::vector<unsigned long long> host(TSVD_STAMP_WORDS * n + 2);
         TSVD_CUDA_OK(cudaDeviceSynchronize());
-        if (n) TSVD_CUDA_OK(cudaMemcpy(host.data(), h->prof.stamps, 2 * n * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+        if (n) TSVD_CUDA_OK(cudaMemcpy(host.data(), h->prof.stamps, TSVD_STAMP_WORDS * n * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
         for (int i = 0; i < TSVD_N_STAGES; ++i) { ms_sum[i] = 0.f; launches[i] = 0; }
         double ns[TSVD_N_STAGES] = {0, 0, 0, 0};
         for (size_t i = 0; i < n; ++i) {
-            const unsigned long long b = host[2 * i], e = host[2 * i + 1];
+            const unsigned long long b = host[TSVD_STAMP_WORDS * i], e = host[TSVD_STAMP_WORDS * i + 1];
             if (b == 0 || e <= b) continue;     // never ran
             ns[h->prof.slot_stage[i]] += (double)(e - b);
             launches[h->prof.slot_stage[i]] += 1;
@@ -287,7 +300,7 @@ static tsvd_status_t ensure_ws(tsvd_handle_s* h, size_t bytes)
 // the decode kernels when the digits of the stage inputs fit in shared memory; everything else
 // runs the tensor-core kernels (which serve every batch size); the CUDA-core kernels remain as
 // the plain reference path, and the index-list kernels (handles packed with index lists, up to
-// TSVD_DECODE_MAX_B tokens) are run on request.  Returns 0 when a forced path cannot serve the request.
+// TSVD_INDEX_MAX_B tokens) are run on request.  Returns 0 when a forced path cannot serve the request.
 static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, unsigned forced, bool wide_x)
 {
     if (forced == TSVD_FLAG_PATH_SIMPLE) return TSVD_FLAG_PATH_SIMPLE;
@@ -377,7 +390,7 @@ extern "C" tsvd_status_t tsvd_reserve(tsvd_handle_t h, int B_max, tsvd_dtype_t d
     TSVD_CUDA_OK(cudaGetDevice(&dev));
     if (dev != h->device) return TSVD_E_CUDA;
     size_t need = 0;
-    const int marks[] = {B_max, 64, TSVD_DECODE_MAX_B};
+    const int marks[] = {B_max, 64, TSVD_DECODE_MAX_B, TSVD_INDEX_MAX_B};
     for (int B : marks) {
         if (B > B_max) continue;
         for (int wide = 0; wide < 2; ++wide) {

@@ -1,4 +1,4 @@
-// Decode path: y = U(diag(S)(V x)) for one to four tokens, bound by streaming the packed codes.
+// Decode path: y = U(diag(S)(V x)) for one to eight tokens, bound by streaming the packed codes.
 //
 // For so few tokens a 128-row tcgen05 tile is almost empty, and what matters is that every SM
 // streams its share of the 2-bit codes (the whole of U and V is read once per forward) with as
@@ -134,107 +134,113 @@ ternary_gemv_kernel(const GemvParams p)
     //      chunks of 8 consecutive columns; all loads of a pass are independent, so a pass costs
     //      about one trip to L2, and the first chunk of each token stays in registers between the
     //      maximum pass and the conversion pass ----
+    // Up to four tokens are converted at a time (eight tokens: two such passes, whose working set
+    // still fits the registers).
     const int n_chunks = p.C_pad >> 3;
-    float keep[NTOK][8];
-    float qscale[NTOK];
+    constexpr int TB = NTOK < 4 ? NTOK : 4;
 #pragma unroll
-    for (int b = 0; b < NTOK; ++b) qscale[b] = 1.f;
-    // tokens beyond the batch re-read token 0 (the loads of all tokens are then unconditional and go
-    // out together); what they read is never used
-    const IN_T* rows[NTOK];
-    bool vec_ok[NTOK];
-#pragma unroll
-    for (int b = 0; b < NTOK; ++b) {
-        rows[b] = in + (size_t)(b < p.B ? b : 0) * p.ld_in;
-        vec_ok[b] = ((reinterpret_cast<uintptr_t>(rows[b])) & 15) == 0;
-    }
-    bool all_vec = true;   // every token's row allows vector loads: one test per chunk, and the loads in a row
-#pragma unroll
-    for (int b = 0; b < NTOK; ++b) all_vec = all_vec && vec_ok[b];
-    auto load_tokens = [&](int ch, float (&v)[NTOK][8]) {
-        if (all_vec && ch * 8 + 8 <= p.C) {
-#pragma unroll
-            for (int b = 0; b < NTOK; ++b) load8<IN_T>(rows[b], ch * 8, 0x7fffffff, true, v[b]);
-        } else {
-#pragma unroll
-            for (int b = 0; b < NTOK; ++b) load8<IN_T>(rows[b], ch * 8, p.C, vec_ok[b], v[b]);
+    for (int b0 = 0; b0 < NTOK; b0 += TB) {
+        float keep[TB][8];
+        float qscale[TB];
+    #pragma unroll
+        for (int b = 0; b < TB; ++b) qscale[b] = 1.f;
+        // tokens beyond the batch re-read token 0 (the loads of all tokens are then unconditional and go
+        // out together); what they read is never used
+        const IN_T* rows[TB];
+        bool vec_ok[TB];
+    #pragma unroll
+        for (int b = 0; b < TB; ++b) {
+            rows[b] = in + (size_t)(b0 + b < p.B ? b0 + b : 0) * p.ld_in;
+            vec_ok[b] = ((reinterpret_cast<uintptr_t>(rows[b])) & 15) == 0;
         }
-    };
-    if constexpr (!kInt) {
-        float amax[NTOK];
-#pragma unroll
-        for (int b = 0; b < NTOK; ++b) amax[b] = 0.f;
+        bool all_vec = true;   // every token's row allows vector loads: one test per chunk, and the loads in a row
+    #pragma unroll
+        for (int b = 0; b < TB; ++b) all_vec = all_vec && vec_ok[b];
+        auto load_tokens = [&](int ch, float (&v)[TB][8]) {
+            if (all_vec && ch * 8 + 8 <= p.C) {
+    #pragma unroll
+                for (int b = 0; b < TB; ++b) load8<IN_T>(rows[b], ch * 8, 0x7fffffff, true, v[b]);
+            } else {
+    #pragma unroll
+                for (int b = 0; b < TB; ++b) load8<IN_T>(rows[b], ch * 8, p.C, vec_ok[b], v[b]);
+            }
+        };
+        if constexpr (!kInt) {
+            float amax[TB];
+    #pragma unroll
+            for (int b = 0; b < TB; ++b) amax[b] = 0.f;
+            for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
+                float v[TB][8];
+                load_tokens(ch, v);
+    #pragma unroll
+                for (int b = 0; b < TB; ++b) {
+    #pragma unroll
+                    for (int e = 0; e < 8; ++e) amax[b] = fmaxf(amax[b], fabsf(v[b][e]));
+                    if (ch == tid) {
+    #pragma unroll
+                        for (int e = 0; e < 8; ++e) keep[b][e] = v[b][e];
+                    }
+                }
+            }
+    #pragma unroll
+            for (int b = 0; b < TB; ++b) {
+                for (int o = 16; o > 0; o >>= 1) amax[b] = fmaxf(amax[b], __shfl_xor_sync(0xffffffffu, amax[b], o));
+                if (lane == 0) wmax[(b0 + b) * GEMV_WARPS + warp] = amax[b];
+            }
+            __syncthreads();
+    #pragma unroll
+            for (int b = 0; b < TB; ++b) {
+                // the sixteen warps' maxima: one per lane of each half-warp, then across its lanes
+                float m = wmax[(b0 + b) * GEMV_WARPS + (lane & (GEMV_WARPS - 1))];
+                for (int o = GEMV_WARPS / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                const int E = tsvd_quant_exponent(m);
+                qscale[b] = tsvd_pow2(8 * ND - 2 - E);
+                if (tid == 0) scale[b0 + b] = tsvd_pow2(E - (8 * ND - 2));   // value = q * scale
+            }
+        } else {
+            if (tid < NTOK) scale[tid] = 1.f;
+        }
+        unsigned range_cnt[TB];   // range diagnostic: the first value of every chunk is sampled
+    #pragma unroll
+        for (int b = 0; b < TB; ++b) range_cnt[b] = 0;
         for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
-            float v[NTOK][8];
-            load_tokens(ch, v);
-#pragma unroll
-            for (int b = 0; b < NTOK; ++b) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) amax[b] = fmaxf(amax[b], fabsf(v[b][e]));
-                if (ch == tid) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) keep[b][e] = v[b][e];
+            float v[TB][8];
+            if (!kInt && ch == tid) {
+    #pragma unroll
+                for (int b = 0; b < TB; ++b)
+    #pragma unroll
+                    for (int e = 0; e < 8; ++e) v[b][e] = keep[b][e];
+            } else {
+                load_tokens(ch, v);
+            }
+    #pragma unroll
+            for (int b = 0; b < TB; ++b) {
+                uint32_t dw[ND][2];
+    #pragma unroll
+                for (int d = 0; d < ND; ++d) dw[d][0] = dw[d][1] = 0u;
+                if (b0 + b < p.B) {
+                    int qv[8];
+                    if constexpr (!kInt) tsvd_range_sample(range_cnt[b], v[b][0], qscale[b]);
+                    if constexpr (ND <= 3) {   // |q| <= 2^22: round by adding a constant, whose image the digit offset absorbs
+    #pragma unroll
+                        for (int e = 0; e < 8; ++e) qv[e] = tsvd_round_bits(v[b][e], qscale[b]);
+                        digits_of<ND, 2>(qv, dw, TSVD_ROUND_BIAS);
+                    } else {
+    #pragma unroll
+                        for (int e = 0; e < 8; ++e) qv[e] = __float2int_rn(v[b][e] * qscale[b]);
+                        digits_of<ND, 2>(qv, dw);
+                    }
                 }
+    #pragma unroll
+                for (int d = 0; d < ND; ++d)
+                    *reinterpret_cast<uint2*>(dig + (size_t)((b0 + b) * ND + d) * dstride + ch * 8) = make_uint2(dw[d][0], dw[d][1]);
             }
         }
-#pragma unroll
-        for (int b = 0; b < NTOK; ++b) {
-            for (int o = 16; o > 0; o >>= 1) amax[b] = fmaxf(amax[b], __shfl_xor_sync(0xffffffffu, amax[b], o));
-            if (lane == 0) wmax[b * GEMV_WARPS + warp] = amax[b];
+        if constexpr (!kInt) {
+    #pragma unroll
+            for (int b = 0; b < TB; ++b)
+                if (tsvd_range_flagged(range_cnt[b]) && lane == 0) atomicOr(p.status, TSVD_DEV_RANGE);
         }
-        __syncthreads();
-#pragma unroll
-        for (int b = 0; b < NTOK; ++b) {
-            // the sixteen warps' maxima: one per lane of each half-warp, then across its lanes
-            float m = wmax[b * GEMV_WARPS + (lane & (GEMV_WARPS - 1))];
-            for (int o = GEMV_WARPS / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            const int E = tsvd_quant_exponent(m);
-            qscale[b] = tsvd_pow2(8 * ND - 2 - E);
-            if (tid == 0) scale[b] = tsvd_pow2(E - (8 * ND - 2));   // value = q * scale
-        }
-    } else {
-        if (tid < NTOK) scale[tid] = 1.f;
-    }
-    unsigned range_cnt[NTOK];   // range diagnostic: the first value of every chunk is sampled
-#pragma unroll
-    for (int b = 0; b < NTOK; ++b) range_cnt[b] = 0;
-    for (int ch = tid; ch < n_chunks; ch += GEMV_THREADS) {
-        float v[NTOK][8];
-        if (!kInt && ch == tid) {
-#pragma unroll
-            for (int b = 0; b < NTOK; ++b)
-#pragma unroll
-                for (int e = 0; e < 8; ++e) v[b][e] = keep[b][e];
-        } else {
-            load_tokens(ch, v);
-        }
-#pragma unroll
-        for (int b = 0; b < NTOK; ++b) {
-            uint32_t dw[ND][2];
-#pragma unroll
-            for (int d = 0; d < ND; ++d) dw[d][0] = dw[d][1] = 0u;
-            if (b < p.B) {
-                int qv[8];
-                if constexpr (!kInt) tsvd_range_sample(range_cnt[b], v[b][0], qscale[b]);
-                if constexpr (ND <= 3) {   // |q| <= 2^22: round by adding a constant, whose image the digit offset absorbs
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) qv[e] = tsvd_round_bits(v[b][e], qscale[b]);
-                    digits_of<ND, 2>(qv, dw, TSVD_ROUND_BIAS);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) qv[e] = __float2int_rn(v[b][e] * qscale[b]);
-                    digits_of<ND, 2>(qv, dw);
-                }
-            }
-#pragma unroll
-            for (int d = 0; d < ND; ++d)
-                *reinterpret_cast<uint2*>(dig + (size_t)(b * ND + d) * dstride + ch * 8) = make_uint2(dw[d][0], dw[d][1]);
-        }
-    }
-    if constexpr (!kInt) {
-#pragma unroll
-        for (int b = 0; b < NTOK; ++b)
-            if (tsvd_range_flagged(range_cnt[b]) && lane == 0) atomicOr(p.status, TSVD_DEV_RANGE);
     }
     __syncthreads();
 
@@ -382,7 +388,8 @@ cudaError_t launch_gemv_tokens(const GemvParams& p, int R_pad, cudaStream_t stre
 {
     if (p.B == 1) return launch_gemv<IN_T, ND, 1, STAGE>(p, R_pad, stream);
     if (p.B == 2) return launch_gemv<IN_T, ND, 2, STAGE>(p, R_pad, stream);
-    return launch_gemv<IN_T, ND, 4, STAGE>(p, R_pad, stream);
+    if (p.B <= 4) return launch_gemv<IN_T, ND, 4, STAGE>(p, R_pad, stream);
+    return launch_gemv<IN_T, ND, 8, STAGE>(p, R_pad, stream);
 }
 
 constexpr int ND_T = 4;   // digits of the intermediate t (fp32), as on the tensor-core path
@@ -393,7 +400,7 @@ inline int digits_for_x(tsvd_dtype_t dt, bool wide) { return dt == TSVD_I8 ? 1 :
 bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x)
 {
     if (B < 1 || B > TSVD_DECODE_MAX_B) return false;
-    const int ntok = B == 3 ? 4 : B;
+    const int ntok = B <= 2 ? B : B <= 4 ? 4 : 8;
     return gemv_smem_bytes(digits_for_x(dt, wide_x), ntok, h->V.C_pad) <= (size_t)GEMV_MAX_SMEM &&
            gemv_smem_bytes(ND_T, ntok, h->U.C_pad) <= (size_t)GEMV_MAX_SMEM;
 }

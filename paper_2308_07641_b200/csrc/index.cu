@@ -244,7 +244,7 @@ tsvd_status_t tsvd_build_index_lists(const int8_t* host, int R, int C, IndexMat*
 
 bool tsvd_index_fits(const tsvd_handle_s* h, int B)
 {
-    if (!h->Vi.row_ptr || !h->Ui.row_ptr || B < 1 || B > TSVD_DECODE_MAX_B) return false;
+    if (!h->Vi.row_ptr || !h->Ui.row_ptr || B < 1 || B > TSVD_INDEX_MAX_B) return false;
     const int ntok = B == 3 ? 4 : B;
     return index_smem_bytes(ntok, h->Vi.C_pad) <= (size_t)IDX_MAX_SMEM &&
            index_smem_bytes(ntok, h->Ui.C_pad) <= (size_t)IDX_MAX_SMEM;

@@ -87,7 +87,7 @@ struct StageProfiler {
     std::vector<Pair> pending;
     float ms[TSVD_N_STAGES] = {0, 0, 0, 0};
     unsigned launches[TSVD_N_STAGES] = {0, 0, 0, 0};
-    unsigned long long* stamps = nullptr;   // mode 2: device, [TSVD_STAMP_SLOTS][2] = {begin, end}
+    unsigned long long* stamps = nullptr;   // mode 2: device, [TSVD_STAMP_SLOTS][TSVD_STAMP_WORDS]: begin, end, spare
     std::vector<int> slot_stage;            // stage of every slot handed out
     void begin(int stage, cudaStream_t s);
     void end(cudaStream_t s);
@@ -95,6 +95,7 @@ struct StageProfiler {
     unsigned long long* slot(int stage);    // mode 2: this launch's pair (null when off or full)
 };
 constexpr int TSVD_STAMP_SLOTS = 1 << 15;
+constexpr int TSVD_STAMP_WORDS = 8;   // begin, end, and six spare words for finer stamps in development builds
 
 struct tsvd_handle_s {
     int device = 0;

@@ -44,6 +44,7 @@ def test_constants_match_the_header(binding):
     def define(name):
         return int(re.search(r"#define\s+" + name + r"\s+(0x[0-9a-fA-F]+|\d+)", hdr).group(1), 0)
     assert define("TSVD_DECODE_MAX_B") == binding.TSVD_DECODE_MAX_B
+    assert define("TSVD_INDEX_MAX_B") == binding.TSVD_INDEX_MAX_B
     assert define("TSVD_FLAG_PATH_DECODE") == binding.TSVD_FLAG_PATH_DECODE
     assert define("TSVD_FLAG_PATH_SIMPLE") == binding.TSVD_FLAG_PATH_SIMPLE
     assert define("TSVD_FLAG_PATH_TENSOR") == binding.TSVD_FLAG_PATH_TENSOR

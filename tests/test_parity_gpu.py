@@ -110,6 +110,10 @@ DECODE = [
     gen.scaled(C["cfg5_d20"], name="dec_i8_b4", M=256, N=384, K=512, B=4),
     gen.scaled(C["cfg5_d50"], name="dec_i8_b1_dense", M=129, N=257, K=255, B=1, density=1.0),
     gen.scaled(C["cfg2"], name="dec_all_zero", M=140, N=130, K=150, B=2, density=0.0),
+    gen.scaled(C["cfg1"], name="dec_f32_b8", M=300, N=333, K=200, B=8, seed=24),
+    gen.scaled(C["cfg3_b4"], name="dec_bf16_b5", M=520, N=2100, K=390, B=5, seed=25),
+    gen.scaled(C["cfg3_b4"], name="dec_bf16_b7", M=512, N=640, K=384, B=7, seed=26),
+    gen.scaled(C["cfg5_d20"], name="dec_i8_b8", M=256, N=384, K=512, B=8),
     gen.scaled(C["cfg2"], name="dec_row_density_varies", M=260, N=300, K=280, B=4, row_density_spread=0.9),
 ]
 
@@ -119,7 +123,7 @@ def test_decode_cases_every_element(spec):
     _util.run_and_check(spec, flags=0x20)
 
 
-def test_decode_is_the_default_up_to_four_tokens_and_refuses_more():
+def test_decode_is_the_default_up_to_eight_tokens_and_refuses_more():
     import torch
     from paper_2308_07641_b200 import binding
     rng = np.random.default_rng(5)
@@ -127,16 +131,16 @@ def test_decode_is_the_default_up_to_four_tokens_and_refuses_more():
     S = np.ones(24, np.float32)
     h = binding.tsvd_pack(U, S, V)
     try:
-        for B in (1, 2, 3, 4):
+        for B in range(1, binding.TSVD_DECODE_MAX_B + 1):
             assert binding.tsvd_plan(h, B, binding.TSVD_BF16)["path"] == "decode"
             assert binding.tsvd_plan(h, B, binding.TSVD_BF16, 0x40)["path"] == "tensor"
-        assert binding.tsvd_plan(h, 5, binding.TSVD_BF16)["path"] == "tensor"
+        assert binding.tsvd_plan(h, 9, binding.TSVD_BF16)["path"] == "tensor"
         plan = binding.tsvd_plan(h, 4, binding.TSVD_I8, 0x20)
         assert (plan["path"], plan["digits_x"], plan["digits_t"]) == ("decode", 1, 4)
-        x = torch.zeros(5 * 36, device="cuda"); y = torch.zeros(5 * 40, device="cuda")
+        x = torch.zeros(9 * 36, device="cuda"); y = torch.zeros(9 * 40, device="cuda")
         L = binding.lib()
-        assert L.tsvd_forward_ex(h, x.data_ptr(), 36, y.data_ptr(), 40, 5, 0, 0x20, None, None) == binding.TSVD_E_TOOBIG
-        assert L.tsvd_forward_ex(h, x.data_ptr(), 36, y.data_ptr(), 40, 4, 0, 0x20, None, None) == binding.TSVD_OK
+        assert L.tsvd_forward_ex(h, x.data_ptr(), 36, y.data_ptr(), 40, 9, 0, 0x20, None, None) == binding.TSVD_E_TOOBIG
+        assert L.tsvd_forward_ex(h, x.data_ptr(), 36, y.data_ptr(), 40, 8, 0, 0x20, None, None) == binding.TSVD_OK
         torch.cuda.synchronize()
     finally:
         binding.tsvd_destroy(h)
@@ -210,7 +214,7 @@ def test_kernels_launched_early_still_see_inputs_written_just_before():
 
 def test_decode_falls_back_when_the_digits_do_not_fit_shared_memory():
     from paper_2308_07641_b200 import binding
-    N = 13000                       # 4 tokens x 4 digits x 13056 columns > 200 KiB
+    N = 13000                       # 4 tokens x 4 digits x 13056 columns > 200 KiB (and so are 8 tokens)
     U = np.zeros((8, 8), np.int8); V = np.zeros((8, N), np.int8); S = np.ones(8, np.float32)
     h = binding.tsvd_pack(U, S, V)
     try:
