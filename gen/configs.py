@@ -154,6 +154,12 @@ def set_entries(x: np.ndarray, x_dtype: str, tokens, cols, value: float) -> np.n
     return out
 
 
+def laplace_matrix(seed: int, M: int, N: int) -> np.ndarray:
+    """A float32 [M, N] matrix of i.i.d. Laplace entries: the random matrix the paper profiles its
+    decomposition on (shape [512, 256] in its Figures 1a and 2a)."""
+    return rng.laplace(seed, 7, M * N).astype(np.float32).reshape(M, N)
+
+
 def make_case(spec: CaseSpec) -> Case:
     U, V, S = make_weights(spec)
     return Case(spec=spec, U=U, V=V, S=S, x=make_x(spec))

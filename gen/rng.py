@@ -71,6 +71,15 @@ def normal(seed: int, tensor_id: int, n: int) -> np.ndarray:
     return out
 
 
+def laplace(seed: int, tensor_id: int, n: int) -> np.ndarray:
+    """float64 standard Laplace variates (density exp(-|x|)/2) by inversion of the distribution."""
+    out = np.empty(n, dtype=np.float64)
+    for s, c in _chunks(n):
+        u = uniform01(seed, tensor_id, 0, s, c) - 0.5
+        out[s:s + c] = -np.sign(u) * np.log1p(-2.0 * np.abs(u))
+    return out
+
+
 def uniform(seed: int, tensor_id: int, n: int, lo: float, hi: float) -> np.ndarray:
     out = np.empty(n, dtype=np.float64)
     for s, c in _chunks(n):
