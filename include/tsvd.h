@@ -155,9 +155,12 @@ tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx, void* y, 
                               tsvd_dtype_t dtype, unsigned flags, void* z_out, void* stream);
 
 /*
- * tsvd_forward_host -- the same map with HOST buffers: copies x to the device,
- * runs tsvd_forward_ex, copies y (and z_out) back, and waits.  x, y, z_out are
- * host pointers (pinned memory makes the copies faster); layout as tsvd_forward.
+ * tsvd_forward_host -- the same map with HOST buffers: copies x to the device, runs
+ * tsvd_forward_ex, copies y (and z_out) back, and waits.  x, y, z_out are host pointers;
+ * layout as tsvd_forward.  Batches of 768 tokens and more are cut into about eight chunks
+ * that are pipelined over three streams of the handle (copy-in, compute, copy-out), so that
+ * with pinned host memory the copies of neighbouring chunks overlap the computation; the
+ * result does not depend on the chunking (tokens are independent).
  */
 tsvd_status_t tsvd_forward_host(tsvd_handle_t h, const void* x, void* y, int B,
                                 tsvd_dtype_t dtype, unsigned flags, void* z_out);
@@ -213,6 +216,29 @@ tsvd_status_t tsvd_reserve(tsvd_handle_t h, int B_max, tsvd_dtype_t dtype);
  * Errors: E_NULL (h), E_NOMEM, E_CUDA.
  */
 tsvd_status_t tsvd_set_bias(tsvd_handle_t h, const float* bias);
+
+/*
+ * tsvd_ternarize -- the ternarisation T(x, theta) of Algorithm 1 (Section "Direct Transition
+ * Algorithm to TSVD form"), the step that turns the singular vectors of the residual into new
+ * columns of U and rows of V in Algorithm 2.  For each of n_vec vectors: the sparsest vector
+ * over {-1,0,+1} whose angle to x is at most theta; it keeps sign(x) on the k largest
+ * magnitudes, k the first index at which (sum of the k largest |x|) / sqrt(k) / ||x|| reaches
+ * cos(theta) (sums and the comparison in double precision), and every entry whose magnitude
+ * equals the k-th largest is kept with it.
+ *
+ *   x      device, float; vector v is the len values at x + v*ldx (ldx >= len)
+ *   theta  angle in radians, 0 <= theta <= pi/2 (the paper uses 0.576)
+ *   t      device, int8; receives vector v at t + v*ldt (ldt >= len)
+ *   nnz    device, int [n_vec], optional: the number of nonzeros of each result, or -1 where no
+ *          ternary vector lies within theta of x (Theorem 1 bounds when that can happen); the
+ *          result is then all zeros
+ *   stream a cudaStream_t; the call is asynchronous; the caller keeps ownership of all buffers
+ * Errors: E_NULL, E_SHAPE (sizes, leading dimensions, theta out of range), E_TOOBIG (len above
+ * TSVD_TERNARIZE_MAX_LEN: a vector is sorted in the shared memory of one SM), E_CUDA.
+ */
+#define TSVD_TERNARIZE_MAX_LEN 32768
+tsvd_status_t tsvd_ternarize(const float* x, int n_vec, int len, int ldx, double theta, int8_t* t, int ldt,
+                             int* nnz, void* stream);
 
 /* Device-side status word of the forwards on this handle since the last read (read after
  * the stream has been synchronised).  Resets the word.  Returns

@@ -37,7 +37,7 @@ DTYPES = {"f32": TSVD_F32, "bf16": TSVD_BF16, "i8": TSVD_I8}
 
 # every symbol include/tsvd.h declares
 EXPORTS = ("tsvd_pack", "tsvd_forward", "tsvd_forward_ex", "tsvd_forward_host", "tsvd_forward_static",
-           "tsvd_reserve", "tsvd_set_bias", "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_index_bytes", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
+           "tsvd_reserve", "tsvd_set_bias", "tsvd_ternarize", "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_index_bytes", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
            "tsvd_launch_count", "tsvd_destroy", "tsvd_strerror")
 
 _lib: Optional[ctypes.CDLL] = None
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.tsvd_reserve.restype = ci
         L.tsvd_set_bias.argtypes = [vp, vp]
         L.tsvd_set_bias.restype = ci
+        L.tsvd_ternarize.argtypes = [vp, ci, ci, ci, ctypes.c_double, vp, ci, vp, vp]
+        L.tsvd_ternarize.restype = ci
         L.tsvd_last_status.argtypes = [vp]
         L.tsvd_last_status.restype = ci
         L.tsvd_info.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci),
@@ -162,6 +164,16 @@ def tsvd_set_bias(h: int, bias: Optional[np.ndarray]) -> None:
         if bias.shape != (tsvd_info(h)["M"],):
             raise TSVDError(TSVD_E_SHAPE, "tsvd_set_bias")
     _check(lib().tsvd_set_bias(h, _np_ptr(bias)), "tsvd_set_bias")
+
+
+TSVD_TERNARIZE_MAX_LEN = 32768
+
+
+def tsvd_ternarize(x_ptr: int, n_vec: int, length: int, ldx: int, theta: float, t_ptr: int, ldt: int,
+                   nnz_ptr: int = 0, stream: int = 0) -> None:
+    """Algorithm 1 on n_vec device vectors (float32 in, int8 out); raw device pointers."""
+    _check(lib().tsvd_ternarize(x_ptr, n_vec, length, ldx, float(theta), t_ptr, ldt, nnz_ptr or None,
+                                stream or None), "tsvd_ternarize")
 
 
 def tsvd_last_status(h: int) -> int:

@@ -148,6 +148,9 @@ static void free_handle(tsvd_handle_s* h)
     if (h->io) cudaFree(h->io);
     if (h->dev_status) cudaFree(h->dev_status);
     if (h->prof.stamps) cudaFree(h->prof.stamps);
+    for (cudaEvent_t e : h->host_events) cudaEventDestroy(e);
+    for (cudaStream_t st : h->host_stream)
+        if (st) cudaStreamDestroy(st);
     (void)cudaGetLastError();
     delete h;
 }
@@ -411,6 +414,16 @@ extern "C" tsvd_status_t tsvd_forward(tsvd_handle_t h, const void* x, void* y, i
     return tsvd_forward_ex(h, x, h->N, y, h->M, B, dtype, 0u, nullptr, stream);
 }
 
+// Host-buffer entry point.  The batch is cut into chunks of whole tiles and pipelined over three
+// streams of the handle: the copy-in of chunk i+1 and the copy-out of chunk i-1 run while chunk i is
+// computed (with pageable host memory the copies stage through the driver and overlap less).
+static tsvd_status_t host_streams(tsvd_handle_s* h)
+{
+    for (int i = 0; i < 3; ++i)
+        if (!h->host_stream[i]) TSVD_CUDA_OK(cudaStreamCreateWithFlags(&h->host_stream[i], cudaStreamNonBlocking));
+    return TSVD_OK;
+}
+
 extern "C" tsvd_status_t tsvd_forward_host(tsvd_handle_t h, const void* x, void* y, int B,
                                            tsvd_dtype_t dtype, unsigned flags, void* z_out)
 {
@@ -419,8 +432,9 @@ extern "C" tsvd_status_t tsvd_forward_host(tsvd_handle_t h, const void* x, void*
     const size_t xs = dtype_size(dtype);
     if (xs == 0) return TSVD_E_DTYPE;
     const bool y_bf16 = (dtype == TSVD_BF16) && !(flags & TSVD_FLAG_OUT_F32);
+    const size_t ys = y_bf16 ? 2 : 4;
     const size_t x_bytes = (size_t)B * h->N * xs;
-    const size_t y_bytes = (size_t)B * h->M * (y_bf16 ? 2 : 4);
+    const size_t y_bytes = (size_t)B * h->M * ys;
     const size_t z_bytes = z_out ? (size_t)B * h->K * 4 : 0;
     // staging buffers live in the handle and only grow
     const size_t x_off = 0, y_off = (x_bytes + 255) & ~(size_t)255;
@@ -432,20 +446,43 @@ extern "C" tsvd_status_t tsvd_forward_host(tsvd_handle_t h, const void* x, void*
         if (cudaMalloc(&h->io, need) != cudaSuccess) { (void)cudaGetLastError(); return TSVD_E_NOMEM; }
         h->io_bytes = need;
     }
+    tsvd_status_t st = host_streams(h);
+    if (st != TSVD_OK) return st;
+    // chunks of whole tiles of both stages (64- and 48-token tiles: multiples of 192), about eight per
+    // call, none below 384 tokens; small batches go in one piece
+    int chunk = B;
+    if (B >= 768) {
+        chunk = ((B + 7) / 8 + 191) / 192 * 192;
+        if (chunk < 384) chunk = 384;
+    }
+    const int n_chunks = (B + chunk - 1) / chunk;
+    while ((int)h->host_events.size() < 2 * n_chunks) {
+        cudaEvent_t e;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { (void)cudaGetLastError(); return TSVD_E_CUDA; }
+        h->host_events.push_back(e);
+    }
     char* base = reinterpret_cast<char*>(h->io);
-    void *dx = base + x_off, *dy = base + y_off, *dz = z_out ? base + z_off : nullptr;
-    tsvd_status_t st = TSVD_OK;
-    cudaStream_t s = nullptr;
+    cudaStream_t s_in = h->host_stream[0], s_run = h->host_stream[1], s_out = h->host_stream[2];
     do {
-        if (cudaMemcpyAsync(dx, x, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) { st = TSVD_E_CUDA; break; }
-        st = tsvd_forward_ex(h, dx, h->N, dy, h->M, B, dtype, flags, dz, s);
-        if (st != TSVD_OK) break;
-        if (cudaMemcpyAsync(y, dy, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) { st = TSVD_E_CUDA; break; }
-        if (z_out && cudaMemcpyAsync(z_out, dz, z_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
-            st = TSVD_E_CUDA; break;
+        for (int c = 0; c < n_chunks && st == TSVD_OK; ++c) {
+            const int b0 = c * chunk, nb = (B - b0 < chunk) ? B - b0 : chunk;
+            const size_t xo = (size_t)b0 * h->N * xs, yo = (size_t)b0 * h->M * ys, zo = (size_t)b0 * h->K * 4;
+            cudaEvent_t e_in = h->host_events[2 * c], e_run = h->host_events[2 * c + 1];
+            if (cudaMemcpyAsync(base + x_off + xo, (const char*)x + xo, (size_t)nb * h->N * xs, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+                cudaEventRecord(e_in, s_in) != cudaSuccess || cudaStreamWaitEvent(s_run, e_in, 0) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+            st = tsvd_forward_ex(h, base + x_off + xo, h->N, base + y_off + yo, h->M, nb, dtype, flags,
+                                 z_out ? base + z_off + zo : nullptr, s_run);
+            if (st != TSVD_OK) break;
+            if (cudaEventRecord(e_run, s_run) != cudaSuccess || cudaStreamWaitEvent(s_out, e_run, 0) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+            if (cudaMemcpyAsync((char*)y + yo, base + y_off + yo, (size_t)nb * h->M * ys, cudaMemcpyDeviceToHost, s_out) != cudaSuccess) { st = TSVD_E_CUDA; break; }
+            if (z_out && cudaMemcpyAsync((char*)z_out + zo, base + z_off + zo, (size_t)nb * h->K * 4, cudaMemcpyDeviceToHost, s_out) != cudaSuccess) {
+                st = TSVD_E_CUDA; break;
+            }
         }
-        if (cudaStreamSynchronize(s) != cudaSuccess) { st = TSVD_E_CUDA; break; }
     } while (0);
+    // everything queued so far is waited for, also after an error
+    const cudaError_t e1 = cudaStreamSynchronize(s_in), e2 = cudaStreamSynchronize(s_run), e3 = cudaStreamSynchronize(s_out);
+    if (st == TSVD_OK && (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess)) st = TSVD_E_CUDA;
     if (st != TSVD_OK) (void)cudaGetLastError();
     return st;
 }

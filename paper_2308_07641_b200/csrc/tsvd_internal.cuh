@@ -110,6 +110,8 @@ struct tsvd_handle_s {
     size_t ws_bytes = 0;
     void* io = nullptr;   // device staging for the host-buffer entry point
     size_t io_bytes = 0;
+    cudaStream_t host_stream[3] = {nullptr, nullptr, nullptr};   // copy-in, compute, copy-out of the host-buffer entry point
+    std::vector<cudaEvent_t> host_events;
     int* dev_status = nullptr;  // device status word: TSVD_DEV_* bits
     StageProfiler prof;
 };

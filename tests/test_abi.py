@@ -53,6 +53,7 @@ def test_constants_match_the_header(binding):
     assert define("TSVD_PACK_INDEX_LISTS") == binding.TSVD_PACK_INDEX_LISTS
     assert define("TSVD_INDEX_MAX_COLUMNS") == binding.TSVD_INDEX_MAX_COLUMNS
     assert define("TSVD_MAX_CONTRACTION") == binding.TSVD_MAX_CONTRACTION
+    assert define("TSVD_TERNARIZE_MAX_LEN") == binding.TSVD_TERNARIZE_MAX_LEN
     assert define("TSVD_FLAG_WIDE_X") == binding.TSVD_FLAG_WIDE_X
     assert int(re.search(r"TSVD_E_RANGE\s*=\s*(\d+)", hdr).group(1)) == binding.TSVD_E_RANGE
     assert define("TSVD_FLAG_PATH_MASK") == (binding.TSVD_FLAG_PATH_SIMPLE | binding.TSVD_FLAG_PATH_DECODE |
@@ -82,6 +83,11 @@ def test_host_side_validation(binding):
     assert lib.tsvd_pack(U.ctypes.data, S.ctypes.data, V.ctypes.data, 2, big, 2, 0, ctypes.byref(h)) == binding.TSVD_E_TOOBIG
     assert h.value is None
     assert lib.tsvd_reserve(None, 1, 0) == binding.TSVD_E_NULL
+    one = ctypes.c_void_p(16)     # never dereferenced: the sizes are checked first
+    assert lib.tsvd_ternarize(None, 1, 4, 4, 0.5, one, 4, None, None) == binding.TSVD_E_NULL
+    assert lib.tsvd_ternarize(one, 1, 4, 3, 0.5, one, 4, None, None) == binding.TSVD_E_SHAPE
+    assert lib.tsvd_ternarize(one, 1, 4, 4, 2.0, one, 4, None, None) == binding.TSVD_E_SHAPE
+    assert lib.tsvd_ternarize(one, 1, binding.TSVD_TERNARIZE_MAX_LEN + 1, 1 << 20, 0.5, one, 1 << 20, None, None) == binding.TSVD_E_TOOBIG
     assert lib.tsvd_set_bias(None, None) == binding.TSVD_E_NULL
     assert lib.tsvd_forward(None, None, None, 1, 0, None) == binding.TSVD_E_NULL
     assert lib.tsvd_info(None, None, None, None, None, None, None) == binding.TSVD_E_NULL

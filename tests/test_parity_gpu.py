@@ -286,6 +286,32 @@ def test_host_buffer_entry_point():
         binding.tsvd_destroy(h)
 
 
+def test_host_buffer_entry_point_pipelined_chunks():
+    """768 tokens and more go through the host entry point in chunks on three streams; every token
+    (and z) must come back as from one forward.  Pinned and pageable host buffers."""
+    import torch
+    from paper_2308_07641_b200 import binding
+    spec = gen.scaled(C["cfg2"], name="host_chunks", M=300, N=200, K=150, B=1000, seed=33)
+    U, V, S = gen.make_weights(spec)
+    x = gen.make_x(spec)
+    ref = oracle.forward(U, S, V, _util.oracle_x(x, "bf16"))
+    h = binding.tsvd_pack(U, S, V)
+    try:
+        y = np.zeros((spec.B, spec.M), np.float32)
+        z = np.zeros((spec.B, spec.K), np.float32)
+        binding.tsvd_forward_host(h, x.ctypes.data, y.ctypes.data, spec.B, binding.TSVD_BF16, 0x1, z.ctypes.data)
+        _util.check_outputs(y.astype(np.float64), z, ref, "bf16", False, "host, pageable")
+        xp = torch.from_numpy(x.view(np.int16)).pin_memory()
+        yp = torch.zeros((spec.B, spec.M), dtype=torch.int16).pin_memory()
+        for _ in range(2):
+            binding.tsvd_forward_host(h, xp.data_ptr(), yp.data_ptr(), spec.B, binding.TSVD_BF16, 0)
+        y16 = yp.view(torch.bfloat16).float().double().numpy()
+        _util.check_outputs(y16, None, ref, "bf16", True, "host, pinned")
+        assert binding.tsvd_last_status(h) == binding.TSVD_OK
+    finally:
+        binding.tsvd_destroy(h)
+
+
 # ---- full-size configurations, sampled token columns -------------------------------------------
 FULL = [
     (C["cfg2"], [0, 1, 777, 2048, 4095]),
