@@ -474,6 +474,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="only the headline workload")
     ap.add_argument("--no-sustained", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer measurement (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     spec = gen.CONFIGS[args.config]
@@ -528,30 +529,35 @@ def main():
     want_sustained = (not args.no_sustained) and spec.name in SUSTAINED
     head = measure(w, args.steps, args.repeats, barrier, dist, world, sustained_s=1.5 if want_sustained else 0.0)
 
-    # end to end: host buffers, copies inside the timed region
-    x_host = torch.from_numpy(w.x_np.view(np.int16) if spec.x_dtype == "bf16" else w.x_np).pin_memory()
-    y_bf16 = w.y.dtype == torch.bfloat16
-    y_host = torch.empty((spec.B, spec.M), dtype=torch.int16 if y_bf16 else torch.float32).pin_memory()
-    dt_code = binding.DTYPES[spec.x_dtype]
-    e2e_steps = max(3, min(args.steps, 20))
-    for _ in range(2):
-        binding.tsvd_forward_host(w.layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        binding.tsvd_forward_host(w.layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
-    torch.cuda.synchronize()
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
-    e2e_s = max_over_ranks(dist, e2e_s, "cuda")
-    e2e = {"value": aggregate_tokens_per_s(world, spec.B, e2e_s * 1e3), "unit": UNIT,
-           "h2d_bytes_per_step": int(x_host.numel() * x_host.element_size()),
-           "d2h_bytes_per_step": int(y_host.numel() * y_host.element_size()), "steps": e2e_steps,
-           "ms_per_step": e2e_s * 1e3}
-    y_e2e = (y_host.view(torch.bfloat16).float() if y_bf16 else y_host).double().numpy()
+    e2e = None
     w.layer.forward(w.x, out=w.y, flags=flags)
     torch.cuda.synchronize()
     y_gpu = w.y.float().double().cpu().numpy()
-    e2e["matches_device_path"] = bool(np.array_equal(y_e2e, y_gpu))
+    if not args.no_e2e:
+        # end to end: host buffers, copies inside the timed region
+        x_host = torch.from_numpy(w.x_np.view(np.int16) if spec.x_dtype == "bf16" else w.x_np).pin_memory()
+        y_bf16 = w.y.dtype == torch.bfloat16
+        y_host = torch.empty((spec.B, spec.M), dtype=torch.int16 if y_bf16 else torch.float32).pin_memory()
+        dt_code = binding.DTYPES[spec.x_dtype]
+        e2e_steps = max(3, min(args.steps, 20))
+        for _ in range(2):
+            binding.tsvd_forward_host(w.layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            binding.tsvd_forward_host(w.layer.handle, x_host.data_ptr(), y_host.data_ptr(), spec.B, dt_code, flags)
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        e2e_s = max_over_ranks(dist, e2e_s, "cuda")
+        e2e = {"value": aggregate_tokens_per_s(world, spec.B, e2e_s * 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": int(x_host.numel() * x_host.element_size()),
+               "d2h_bytes_per_step": int(y_host.numel() * y_host.element_size()), "steps": e2e_steps,
+               "ms_per_step": e2e_s * 1e3}
+        y_e2e = (y_host.view(torch.bfloat16).float() if y_bf16 else y_host).double().numpy()
+        w.layer.forward(w.x, out=w.y, flags=flags)
+        torch.cuda.synchronize()
+        y_gpu = w.y.float().double().cpu().numpy()
+        e2e["matches_device_path"] = bool(np.array_equal(y_e2e, y_gpu))
 
     if rank != 0:
         w.close()

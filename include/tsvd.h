@@ -155,6 +155,38 @@ tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx, void* y, 
                               tsvd_dtype_t dtype, unsigned flags, void* z_out, void* stream);
 
 /*
+ * tsvd_forward_v -- the first two rows of Table S1 alone: t = diag(S)(V x), fp32, for B columns.
+ * The convolution forms of a TSVD layer (Section "TSVD in Convolution Layer") apply V(.) and U(.) as
+ * two convolutions with the channel-wise scale between them; each of the two is this call on the
+ * patches of its input (see tsvd_im2col), with the ternary matrix of that stage packed as the V of
+ * a handle (S = 1 and a 1-row U of zeros for the stage that has no scale).
+ *
+ *   x      device, B columns at x + b*ldx (ldx >= N), 16-byte aligned, dtype as tsvd_forward
+ *   t_out  device, float, column b at t_out + b*ldt (ldt >= K), 16-byte aligned
+ *   flags  TSVD_FLAG_PATH_SIMPLE / _DECODE / _TENSOR, TSVD_FLAG_WIDE_X (not _INDEX, not _OUT_F32)
+ * Asynchronous on `stream`; same scratch rules as tsvd_forward.
+ * Errors: as tsvd_forward_ex; E_DTYPE for TSVD_FLAG_PATH_INDEX.
+ */
+tsvd_status_t tsvd_forward_v(tsvd_handle_t h, const void* x, int ldx, float* t_out, int ldt, int B,
+                             tsvd_dtype_t dtype, unsigned flags, void* stream);
+
+/*
+ * tsvd_im2col -- the patches of an image batch, so that a convolution with a ternary kernel becomes
+ * the ternary matrix product of this library (Section "TSVD in Convolution Layer": V(.) and U(.) in
+ * convolution form with kernels [K1,K2], [1,1], [K1,1] or [1,K2]).
+ *
+ *   x    device, n_img images in NHWC layout: x[((n*H + h)*W + w)*C + c], dtype as given
+ *   out  device, same dtype: row (n, ho, wo) at out + ((n*Ho + ho)*Wo + wo)*ld_out holds the k1*k2*C
+ *        values x[n, ho*stride_h + a*dil_h - pad_h, wo*stride_w + b*dil_w - pad_w, c] at index
+ *        (a*k2 + b)*C + c, zero where the position lies outside the image;
+ *        Ho = (H + 2 pad_h - dil_h (k1-1) - 1) / stride_h + 1, Wo likewise; ld_out >= k1*k2*C
+ * Asynchronous on `stream`; the caller owns both buffers.  Errors: E_NULL, E_SHAPE, E_DTYPE, E_CUDA.
+ */
+tsvd_status_t tsvd_im2col(const void* x, tsvd_dtype_t dtype, int n_img, int H, int W, int C, int k1, int k2,
+                          int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w, void* out,
+                          long long ld_out, void* stream);
+
+/*
  * tsvd_forward_host -- the same map with HOST buffers: copies x to the device, runs
  * tsvd_forward_ex, copies y (and z_out) back, and waits.  x, y, z_out are host pointers;
  * layout as tsvd_forward.  Batches of 768 tokens and more are cut into about eight chunks

@@ -332,8 +332,8 @@ extern "C" tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, u
     return TSVD_OK;
 }
 
-extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx, void* y, int ldy, int B,
-                                         tsvd_dtype_t dtype, unsigned flags, void* z_out, void* stream)
+static tsvd_status_t forward_impl(tsvd_handle_t h, const void* x, int ldx, void* y, int ldy, int B, tsvd_dtype_t dtype,
+                                  unsigned flags, void* z_out, void* stream, bool v_only, float** t_where)
 {
     if (!h || !x || !y) return TSVD_E_NULL;
     if (B < 1) return TSVD_E_SHAPE;
@@ -343,7 +343,7 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     if (flags & ~known) return TSVD_E_DTYPE;
     const unsigned path = flags & TSVD_FLAG_PATH_MASK;
     if (path & (path - 1)) return TSVD_E_DTYPE;  // at most one forced path
-    if (ldx < h->N || ldy < h->M) return TSVD_E_SHAPE;
+    if (ldx < h->N || ldy < (v_only ? h->K : h->M)) return TSVD_E_SHAPE;
     if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)z_out & 3)) return TSVD_E_ALIGN;
 
     int dev = 0;
@@ -356,6 +356,9 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     a.z_out = z_out;
     a.test_stall = (flags & TSVD_FLAG_TEST_STALL) != 0;
     a.wide_x = (flags & TSVD_FLAG_WIDE_X) != 0;
+    a.v_only = v_only;
+    a.t_where = t_where;
+    if (v_only && path == TSVD_FLAG_PATH_INDEX) return TSVD_E_DTYPE;   // the index-list kernels run whole forwards only
     a.stream = (cudaStream_t)stream;
 
     const unsigned chosen = choose_path(h, B, dtype, path, a.wide_x);
@@ -380,6 +383,25 @@ extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx
     a.t = reinterpret_cast<float*>(h->ws);
     a.t_ld = h->V.R_pad;
     return tsvd_forward_simple(a);
+}
+
+extern "C" tsvd_status_t tsvd_forward_ex(tsvd_handle_t h, const void* x, int ldx, void* y, int ldy, int B,
+                                         tsvd_dtype_t dtype, unsigned flags, void* z_out, void* stream)
+{
+    return forward_impl(h, x, ldx, y, ldy, B, dtype, flags, z_out, stream, false, nullptr);
+}
+
+extern "C" tsvd_status_t tsvd_forward_v(tsvd_handle_t h, const void* x, int ldx, float* t_out, int ldt, int B,
+                                        tsvd_dtype_t dtype, unsigned flags, void* stream)
+{
+    if (!t_out) return TSVD_E_NULL;
+    float* t = nullptr;
+    const tsvd_status_t st = forward_impl(h, x, ldx, t_out, ldt, B, dtype, flags, nullptr, stream, true, &t);
+    if (st != TSVD_OK) return st;
+    // the stage wrote all padded rows into the handle's scratch: the K real ones go to the caller
+    TSVD_CUDA_OK(cudaMemcpy2DAsync(t_out, (size_t)ldt * sizeof(float), t, (size_t)h->V.R_pad * sizeof(float),
+                                   (size_t)h->K * sizeof(float), (size_t)B, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return TSVD_OK;
 }
 
 // The largest scratch any path asks for with up to B_max tokens of this dtype: every path's need

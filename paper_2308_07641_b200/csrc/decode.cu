@@ -432,6 +432,7 @@ tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws)
     }
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
+    if (a.v_only) { *a.t_where = t; return TSVD_OK; }
 
     GemvParams q{};
     q.units = h->U.units; q.R = h->M; q.C = h->K; q.C_pad = h->U.C_pad;

@@ -153,6 +153,7 @@ tsvd_status_t tsvd_forward_simple(const ForwardArgs& a)
     }
     h->prof.end(a.stream);
     if (e != cudaSuccess) return TSVD_E_CUDA;
+    if (a.v_only) { *a.t_where = a.t; return TSVD_OK; }
     h->prof.begin(3, a.stream);
     // U-stage: y[b,m] = sum_k U[m,k] t[b,k]
     const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;

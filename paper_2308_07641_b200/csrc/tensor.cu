@@ -969,6 +969,7 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
     e = launch_gemm<NDX, EPI_ACC, SMALL_TOK>(p, v_tiles, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
+    if (a.v_only) { *a.t_where = w.t; return TSVD_OK; }
 
     h->prof.begin(2, st);
     e = launch_digitise<float, ND_T, SMALL_TOK>(w.t, h->V.R_pad, a.B, h->K, KBu, p.tmax, w.Dt, w.scale_t, w.yacc,
@@ -1060,6 +1061,7 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     else e = launch_gemm<1, EPI_V>(p, v_tiles, st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
+    if (a.v_only) { *a.t_where = w.t; return TSVD_OK; }
 
     // stage 2: t -> digits (each token's scale comes from its own max |t|)
     h->prof.begin(2, st);

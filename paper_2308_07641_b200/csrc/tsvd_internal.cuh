@@ -183,6 +183,8 @@ struct ForwardArgs {
     void* z_out;
     bool test_stall = false;   // TSVD_FLAG_TEST_STALL
     bool wide_x = false;       // TSVD_FLAG_WIDE_X: bf16 activations as four digits
+    bool v_only = false;       // stop after the V-stage and its scale (tsvd_forward_v)
+    float** t_where = nullptr; // v_only: receives where t = S*(V x) was written, [B][R_pad of V] fp32
     float* t;        // scratch [B][t_ld] fp32: S * (V x)
     int t_ld;
     cudaStream_t stream;

@@ -1,0 +1,96 @@
+"""GPU parity of the convolution forms (Section "TSVD in Convolution Layer", Eq. 5): the library's
+patch gather and single-stage forward, composed by TSVDConv2d, against the CPU checker's staged
+evaluation V(.) -> diag(s)(.) -> U(.), element by element (fp32 outputs: maximum norm, 1e-5)."""
+import numpy as np
+import pytest
+
+import gen
+from oracle import conv as oc
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2308_07641_b200 import build
+    build.build()
+
+
+def _layer(seed, form, C_out, C_in, K1, K2, K, density=0.28):
+    M, N = oc.matrix_shape(form, C_out, C_in, K1, K2)
+    U = gen.rng.ternary(seed, 1, M * K, density).reshape(M, K)
+    V = gen.rng.ternary(seed, 2, K * N, density).reshape(K, N)
+    g = np.random.default_rng(seed)
+    S = (np.exp(0.5 * g.standard_normal(K)) * g.choice([-1.0, 1.0], K)).astype(np.float32)
+    return U, S, V
+
+
+def _x(seed, shape, x_dtype):
+    n = int(np.prod(shape))
+    if x_dtype == "i8":
+        return gen.rng.int8_uniform(seed, 4, n, -128, 127).reshape(shape)
+    v = gen.rng.normal(seed, 4, n).astype(np.float32).reshape(shape)
+    return gen.rng.f32_to_bf16_bits(v).reshape(shape) if x_dtype == "bf16" else v
+
+
+def _run(form, geom, x_dtype, shape=(2, 13, 11), C_in=24, C_out=40, K1=3, K2=3, K=50, flags=0, seed=0):
+    import torch
+    from paper_2308_07641_b200 import device_activations
+    from paper_2308_07641_b200.conv import TSVDConv2d
+    stride, pad, dil = geom
+    U, S, V = _layer(100 + seed + form, form, C_out, C_in, K1, K2, K)
+    x = _x(200 + seed, shape + (C_in,), x_dtype)
+    layer = TSVDConv2d(U, S, V, form, C_out, C_in, K1, K2, stride, pad, dil)
+    try:
+        xt = device_activations(x.reshape(-1, C_in), x_dtype).view(*shape, C_in)
+        y = layer.forward(xt, flags).double().cpu().numpy()
+        torch.cuda.synchronize()
+        assert layer.status() == 0
+    finally:
+        layer.close()
+    ref = oc.conv2d_tsvd(gen.widen_x(x, x_dtype), U, S, V, form, C_out, C_in, K1, K2, stride, pad, dil)
+    assert y.shape == ref.shape
+    assert np.abs(y - ref).max() <= 1e-5 * np.abs(ref).max(), (form, geom, x_dtype)
+
+
+GEOMS = [((1, 1), (0, 0), (1, 1)), ((2, 2), (1, 1), (1, 1)), ((1, 2), (2, 0), (2, 1)), ((2, 1), (1, 2), (1, 2))]
+
+
+@pytest.mark.parametrize("x_dtype", ["f32", "bf16", "i8"])
+@pytest.mark.parametrize("geom", GEOMS, ids=lambda g: "s%d%d_p%d%d_d%d%d" % (g[0] + g[1] + g[2]))
+@pytest.mark.parametrize("form", [0, 1, 2, 3])
+def test_four_forms(form, geom, x_dtype):
+    _run(form, geom, x_dtype)
+
+
+@pytest.mark.parametrize("form", [0, 1, 2, 3])
+def test_rectangular_kernels_and_ragged_channels(form):
+    _run(form, ((1, 1), (1, 0), (1, 1)), "f32", shape=(1, 9, 17), C_in=7, C_out=13, K1=2, K2=5, K=19, seed=7)
+
+
+@pytest.mark.parametrize("flags", [0x10, 0x20, 0x40], ids=["simple", "decode", "tensor"])
+def test_every_kernel_family_serves_a_stage(flags):
+    # one image of 3 x 4 pixels: with a 3x3 kernel and no padding 2 output pixels, within the decode limit
+    _run(0, ((1, 1), (0, 0), (1, 1)), "f32", shape=(1, 3, 4), flags=flags, seed=3)
+    _run(1, ((1, 1), (1, 1), (1, 1)), "bf16", shape=(1, 2, 3), flags=flags, seed=4)
+
+
+def test_pointwise_form_is_the_linear_layer():
+    """A [1,1] kernel: the convolution is the linear map on every pixel, and costs no patch gather."""
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear, binding, device_activations
+    from paper_2308_07641_b200.conv import TSVDConv2d
+    U, S, V = _layer(9, 0, 48, 32, 1, 1, 64)
+    x = _x(9, (2, 5, 6, 32), "f32")
+    conv = TSVDConv2d(U, S, V, 0, 48, 32, 1, 1)
+    lin = TSVDLinear(U, S, V)
+    try:
+        n0 = binding.tsvd_launch_count()
+        y = conv.forward(device_activations(x.reshape(-1, 32), "f32").view(2, 5, 6, 32))
+        torch.cuda.synchronize()
+        assert binding.tsvd_launch_count() - n0 <= 8          # two stages of at most four kernels, no gather
+        y_lin = lin.forward(device_activations(x.reshape(-1, 32), "f32"))
+        err = (y.view(-1, 48) - y_lin).abs().max().item()
+        assert err <= 1e-5 * y_lin.abs().max().item()
+    finally:
+        conv.close(); lin.close()
