@@ -15,7 +15,8 @@
  * a CUDA device they return TSVD_E_CUDA.
  *
  * Arithmetic of the fast kernels (tensor-core, decode and index-list paths), which is
- * what bounds their accuracy.  Per token, the activations are rounded once to a
+ * what bounds their accuracy.  Per token (the decode kernels: per token and quarter of
+ * the columns, from three tokens and 1024 columns on), the activations are rounded once to a
  * multiple of 2^(E-22) (bf16 activations; 2^(E-30) with TSVD_FLAG_WIDE_X) or 2^(E-30)
  * (fp32 activations), where 2^E is the power of two just above the token's largest
  * magnitude; int8 activations are used as they are.  From there the V-stage is exact
@@ -278,7 +279,7 @@ tsvd_status_t tsvd_ternarize(const float* x, int n_vec, int len, int ldx, double
  *   TSVD_E_RANGE   if some token's dynamic range was wider than the fixed-point digits
  *                  resolve: while converting a stage's input the kernels sample one value
  *                  in eight, and raise this when, among at least 32 nonzero samples of a
- *                  token that one warp converted, fewer than a quarter reach 2^12
+ *                  token that one warp or one CTA converted, fewer than a quarter reach 2^12
  *                  quantisation steps (most entries then keep fewer than 12 bits; for a
  *                  normally distributed bulk this happens from an outlier of about 2^10
  *                  times the bulk's scale with three digits, 2^18 with four).  y is still

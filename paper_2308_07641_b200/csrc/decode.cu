@@ -357,6 +357,335 @@ ternary_gemv_kernel(const GemvParams p)
     tsvd_stamp_end(p.stamp);
 }
 
+#ifdef TSVD_PHASES   // development builds: finer time stamps from one warp of a middle CTA
+#define PH(k) do { if (p.stamp && blockIdx.x == (gridDim.x / 2) && tid == 96) p.stamp[2 + (k)] = tsvd_globaltimer(); } while (0)
+#else
+#define PH(k) do { } while (0)
+#endif
+
+// ---------------------------------------------------------------------------------------
+// Cluster form of the same stage, for contractions of 1024 columns and more.  In the kernel
+// above every CTA reads and converts the whole stage input; at four tokens that takes longer than
+// streaming the CTA's codes.  Here four CTAs of a thread-block cluster share a tile of 128 rows
+// and split its CONTRACTION: each reads and converts only its quarter of the columns (with its
+// own power-of-two scale per token: a finer scale than one per token, never a coarser one),
+// contracts all 128 rows against that quarter, and the four partial results meet through
+// distributed shared memory: CTA c of the cluster finishes rows 32c .. 32c+31, every CTA stores
+// its partial sums of those rows into a slot of CTA c's shared memory, one cluster barrier, and
+// the owner adds the four slots in a fixed order (deterministic; for int8 activations the slots
+// hold the exact integers).  No global atomics, no second pass over the input.
+// ---------------------------------------------------------------------------------------
+constexpr int CLUSTER_CTAS = 4;
+constexpr int CLUSTER_ROWS = 128;           // rows of a cluster's tile = rows every CTA of it contracts
+constexpr int CLUSTER_OWN = CLUSTER_ROWS / CLUSTER_CTAS;   // rows a CTA finishes
+constexpr int CLUSTER_MIN_GROUPS = 16;      // use this form from 1024 columns on
+constexpr int CLUSTER_MIN_TOKENS = 3;        // and from three tokens on
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// address of `local` (a shared-memory address of this CTA) in the shared memory of CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_map(const void* local, uint32_t rank)
+{
+    uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(local)), r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_store(uint32_t remote, uint32_t bits)
+{
+    asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(remote), "r"(bits) : "memory");
+}
+__device__ __forceinline__ void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+
+__host__ __device__ inline int cluster_slab_groups(int C_pad) { return ((C_pad >> 6) + CLUSTER_CTAS - 1) / CLUSTER_CTAS; }
+
+// grid: (R_pad / 128) * 4 CTAs of 512 threads in clusters of 4.  Dynamic shared memory:
+//   digits [NTOK*ND][slab + 64] int8 | sums [4 column parts][NTOK*ND][128] int32 | slots [4][NTOK][32] | scale [NTOK] |
+//   max bits [NTOK] | range counts [NTOK]
+// Warp w: rows 32 (w % 4) .. +31 of the tile (two MMA row tiles), column part w / 4 of the CTA's slab:
+// per round of 16 groups it takes groups 4 (w / 4) .. +3.
+template <typename IN_T, int ND, int NTOK, int STAGE>
+__global__ void __launch_bounds__(GEMV_THREADS, NTOK <= 2 ? 2 : 1)
+ternary_gemv_cluster_kernel(const GemvParams p)
+{
+    extern __shared__ __align__(16) uint8_t smem[];
+    constexpr bool kInt = sizeof(IN_T) == 1;
+    constexpr bool kIntSlots = kInt && STAGE == STAGE_V;   // exact integer partial sums
+    constexpr int NCOL = NTOK * ND;
+    constexpr int NT = (NCOL + 7) / 8;
+    const int n_groups = p.C_pad >> 6;
+    const int gq = cluster_slab_groups(p.C_pad);
+    const uint32_t rank = cluster_rank();
+    const int g0 = (int)rank * gq, g1 = min(n_groups, g0 + gq);      // this CTA's column groups
+    const int dstride = gq * 64 + GEMV_DIG_PAD;
+    int8_t* dig = reinterpret_cast<int8_t*>(smem);
+    int* red = reinterpret_cast<int*>(smem + (size_t)NCOL * dstride);
+    uint32_t* slots = reinterpret_cast<uint32_t*>(red + 4 * NCOL * CLUSTER_ROWS);   // [4][NTOK][32]
+    float* scale = reinterpret_cast<float*>(slots + CLUSTER_CTAS * NTOK * CLUSTER_OWN);
+    unsigned* smax = reinterpret_cast<unsigned*>(scale + NTOK);
+    unsigned* srange = smax + NTOK;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, q = lane & 3;
+    const int rp = warp & 3, cp = warp >> 2;
+    const int tile = blockIdx.x / CLUSTER_CTAS;
+    const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
+    if (tid < NTOK) { smax[tid] = 0u; srange[tid] = 0u; }
+
+    // this lane's codes of the first round, requested before the wait (they travel from HBM meanwhile)
+    constexpr int GROUP_WORDS = 128 * 4;
+    const uint32_t* wp = reinterpret_cast<const uint32_t*>(p.units) +
+                         (tsvd_unit_index(tile * CLUSTER_ROWS + rp * 32, g0 + cp * GEMV_PRE, p.C_pad) + g) * 4 + q;
+    uint32_t w[GEMV_PRE][2][2];
+#pragma unroll
+    for (int i = 0; i < GEMV_PRE; ++i) {
+        const bool there = g0 + cp * GEMV_PRE + i < g1;
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int r = 0; r < 2; ++r)
+                w[i][h][r] = there ? ld_stream_now(wp + i * GROUP_WORDS + (16 * h + 8 * r) * 4) : 0u;
+    }
+    pdl_wait();
+    pdl_launch_dependents();
+    tsvd_stamp_begin(p.stamp);
+    PH(0);
+    __syncthreads();   // the cleared maxima and counts
+
+    // ---- this CTA's quarter of the stage input as fixed-point digits: item = (token, chunk of 8 columns) ----
+    const int slab_chunks = (g1 - g0) * 8;                    // chunks of 8 columns in the slab
+    const int n_items = NTOK * slab_chunks;
+    constexpr int MAX_KEEP = 2;                               // items a thread keeps between the passes
+    float keep[MAX_KEEP][8];
+    auto load_item = [&](int it, float (&v)[8]) {
+        const int b = it / slab_chunks, ch = it - b * slab_chunks;
+        const IN_T* row = in + (size_t)(b < p.B ? b : 0) * p.ld_in;
+        const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+        load8<IN_T>(row, g0 * 64 + ch * 8, p.C, vec_ok, v);
+    };
+    // (all 32 lanes of a warp run the same number of trips when this holds: n_items is then a multiple of 32)
+    const bool warp_one_token = (slab_chunks & 31) == 0;
+    if constexpr (!kInt) {
+        int k = 0;
+        for (int it = tid; it < n_items; it += GEMV_THREADS, ++k) {
+            float v[8];
+            load_item(it, v);
+            float m = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) m = fmaxf(m, fabsf(v[e]));
+            if (k < MAX_KEEP) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) keep[k][e] = v[e];
+            }
+            // non-negative floats order as their bits; when a warp's 32 items belong to one token
+            // (slabs of whole multiples of 256 columns) the warp reduces first
+            unsigned mb = __float_as_uint(m);
+            if (warp_one_token) {
+                mb = __reduce_max_sync(0xffffffffu, mb);
+                if (lane == 0 && mb) atomicMax(&smax[it / slab_chunks], mb);
+            } else if (mb) {
+                atomicMax(&smax[it / slab_chunks], mb);
+            }
+        }
+        __syncthreads();
+    }
+    PH(1);
+    {
+        int k = 0;
+        for (int it = tid; it < n_items; it += GEMV_THREADS, ++k) {
+            const int b = it / slab_chunks, ch = it - b * slab_chunks;
+            float v[8];
+            if (!kInt && k < MAX_KEEP) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[e] = keep[k][e];
+            } else {
+                load_item(it, v);
+            }
+            uint32_t dw[ND][2];
+#pragma unroll
+            for (int d = 0; d < ND; ++d) dw[d][0] = dw[d][1] = 0u;
+            if (b < p.B) {
+                int qv[8];
+                float qscale = 1.f;
+                if constexpr (!kInt) {
+                    const int E = tsvd_quant_exponent(__uint_as_float(smax[b]));
+                    qscale = tsvd_pow2(8 * ND - 2 - E);
+                    unsigned cnt = 0;
+                    tsvd_range_sample(cnt, v[0], qscale);
+                    if (warp_one_token) {
+                        cnt = __reduce_add_sync(0xffffffffu, cnt);
+                        if (lane == 0 && cnt) atomicAdd(&srange[b], cnt);
+                    } else if (cnt) {
+                        atomicAdd(&srange[b], cnt);
+                    }
+                }
+                if constexpr (ND <= 3) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) qv[e] = tsvd_round_bits(v[e], qscale);
+                    digits_of<ND, 2>(qv, dw, TSVD_ROUND_BIAS);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) qv[e] = __float2int_rn(v[e] * qscale);
+                    digits_of<ND, 2>(qv, dw);
+                }
+            }
+#pragma unroll
+            for (int d = 0; d < ND; ++d)
+                *reinterpret_cast<uint2*>(dig + (size_t)(b * ND + d) * dstride + ch * 8) = make_uint2(dw[d][0], dw[d][1]);
+        }
+    }
+    if (tid < NTOK) {
+        float sc = 1.f;
+        if constexpr (!kInt) sc = tsvd_pow2(tsvd_quant_exponent(__uint_as_float(smax[tid])) - (8 * ND - 2));
+        scale[tid] = sc;
+    }
+    __syncthreads();
+    if constexpr (!kInt) {
+        if (tid < NTOK) {   // range diagnostic on this CTA's samples of the token
+            const unsigned tot = srange[tid], nz = tot & 0xffffu, big = tot >> 16;
+            if (nz >= 32u && 4u * big < nz) atomicOr(p.status, TSVD_DEV_RANGE);
+        }
+    }
+
+    PH(2);
+    // ---- stream the codes of this warp's rows and column part ----
+    int acc[2][NT][4];
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[h][j][c] = 0;
+    bool col_there[NT];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) col_there[j] = 8 * j + g < NCOL;
+    const int8_t* dp = dig + (size_t)g * dstride + cp * (GEMV_PRE * 64) + q * 16;
+    constexpr int ROUND = 4 * GEMV_PRE;     // column groups the CTA's four column parts cover per round
+#pragma unroll 1
+    for (int rb = g0; rb < g1; rb += ROUND) {
+        const int first = rb + cp * GEMV_PRE;          // this warp's first group of the round
+        wp += ROUND * GROUP_WORDS;
+        const bool more = rb + ROUND < g1;
+#pragma unroll
+        for (int i = 0; i < GEMV_PRE; ++i) {
+            if (first + i < g1) {
+                uint4 xd[NT];
+#pragma unroll
+                for (int j = 0; j < NT; ++j)
+                    xd[j] = col_there[j] ? *reinterpret_cast<const uint4*>(dp + (size_t)(8 * j) * dstride + i * 64)
+                                         : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t e0[4], e1[4];
+                    tsvd_expand16(w[i][h][0], e0);
+                    tsvd_expand16(w[i][h][1], e1);
+                    if (more && first + ROUND + i < g1) {   // the group's codes are in e0/e1: request the next round's
+#pragma unroll
+                        for (int r = 0; r < 2; ++r) w[i][h][r] = ld_stream_now(wp + i * GROUP_WORDS + (16 * h + 8 * r) * 4);
+                    }
+#pragma unroll
+                    for (int j = 0; j < NT; ++j) {
+                        mma_s8(acc[h][j], e0[0], e1[0], e0[1], e1[1], xd[j].x, xd[j].y);
+                        mma_s8(acc[h][j], e0[2], e1[2], e0[3], e1[3], xd[j].z, xd[j].w);
+                    }
+                }
+            }
+        }
+        dp += ROUND * 64;
+    }
+    PH(3);
+    // every warp owns its rows of its column part's plane of `red`: plain stores, summed below
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int n = 8 * j + 2 * q + (c & 1), r = rp * 32 + 16 * h + g + 8 * (c >> 1);
+                if (n < NCOL) red[(cp * NCOL + n) * CLUSTER_ROWS + r] = acc[h][j][c];
+            }
+    __syncthreads();
+    PH(4);
+
+    // ---- this CTA's partial result of every row goes to the CTA that finishes the row ----
+    for (int it = tid; it < NTOK * CLUSTER_ROWS; it += GEMV_THREADS) {
+        const int b = it / CLUSTER_ROWS, r = it % CLUSTER_ROWS;
+        int a[ND];
+#pragma unroll
+        for (int d = 0; d < ND; ++d) {   // the four column parts: exact integer additions
+            const int* rr = red + (b * ND + d) * CLUSTER_ROWS + r;
+            a[d] = rr[0] + rr[NCOL * CLUSTER_ROWS] + rr[2 * NCOL * CLUSTER_ROWS] + rr[3 * NCOL * CLUSTER_ROWS];
+        }
+        uint32_t bits;
+        if constexpr (kIntSlots) {
+            bits = (uint32_t)a[0];
+        } else {
+            float f;
+            if constexpr (ND == 1) f = (float)a[0];
+            else if constexpr (ND == 2) f = (float)(a[0] + (a[1] << 8));
+            else {
+                const int lo = a[0] + (a[1] << 8);
+                int hi = a[2];
+                if constexpr (ND == 4) hi += a[3] << 8;
+                f = fmaf((float)hi, 65536.f, (float)lo);
+            }
+            bits = __float_as_uint(f * scale[b]);   // a power of two: exact
+        }
+        const uint32_t owner = (uint32_t)(r / CLUSTER_OWN);
+        cluster_store(cluster_map(slots + ((int)rank * NTOK + b) * CLUSTER_OWN + (r % CLUSTER_OWN), owner), bits);
+    }
+    cluster_barrier();
+    PH(5);
+
+    // ---- thread (token, own row): the four partial results in a fixed order -> the stage's output ----
+    if (tid < NTOK * CLUSTER_OWN) {
+        const int b = tid / CLUSTER_OWN, r = tid % CLUSTER_OWN;
+        const int orow = tile * CLUSTER_ROWS + (int)rank * CLUSTER_OWN + r;
+        if (b < p.B) {
+            float val;
+            int zi = 0;
+            if constexpr (kIntSlots) {
+#pragma unroll
+                for (int c = 0; c < CLUSTER_CTAS; ++c) zi += (int)slots[(c * NTOK + b) * CLUSTER_OWN + r];
+                val = (float)zi;
+            } else {
+                val = 0.f;
+#pragma unroll
+                for (int c = 0; c < CLUSTER_CTAS; ++c) val += __uint_as_float(slots[(c * NTOK + b) * CLUSTER_OWN + r]);
+            }
+            if constexpr (STAGE == STAGE_V) {
+                reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + orow] = p.S[orow] * val;   // the K multiplications
+                if (p.z_out && orow < p.R) {
+                    if (p.z_int) reinterpret_cast<int*>(p.z_out)[(size_t)b * p.z_ld + orow] = zi;
+                    else reinterpret_cast<float*>(p.z_out)[(size_t)b * p.z_ld + orow] = val;
+                }
+            } else if (orow < p.R) {
+                const float yv = p.bias ? val + __ldg(p.bias + orow) : val;
+                if (p.out_bf16)
+                    reinterpret_cast<__nv_bfloat16*>(p.out)[(size_t)b * p.ld_out + orow] = __float2bfloat16_rn(yv);
+                else
+                    reinterpret_cast<float*>(p.out)[(size_t)b * p.ld_out + orow] = yv;
+            }
+        }
+    }
+    tsvd_stamp_end(p.stamp);
+}
+
+size_t gemv_cluster_smem_bytes(int nd, int ntok, int C_pad)
+{
+    const size_t ncol = (size_t)ntok * nd;
+    return ncol * (cluster_slab_groups(C_pad) * 64 + GEMV_DIG_PAD) + 4 * ncol * CLUSTER_ROWS * sizeof(int) +
+           (size_t)CLUSTER_CTAS * ntok * CLUSTER_OWN * 4 + (size_t)ntok * 12;
+}
+// (at one and two tokens the exchange between the four CTAs costs more than the shared conversion saves)
+inline bool use_cluster_form(int C_pad, int B) { return B >= CLUSTER_MIN_TOKENS && (C_pad >> 6) >= CLUSTER_MIN_GROUPS; }
+
 size_t gemv_smem_bytes(int nd, int ntok, int C_pad)
 {
     return (size_t)ntok * nd * (C_pad + GEMV_DIG_PAD) + (size_t)ntok * nd * GEMV_ROWS * sizeof(int) +
@@ -383,9 +712,48 @@ cudaError_t launch_gemv(const GemvParams& p, int R_pad, cudaStream_t stream)
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
+template <typename IN_T, int ND, int NTOK, int STAGE>
+cudaError_t launch_gemv_cluster(const GemvParams& p, int R_pad, cudaStream_t stream)
+{
+    static bool attr_set[64] = {};   // per instantiation and device
+    const size_t smem = gemv_cluster_smem_bytes(ND, NTOK, p.C_pad);
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(ternary_gemv_cluster_kernel<IN_T, ND, NTOK, STAGE>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, GEMV_MAX_SMEM);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(R_pad / CLUSTER_ROWS * CLUSTER_CTAS));
+    cfg.blockDim = dim3(GEMV_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CLUSTER_CTAS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, ternary_gemv_cluster_kernel<IN_T, ND, NTOK, STAGE>, (const GemvParams)p);
+    tsvd_count_launch();
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 template <typename IN_T, int ND, int STAGE>
 cudaError_t launch_gemv_tokens(const GemvParams& p, int R_pad, cudaStream_t stream)
 {
+    if (use_cluster_form(p.C_pad, p.B)) {
+        if (p.B == 1) return launch_gemv_cluster<IN_T, ND, 1, STAGE>(p, R_pad, stream);
+        if (p.B == 2) return launch_gemv_cluster<IN_T, ND, 2, STAGE>(p, R_pad, stream);
+        if (p.B <= 4) return launch_gemv_cluster<IN_T, ND, 4, STAGE>(p, R_pad, stream);
+        return launch_gemv_cluster<IN_T, ND, 8, STAGE>(p, R_pad, stream);
+    }
     if (p.B == 1) return launch_gemv<IN_T, ND, 1, STAGE>(p, R_pad, stream);
     if (p.B == 2) return launch_gemv<IN_T, ND, 2, STAGE>(p, R_pad, stream);
     if (p.B <= 4) return launch_gemv<IN_T, ND, 4, STAGE>(p, R_pad, stream);
@@ -401,8 +769,10 @@ bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_
 {
     if (B < 1 || B > TSVD_DECODE_MAX_B) return false;
     const int ntok = B <= 2 ? B : B <= 4 ? 4 : 8;
-    return gemv_smem_bytes(digits_for_x(dt, wide_x), ntok, h->V.C_pad) <= (size_t)GEMV_MAX_SMEM &&
-           gemv_smem_bytes(ND_T, ntok, h->U.C_pad) <= (size_t)GEMV_MAX_SMEM;
+    auto need = [&](int nd, int C_pad) {
+        return use_cluster_form(C_pad, B) ? gemv_cluster_smem_bytes(nd, ntok, C_pad) : gemv_smem_bytes(nd, ntok, C_pad);
+    };
+    return need(digits_for_x(dt, wide_x), h->V.C_pad) <= (size_t)GEMV_MAX_SMEM && need(ND_T, h->U.C_pad) <= (size_t)GEMV_MAX_SMEM;
 }
 
 size_t tsvd_decode_ws_bytes(const tsvd_handle_s* h, int B) { return (size_t)B * h->V.R_pad * sizeof(float); }

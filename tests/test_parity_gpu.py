@@ -147,10 +147,11 @@ def test_decode_is_the_default_up_to_eight_tokens_and_refuses_more():
 
 
 def test_decode_and_tensor_paths_agree_bit_for_bit():
-    """Both quantise the stage inputs the same way and add exact integers: identical outputs."""
+    """Below 1024 columns both quantise each token with one scale and add exact integers: identical
+    outputs.  (From 1024 columns on the decode kernels scale each quarter of the columns on its own.)"""
     import torch
     from paper_2308_07641_b200 import TSVDLinear
-    spec = gen.scaled(C["cfg3_b4"], name="agree", M=700, N=900, K=520, B=4, seed=31)
+    spec = gen.scaled(C["cfg3_b4"], name="agree", M=700, N=700, K=520, B=4, seed=31)
     U, V, S = gen.make_weights(spec)
     x = _util.torch_x(gen.make_x(spec), spec.x_dtype)
     layer = TSVDLinear(U, S, V)
@@ -159,6 +160,31 @@ def test_decode_and_tensor_paths_agree_bit_for_bit():
         y_ten = layer.forward(x, flags=0x40 | 0x1).clone()
         torch.cuda.synchronize()
         assert torch.equal(y_dec, y_ten)
+    finally:
+        layer.close()
+
+
+@pytest.mark.parametrize("B", [1, 2, 3, 4, 6, 8])
+@pytest.mark.parametrize("x_dtype,base", [("bf16", "cfg3_b4"), ("f32", "cfg1"), ("i8", "cfg5_d20")])
+def test_decode_cluster_form_long_contractions(B, x_dtype, base):
+    """From 1024 columns on four CTAs of a cluster split the contraction of a 128-row tile; ragged
+    column counts leave the last quarter short, and 17 or 18 column groups do not divide by four."""
+    for (M, N, K) in ((300, 1100, 1030), (200, 2300, 1100)):
+        spec = gen.scaled(C[base], name=f"cluster_{x_dtype}_B{B}_{N}", M=M, N=N, K=K, B=B, seed=90 + B)
+        _util.run_and_check(spec, flags=0x20)
+
+
+def test_decode_cluster_form_runs_back_to_back_and_is_deterministic():
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear
+    spec = gen.scaled(C["cfg3_b4"], name="cluster_repeat", M=1000, N=4096, K=2048, B=4, seed=97)
+    U, V, S = gen.make_weights(spec)
+    x = _util.torch_x(gen.make_x(spec), "bf16")
+    layer = TSVDLinear(U, S, V)
+    try:
+        ys = [layer.forward(x, flags=0x20 | 0x1).clone() for _ in range(6)]
+        torch.cuda.synchronize()
+        assert all(torch.equal(ys[0], y) for y in ys[1:])
     finally:
         layer.close()
 
@@ -214,14 +240,24 @@ def test_kernels_launched_early_still_see_inputs_written_just_before():
 
 def test_decode_falls_back_when_the_digits_do_not_fit_shared_memory():
     from paper_2308_07641_b200 import binding
-    N = 13000                       # 4 tokens x 4 digits x 13056 columns > 200 KiB (and so are 8 tokens)
+    N = 13000                       # 2 tokens x 4 digits x 13056 columns fit 200 KiB; so do 4 and 8 tokens on a quarter each
     U = np.zeros((8, 8), np.int8); V = np.zeros((8, N), np.int8); S = np.ones(8, np.float32)
     h = binding.tsvd_pack(U, S, V)
     try:
-        assert binding.tsvd_plan(h, 4, binding.TSVD_F32)["path"] == "tensor"
+        for B in (1, 2, 4, 8):
+            assert binding.tsvd_plan(h, B, binding.TSVD_F32)["path"] == "decode"
+    finally:
+        binding.tsvd_destroy(h)
+    N = 40000                       # 40064 padded columns x 4 digits: one token fits, two do not; a quarter at four tokens fits, at eight not
+    V = np.zeros((8, N), np.int8)
+    h = binding.tsvd_pack(U, S, V)
+    try:
         assert binding.tsvd_plan(h, 1, binding.TSVD_F32)["path"] == "decode"
+        assert binding.tsvd_plan(h, 2, binding.TSVD_F32)["path"] == "tensor"
+        assert binding.tsvd_plan(h, 4, binding.TSVD_F32)["path"] == "decode"
+        assert binding.tsvd_plan(h, 8, binding.TSVD_F32)["path"] == "tensor"
         with pytest.raises(binding.TSVDError) as ei:
-            binding.tsvd_plan(h, 4, binding.TSVD_F32, 0x20)
+            binding.tsvd_plan(h, 8, binding.TSVD_F32, 0x20)
         assert ei.value.status == binding.TSVD_E_TOOBIG
     finally:
         binding.tsvd_destroy(h)
