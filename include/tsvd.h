@@ -84,8 +84,9 @@ typedef enum {
  * codes against fixed-point digits of the stage's input held in shared memory) serve batches
  * of at most this many tokens, and are what a forward of so few tokens runs by default.
  * Forcing them for a larger batch, or for a contraction too long for the digits to fit in
- * shared memory (about 10,000 columns at four tokens, 6,000 at eight), returns TSVD_E_TOOBIG. */
-#define TSVD_DECODE_MAX_B 8
+ * shared memory (about 13,000 columns at one token, 40,000 at four, 12,000 at sixteen; nine to
+ * sixteen tokens also need 1024 columns or more in both stages), returns TSVD_E_TOOBIG. */
+#define TSVD_DECODE_MAX_B 16
 /* the index-list kernels serve at most this many tokens */
 #define TSVD_INDEX_MAX_B 4
 /* Test hook for the bounded device-side waits: with B > 64 the V-stage kernel's copy

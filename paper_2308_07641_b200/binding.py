@@ -24,7 +24,7 @@ TSVD_STATIC_SCRATCH_BYTES = 4 << 20
 TSVD_FLAG_OUT_F32 = 0x1
 TSVD_FLAG_PATH_SIMPLE = 0x10
 TSVD_FLAG_PATH_DECODE = 0x20
-TSVD_DECODE_MAX_B = 8        # largest batch the decode kernels serve (tsvd.h)
+TSVD_DECODE_MAX_B = 16       # largest batch the decode kernels serve (tsvd.h)
 TSVD_INDEX_MAX_B = 4         # largest batch the index-list kernels serve
 TSVD_FLAG_PATH_TENSOR = 0x40
 TSVD_FLAG_PATH_INDEX = 0x80      # index-list kernels, for handles packed with TSVD_PACK_INDEX_LISTS

@@ -29,7 +29,7 @@ constexpr int GEMV_THREADS = 512, GEMV_WARPS = GEMV_THREADS / 32;
 constexpr int GEMV_ROWS = 32;       // rows per CTA: two MMA row tiles
 constexpr int GEMV_PRE = 4;         // column groups a warp has in flight at a time
 constexpr int GEMV_DIG_PAD = 64;    // bytes between digit rows beyond C_pad: eight rows x four quarters hit all banks
-constexpr int GEMV_MAX_SMEM = 200 * 1024;
+constexpr int GEMV_MAX_SMEM = 224 * 1024;
 
 enum { STAGE_V = 0, STAGE_U = 1 };
 
@@ -575,24 +575,25 @@ ternary_gemv_cluster_kernel(const GemvParams p)
 #pragma unroll
         for (int i = 0; i < GEMV_PRE; ++i) {
             if (first + i < g1) {
-                uint4 xd[NT];
-#pragma unroll
-                for (int j = 0; j < NT; ++j)
-                    xd[j] = col_there[j] ? *reinterpret_cast<const uint4*>(dp + (size_t)(8 * j) * dstride + i * 64)
-                                         : make_uint4(0, 0, 0, 0);
+                uint32_t e0[2][4], e1[2][4];   // sixteen entries of rows 16h + g and 16h + g + 8 as int8
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    uint32_t e0[4], e1[4];
-                    tsvd_expand16(w[i][h][0], e0);
-                    tsvd_expand16(w[i][h][1], e1);
-                    if (more && first + ROUND + i < g1) {   // the group's codes are in e0/e1: request the next round's
+                    tsvd_expand16(w[i][h][0], e0[h]);
+                    tsvd_expand16(w[i][h][1], e1[h]);
+                    if (more && first + ROUND + i < g1) {   // the group's codes are expanded: request the next round's
 #pragma unroll
                         for (int r = 0; r < 2; ++r) w[i][h][r] = ld_stream_now(wp + i * GROUP_WORDS + (16 * h + 8 * r) * 4);
                     }
+                }
 #pragma unroll
-                    for (int j = 0; j < NT; ++j) {
-                        mma_s8(acc[h][j], e0[0], e1[0], e0[1], e1[1], xd[j].x, xd[j].y);
-                        mma_s8(acc[h][j], e0[2], e1[2], e0[3], e1[3], xd[j].z, xd[j].w);
+                for (int j = 0; j < NT; ++j) {
+                    // digits of columns 16q .. 16q+15 of this group, (token, digit) pair 8j + g
+                    const uint4 xd = col_there[j] ? *reinterpret_cast<const uint4*>(dp + (size_t)(8 * j) * dstride + i * 64)
+                                                  : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        mma_s8(acc[h][j], e0[h][0], e1[h][0], e0[h][1], e1[h][1], xd.x, xd.y);
+                        mma_s8(acc[h][j], e0[h][2], e1[h][2], e0[h][3], e1[h][3], xd.z, xd.w);
                     }
                 }
             }
@@ -752,8 +753,10 @@ cudaError_t launch_gemv_tokens(const GemvParams& p, int R_pad, cudaStream_t stre
         if (p.B == 1) return launch_gemv_cluster<IN_T, ND, 1, STAGE>(p, R_pad, stream);
         if (p.B == 2) return launch_gemv_cluster<IN_T, ND, 2, STAGE>(p, R_pad, stream);
         if (p.B <= 4) return launch_gemv_cluster<IN_T, ND, 4, STAGE>(p, R_pad, stream);
-        return launch_gemv_cluster<IN_T, ND, 8, STAGE>(p, R_pad, stream);
+        if (p.B <= 8) return launch_gemv_cluster<IN_T, ND, 8, STAGE>(p, R_pad, stream);
+        return launch_gemv_cluster<IN_T, ND, 16, STAGE>(p, R_pad, stream);
     }
+    if (p.B > 8) return cudaErrorInvalidValue;   // (tsvd_decode_fits keeps such requests away)
     if (p.B == 1) return launch_gemv<IN_T, ND, 1, STAGE>(p, R_pad, stream);
     if (p.B == 2) return launch_gemv<IN_T, ND, 2, STAGE>(p, R_pad, stream);
     if (p.B <= 4) return launch_gemv<IN_T, ND, 4, STAGE>(p, R_pad, stream);
@@ -768,7 +771,9 @@ inline int digits_for_x(tsvd_dtype_t dt, bool wide) { return dt == TSVD_I8 ? 1 :
 bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x)
 {
     if (B < 1 || B > TSVD_DECODE_MAX_B) return false;
-    const int ntok = B <= 2 ? B : B <= 4 ? 4 : 8;
+    const int ntok = B <= 2 ? B : B <= 4 ? 4 : B <= 8 ? 8 : 16;
+    // nine to sixteen tokens: the cluster form only
+    if (B > 8 && !(use_cluster_form(h->V.C_pad, B) && use_cluster_form(h->U.C_pad, B))) return false;
     auto need = [&](int nd, int C_pad) {
         return use_cluster_form(C_pad, B) ? gemv_cluster_smem_bytes(nd, ntok, C_pad) : gemv_smem_bytes(nd, ntok, C_pad);
     };

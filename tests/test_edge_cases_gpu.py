@@ -2,7 +2,7 @@
 CPU checker at the stated tolerances, on every kernel family:
 
   tensor  (B > 64: 192-column tiles)      small  (5..64 tokens: split contraction)
-  decode  (1..8 tokens)                   index  (1..4 tokens, index lists)      simple (CUDA cores)
+  decode  (1..16 tokens)                  index  (1..4 tokens, index lists)      simple (CUDA cores)
 
 Cases: S with negative, zero and widely spread entries (S comes from a pseudo-inverse, Eq. 4);
 tokens with outliers 2^8 .. 2^20 above their bulk; an all-zero token inside a batch; int8
@@ -25,7 +25,7 @@ OK, RANGE = 0, 10
 SIMPLE, DECODE, TENSOR, INDEX, WIDE = 0x10, 0x20, 0x40, 0x80, 0x200
 
 # (family name, forced path flag, batch, tsvd_pack flags)
-FAMILIES = [("tensor", TENSOR, 150, 0), ("small", TENSOR, 23, 0), ("decode", DECODE, 3, 0), ("decode8", DECODE, 7, 0),
+FAMILIES = [("tensor", TENSOR, 150, 0), ("small", TENSOR, 23, 0), ("decode", DECODE, 3, 0), ("decode8", DECODE, 7, 0), ("decode16", DECODE, 13, 0),
             ("index", INDEX, 4, 1), ("simple", SIMPLE, 11, 0)]
 FAST = [f for f in FAMILIES if f[0] != "simple"]
 
@@ -40,6 +40,8 @@ def _spec(base, name, B, **kw):
     kw.setdefault("M", 520)
     kw.setdefault("N", 1100)
     kw.setdefault("K", 650)
+    if B == 13:       # the decode16 family: nine to sixteen tokens need 1024+ columns in both stages
+        kw["N"], kw["K"] = max(kw["N"], 1100), max(kw["K"], 1030)
     return gen.scaled(C[base], name=name, B=B, **kw)
 
 
