@@ -19,7 +19,9 @@ Readings where the paper is silent:
   * stride, padding and dilation of the layer go, per direction, to the stage whose kernel spans
     that direction (to V(.) where neither does); the other stage has stride 1 and no padding there.
     Zero padding of the intermediate is exact because the stages have no bias;
-  * groups = 1 (the depth-wise layers of the listing, rank 5, are not covered).
+  * groups: a grouped layer (the depth-wise layers of the listing: groups = channels, rank 5) is one
+    independent TSVD per group on that group's channels, each with its own U, S, V of equal shapes
+    (`conv2d_tsvd_grouped`); the listing's "rank" is read as the rank of each group.
 
 Nothing in the GPU library imports this module, and this module imports nothing of it.
 Pins: tests/test_conv_pins.py.
@@ -139,3 +141,25 @@ def conv2d_dense(x: np.ndarray, W: np.ndarray, stride: Pair = (1, 1), padding: P
     C_out, C_in, K1, K2 = W.shape
     pa = _patches(np.asarray(x, dtype=np.float64), (K1, K2), stride, padding, dilation)
     return np.einsum("nhwcab,ocab->nhwo", pa, np.asarray(W, dtype=np.float64))
+
+
+def conv2d_tsvd_grouped(x: np.ndarray, Us, Ss, Vs, form: int, C_out: int, C_in: int, K1: int, K2: int,
+                        stride: Pair = (1, 1), padding: Pair = (0, 0), dilation: Pair = (1, 1)) -> np.ndarray:
+    """A grouped layer: group g maps input channels [g*C_in/G, (g+1)*C_in/G) to output channels
+    [g*C_out/G, (g+1)*C_out/G) by its own TSVD (Us[g], Ss[g], Vs[g]); G = len(Us)."""
+    G = len(Us)
+    ci, co = C_in // G, C_out // G
+    assert ci * G == C_in and co * G == C_out
+    outs = [conv2d_tsvd(np.ascontiguousarray(x[..., g * ci:(g + 1) * ci]), Us[g], Ss[g], Vs[g], form, co, ci, K1, K2,
+                        stride, padding, dilation) for g in range(G)]
+    return np.concatenate(outs, axis=-1)
+
+
+def conv2d_dense_grouped(x: np.ndarray, W: np.ndarray, groups: int, stride: Pair = (1, 1), padding: Pair = (0, 0),
+                         dilation: Pair = (1, 1)) -> np.ndarray:
+    """Plain grouped correlation; W [C_out, C_in / groups, K1, K2]."""
+    C_out = W.shape[0]
+    ci, co = W.shape[1], C_out // groups
+    outs = [conv2d_dense(x[..., g * ci:(g + 1) * ci], W[g * co:(g + 1) * co], stride, padding, dilation)
+            for g in range(groups)]
+    return np.concatenate(outs, axis=-1)

@@ -86,3 +86,33 @@ def test_pointwise_kernel_is_the_linear_layer():
     x = g.standard_normal((3, 2, 2, 4))
     y = oc.conv2d_tsvd(x, U, S, V, 0, 6, 4, 1, 1)
     assert np.abs(y.reshape(12, 6) - oracle.forward(U, S, V, x.reshape(12, 4)).y).max() < 1e-13
+
+
+def test_grouped_and_depthwise_layers():
+    """Groups are independent layers on their own channels: against nested loops over the grouped
+    kernel that the per-group U diag(S) V reshape to (a depth-wise 7x7 layer of rank 5 among them)."""
+    g = np.random.default_rng(21)
+    for (G, co, ci, K1, K2, K, form, geom) in [(6, 1, 1, 7, 7, 5, 0, ((1, 1), (3, 3), (1, 1))),
+                                               (3, 2, 4, 3, 3, 6, 2, ((2, 1), (1, 1), (1, 1))),
+                                               (2, 3, 2, 2, 3, 4, 1, ((1, 2), (0, 1), (1, 1)))]:
+        stride, pad, dil = geom
+        M, N = oc.matrix_shape(form, co, ci, K1, K2)
+        Us = [g.integers(-1, 2, (M, K)).astype(np.int8) for _ in range(G)]
+        Vs = [g.integers(-1, 2, (K, N)).astype(np.int8) for _ in range(G)]
+        Ss = [(g.integers(-16, 17, K) / 8.0).astype(np.float32) for _ in range(G)]
+        x = g.integers(-20, 21, (2, 9, 8, G * ci)) / 4.0
+        Wk = np.concatenate([oc.matrix_to_kernel((Us[i] * Ss[i].astype(np.float64)[None, :]) @ Vs[i].astype(np.float64),
+                                                 form, co, ci, K1, K2) for i in range(G)], axis=0)
+        got = oc.conv2d_tsvd_grouped(x, Us, Ss, Vs, form, G * co, G * ci, K1, K2, stride, pad, dil)
+        assert np.array_equal(got, oc.conv2d_dense_grouped(x, Wk, G, stride, pad, dil))
+        # the grouped correlation itself, by nested loops on one output position per channel
+        n, Ho, Wo, Co = got.shape
+        for o in range(Co):
+            grp = o // co
+            ho, wo = Ho // 2, Wo // 3
+            acc = 0.0
+            for c, a, b in itertools.product(range(ci), range(K1), range(K2)):
+                h, w = ho * stride[0] + a * dil[0] - pad[0], wo * stride[1] + b * dil[1] - pad[1]
+                if 0 <= h < 9 and 0 <= w < 8:
+                    acc += Wk[o, c, a, b] * x[1, h, w, grp * ci + c]
+            assert abs(got[1, ho, wo, o] - acc) < 1e-12
