@@ -12,7 +12,11 @@ The kernel W [C_out, C_in, K1, K2] is decomposed as one of the four matrices of 
 
 with rows ordered (c_out, a, b) and columns (c_in, a, b) as the products are written there.  Per
 direction, the layer's stride, padding and dilation go to the stage whose kernel spans that direction
-(to V(.) where neither does).  Images are NHWC; groups = 1; no bias inside the stages.
+(to V(.) where neither does).  Images are NHWC; no bias inside the stages.  A grouped layer (the
+depth-wise layers of the paper's listing: one TSVD of rank 5 per channel) is passed as lists of
+per-group U, S, V and runs as one layer whose matrices are block-diagonal: group g's ternary entries
+sit at its own channels and its own rank components, zeros elsewhere, so both stages stay the same two
+ternary products.
 """
 from __future__ import annotations
 
@@ -35,14 +39,17 @@ def _out(L: int, k: int, s: int, p: int, d: int) -> int:
 
 class TSVDConv2d:
     """A convolution layer in TSVD form.  U int8 [M, K], S float32 [K], V int8 [K, N] with [M, N] the
-    shape of the chosen matrix of Eq. 5."""
+    shape of the chosen matrix of Eq. 5; or, for a grouped layer, lists of G such triples of equal
+    shapes, each for C_out/G output and C_in/G input channels."""
 
     def __init__(self, U, S, V, form: int, C_out: int, C_in: int, K1: int, K2: int, stride: Pair = (1, 1),
                  padding: Pair = (0, 0), dilation: Pair = (1, 1)):
+        (v1, v2), (u1, u2) = _stage_kernels(form, K1, K2)
+        if isinstance(U, (list, tuple)):
+            U, S, V = self._block_diagonal(U, S, V, C_out, C_in, (v1, v2), (u1, u2))
         U = np.ascontiguousarray(U, dtype=np.int8)
         V = np.ascontiguousarray(V, dtype=np.int8)
         S = np.ascontiguousarray(S, dtype=np.float32)
-        (v1, v2), (u1, u2) = _stage_kernels(form, K1, K2)
         K = S.shape[0]
         if U.shape != (C_out * u1 * u2, K) or V.shape != (K, C_in * v1 * v2):
             raise binding.TSVDError(binding.TSVD_E_SHAPE, "TSVDConv2d")
@@ -62,6 +69,27 @@ class TSVDConv2d:
         # matrix of each handle is a single row of zeros.
         self.h_v = binding.tsvd_pack(np.zeros((1, K), np.int8), S, np.ascontiguousarray(Vp))
         self.h_u = binding.tsvd_pack(np.zeros((1, C_out), np.int8), np.ones(C_out, np.float32), np.ascontiguousarray(Up))
+
+    @staticmethod
+    def _block_diagonal(Us, Ss, Vs, C_out, C_in, kv, ku):
+        """G per-group layers as one: rank components concatenated, group g's entries at its channels."""
+        G = len(Us)
+        co, ci = C_out // G, C_in // G
+        Kg = np.asarray(Ss[0]).shape[0]
+        if co * G != C_out or ci * G != C_in or len(Ss) != G or len(Vs) != G:
+            raise binding.TSVDError(binding.TSVD_E_SHAPE, "TSVDConv2d")
+        (v1, v2), (u1, u2) = kv, ku
+        U = np.zeros((C_out, u1, u2, G * Kg), np.int8)
+        V = np.zeros((G * Kg, C_in, v1, v2), np.int8)
+        S = np.zeros(G * Kg, np.float32)
+        for g in range(G):
+            Ug, Vg = np.asarray(Us[g], dtype=np.int8), np.asarray(Vs[g], dtype=np.int8)
+            if Ug.shape != (co * u1 * u2, Kg) or Vg.shape != (Kg, ci * v1 * v2):
+                raise binding.TSVDError(binding.TSVD_E_SHAPE, "TSVDConv2d")
+            U[g * co:(g + 1) * co, :, :, g * Kg:(g + 1) * Kg] = Ug.reshape(co, u1, u2, Kg)
+            V[g * Kg:(g + 1) * Kg, g * ci:(g + 1) * ci] = Vg.reshape(Kg, ci, v1, v2)
+            S[g * Kg:(g + 1) * Kg] = np.asarray(Ss[g], dtype=np.float32)
+        return U.reshape(C_out * u1 * u2, G * Kg), S, V.reshape(G * Kg, C_in * v1 * v2)
 
     def forward(self, x, flags: int = 0):
         """x: CUDA tensor [n, H, W, C_in] (float32, bfloat16 or int8), contiguous.  Returns float32

@@ -94,3 +94,27 @@ def test_pointwise_form_is_the_linear_layer():
         assert err <= 1e-5 * y_lin.abs().max().item()
     finally:
         conv.close(); lin.close()
+
+
+@pytest.mark.parametrize("case", [(12, 1, 1, 7, 7, 5, 0, ((1, 1), (3, 3), (1, 1)), "f32"),      # depth-wise 7x7, rank 5 per channel
+                                  (4, 6, 3, 3, 3, 10, 2, ((2, 2), (1, 1), (1, 1)), "bf16"),
+                                  (3, 4, 8, 2, 3, 9, 1, ((1, 1), (1, 1), (1, 2)), "i8")],
+                         ids=["depthwise_7x7_rank5", "grouped_form2", "grouped_form1"])
+def test_grouped_and_depthwise_layers(case):
+    import torch
+    from paper_2308_07641_b200 import device_activations
+    from paper_2308_07641_b200.conv import TSVDConv2d
+    G, co, ci, K1, K2, K, form, (stride, pad, dil), x_dtype = case
+    layers = [_layer(300 + g, form, co, ci, K1, K2, K) for g in range(G)]
+    Us, Ss, Vs = [l[0] for l in layers], [l[1] for l in layers], [l[2] for l in layers]
+    x = _x(301, (2, 14, 11, G * ci), x_dtype)
+    conv = TSVDConv2d(Us, Ss, Vs, form, G * co, G * ci, K1, K2, stride, pad, dil)
+    try:
+        y = conv.forward(device_activations(x.reshape(-1, G * ci), x_dtype).view(2, 14, 11, G * ci)).double().cpu().numpy()
+        torch.cuda.synchronize()
+        assert conv.status() == 0
+    finally:
+        conv.close()
+    ref = oc.conv2d_tsvd_grouped(gen.widen_x(x, x_dtype), Us, Ss, Vs, form, G * co, G * ci, K1, K2, stride, pad, dil)
+    assert y.shape == ref.shape
+    assert np.abs(y - ref).max() <= 1e-5 * np.abs(ref).max()
