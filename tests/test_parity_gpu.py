@@ -174,6 +174,18 @@ def test_decode_cluster_form_long_contractions(B, x_dtype, base):
         _util.run_and_check(spec, flags=0x20)
 
 
+@pytest.mark.parametrize("B", [1, 2, 4, 7])
+@pytest.mark.parametrize("x_dtype,base", [("bf16", "cfg3_b4"), ("i8", "cfg5_d20")])
+def test_decode_contractions_longer_than_one_round(B, x_dtype, base):
+    """More than 4096 columns: a warp of the single-CTA kernel, and more than 4096 columns per quarter a
+    warp of the cluster form, comes back for further rounds of column groups (codes requested one round
+    ahead).  9000 columns = 142 groups (three rounds; quarters of 36, 36, 36, 34), 17000 columns per
+    quarter more than one round as well."""
+    for (M, N, K) in ((150, 9000, 140), (140, 17000, 130)):
+        spec = gen.scaled(C[base], name=f"rounds_{x_dtype}_B{B}_{N}", M=M, N=N, K=K, B=B, seed=120 + B, density=0.1)
+        _util.run_and_check(spec, flags=0x20)
+
+
 def test_decode_cluster_form_runs_back_to_back_and_is_deterministic():
     import torch
     from paper_2308_07641_b200 import TSVDLinear
