@@ -212,7 +212,7 @@ def sample_tokens(B):
     return sorted({0, 1, B // 2, B - 2, B - 1, 47, 48, 63, 64} & set(range(B)))
 
 
-def cpu_baseline(spec, U, S, V, x_np, target_s=10.0):
+def cpu_baseline(spec, U, S, V, x_np, target_s=15.0):
     """Time the CPU checker, as it stands, on a bounded sample of the workload's tokens."""
     import oracle
     cores = oracle.threads()
