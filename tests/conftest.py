@@ -13,7 +13,7 @@ def pytest_configure(config):
 
 
 def pytest_collection_modifyitems(config, items):
-    # GPU tests fail (not skip) on a GPU machine when the CUDA library is missing; on a
+    # GPU tests fail (not skip) on a machine with a GPU when the CUDA library is missing; on a
     # machine without a device they are skipped so that `-m "not gpu"` is not needed locally.
     try:
         import torch
