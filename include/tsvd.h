@@ -61,8 +61,10 @@ typedef enum {
     TSVD_E_TIMEOUT = 7, /* a bounded device-side wait gave up                      */
     TSVD_E_NOMEM = 8,   /* host or device allocation failed                        */
     TSVD_E_TOOBIG = 9,  /* request exceeds a fixed capacity (tsvd_forward_static, TSVD_MAX_CONTRACTION) */
-    TSVD_E_RANGE = 10   /* tsvd_last_status only: a token's dynamic range exceeded what the
+    TSVD_E_RANGE = 10,  /* tsvd_last_status only: a token's dynamic range exceeded what the
                            fixed-point digits resolve (see the note on arithmetic above)   */
+    TSVD_E_INTERNAL = 11 /* tsvd_last_status only, builds with -DTSVD_CHECK_BOUNDS: a kernel found
+                           one of its ring or tile indices outside its range              */
 } tsvd_status_t;
 
 /* Longest contraction (N and K) a handle may have: the digit sums of a row are combined in

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libtsvd.so")
 TSVD_F32, TSVD_BF16, TSVD_I8 = 0, 1, 2
 TSVD_OK = 0
 (TSVD_E_NULL, TSVD_E_SHAPE, TSVD_E_VALUE, TSVD_E_DTYPE, TSVD_E_ALIGN, TSVD_E_CUDA,
- TSVD_E_TIMEOUT, TSVD_E_NOMEM, TSVD_E_TOOBIG, TSVD_E_RANGE) = range(1, 11)
+ TSVD_E_TIMEOUT, TSVD_E_NOMEM, TSVD_E_TOOBIG, TSVD_E_RANGE, TSVD_E_INTERNAL) = range(1, 12)
 TSVD_MAX_CONTRACTION = 65280
 TSVD_STATIC_SCRATCH_BYTES = 4 << 20
 TSVD_FLAG_OUT_F32 = 0x1
@@ -47,6 +47,14 @@ class TSVDError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
         super().__init__(f"{what}: {tsvd_strerror(status)} (status {status})")
+
+
+def use_library(path: Optional[str]) -> None:
+    """Make the binding call the library at `path` (e.g. a checked build, see build.build_checked)
+    from now on; None goes back to the regular libtsvd.so.  Handles do not carry over."""
+    global _lib, LIB_PATH
+    LIB_PATH = path or os.path.join(_HERE, "libtsvd.so")
+    _lib = None
 
 
 def lib() -> ctypes.CDLL:

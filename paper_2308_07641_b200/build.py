@@ -43,5 +43,21 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_checked() -> str:
+    """A second library, libtsvd_checked.so, compiled with -DTSVD_CHECK_BOUNDS: the contraction kernel
+    checks its ring and tile indices and reports a violation through the status word
+    (tsvd_last_status: TSVD_E_INTERNAL).  For development and for the test that runs it."""
+    out = os.path.join(HERE, "libtsvd_checked.so")
+    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
+    if os.path.exists(out) and all(os.path.getmtime(d) <= os.path.getmtime(out) for d in deps):
+        return out
+    nvcc = os.environ.get("NVCC", "nvcc")
+    tmp = out + f".{os.getpid()}.tmp"
+    subprocess.check_call([nvcc] + NVCC_FLAGS + ["-DTSVD_CHECK_BOUNDS", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+                                                 "-o", tmp] + sources() + ["-lcudart"])
+    os.replace(tmp, out)
+    return out
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

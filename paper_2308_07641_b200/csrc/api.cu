@@ -24,6 +24,7 @@ extern "C" const char* tsvd_strerror(tsvd_status_t s)
         case TSVD_E_NOMEM: return "out of memory";
         case TSVD_E_TOOBIG: return "request exceeds a fixed capacity (static scratch, contraction length or index width)";
         case TSVD_E_RANGE: return "a token's dynamic range exceeded what the fixed-point digits resolve";
+        case TSVD_E_INTERNAL: return "a checked build found an index outside its range";
     }
     return "unknown status";
 }
@@ -254,6 +255,7 @@ extern "C" tsvd_status_t tsvd_last_status(tsvd_handle_t h)
     int word = 0;
     TSVD_CUDA_OK(cudaMemcpy(&word, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost));
     if (word) TSVD_CUDA_OK(cudaMemset(h->dev_status, 0, sizeof(int)));
+    if (word & TSVD_DEV_BOUNDS) return TSVD_E_INTERNAL;
     if (word & TSVD_DEV_TIMEOUT) return TSVD_E_TIMEOUT;
     return (word & TSVD_DEV_RANGE) ? TSVD_E_RANGE : TSVD_OK;
 }

@@ -435,6 +435,8 @@ ternary_mma_kernel(const GemmParams p)
                     const uint32_t bytes = (uint32_t)min(STEP_BLOCKS, tc.kb1 - kb) * blk_bytes;
                     if (!mbar_wait(&empty[slot * empty_stride], phase ^ 1, abort_flag)) { alive = false; break; }
                     if (is_b && p.test_stall) { alive = false; break; }   // nothing will ever land
+                    TSVD_BOUND(p.status, slot < depth && bytes <= slot_bytes && kb + (int)(bytes / blk_bytes) <= KB &&
+                                             tc.rt < p.row_tiles && tc.jt < p.j_tiles);
                     if (elect_one()) {
                         if (copy) {
                             mbar_arrive_expect_tx(&full[slot], bytes);
@@ -481,6 +483,7 @@ ternary_mma_kernel(const GemmParams p)
                     tc_fence_after_sync();
                     const uint32_t a_tmem = tmem_base + (uint32_t)A_COL0 + aslot * (uint32_t)A_SLOT_COLS;
                     const uint64_t b_desc = b_desc0 + (uint64_t)(slot * (B_SLOT_BYTES >> 4));
+                    TSVD_BOUND(p.status, slot < nb && aslot < (uint32_t)NA && nblk >= 1 && nblk <= STEP_BLOCKS);
                     const uint32_t cur = slot;
                     if (++slot == nb) { slot = 0; phase ^= 1; }
                     aslot = (aslot + 1) & (NA - 1);
@@ -524,6 +527,7 @@ ternary_mma_kernel(const GemmParams p)
                 if (it % EXP_GROUPS != group) continue;
                 const int nblk = min(STEP_BLOCKS, kb1 - kb);
                 const int sp = it % NP, sa = it % NA;
+                TSVD_BOUND(p.status, sb < nb && r < BLOCK_R && A_COL0 + sa * A_SLOT_COLS + STEP_BLOCKS * A_BLOCK_COLS <= TMEM_COLS);
                 if (!mbar_wait(&pfull_bar[sp], (it / NP) & 1, abort_flag)) { alive = false; break; }
                 const uint4* packed = reinterpret_cast<const uint4*>(p_tiles + sp * P_SLOT_BYTES);
                 const uint32_t a_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(A_COL0 + sa * A_SLOT_COLS);
@@ -576,6 +580,7 @@ ternary_mma_kernel(const GemmParams p)
             const TileCoord tc = tile_coord(p, tile);
             const int rt = tc.rt, jt = tc.jt;
             const int row = rt * BLOCK_R + row_in;
+            TSVD_BOUND(p.status, rt < p.row_tiles && jt < p.j_tiles && row < p.row_tiles * BLOCK_R);
             const uint32_t buf = local & 1;
             // this warp takes its share of the groups of 8 tokens
             constexpr int N_GROUPS = TOK / 8;

@@ -119,6 +119,16 @@ struct tsvd_handle_s {
 // bits of the device status word
 constexpr int TSVD_DEV_TIMEOUT = 1;   // a bounded wait gave up
 constexpr int TSVD_DEV_RANGE = 2;     // a token's dynamic range exceeded what the digits resolve
+constexpr int TSVD_DEV_BOUNDS = 4;    // checked builds (-DTSVD_CHECK_BOUNDS): a ring or tile index left its range
+
+// Index checks of the contraction kernel's rings and tiles, compiled in with -DTSVD_CHECK_BOUNDS: a
+// violated bound raises TSVD_DEV_BOUNDS in the device status word (and nothing else: the access still
+// happens, so a checked build is for finding a wrong index, not for surviving one).
+#ifdef TSVD_CHECK_BOUNDS
+#define TSVD_BOUND(status, cond) do { if (!(cond)) atomicOr((status), TSVD_DEV_BOUNDS); } while (0)
+#else
+#define TSVD_BOUND(status, cond) do { } while (0)
+#endif
 
 // Programmatic dependent launch: a kernel launched with this configuration may be set up, and
 // run up to its pdl_wait(), while the kernel before it in the stream is still running;

@@ -61,8 +61,8 @@ def test_constants_match_the_header(binding):
 
 
 def test_strerror_covers_all_codes(binding):
-    seen = {binding.tsvd_strerror(i) for i in range(0, 11)}
-    assert len(seen) == 11 and "unknown status" not in seen
+    seen = {binding.tsvd_strerror(i) for i in range(0, 12)}
+    assert len(seen) == 12 and "unknown status" not in seen
     assert binding.tsvd_strerror(99) == "unknown status"
 
 

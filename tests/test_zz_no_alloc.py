@@ -21,7 +21,7 @@ from tests import _util
 pytestmark = pytest.mark.gpu
 
 
-def _forward_pair(binding, h, x_np, x_dtype, M):
+def _forward_pair(binding, h, x_np, x_dtype, M, check_memory=True):
     import torch
     x = _util.torch_x(x_np, x_dtype)
     B = x.shape[0]
@@ -35,7 +35,8 @@ def _forward_pair(binding, h, x_np, x_dtype, M):
     binding.tsvd_forward_static(h, x.data_ptr(), y_sta.data_ptr(), B, dt)
     torch.cuda.synchronize()
     free_after, _ = torch.cuda.mem_get_info()
-    assert free_after == free_before, "tsvd_forward_static changed the device memory in use"
+    if check_memory:
+        assert free_after == free_before, "tsvd_forward_static changed the device memory in use"
     return y_ref.double().cpu().numpy(), y_sta.double().cpu().numpy()
 
 
@@ -48,7 +49,9 @@ def test_static_matches_forward_on_two_calls_in_a_row(x_dtype, base):
     x = gen.make_x(spec)
     h = binding.tsvd_pack(U, S, V)
     try:
-        _forward_pair(binding, h, x[:1], x_dtype, spec.M)      # first call on the device: address look-up
+        # first call in the process: the CUDA runtime loads the kernels and places the fixed array now
+        # (lazy module loading), so the memory in use is compared on the calls after it
+        _forward_pair(binding, h, x[:1], x_dtype, spec.M, check_memory=False)
         for xs in (x, x[5:24]):              # second call: other inputs, smaller batch
             y_ref, y_sta = _forward_pair(binding, h, xs, x_dtype, spec.M)
             err = np.abs(y_sta - y_ref)
