@@ -208,7 +208,7 @@ size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool
 int tsvd_tensor_digits_x(tsvd_dtype_t dt, bool wide_x);
 int tsvd_tensor_digits_t();
 
-// decode.cu -- one to four tokens, bound by streaming the packed codes
+// decode.cu -- one to sixteen tokens, bound by streaming the packed codes
 bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x);
 size_t tsvd_decode_ws_bytes(const tsvd_handle_s* h, int B);
 tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws);
