@@ -1,4 +1,5 @@
-// Decode path: y = U(diag(S)(V x)) for one to eight tokens, bound by streaming the packed codes.
+// Decode path: y = U(diag(S)(V x)) for one to sixteen tokens, bound by streaming the packed codes (a single-CTA
+// kernel per 32 rows, described first; from three tokens on a cluster form, described where it is defined).
 //
 // For so few tokens a 128-row tcgen05 tile is almost empty, and what matters is that every SM
 // streams its share of the 2-bit codes (the whole of U and V is read once per forward) with as
