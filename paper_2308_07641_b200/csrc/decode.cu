@@ -754,7 +754,9 @@ cudaError_t launch_gemv_tokens(const GemvParams& p, int R_pad, cudaStream_t stre
         if (p.B == 1) return launch_gemv_cluster<IN_T, ND, 1, STAGE>(p, R_pad, stream);
         if (p.B == 2) return launch_gemv_cluster<IN_T, ND, 2, STAGE>(p, R_pad, stream);
         if (p.B <= 4) return launch_gemv_cluster<IN_T, ND, 4, STAGE>(p, R_pad, stream);
+        if (p.B <= 6) return launch_gemv_cluster<IN_T, ND, 6, STAGE>(p, R_pad, stream);
         if (p.B <= 8) return launch_gemv_cluster<IN_T, ND, 8, STAGE>(p, R_pad, stream);
+        if (p.B <= 12) return launch_gemv_cluster<IN_T, ND, 12, STAGE>(p, R_pad, stream);
         return launch_gemv_cluster<IN_T, ND, 16, STAGE>(p, R_pad, stream);
     }
     if (p.B > 8) return cudaErrorInvalidValue;   // (tsvd_decode_fits keeps such requests away)
@@ -772,11 +774,12 @@ inline int digits_for_x(tsvd_dtype_t dt, bool wide) { return dt == TSVD_I8 ? 1 :
 bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x)
 {
     if (B < 1 || B > TSVD_DECODE_MAX_B) return false;
-    const int ntok = B <= 2 ? B : B <= 4 ? 4 : B <= 8 ? 8 : 16;
+    int ntok = B <= 2 ? B : B <= 4 ? 4 : B <= 8 ? 8 : B <= 12 ? 12 : 16;   // tokens of the instantiation that serves B
     // nine to sixteen tokens: the cluster form only
     if (B > 8 && !(use_cluster_form(h->V.C_pad, B) && use_cluster_form(h->U.C_pad, B))) return false;
     auto need = [&](int nd, int C_pad) {
-        return use_cluster_form(C_pad, B) ? gemv_cluster_smem_bytes(nd, ntok, C_pad) : gemv_smem_bytes(nd, ntok, C_pad);
+        if (!use_cluster_form(C_pad, B)) return gemv_smem_bytes(nd, ntok, C_pad);
+        return gemv_cluster_smem_bytes(nd, (B == 5 || B == 6) ? 6 : ntok, C_pad);   // (the cluster form also has six)
     };
     return need(digits_for_x(dt, wide_x), h->V.C_pad) <= (size_t)GEMV_MAX_SMEM && need(ND_T, h->U.C_pad) <= (size_t)GEMV_MAX_SMEM;
 }
