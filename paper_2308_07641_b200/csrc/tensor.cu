@@ -225,6 +225,142 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     tsvd_stamp_end(stamp);
 }
 
+// The same conversion for rows of at most 4096 padded values, 16-byte aligned and a multiple of 16
+// long, as a grid that stays resident: a block of 256 threads (a chunk of 16 values per thread) walks
+// over tokens blockIdx.x, blockIdx.x + gridDim.x, ... and holds the next token's chunk in registers,
+// still in the input type, while it reduces, converts and stores the current one, so that a token's
+// trip to memory is hidden behind the token before it.  Same digits, scales, cleared words and range
+// flag as digitise_kernel.
+template <typename IN_T>
+struct RawChunk16 { uint4 u[sizeof(IN_T)]; };   // 16 values of 1, 2 or 4 bytes
+
+template <typename IN_T>
+__device__ __forceinline__ void raw_zero(RawChunk16<IN_T>& r)
+{
+#pragma unroll
+    for (int i = 0; i < (int)sizeof(IN_T); ++i) r.u[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+template <typename IN_T>
+__device__ __forceinline__ void raw_load(const IN_T* __restrict__ p, RawChunk16<IN_T>& r)
+{
+    const uint4* p4 = reinterpret_cast<const uint4*>(p);
+#pragma unroll
+    for (int i = 0; i < (int)sizeof(IN_T); ++i) r.u[i] = __ldg(p4 + i);
+}
+template <typename IN_T>
+__device__ __forceinline__ void raw_unpack(const RawChunk16<IN_T>& r, float (&v)[16])
+{
+    if constexpr (sizeof(IN_T) == 4) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[4 * i] = __uint_as_float(r.u[i].x); v[4 * i + 1] = __uint_as_float(r.u[i].y);
+            v[4 * i + 2] = __uint_as_float(r.u[i].z); v[4 * i + 3] = __uint_as_float(r.u[i].w);
+        }
+    } else if constexpr (sizeof(IN_T) == 2) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t w[4] = {r.u[i].x, r.u[i].y, r.u[i].z, r.u[i].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {   // bf16 -> fp32 is a 16-bit shift
+                v[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+                v[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+            }
+        }
+    } else {
+        const uint32_t w[4] = {r.u[0].x, r.u[0].y, r.u[0].z, r.u[0].w};
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = (float)(int)(int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xFF);
+    }
+}
+
+template <typename IN_T, int ND, int TOK>
+__global__ void __launch_bounds__(256, 4)
+digitise_stream_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
+                       int8_t* __restrict__ D, float* __restrict__ scale_out, int* __restrict__ zero_buf,
+                       int zero_per_token, int zero_total, int* __restrict__ status,
+                       unsigned long long* __restrict__ stamp)
+{
+    constexpr int NT = ND * TOK;
+    constexpr bool kInt = sizeof(IN_T) == 1;
+    static_assert(TOK % 8 == 0, "digit rows of one token must share their swizzle term");
+    pdl_wait();                 // nothing is read or written before the kernel ahead has completed
+    pdl_launch_dependents();
+    tsvd_stamp_begin(stamp);
+    __shared__ float red[2][8];
+    const int ch = threadIdx.x;                   // this thread's chunk of every row
+    const bool has = ch < KB * (BLOCK_C / 16);    // ... lies in the padded row
+    const bool inside = ch * 16 < C;              // ... and holds values (C is a multiple of 16)
+    const int kb = ch >> 3, cc = ch & 7;          // contraction block, 16-byte chunk of its 128-byte row
+    const IN_T* col = in + ch * 16;
+    RawChunk16<IN_T> nxt;
+    raw_zero(nxt);
+    int b = blockIdx.x;
+    if (b < B && inside) raw_load(col + (size_t)b * ld_in, nxt);
+    for (int par = 0; b < B_pad; b += gridDim.x, par ^= 1) {
+        const RawChunk16<IN_T> cur = nxt;
+        const int bn = b + gridDim.x;
+        raw_zero(nxt);
+        if (bn < B && inside) raw_load(col + (size_t)bn * ld_in, nxt);
+
+        if (zero_buf)   // clear this token's slice of the accumulators a later kernel adds into
+            for (int i = threadIdx.x; i < zero_per_token; i += 256)
+                if ((size_t)b * zero_per_token + i < (size_t)zero_total) zero_buf[(size_t)b * zero_per_token + i] = 0;
+
+        const bool live = b < B;
+        float v[16];
+        raw_unpack(cur, v);     // zeros for a dead token and outside the row
+        float qscale = 1.f;
+        if constexpr (!kInt) {
+            float amax = 0.f;
+#pragma unroll
+            for (int e = 0; e < 16; ++e) amax = fmaxf(amax, fabsf(v[e]));
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            // the two halves of `red` alternate: a warp may write the next token's maximum while
+            // another still reads this one's, never the one after (the barrier between them)
+            if ((threadIdx.x & 31) == 0) red[par][threadIdx.x >> 5] = amax;
+            __syncthreads();
+#pragma unroll
+            for (int w = 0; w < 8; ++w) amax = fmaxf(amax, red[par][w]);
+            const int E = tsvd_quant_exponent(amax);
+            qscale = tsvd_pow2(8 * ND - 2 - E);
+            if (threadIdx.x == 0) scale_out[b] = tsvd_pow2(E - (8 * ND - 2));   // value = q * scale
+        } else {
+            if (threadIdx.x == 0) scale_out[b] = 1.f;
+        }
+
+        unsigned range_cnt = 0;
+        if (has) {
+            uint32_t dig[ND][4];
+#pragma unroll
+            for (int d = 0; d < ND; ++d)
+#pragma unroll
+                for (int w = 0; w < 4; ++w) dig[d][w] = 0;
+            if (live) {
+                int q[16];
+                if constexpr (!kInt) tsvd_range_sample(range_cnt, v[0], qscale);
+                if constexpr (ND <= 3) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) q[e] = tsvd_round_bits(v[e], qscale);
+                    digits_of<ND, 4>(q, dig, TSVD_ROUND_BIAS);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) q[e] = __float2int_rn(v[e] * qscale);
+                    digits_of<ND, 4>(q, dig);
+                }
+            }
+            const int jt = b / TOK, b_in = b % TOK;
+            int8_t* dst = D + ((size_t)jt * KB + kb) * (size_t)(NT * 128) + b_in * 128 + ((cc ^ (b_in & 7)) << 4);
+#pragma unroll
+            for (int d = 0; d < ND; ++d)
+                *reinterpret_cast<uint4*>(dst + d * (TOK * 128)) = make_uint4(dig[d][0], dig[d][1], dig[d][2], dig[d][3]);
+        }
+        if constexpr (!kInt) {
+            if (tsvd_range_flagged(range_cnt) && (threadIdx.x & 31) == 0) atomicOr(status, TSVD_DEV_RANGE);
+        }
+    }
+    tsvd_stamp_end(stamp);
+}
+
 // ---------------------------------------------------------------------------------------
 // The contraction kernel (persistent: one CTA per SM walks over the tiles).  Tile (rt, jt) is
 // the 128 x (ND*TOK) integer block
@@ -781,6 +917,19 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
 {
     const int B_pad = (B + TOK - 1) / TOK * TOK;
     const int zero_per_token = (zero_total + B_pad - 1) / B_pad;   // every token slot clears a share
+    // rows of 1024 to 4096 padded values that vector loads can read whole, without a maximum given:
+    // the resident form, as many blocks as the GPU holds at one time
+    if (!amax_bits && KB >= 8 && KB <= 32 && C % 16 == 0 &&
+        ((((uintptr_t)in) | ((size_t)ld_in * sizeof(IN_T))) & 15) == 0) {
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int resident = 4 * sms;
+        PdlLaunch cfg((unsigned)(B_pad < resident ? B_pad : resident), 256, 0, stream);
+        const cudaError_t e = cudaLaunchKernelEx(&cfg.cfg, digitise_stream_kernel<IN_T, ND, TOK>, in, ld_in, B, B_pad, C, KB, D,
+                                                 scale, zero_buf, zero_per_token, zero_total, status, stamp);
+        tsvd_count_launch();
+        return e != cudaSuccess ? e : cudaGetLastError();
+    }
     // one warp per token when that gives enough warps to fill the GPU, or for short rows
     PdlLaunch cfg((B_pad * 32 >= 148 * 1024 || KB < 8) ? (unsigned)((B_pad + 7) / 8) : (unsigned)B_pad, 256, 0, stream);
     cudaError_t e;
