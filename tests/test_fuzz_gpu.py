@@ -41,3 +41,26 @@ def _case(i):
 def test_random_case_default_path(i):
     spec, weights, bias = _case(i)
     _util.run_and_check(spec, weights=weights, bias=bias, expect_status=(0, 10))
+
+
+def _stream_case(i):
+    """Aligned rows of 1024 to 4096 values and batches around and beyond 4 x 148 token slots: the regime
+    of the digit conversion that keeps its blocks resident and walks them over the tokens."""
+    g = np.random.default_rng(9100 + i)
+    M = int(g.integers(1, 400))
+    N = 16 * int(g.integers(64, 257))
+    K = 16 * int(g.integers(64, 257)) if i % 2 == 0 else int(g.integers(1030, 4096))
+    B = (591, 592, 593, 640, 1183, 1185, 1300, 1777, 2049)[i % 9]
+    x_dtype = ("bf16", "f32", "i8")[i % 3]
+    base = {"bf16": "cfg2", "f32": "cfg1", "i8": "cfg5_d20"}[x_dtype]
+    spec = gen.scaled(gen.CONFIGS[base], name=f"stream{i}_{x_dtype}_{M}x{N}x{K}_B{B}", M=M, N=N, K=K, B=B,
+                      density=float(g.choice([0.05, 0.28, 0.6])), seed=9100 + i)
+    U, V, S = gen.make_weights(spec)
+    S = (S * g.choice([-1.0, 1.0], K)).astype(np.float32)
+    return spec, (U, V, S), (0x200 if x_dtype == "bf16" and i % 2 == 0 else 0)
+
+
+@pytest.mark.parametrize("i", range(12))
+def test_random_case_resident_digit_conversion(i):
+    spec, weights, flags = _stream_case(i)
+    _util.run_and_check(spec, weights=weights, flags=flags, expect_status=(0, 10))
