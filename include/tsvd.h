@@ -191,6 +191,24 @@ tsvd_status_t tsvd_im2col(const void* x, tsvd_dtype_t dtype, int n_img, int H, i
                           long long ld_out, void* stream);
 
 /*
+ * tsvd_forward_v_patches -- tsvd_im2col and tsvd_forward_v in one call, without the patch matrix: the
+ * stage's tokens are the patches of the image batch at x, read in place while they are converted for the
+ * tensor-core kernels (Section "TSVD in Convolution Layer": V(.) or U(.) as a convolution).  The result
+ * is, bit for bit, that of tsvd_forward_v on the output of tsvd_im2col.
+ *
+ *   x      device, n_img NHWC images of dtype `dtype`, 16-byte aligned; C a multiple of 16
+ *   geometry as tsvd_im2col; k1*k2*C must equal the handle's N; B = n_img*Ho*Wo tokens
+ *   t_out  device, float, row (n, ho, wo) at t_out + ((n*Ho + ho)*Wo + wo)*ldt (ldt >= K), 16-byte aligned
+ *   flags  TSVD_FLAG_WIDE_X; TSVD_FLAG_PATH_TENSOR to take the tensor-core kernels for 16 tokens and fewer
+ * Asynchronous on `stream`; same scratch rules as tsvd_forward.
+ * Errors: as tsvd_forward_v; E_SHAPE also when C is not a multiple of 16, when k1*k2*C != N, or when
+ * the batch would not run on the tensor-core kernels (use tsvd_im2col + tsvd_forward_v there).
+ */
+tsvd_status_t tsvd_forward_v_patches(tsvd_handle_t h, const void* x, tsvd_dtype_t dtype, int n_img, int H, int W, int C,
+                                     int k1, int k2, int stride_h, int stride_w, int pad_h, int pad_w, int dil_h,
+                                     int dil_w, float* t_out, int ldt, unsigned flags, void* stream);
+
+/*
  * tsvd_forward_host -- the same map with HOST buffers: copies x to the device, runs
  * tsvd_forward_ex, copies y (and z_out) back, and waits.  x, y, z_out are host pointers;
  * layout as tsvd_forward.  Batches of 768 tokens and more are cut into about eight chunks

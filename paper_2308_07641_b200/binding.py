@@ -37,7 +37,7 @@ DTYPES = {"f32": TSVD_F32, "bf16": TSVD_BF16, "i8": TSVD_I8}
 
 # every symbol include/tsvd.h declares
 EXPORTS = ("tsvd_pack", "tsvd_forward", "tsvd_forward_ex", "tsvd_forward_host", "tsvd_forward_static",
-           "tsvd_reserve", "tsvd_set_bias", "tsvd_ternarize", "tsvd_forward_v", "tsvd_im2col", "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_index_bytes", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
+           "tsvd_reserve", "tsvd_set_bias", "tsvd_ternarize", "tsvd_forward_v", "tsvd_forward_v_patches", "tsvd_im2col", "tsvd_last_status", "tsvd_plan", "tsvd_info", "tsvd_index_bytes", "tsvd_unpack", "tsvd_profile_enable", "tsvd_profile_read",
            "tsvd_launch_count", "tsvd_destroy", "tsvd_strerror")
 
 _lib: Optional[ctypes.CDLL] = None
@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.tsvd_ternarize.restype = ci
         L.tsvd_forward_v.argtypes = [vp, vp, ci, vp, ci, ci, ci, cu, vp]
         L.tsvd_forward_v.restype = ci
+        L.tsvd_forward_v_patches.argtypes = [vp, vp, ci] + [ci] * 12 + [vp, ci, cu, vp]
+        L.tsvd_forward_v_patches.restype = ci
         L.tsvd_im2col.argtypes = [vp, ci] + [ci] * 12 + [vp, ctypes.c_longlong, vp]
         L.tsvd_im2col.restype = ci
         L.tsvd_last_status.argtypes = [vp]
@@ -185,6 +187,13 @@ def tsvd_forward_v(h: int, x_ptr: int, ldx: int, t_ptr: int, ldt: int, B: int, d
                    stream: int = 0) -> None:
     """t = diag(S)(V x) only (fp32 [B][K]); raw device pointers."""
     _check(lib().tsvd_forward_v(h, x_ptr, ldx, t_ptr, ldt, B, dtype, flags, stream or None), "tsvd_forward_v")
+
+
+def tsvd_forward_v_patches(h: int, x_ptr: int, dtype: int, n_img: int, H: int, W: int, C: int, k1: int, k2: int, stride,
+                           pad, dil, t_ptr: int, ldt: int, flags: int = 0, stream: int = 0) -> None:
+    """t = diag(S)(V patches) with the patches of an NHWC image batch read in place; raw device pointers."""
+    _check(lib().tsvd_forward_v_patches(h, x_ptr, dtype, n_img, H, W, C, k1, k2, stride[0], stride[1], pad[0], pad[1],
+                                        dil[0], dil[1], t_ptr, ldt, flags, stream or None), "tsvd_forward_v_patches")
 
 
 def tsvd_im2col(x_ptr: int, dtype: int, n_img: int, H: int, W: int, C: int, k1: int, k2: int, stride, pad, dil,

@@ -1,7 +1,9 @@
 """The convolution forms of a TSVD layer (Section "TSVD in Convolution Layer" of the paper) on the
-current CUDA device, composed from the library's calls: `tsvd_im2col` gathers the patches of a
-stage's input, `tsvd_forward_v` applies that stage's ternary matrix (and, for V(.), the channel-wise
-scale diag(s)(.)).  Marshalling and index bookkeeping only; the arithmetic runs in the library.
+current CUDA device, composed from the library's calls: `tsvd_forward_v` applies a stage's ternary
+matrix (and, for V(.), the channel-wise scale diag(s)(.)) to the patches of the stage's input, which
+`tsvd_forward_v_patches` reads in place (channels a multiple of 16, tensor-core kernels) and
+`tsvd_im2col` gathers into a patch matrix otherwise.  Marshalling and index bookkeeping only; the
+arithmetic runs in the library.
 
 The kernel W [C_out, C_in, K1, K2] is decomposed as one of the four matrices of Eq. 5:
 
@@ -102,26 +104,37 @@ class TSVDConv2d:
         stream = torch.cuda.current_stream(x.device).cuda_stream
         (v1, v2), (u1, u2) = self.kv, self.ku
         Hv, Wv = _out(H, v1, self.sv[0], self.pv[0], self.dv[0]), _out(W, v2, self.sv[1], self.pv[1], self.dv[1])
-        if (v1, v2) == (1, 1) and self.sv == (1, 1) and self.pv == (0, 0):
-            cols = x.view(n * H * W, self.C_in)                 # a [1,1] stage reads the pixels as they are
-        else:
-            cols = torch.empty((n * Hv * Wv, v1 * v2 * self.C_in), dtype=x.dtype, device=x.device)
-            binding.tsvd_im2col(x.data_ptr(), dt, n, H, W, self.C_in, v1, v2, self.sv, self.pv, self.dv,
-                                cols.data_ptr(), cols.stride(0), stream)
         t = torch.empty((n * Hv * Wv, self.K), dtype=torch.float32, device=x.device)
-        binding.tsvd_forward_v(self.h_v, cols.data_ptr(), cols.stride(0), t.data_ptr(), t.stride(0), cols.shape[0], dt,
-                               flags, stream)
+        self._stage(self.h_v, x, dt, n, H, W, self.C_in, (v1, v2), self.sv, self.pv, self.dv, t, flags, stream)
         Ho, Wo = _out(Hv, u1, self.su[0], self.pu[0], self.du[0]), _out(Wv, u2, self.su[1], self.pu[1], self.du[1])
-        if (u1, u2) == (1, 1) and self.su == (1, 1) and self.pu == (0, 0):
-            cols_u = t
-        else:
-            cols_u = torch.empty((n * Ho * Wo, u1 * u2 * self.K), dtype=torch.float32, device=x.device)
-            binding.tsvd_im2col(t.data_ptr(), binding.TSVD_F32, n, Hv, Wv, self.K, u1, u2, self.su, self.pu, self.du,
-                                cols_u.data_ptr(), cols_u.stride(0), stream)
         y = torch.empty((n * Ho * Wo, self.C_out), dtype=torch.float32, device=x.device)
-        binding.tsvd_forward_v(self.h_u, cols_u.data_ptr(), cols_u.stride(0), y.data_ptr(), y.stride(0), cols_u.shape[0],
-                               binding.TSVD_F32, flags, stream)
+        self._stage(self.h_u, t, binding.TSVD_F32, n, Hv, Wv, self.K, (u1, u2), self.su, self.pu, self.du, y, flags, stream)
         return y.view(n, Ho, Wo, self.C_out)
+
+    @staticmethod
+    def _stage(handle, img, dt, n, H, W, C, kernel, stride, pad, dil, out, flags, stream):
+        """One ternary stage as a convolution over `img` (NHWC, C channels) into `out` [pixels, rank].  A
+        [1,1] stage without stride or padding reads the pixels as they are; otherwise the patches are read in
+        place when the library can do that (tensor-core kernels, channels a multiple of 16), else gathered
+        into a patch matrix first."""
+        import torch
+        k1, k2 = kernel
+        B = out.shape[0]
+        if kernel == (1, 1) and stride == (1, 1) and pad == (0, 0):
+            binding.tsvd_forward_v(handle, img.data_ptr(), C, out.data_ptr(), out.stride(0), B, dt, flags, stream)
+            return
+        forced = flags & (binding.TSVD_FLAG_PATH_SIMPLE | binding.TSVD_FLAG_PATH_DECODE)
+        if C % 16 == 0 and not forced and (B > binding.TSVD_DECODE_MAX_B or flags & binding.TSVD_FLAG_PATH_TENSOR):
+            try:
+                binding.tsvd_forward_v_patches(handle, img.data_ptr(), dt, n, H, W, C, k1, k2, stride, pad, dil,
+                                               out.data_ptr(), out.stride(0), flags, stream)
+                return
+            except binding.TSVDError as e:
+                if e.status != binding.TSVD_E_SHAPE:      # "not in place for this call": gather first
+                    raise
+        cols = torch.empty((B, k1 * k2 * C), dtype=img.dtype, device=img.device)
+        binding.tsvd_im2col(img.data_ptr(), dt, n, H, W, C, k1, k2, stride, pad, dil, cols.data_ptr(), cols.stride(0), stream)
+        binding.tsvd_forward_v(handle, cols.data_ptr(), cols.stride(0), out.data_ptr(), out.stride(0), B, dt, flags, stream)
 
     __call__ = forward
 

@@ -335,7 +335,8 @@ extern "C" tsvd_status_t tsvd_plan(tsvd_handle_t h, int B, tsvd_dtype_t dtype, u
 }
 
 static tsvd_status_t forward_impl(tsvd_handle_t h, const void* x, int ldx, void* y, int ldy, int B, tsvd_dtype_t dtype,
-                                  unsigned flags, void* z_out, void* stream, bool v_only, float** t_where)
+                                  unsigned flags, void* z_out, void* stream, bool v_only, float** t_where,
+                                  const PatchGather* gather = nullptr)
 {
     if (!h || !x || !y) return TSVD_E_NULL;
     if (B < 1) return TSVD_E_SHAPE;
@@ -360,11 +361,13 @@ static tsvd_status_t forward_impl(tsvd_handle_t h, const void* x, int ldx, void*
     a.wide_x = (flags & TSVD_FLAG_WIDE_X) != 0;
     a.v_only = v_only;
     a.t_where = t_where;
+    a.gather = gather;
     if (v_only && path == TSVD_FLAG_PATH_INDEX) return TSVD_E_DTYPE;   // the index-list kernels run whole forwards only
     a.stream = (cudaStream_t)stream;
 
     const unsigned chosen = choose_path(h, B, dtype, path, a.wide_x);
     if (chosen == 0u) return TSVD_E_TOOBIG;
+    if (gather && chosen != TSVD_FLAG_PATH_TENSOR) return TSVD_E_SHAPE;   // only those kernels read patches in place
     if (chosen == TSVD_FLAG_PATH_TENSOR) {
         tsvd_status_t st = ensure_ws(h, tsvd_tensor_ws_bytes(h, B, dtype, a.wide_x));
         if (st != TSVD_OK) return st;
@@ -401,6 +404,29 @@ extern "C" tsvd_status_t tsvd_forward_v(tsvd_handle_t h, const void* x, int ldx,
     const tsvd_status_t st = forward_impl(h, x, ldx, t_out, ldt, B, dtype, flags, nullptr, stream, true, &t);
     if (st != TSVD_OK) return st;
     // the stage wrote all padded rows into the handle's scratch: the K real ones go to the caller
+    TSVD_CUDA_OK(cudaMemcpy2DAsync(t_out, (size_t)ldt * sizeof(float), t, (size_t)h->V.R_pad * sizeof(float),
+                                   (size_t)h->K * sizeof(float), (size_t)B, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return TSVD_OK;
+}
+
+extern "C" tsvd_status_t tsvd_forward_v_patches(tsvd_handle_t h, const void* x, tsvd_dtype_t dtype, int n_img, int H, int W,
+                                                int C, int k1, int k2, int stride_h, int stride_w, int pad_h, int pad_w,
+                                                int dil_h, int dil_w, float* t_out, int ldt, unsigned flags, void* stream)
+{
+    if (!h || !x || !t_out) return TSVD_E_NULL;
+    if (n_img < 1 || H < 1 || W < 1 || C < 1 || k1 < 1 || k2 < 1 || stride_h < 1 || stride_w < 1 || pad_h < 0 || pad_w < 0 ||
+        dil_h < 1 || dil_w < 1)
+        return TSVD_E_SHAPE;
+    const int Ho = (H + 2 * pad_h - dil_h * (k1 - 1) - 1) / stride_h + 1;
+    const int Wo = (W + 2 * pad_w - dil_w * (k2 - 1) - 1) / stride_w + 1;
+    const long long feat = (long long)k1 * k2 * C, B = (long long)n_img * Ho * Wo;
+    if (Ho < 1 || Wo < 1 || feat != h->N || B > 0x7fffffffLL || C % 16 != 0) return TSVD_E_SHAPE;
+    PatchGather g;
+    g.H = H; g.W = W; g.C = C; g.k2 = k2; g.sh = stride_h; g.sw = stride_w; g.ph = pad_h; g.pw = pad_w;
+    g.dh = dil_h; g.dw = dil_w; g.Ho = Ho; g.Wo = Wo; g.feat = (int)feat;
+    float* t = nullptr;
+    const tsvd_status_t st = forward_impl(h, x, h->N, t_out, ldt, (int)B, dtype, flags, nullptr, stream, true, &t, &g);
+    if (st != TSVD_OK) return st;
     TSVD_CUDA_OK(cudaMemcpy2DAsync(t_out, (size_t)ldt * sizeof(float), t, (size_t)h->V.R_pad * sizeof(float),
                                    (size_t)h->K * sizeof(float), (size_t)B, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
     return TSVD_OK;

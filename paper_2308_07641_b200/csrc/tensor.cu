@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(256, 4)   // <= 64 registers: a batch of 4096 
 digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                 const unsigned* __restrict__ amax_bits, int8_t* __restrict__ D, float* __restrict__ scale_out,
                 int* __restrict__ zero_buf, int zero_per_token, int zero_total, int* __restrict__ status,
-                unsigned long long* __restrict__ stamp)
+                unsigned long long* __restrict__ stamp, const PatchGather pg)
 {
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
@@ -106,7 +106,25 @@ digitise_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C,
     const IN_T* row = in + (size_t)b * ld_in;
     const bool vec_ok = ((((uintptr_t)in) | ((size_t)ld_in * sizeof(IN_T))) & 15) == 0;
     const int n_chunks = KB * PER_BLOCK;
+    // tokens that are image patches: (image, output row, output column) of this token
+    int pg_n = 0, pg_ho = 0, pg_wo = 0;
+    if (pg.C) {
+        pg_wo = b % pg.Wo;
+        pg_ho = (b / pg.Wo) % pg.Ho;
+        pg_n = b / (pg.Wo * pg.Ho);
+    }
     auto load_chunk = [&](int ch, float (&v)[CH]) {
+        if (pg.C) {   // a chunk lies inside one run of channels (or past the row's end, or outside the image: zeros)
+            const IN_T* p = ch * CH < pg.feat ? tsvd_patch_ptr<IN_T>(pg, in, pg_n, pg_ho, pg_wo, ch * CH) : nullptr;
+            if (p) {
+                if constexpr (CH == 16) load16<IN_T>(p, 0, CH, true, v);
+                else load8<IN_T>(p, 0, CH, true, v);
+            } else {
+#pragma unroll
+                for (int e = 0; e < CH; ++e) v[e] = 0.f;
+            }
+            return;
+        }
         if constexpr (CH == 16) load16<IN_T>(row, ch * CH, C, vec_ok, v);
         else load8<IN_T>(row, ch * CH, C, vec_ok, v);
     };
@@ -278,7 +296,7 @@ __global__ void __launch_bounds__(256, 4)
 digitise_stream_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad, int C, int KB,
                        int8_t* __restrict__ D, float* __restrict__ scale_out, int* __restrict__ zero_buf,
                        int zero_per_token, int zero_total, int* __restrict__ status,
-                       unsigned long long* __restrict__ stamp)
+                       unsigned long long* __restrict__ stamp, const PatchGather pg)
 {
     constexpr int NT = ND * TOK;
     constexpr bool kInt = sizeof(IN_T) == 1;
@@ -292,15 +310,22 @@ digitise_stream_kernel(const IN_T* __restrict__ in, int ld_in, int B, int B_pad,
     const bool inside = ch * 16 < C;              // ... and holds values (C is a multiple of 16)
     const int kb = ch >> 3, cc = ch & 7;          // contraction block, 16-byte chunk of its 128-byte row
     const IN_T* col = in + ch * 16;
+    // where this thread's chunk of token t lies (null: nothing to load): a row of a matrix, or a run of
+    // channels of an image patch
+    auto chunk_of = [&](int t) -> const IN_T* {
+        if (t >= B || !inside) return nullptr;
+        if (pg.C) return tsvd_patch_ptr<IN_T>(pg, in, t / (pg.Wo * pg.Ho), (t / pg.Wo) % pg.Ho, t % pg.Wo, ch * 16);
+        return col + (size_t)t * ld_in;
+    };
     RawChunk16<IN_T> nxt;
     raw_zero(nxt);
     int b = blockIdx.x;
-    if (b < B && inside) raw_load(col + (size_t)b * ld_in, nxt);
+    if (const IN_T* p0 = chunk_of(b)) raw_load(p0, nxt);
     for (int par = 0; b < B_pad; b += gridDim.x, par ^= 1) {
         const RawChunk16<IN_T> cur = nxt;
         const int bn = b + gridDim.x;
         raw_zero(nxt);
-        if (bn < B && inside) raw_load(col + (size_t)bn * ld_in, nxt);
+        if (const IN_T* pn = chunk_of(bn)) raw_load(pn, nxt);
 
         if (zero_buf)   // clear this token's slice of the accumulators a later kernel adds into
             for (int i = threadIdx.x; i < zero_per_token; i += 256)
@@ -913,8 +938,9 @@ ternary_mma_kernel(const GemmParams p)
 template <typename IN_T, int ND, int TOK = tokens_per_tile(ND)>
 cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, const unsigned* amax_bits,
                             int8_t* D, float* scale, int* zero_buf, int zero_total, int* status,
-                            unsigned long long* stamp, cudaStream_t stream)
+                            unsigned long long* stamp, cudaStream_t stream, const PatchGather* gather = nullptr)
 {
+    const PatchGather pg = gather ? *gather : PatchGather();
     const int B_pad = (B + TOK - 1) / TOK * TOK;
     const int zero_per_token = (zero_total + B_pad - 1) / B_pad;   // every token slot clears a share
     // rows of 1024 to 4096 padded values that vector loads can read whole, without a maximum given:
@@ -922,13 +948,13 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
     // half of a block's threads without a chunk: there a batch large enough for the warp-per-token
     // form below keeps that form, which measured 4% faster on a convolution's 25088 patches of 1152)
     if (!amax_bits && KB >= 8 && KB <= 32 && (KB >= 16 || B_pad * 32 < 148 * 1024) && C % 16 == 0 &&
-        ((((uintptr_t)in) | ((size_t)ld_in * sizeof(IN_T))) & 15) == 0) {
+        ((((uintptr_t)in) | ((size_t)(gather ? 16 : ld_in) * sizeof(IN_T))) & 15) == 0) {
         int dev = 0, sms = 148;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         const int resident = 4 * sms;
         PdlLaunch cfg((unsigned)(B_pad < resident ? B_pad : resident), 256, 0, stream);
         const cudaError_t e = cudaLaunchKernelEx(&cfg.cfg, digitise_stream_kernel<IN_T, ND, TOK>, in, ld_in, B, B_pad, C, KB, D,
-                                                 scale, zero_buf, zero_per_token, zero_total, status, stamp);
+                                                 scale, zero_buf, zero_per_token, zero_total, status, stamp, pg);
         tsvd_count_launch();
         return e != cudaSuccess ? e : cudaGetLastError();
     }
@@ -940,13 +966,13 @@ cudaError_t launch_digitise(const IN_T* in, int ld_in, int B, int C, int KB, con
         // round and the row still fits the registers (three chunks of 8 per lane)
         if ((KB * 8) % 32 != 0 && KB * 16 <= 3 * 32)
             e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK, 8>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                                   scale, zero_buf, zero_per_token, zero_total, status, stamp);
+                                   scale, zero_buf, zero_per_token, zero_total, status, stamp, pg);
         else
             e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 32, TOK, 16>, in, ld_in, B, B_pad, C, KB, amax_bits,
-                                   D, scale, zero_buf, zero_per_token, zero_total, status, stamp);
+                                   D, scale, zero_buf, zero_per_token, zero_total, status, stamp, pg);
     } else {
         e = cudaLaunchKernelEx(&cfg.cfg, digitise_kernel<IN_T, ND, 256, TOK, 16>, in, ld_in, B, B_pad, C, KB, amax_bits, D,
-                               scale, zero_buf, zero_per_token, zero_total, status, stamp);
+                               scale, zero_buf, zero_per_token, zero_total, status, stamp, pg);
     }
     tsvd_count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
@@ -1107,7 +1133,7 @@ tsvd_status_t forward_small(const ForwardArgs& a, const SmallWs& w)
 
     h->prof.begin(0, st);
     e = launch_digitise<IN_T, NDX, SMALL_TOK>((const IN_T*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                              w.zacc, w.zacc_ints, h->dev_status, h->prof.slot(0), st);
+                                              w.zacc, w.zacc_ints, h->dev_status, h->prof.slot(0), st, a.gather);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
@@ -1184,19 +1210,19 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     switch (a.dtype) {
         case TSVD_F32:
             e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, nullptr, 0,
-                                          h->dev_status, stamp0, st);
+                                          h->dev_status, stamp0, st, a.gather);
             break;
         case TSVD_BF16:
             if (wide_bf16)
                 e = launch_digitise<__nv_bfloat16, 4>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
-                                                      w.scale_x, nullptr, 0, h->dev_status, stamp0, st);
+                                                      w.scale_x, nullptr, 0, h->dev_status, stamp0, st, a.gather);
             else
                 e = launch_digitise<__nv_bfloat16, 3>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
-                                                      w.scale_x, nullptr, 0, h->dev_status, stamp0, st);
+                                                      w.scale_x, nullptr, 0, h->dev_status, stamp0, st, a.gather);
             break;
         case TSVD_I8:
             e = launch_digitise<int8_t, 1>((const int8_t*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
-                                           nullptr, 0, h->dev_status, stamp0, st);
+                                           nullptr, 0, h->dev_status, stamp0, st, a.gather);
             break;
         default:
             return TSVD_E_DTYPE;

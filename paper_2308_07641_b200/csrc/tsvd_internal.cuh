@@ -181,6 +181,26 @@ tsvd_status_t tsvd_pack_matrix(const int8_t* host, int R, int C, PackedMat* out,
 tsvd_status_t tsvd_unpack_matrix(const PackedMat& pm, int8_t* host);
 
 // simple.cu -- CUDA-core reference kernels
+// A stage input given as the patches of an NHWC image batch instead of a matrix: token b = (n, ho, wo)
+// reads, for kernel position (a, b2), the C channels of pixel (ho*sh + a*dh - ph, wo*sw + b2*dw - pw) of
+// image n (zeros outside the image); its row is the k1*k2 runs of C values in the order (a, b2, channel).
+// C = 0: off.  C is a multiple of 16, so that a 16-value chunk never straddles two runs.
+struct PatchGather {
+    int H = 0, W = 0, C = 0, k2 = 0, sh = 0, sw = 0, ph = 0, pw = 0, dh = 0, dw = 0, Ho = 0, Wo = 0, feat = 0;
+};
+#ifdef __CUDACC__
+// Where the values feat0 .. (a chunk inside one run) of token (n, ho, wo) lie; null outside the image.
+template <typename T>
+__device__ __forceinline__ const T* tsvd_patch_ptr(const PatchGather& g, const T* img, int n, int ho, int wo, int feat0)
+{
+    const int ab = feat0 / g.C, c0 = feat0 - ab * g.C;
+    const int a = ab / g.k2, b2 = ab - a * g.k2;
+    const int h = ho * g.sh + a * g.dh - g.ph, w = wo * g.sw + b2 * g.dw - g.pw;
+    if (h < 0 || h >= g.H || w < 0 || w >= g.W) return nullptr;
+    return img + (((long long)n * g.H + h) * g.W + w) * g.C + c0;
+}
+#endif
+
 struct ForwardArgs {
     tsvd_handle_s* h;
     const void* x;
@@ -195,6 +215,7 @@ struct ForwardArgs {
     bool wide_x = false;       // TSVD_FLAG_WIDE_X: bf16 activations as four digits
     bool v_only = false;       // stop after the V-stage and its scale (tsvd_forward_v)
     float** t_where = nullptr; // v_only: receives where t = S*(V x) was written, [B][R_pad of V] fp32
+    const PatchGather* gather = nullptr;   // the tokens are patches of the image batch at x (tensor-core path only)
     float* t;        // scratch [B][t_ld] fp32: S * (V x)
     int t_ld;
     cudaStream_t stream;

@@ -90,6 +90,7 @@ def test_host_side_validation(binding):
     assert lib.tsvd_ternarize(one, 1, binding.TSVD_TERNARIZE_MAX_LEN + 1, 1 << 20, 0.5, one, 1 << 20, None, None) == binding.TSVD_E_TOOBIG
     assert lib.tsvd_set_bias(None, None) == binding.TSVD_E_NULL
     assert lib.tsvd_forward_v(None, one, 4, one, 4, 1, 0, 0, None) == binding.TSVD_E_NULL
+    assert lib.tsvd_forward_v_patches(None, one, 0, 1, 4, 4, 16, 1, 1, 1, 1, 0, 0, 1, 1, one, 4, 0, None) == binding.TSVD_E_NULL
     assert lib.tsvd_im2col(None, 0, 1, 4, 4, 1, 1, 1, 1, 1, 0, 0, 1, 1, one, 1, None) == binding.TSVD_E_NULL
     assert lib.tsvd_im2col(one, 0, 1, 2, 2, 1, 3, 3, 1, 1, 0, 0, 1, 1, one, 9, None) == binding.TSVD_E_SHAPE   # kernel larger than the image
     assert lib.tsvd_im2col(one, 0, 1, 4, 4, 2, 3, 3, 1, 1, 0, 0, 1, 1, one, 17, None) == binding.TSVD_E_SHAPE  # ld_out < k1*k2*C
