@@ -476,7 +476,18 @@ ternary_mma_kernel(const GemmParams p)
 {
     constexpr int EPI_SHARES = EPI_WARPS / 4;
     constexpr int NT = ND * TOK;
-    static_assert(NT % 16 == 0 && NT <= NT_MAX && TOK % 16 == 0, "tile shape");
+    // Tiles of up to 192 columns have two accumulator buffers, so that a tile is drained while the next
+    // is contracted.  WIDE: one buffer of 256 columns, for launches in which no CTA has a second tile
+    // anyway; the digit ring then holds three steps of 64 KiB in the same 192 KiB.
+    constexpr bool WIDE = NT > NT_MAX;
+    static_assert(NT % 16 == 0 && NT <= 256 && TOK % 16 == 0, "tile shape");
+    static_assert(!WIDE || EPI != EPI_ACC, "wide tiles: whole contractions only");
+    constexpr uint32_t N_ACC = WIDE ? 1 : 2;
+    constexpr uint32_t ACC_COLS = WIDE ? 256 : NT_MAX;
+    constexpr uint32_t A_COL0 = N_ACC * ACC_COLS;
+    constexpr uint32_t B_SLOT_BYTES = STEP_BLOCKS * (WIDE ? 256 : NT_MAX) * BLOCK_C;
+    static_assert(A_COL0 + NA * A_SLOT_COLS <= TMEM_COLS, "tensor memory budget");
+    static_assert((WIDE ? 3 : NB) * B_SLOT_BYTES <= NB * ::B_SLOT_BYTES, "digit ring inside its share of shared memory");
     constexpr uint32_t B_TILE_BYTES = NT * BLOCK_C;
     constexpr uint32_t IDESC = umma_idesc_s8(BLOCK_R, NT);
 
@@ -503,7 +514,7 @@ ternary_mma_kernel(const GemmParams p)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* b_tiles = smem;                                 // NB x 48 KiB, 1024-aligned
-    uint8_t* p_tiles = b_tiles + NB * B_SLOT_BYTES;          // NP x 8 KiB
+    uint8_t* p_tiles = b_tiles + NB * ::B_SLOT_BYTES;        // NP x 8 KiB
     uint64_t* bars = reinterpret_cast<uint64_t*>(p_tiles + NP * P_SLOT_BYTES);
     uint64_t* pfull_bar = bars;                      // [NP] packed codes landed
     uint64_t* pempty_bar = pfull_bar + NP;           // [NP] expanders have read them
@@ -632,8 +643,8 @@ ternary_mma_kernel(const GemmParams p)
             bool ready = mbar_test_wait(&ready_bar[0], 0);
             bool alive = true;
             for (int L = 0, tile = tile_first; L < tile_count && alive; ++L, tile += tile_step) {
-                const uint32_t buf = (uint32_t)L & 1u;
-                if (!mbar_wait(&accempty_bar[buf], (((uint32_t)L >> 1) & 1) ^ 1, abort_flag)) break;
+                const uint32_t buf = (uint32_t)L % N_ACC;
+                if (!mbar_wait(&accempty_bar[buf], (((uint32_t)L / N_ACC) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)ACC_COLS;
                 int kb0, kb1;
@@ -742,7 +753,7 @@ ternary_mma_kernel(const GemmParams p)
             const int rt = tc.rt, jt = tc.jt;
             const int row = rt * BLOCK_R + row_in;
             TSVD_BOUND(p.status, rt < p.row_tiles && jt < p.j_tiles && row < p.row_tiles * BLOCK_R);
-            const uint32_t buf = local & 1;
+            const uint32_t buf = local % N_ACC;
             // this warp takes its share of the groups of 8 tokens
             constexpr int N_GROUPS = TOK / 8;
             constexpr int MY_GROUPS = N_GROUPS / EPI_SHARES;
@@ -751,7 +762,7 @@ ternary_mma_kernel(const GemmParams p)
             if constexpr (EPI == EPI_V) s_row = p.S[row];
             if constexpr (EPI == EPI_U_F32 || EPI == EPI_U_BF16) s_row = p.bias ? __ldg(p.bias + row) : 0.f;
             const bool row_ok = row < p.R;
-            if (!mbar_wait(&accfull_bar[buf], (local >> 1) & 1, abort_flag)) break;
+            if (!mbar_wait(&accfull_bar[buf], (local / N_ACC) & 1, abort_flag)) break;
             tc_fence_after_sync();
             const uint32_t t_lane = tmem_base + buf * (uint32_t)ACC_COLS + ((uint32_t)(lane_grp * 32) << 16);
 #pragma unroll
@@ -1000,7 +1011,9 @@ cudaError_t launch_gemm_w(const GemmParams& p, int row_tiles, cudaStream_t strea
     q.nb = NB;
     q.resident = 0;
     const int steps = (q.KB + STEP_BLOCKS - 1) / STEP_BLOCKS;
-    if (q.ksplit == 1 && steps <= NB) {
+    if (ND * TOK > NT_MAX) {
+        q.nb = 3;   // tiles of 256 columns: three steps of 64 KiB fill the digit ring
+    } else if (q.ksplit == 1 && steps <= NB) {
         q.nb = steps * (NB / steps);
         q.resident = 1;
     }
@@ -1035,6 +1048,25 @@ constexpr int ND_T = 4;
 // take tiles of 128 tokens where that leaves fewer padded tokens, e.g. 256 tokens as 2 x 128 instead of
 // 192 + 64 (V-stage of a 8192 x 4096 matrix at 256 tokens: 14.1 -> 12.0 us).
 constexpr int TOK_I8_NARROW = 128;
+// Tokens per tile of the U-stage: 48 (four digits, 192 columns, two accumulator buffers), or 64 (256
+// columns, one buffer) when that brings the number of tiles down to at most one per SM, where nothing
+// would overlap with a second buffer anyway (4096 rows x 256 tokens: 32 x 6 = 192 tiles in two rounds
+// against 32 x 4 = 128 in one).
+constexpr int TOK_T_WIDE = 64;
+inline int tokens_of_t_tile(const tsvd_handle_s* h, int B)
+{
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0, n = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        sms = n;
+    }
+    const int rows = h->U.R_pad / BLOCK_R;
+    const int regular = tokens_per_tile(ND_T);
+    const long long tiles_regular = (long long)rows * ((B + regular - 1) / regular);
+    const long long tiles_wide = (long long)rows * ((B + TOK_T_WIDE - 1) / TOK_T_WIDE);
+    return tiles_regular > sms && tiles_wide <= sms ? TOK_T_WIDE : regular;
+}
 inline int tokens_of_x_tile(int ndx, int B)
 {
     const int wide_tile = tokens_per_tile(ndx);
@@ -1052,7 +1084,7 @@ struct TensorWs {
 TensorWs carve(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide, void* base)
 {
     const int ndx = digits_for_x(dt, wide);
-    const int tokx = tokens_of_x_tile(ndx, B), tokt = tokens_per_tile(ND_T);
+    const int tokx = tokens_of_x_tile(ndx, B), tokt = tokens_of_t_tile(h, B);
     const size_t Bx = align_up(B, tokx), Bt = align_up(B, tokt);
     const size_t Bmax = Bx > Bt ? Bx : Bt;
     const size_t KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
@@ -1266,8 +1298,13 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
 
     // stage 2: t -> digits (each token's scale comes from its own max |t|)
     h->prof.begin(2, st);
-    e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, 0,
-                                     h->dev_status, h->prof.slot(2), st);
+    const bool wide_t = tokens_of_t_tile(h, a.B) == TOK_T_WIDE;
+    if (wide_t)
+        e = launch_digitise<float, ND_T, TOK_T_WIDE>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, 0,
+                                                     h->dev_status, h->prof.slot(2), st);
+    else
+        e = launch_digitise<float, ND_T>(w.t, h->V.R_pad, a.B, h->K, KBu, nullptr, w.Dt, w.scale_t, nullptr, 0,
+                                         h->dev_status, h->prof.slot(2), st);
     h->prof.end(st);
     if (e != cudaSuccess) return TSVD_E_CUDA;
 
@@ -1278,8 +1315,14 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     const int u_tiles = h->U.R_pad / BLOCK_R;
     const bool bf16_out = (a.dtype == TSVD_BF16) && !a.out_f32;
     h->prof.begin(3, st);
-    if (bf16_out) e = launch_gemm<ND_T, EPI_U_BF16>(q, u_tiles, st);
-    else e = launch_gemm<ND_T, EPI_U_F32>(q, u_tiles, st);
+    if (wide_t) {
+        if (bf16_out) e = launch_gemm<ND_T, EPI_U_BF16, TOK_T_WIDE>(q, u_tiles, st);
+        else e = launch_gemm<ND_T, EPI_U_F32, TOK_T_WIDE>(q, u_tiles, st);
+    } else if (bf16_out) {
+        e = launch_gemm<ND_T, EPI_U_BF16>(q, u_tiles, st);
+    } else {
+        e = launch_gemm<ND_T, EPI_U_F32>(q, u_tiles, st);
+    }
     h->prof.end(st);
     return e == cudaSuccess ? TSVD_OK : TSVD_E_CUDA;
 }
