@@ -28,6 +28,7 @@ CASES = [
     gen.scaled(C["cfg2"], name="chk_small_batch_split", M=520, N=2100, K=390, B=40, seed=403),      # split contraction, last-arriver tail
     gen.scaled(C["cfg5_d20"], name="chk_int8", M=256, N=384, K=1200, B=100, seed=404),
     gen.scaled(C["cfg1"], name="chk_f32_ragged", M=129, N=130, K=127, B=65, seed=405),
+    gen.scaled(C["cfg2"], name="chk_wide_u_tiles", M=2560, N=330, K=1300, B=400, seed=406),         # U-stage: one round of 256-column tiles
 ]
 
 

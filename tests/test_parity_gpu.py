@@ -417,3 +417,19 @@ def test_small_batch_with_many_row_tiles_runs_unsplit():
     """More output tiles than SMs: the contraction is not split (every part is the last one)."""
     spec = gen.scaled(C["cfg5_d20"], name="unsplit", M=128 * 80, N=256, K=128 * 80, B=17, seed=52)
     _util.run_and_check(spec, sample_tokens=[0, 8, 16])
+
+
+@pytest.mark.parametrize("B", [385, 400, 448])
+@pytest.mark.parametrize("x_dtype,base", [("bf16", "cfg2"), ("f32", "cfg1"), ("i8", "cfg5_d20")])
+def test_u_stage_in_one_round_of_256_column_tiles(B, x_dtype, base):
+    """20 row tiles x 9 or 10 token tiles of 48 are more tiles than SMs, 20 x 7 of 64 tokens are not: the
+    U-stage then runs tiles of 256 columns on one accumulator buffer (ragged last tile at 385 and 400)."""
+    spec = gen.scaled(C[base], name=f"wide_u_{x_dtype}_B{B}", M=2560 - 7, N=330, K=1300, B=B, seed=53)
+    _util.run_and_check(spec, sample_tokens=[0, 1, 47, 48, 63, 64, 191, 192, B - 2, B - 1])
+
+
+@pytest.mark.parametrize("B", [100, 128, 200, 256, 300])
+def test_int8_v_stage_in_tiles_of_128_tokens(B):
+    """int8 activations: 128-token tiles where they leave fewer padded tokens than 192-token ones (z bit-exact)."""
+    spec = gen.scaled(C["cfg5_d20"], name=f"narrow_i8_B{B}", M=200, N=1500, K=700, B=B, seed=54)
+    _util.run_and_check(spec)
