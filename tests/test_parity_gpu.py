@@ -360,15 +360,16 @@ def test_host_buffer_entry_point_pipelined_chunks():
         binding.tsvd_destroy(h)
 
 
-# ---- full-size configurations, sampled token columns -------------------------------------------
+# ---- full-size configurations: every token (None) where the checker needs seconds, else sampled token
+#      columns (cfg4 is also compared on 130 tokens with the numeric edge cases) -------------------
 FULL = [
-    (C["cfg2"], [0, 1, 777, 2048, 4095]),
+    (C["cfg2"], None),
     (C["cfg3_b1"], None),
     (C["cfg3_b4"], None),
     (C["cfg3_b16"], None),
     (C["cfg4"], [0, 1023, 2047]),
     (C["cfg5_d05"], [0, 100, 255]),
-    (C["cfg5_d20"], [0, 100, 255]),
+    (C["cfg5_d20"], None),
     (C["cfg5_d50"], [0, 100, 255]),
 ]
 
