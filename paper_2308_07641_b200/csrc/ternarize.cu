@@ -54,9 +54,11 @@ ternarize_kernel(const float* __restrict__ x, int len, int ldx, int P, double co
     if (tid == 0) first_k = 0x7fffffff;
     const double norm = sqrt(block_sum(sq, red));   // (its barriers also publish keys and first_k)
 
-    // bitonic sort, descending
+    // bitonic sort, descending.  Exchanges at distance 32 and more go through shared memory with a
+    // block-wide barrier each; the last five of every stage (distance 16 .. 1) stay inside the 32
+    // consecutive keys a warp holds per round, so they run in registers with shuffles.
     for (int k = 2; k <= P; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
+        for (int j = k >> 1; j >= 32; j >>= 1) {
             for (int i = tid; i < P; i += TERN_THREADS) {
                 const int l = i ^ j;
                 if (l > i) {
@@ -67,7 +69,19 @@ ternarize_kernel(const float* __restrict__ x, int len, int ldx, int P, double co
             }
             __syncthreads();
         }
+        for (int i = tid; i < P; i += TERN_THREADS) {       // (P is a multiple of the block: whole warps)
+            float a = keys[i];
+            const bool desc = (i & k) == 0;
+            for (int j = (k >> 1) < 16 ? (k >> 1) : 16; j > 0; j >>= 1) {
+                const float b = __shfl_xor_sync(0xffffffffu, a, j);
+                const bool lower = (i & j) == 0;             // this lane holds the lower index of the pair
+                a = (desc == lower) ? fmaxf(a, b) : fminf(a, b);
+            }
+            keys[i] = a;
+        }
+        if (k >= 32) __syncthreads();   // below that a thread only ever touches its own keys
     }
+    __syncthreads();
 
     // prefix sums in double: thread `tid` owns the run [tid * run, tid * run + run)
     const int run = P / TERN_THREADS;
