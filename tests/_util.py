@@ -5,7 +5,6 @@ import numpy as np
 
 import gen
 import oracle
-from gen import rng
 
 # Tolerances (stated for this map's outputs):
 #   int8 activations: z = V x bit-exact int32
@@ -23,7 +22,6 @@ def torch_x(case_x: np.ndarray, x_dtype: str):
 def run_gpu(layer, x_np: np.ndarray, x_dtype: str, flags: int = 0, want_z: bool = True):
     """Forward through TSVDLinear; returns (y as float64 numpy [B,M], z numpy or None, y_is_bf16)."""
     import torch
-    from paper_2308_07641_b200 import TSVD_FLAG_OUT_F32
     x = torch_x(x_np, x_dtype)
     B = x.shape[0]
     K = layer.info["K"]

@@ -6,7 +6,6 @@ import numpy as np
 import pytest
 
 import gen
-import oracle
 from tests import _util
 
 pytestmark = pytest.mark.gpu

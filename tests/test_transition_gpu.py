@@ -9,7 +9,6 @@ import numpy as np
 import pytest
 
 import gen
-import oracle
 from oracle import transition as otr
 from tests import _util
 
