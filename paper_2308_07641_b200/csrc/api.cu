@@ -313,6 +313,13 @@ static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, u
     if (forced == TSVD_FLAG_PATH_INDEX) return tsvd_index_fits(h, B) ? TSVD_FLAG_PATH_INDEX : 0u;
     const bool fits = tsvd_decode_fits(h, B, dtype, wide_x);
     if (forced == TSVD_FLAG_PATH_DECODE) return fits ? TSVD_FLAG_PATH_DECODE : 0u;
+    // The cluster kernels of the tensor-core path (one launch per stage, nine to sixty-four tokens) are
+    // the faster ones from nine tokens on, and from five where the decode kernels would run their
+    // single-CTA form (a contraction under 1024 columns): measured, bf16, microseconds per forward,
+    // decode / cluster-tensor: 768^3 at 5 and 8 tokens 10.9 / 7.7 and 11.2 / 7.7; 4096^3 at 6, 8, 9 and 16
+    // tokens 11.5 / 13.1, 12.9 / 13.1, 16.5 / 14.1 and 21.2 / 14.6; at four tokens and fewer the decode
+    // kernels win everywhere (4096^3: 9.1 / 13.0).
+    if (tsvd_mid_fits(h, B, dtype, wide_x) && (B >= 9 || !tsvd_decode_cluster_form(h, B))) return TSVD_FLAG_PATH_TENSOR;
     return fits ? TSVD_FLAG_PATH_DECODE : TSVD_FLAG_PATH_TENSOR;
 }
 

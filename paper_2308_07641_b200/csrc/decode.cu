@@ -784,6 +784,11 @@ bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_
     return need(digits_for_x(dt, wide_x), h->V.C_pad) <= (size_t)GEMV_MAX_SMEM && need(ND_T, h->U.C_pad) <= (size_t)GEMV_MAX_SMEM;
 }
 
+bool tsvd_decode_cluster_form(const tsvd_handle_s* h, int B)
+{
+    return use_cluster_form(h->V.C_pad, B) && use_cluster_form(h->U.C_pad, B);
+}
+
 size_t tsvd_decode_ws_bytes(const tsvd_handle_s* h, int B) { return (size_t)B * h->V.R_pad * sizeof(float); }
 
 tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws)

@@ -1233,6 +1233,7 @@ size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool
 tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
 {
     tsvd_handle_s* h = a.h;
+    if (tsvd_mid_fits(h, a.B, a.dtype, a.wide_x)) return tsvd_forward_mid(a, ws);   // (its scratch is the smaller)
     if (a.B <= SMALL_MAX_B) {
         // small batches: 16-token tiles, the contraction split across CTAs
         const SmallWs sw = carve_small(h, a.B, a.dtype, a.wide_x, ws);

@@ -229,8 +229,14 @@ size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool
 int tsvd_tensor_digits_x(tsvd_dtype_t dt, bool wide_x);
 int tsvd_tensor_digits_t();
 
+// midbatch.cu -- nine to sixty-four tokens: one launch per stage, clusters share a row tile's contraction
+bool tsvd_mid_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x);
+size_t tsvd_mid_ws_bytes(const tsvd_handle_s* h, int B);
+tsvd_status_t tsvd_forward_mid(const ForwardArgs& a, void* ws);
+
 // decode.cu -- one to sixteen tokens, bound by streaming the packed codes
 bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x);
+bool tsvd_decode_cluster_form(const tsvd_handle_s* h, int B);   // both stages would run the cluster form
 size_t tsvd_decode_ws_bytes(const tsvd_handle_s* h, int B);
 tsvd_status_t tsvd_forward_decode(const ForwardArgs& a, void* ws);
 

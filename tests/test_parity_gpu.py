@@ -123,7 +123,7 @@ def test_decode_cases_every_element(spec):
     _util.run_and_check(spec, flags=0x20)
 
 
-def test_decode_is_the_default_up_to_eight_tokens_and_refuses_more():
+def test_decode_is_the_default_up_to_four_tokens_and_refuses_more_than_eight():
     import torch
     from paper_2308_07641_b200 import binding
     rng = np.random.default_rng(5)
@@ -131,8 +131,11 @@ def test_decode_is_the_default_up_to_eight_tokens_and_refuses_more():
     S = np.ones(24, np.float32)
     h = binding.tsvd_pack(U, S, V)
     try:
-        for B in range(1, 9):         # (nine to sixteen tokens only where both contractions have 1024+ columns)
-            assert binding.tsvd_plan(h, B, binding.TSVD_BF16)["path"] == "decode"
+        for B in range(1, 9):
+            # contractions under 1024 columns: the decode kernels by default up to four tokens, from five on
+            # the cluster kernels of the tensor-core path; the decode kernels on request up to eight
+            assert binding.tsvd_plan(h, B, binding.TSVD_BF16)["path"] == ("decode" if B <= 4 else "tensor")
+            assert binding.tsvd_plan(h, B, binding.TSVD_BF16, 0x20)["path"] == "decode"
             assert binding.tsvd_plan(h, B, binding.TSVD_BF16, 0x40)["path"] == "tensor"
         assert binding.tsvd_plan(h, 9, binding.TSVD_BF16)["path"] == "tensor"
         plan = binding.tsvd_plan(h, 4, binding.TSVD_I8, 0x20)
