@@ -84,15 +84,19 @@ typedef enum {
 #define TSVD_FLAG_WIDE_X 0x200u
 /* The decode kernels (two launches, one per stage; each CTA streams 32 rows of the packed
  * codes against fixed-point digits of the stage's input held in shared memory) serve batches
- * of at most this many tokens, and are what a forward of so few tokens runs by default.
- * Forcing them for a larger batch, or for a contraction too long for the digits to fit in
+ * of at most this many tokens.  They are the default up to four tokens, and up to eight where
+ * both contractions have 1024 columns or more; beyond that, up to 64 tokens, the default is a
+ * pair of cluster kernels of the tensor-core path (TSVD_FLAG_PATH_TENSOR; one launch per stage,
+ * contractions of up to 8192 columns), and the tile kernels of that path otherwise.
+ * Forcing the decode kernels for a larger batch, or for a contraction too long for the digits to fit in
  * shared memory (about 13,000 columns at one token, 40,000 at four, 12,000 at sixteen; nine to
  * sixteen tokens also need 1024 columns or more in both stages), returns TSVD_E_TOOBIG. */
 #define TSVD_DECODE_MAX_B 16
 /* the index-list kernels serve at most this many tokens */
 #define TSVD_INDEX_MAX_B 4
-/* Test hook for the bounded device-side waits: with B > 64 the V-stage kernel's copy
- * producer withholds the activation digits, so every wait on them runs out (after a few
+/* Test hook for the bounded device-side waits: the V-stage kernel of the tensor-core path
+ * withholds the activation digits (B > 64: its copy producer; fewer tokens: the converting warps
+ * never declare them ready), so every wait on them runs out (after a few
  * milliseconds instead of the usual ~2 s); all CTAs then leave through their normal exit,
  * y is unspecified, and tsvd_last_status reports TSVD_E_TIMEOUT.  No fault, no hang: the
  * context and the handle stay usable. */

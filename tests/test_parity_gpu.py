@@ -382,14 +382,16 @@ def test_full_size_sampled(spec, sample):
     _util.run_and_check(spec, sample_tokens=sample)
 
 
-def test_bounded_wait_gives_up_and_reports_timeout():
-    """Failure detection without a fault: a forward whose copy producer withholds its data (test
-    hook) must end by itself, report TSVD_E_TIMEOUT through the handle's status word, and leave
-    the context and the handle usable for a correct forward right after."""
+@pytest.mark.parametrize("B", [200, 20], ids=["tile_kernels", "cluster_kernels"])
+def test_bounded_wait_gives_up_and_reports_timeout(B):
+    """Failure detection without a fault: a forward whose digits are withheld (test hook: by the copy
+    producer of the tile kernels, by the converting warps of the cluster kernels) must end by itself,
+    report TSVD_E_TIMEOUT through the handle's status word, and leave the context and the handle usable
+    for a correct forward right after."""
     import time
     import torch
     from paper_2308_07641_b200 import TSVDLinear, binding
-    spec = gen.scaled(C["cfg2"], name="stall", M=256, N=256, K=256, B=200, seed=41)
+    spec = gen.scaled(C["cfg2"], name="stall", M=256, N=256, K=256, B=B, seed=41)
     U, V, S = gen.make_weights(spec)
     x = gen.make_x(spec)
     layer = TSVDLinear(U, S, V)
