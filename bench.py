@@ -497,6 +497,11 @@ def roofline_of(w, peaks, peaks_src, ms_per_step, stage_ms, stage_n, sm_mhz):
         int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
         out["step_tensor_frac"] = all_ops / (ms_per_step * 1e-3) / 1e12 / int8_peak
         out["step_useful_frac_of_bf16_peak"] = single / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"]
+        if spec.B <= 32:
+            # up to 32 tokens the tensor-core path runs one cluster kernel per stage and streaming the packed
+            # codes is the other bound worth quoting
+            out["step_hbm_gbs"] = float(info["packed_bytes"]) / (ms_per_step * 1e-3) / 1e9
+            out["step_hbm_frac"] = out["step_hbm_gbs"] / peaks["hbm_gbs"]
     return out
 
 

@@ -85,9 +85,9 @@ typedef enum {
 /* The decode kernels (two launches, one per stage; each CTA streams 32 rows of the packed
  * codes against fixed-point digits of the stage's input held in shared memory) serve batches
  * of at most this many tokens.  They are the default up to four tokens, and up to eight where
- * both contractions have 1024 columns or more; beyond that, up to 64 tokens, the default is a
+ * both contractions have 1024 columns or more; beyond that, up to 32 tokens, the default is a
  * pair of cluster kernels of the tensor-core path (TSVD_FLAG_PATH_TENSOR; one launch per stage,
- * contractions of up to 8192 columns), and the tile kernels of that path otherwise.
+ * contractions of up to 4096 columns), and the tile kernels of that path otherwise.
  * Forcing the decode kernels for a larger batch, or for a contraction too long for the digits to fit in
  * shared memory (about 13,000 columns at one token, 40,000 at four, 12,000 at sixteen; nine to
  * sixteen tokens also need 1024 columns or more in both stages), returns TSVD_E_TOOBIG. */

@@ -313,7 +313,7 @@ static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, u
     if (forced == TSVD_FLAG_PATH_INDEX) return tsvd_index_fits(h, B) ? TSVD_FLAG_PATH_INDEX : 0u;
     const bool fits = tsvd_decode_fits(h, B, dtype, wide_x);
     if (forced == TSVD_FLAG_PATH_DECODE) return fits ? TSVD_FLAG_PATH_DECODE : 0u;
-    // The cluster kernels of the tensor-core path (one launch per stage, nine to sixty-four tokens) are
+    // The cluster kernels of the tensor-core path (one launch per stage, up to thirty-two tokens) are
     // the faster ones from nine tokens on, and from five where the decode kernels would run their
     // single-CTA form (a contraction under 1024 columns): measured, bf16, microseconds per forward,
     // decode / cluster-tensor: 768^3 at 5 and 8 tokens 10.9 / 7.7 and 11.2 / 7.7; 4096^3 at 6, 8, 9 and 16

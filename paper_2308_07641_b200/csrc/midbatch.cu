@@ -1,23 +1,21 @@
-// Nine to sixty-four tokens: one launch per stage (Table S1 rows "V(.)" with its scale, and "U(.)"),
+// Five to thirty-two tokens: one launch per stage (Table S1 rows "V(.)" with its scale, and "U(.)"),
 // the contraction on tcgen05 with the work of a 128-row tile shared by the CTAs of a thread-block cluster.
 //
 // For so few tokens neither of the other forms fits well: the warp-level MMA of the decode kernels is
 // a quarter as fast and at sixteen tokens its instructions, not the packed codes, set the time; the
 // tile kernels of the large batches need a launch for each conversion to digits and, to occupy the
 // SMs, a contraction split over CTAs whose parts meet through global atomics (four launches).  Here a
-// cluster of 4 or 8 CTAs takes one tile of 128 rows and splits its contraction: every CTA
+// cluster of 4 CTAs takes one tile of 128 rows and splits its contraction: every CTA
 //   - expands its slab of the packed codes (at most eight blocks of 128 columns) straight into tensor
 //     memory, where the whole slab's A operand fits beside the accumulator (4 warps, thread = row),
 //   - converts the same slab of the stage's input into digits in shared memory, a warp per token, with a
-//     power-of-two scale per token and slab (never coarser than one scale per token) (8 warps),
+//     power-of-two scale per token and slab (never coarser than one scale per token) (16 warps),
 //   - contracts them with tcgen05.mma (M = 128, N = digits x tokens <= 256; one thread issues),
 //   - and sends its partial results, as float (the exact integers for int8 activations in the V-stage),
 //     to the CTA that owns the row through distributed shared memory; after one cluster barrier the
 //     owner adds the parts in a fixed order and applies S, or the bias, and the output rounding.
 // No global atomics, no scratch besides t = S*(V x); deterministic.  Results agree with the other
 // kernel families within the tolerance, not bit for bit (the per-slab scales).
-#include <initializer_list>
-
 #include "digits.cuh"
 #include "sm100_ptx.cuh"
 #include "tsvd_internal.cuh"
@@ -26,13 +24,18 @@ namespace {
 
 using namespace ptx;
 
-constexpr int MID_THREADS = 416;       // warps 0-3: expand, then epilogue; 4-11: convert; 12: tensor memory and MMA issue
-constexpr int MID_CONV_WARPS = 8;
+constexpr int MID_THREADS = 672;       // warps 0-3: expand, then epilogue; 4: tensor memory and MMA issue; 5-20: convert
+constexpr int MID_CONV_WARPS = 16;
+constexpr int MID_MMA_WARP = 4, MID_CONV_WARP0 = 5;
 constexpr int MID_MAX_BLOCKS = 8;      // blocks of 128 columns per CTA: 32 tensor-memory columns of A each
 constexpr int MID_A_COL0 = 256;        // accumulator: columns 0 .. N-1 (N <= 256); A operand from here
 constexpr int MID_TMEM_COLS = 512;
 constexpr int MID_DIGIT_BYTES_MAX = 160 * 1024;
-constexpr int MID_MAX_B = 64, MID_MIN_B = 5;   // (five to eight tokens: only where the decode kernels have no cluster form)
+// Five to thirty-two tokens (five to eight: only where the decode kernels have no cluster form).  With 64-token
+// tiles the digits of a slab of 1024 columns no longer fit shared memory, and clusters of eight CTAs on half the
+// slab measured far slower (4096^3 at 48 and 64 tokens: 57 and 64 us against 29 us for 65 tokens on the tile kernels).
+constexpr int MID_MAX_B = 32, MID_MIN_B = 5;
+constexpr int MID_CL = 4;
 
 enum { MID_STAGE_V = 0, MID_STAGE_U = 1 };
 
@@ -111,7 +114,7 @@ ternary_cluster_mma_kernel(const MidParams p)
         u_next[0] = __ldg(my_units);
         u_next[1] = __ldg(my_units + 128);
     }
-    if (warp == 12) {
+    if (warp == MID_MMA_WARP) {
         tmem_alloc(tmem_slot, MID_TMEM_COLS);
         tmem_relinquish();
     }
@@ -123,7 +126,6 @@ ternary_cluster_mma_kernel(const MidParams p)
     // converting warps) and the output written (by everyone, after the cluster barrier) only after that
     // kernel has completed; expanding the codes into tensor memory depends on nothing it does.
     pdl_launch_dependents();
-    tsvd_stamp_begin(p.stamp);
 
     if (warp < 4) {
         // ---- expanders: thread = row of the tile = tensor-memory lane ----
@@ -149,14 +151,15 @@ ternary_cluster_mma_kernel(const MidParams p)
             __syncwarp();
             if (lane == 0) mbar_arrive(&a_ready[j]);
         }
-    } else if (warp < 4 + MID_CONV_WARPS) {
+    } else if (warp >= MID_CONV_WARP0) {
         // ---- digits of the slab, a warp per token: a lane holds its (up to two) chunks of 16 values
         //      between the maximum and the conversion ----
         pdl_wait();
+        if (warp == MID_CONV_WARP0) tsvd_stamp_begin_any(p.stamp);
         const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
         const int col0 = kb0 * 128;
         const int n_chunks = n_blk * 8;
-        for (int tb = warp - 4; tb < TOK; tb += MID_CONV_WARPS) {
+        for (int tb = warp - MID_CONV_WARP0; tb < TOK; tb += MID_CONV_WARPS) {
             const bool live = tb < p.B;
             const IN_T* row = in + (size_t)(live ? tb : 0) * p.ld_in;
             const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
@@ -339,23 +342,20 @@ ternary_cluster_mma_kernel(const MidParams p)
     __syncthreads();
     if (ctl[0] && tid == 0) atomicOr(p.status, TSVD_DEV_TIMEOUT);
     tsvd_stamp_end(p.stamp);
-    if (warp == 12) {
+    if (warp == MID_MMA_WARP) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, MID_TMEM_COLS);
     }
 }
 
 // ---- host side ----------------------------------------------------------------------------------
-inline int mid_tok(int B) { return B <= 16 ? 16 : B <= 32 ? 32 : 64; }
+inline int mid_tok(int B) { return B <= 16 ? 16 : 32; }
 
 // cluster size for a stage (0: this form does not serve it): slabs of at most eight blocks whose digits fit
 inline int mid_cluster(int KB, int nt)
 {
-    for (int cl : {4, 8}) {
-        const int cap = (KB + cl - 1) / cl;
-        if (cap <= MID_MAX_BLOCKS && (size_t)cap * nt * 128 <= (size_t)MID_DIGIT_BYTES_MAX) return cl;
-    }
-    return 0;
+    const int cap = (KB + MID_CL - 1) / MID_CL;
+    return cap <= MID_MAX_BLOCKS && (size_t)cap * nt * 128 <= (size_t)MID_DIGIT_BYTES_MAX ? MID_CL : 0;
 }
 
 inline size_t mid_smem_bytes(int KB, int nt, int tok, int cl)
@@ -400,18 +400,9 @@ template <typename IN_T, int ND, int STAGE>
 cudaError_t launch_mid(const MidParams& p, int R_pad, cudaStream_t stream)
 {
     const int tok = mid_tok(p.B);
-    const int cl = mid_cluster(p.KB, ND * tok);
-    if (cl == 4) {
-        if (tok == 16) return launch_mid_cl<IN_T, ND, 16, STAGE, 4>(p, R_pad, stream);
-        if (tok == 32) return launch_mid_cl<IN_T, ND, 32, STAGE, 4>(p, R_pad, stream);
-        return launch_mid_cl<IN_T, ND, 64, STAGE, 4>(p, R_pad, stream);
-    }
-    if (cl == 8) {
-        if (tok == 16) return launch_mid_cl<IN_T, ND, 16, STAGE, 8>(p, R_pad, stream);
-        if (tok == 32) return launch_mid_cl<IN_T, ND, 32, STAGE, 8>(p, R_pad, stream);
-        return launch_mid_cl<IN_T, ND, 64, STAGE, 8>(p, R_pad, stream);
-    }
-    return cudaErrorInvalidConfiguration;
+    if (mid_cluster(p.KB, ND * tok) != MID_CL) return cudaErrorInvalidConfiguration;
+    if (tok == 16) return launch_mid_cl<IN_T, ND, 16, STAGE, MID_CL>(p, R_pad, stream);
+    return launch_mid_cl<IN_T, ND, 32, STAGE, MID_CL>(p, R_pad, stream);
 }
 
 constexpr int ND_T = 4;   // digits of the intermediate t (fp32), as on the other paths

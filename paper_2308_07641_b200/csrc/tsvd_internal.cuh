@@ -165,6 +165,11 @@ __device__ __forceinline__ void tsvd_stamp_begin(unsigned long long* s)
 {
     if (s && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) s[0] = tsvd_globaltimer();
 }
+// the same from any one warp of the grid's first CTA (lane 0 writes)
+__device__ __forceinline__ void tsvd_stamp_begin_any(unsigned long long* s)
+{
+    if (s && blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0) s[0] = tsvd_globaltimer();
+}
 __device__ __forceinline__ void tsvd_stamp_end(unsigned long long* s)   // every warp, at its end
 {
     if (s && (threadIdx.x & 31) == 0) atomicMax(s + 1, tsvd_globaltimer());
@@ -229,7 +234,7 @@ size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool
 int tsvd_tensor_digits_x(tsvd_dtype_t dt, bool wide_x);
 int tsvd_tensor_digits_t();
 
-// midbatch.cu -- nine to sixty-four tokens: one launch per stage, clusters share a row tile's contraction
+// midbatch.cu -- five to thirty-two tokens: one launch per stage, clusters share a row tile's contraction
 bool tsvd_mid_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x);
 size_t tsvd_mid_ws_bytes(const tsvd_handle_s* h, int B);
 tsvd_status_t tsvd_forward_mid(const ForwardArgs& a, void* ws);
