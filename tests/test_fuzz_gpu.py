@@ -64,3 +64,30 @@ def _stream_case(i):
 def test_random_case_resident_digit_conversion(i):
     spec, weights, flags = _stream_case(i)
     _util.run_and_check(spec, weights=weights, flags=flags, expect_status=(0, 10))
+
+
+def _cluster_case(i):
+    """Five to 32 tokens on contractions of up to 4096 columns: the cluster kernels of the tensor-core path
+    (slabs of zero to eight blocks per CTA, ragged rows and columns, every activation type, bias)."""
+    g = np.random.default_rng(9500 + i)
+    M = int(g.integers(1, 900))
+    N = int(g.choice([1, 100, 128, 129, 500, 512, 513, 1024, 2000, 3000, 4096]))
+    K = int(g.choice([1, 127, 128, 300, 640, 1030, 2500, 4096]))
+    B = int(g.choice([5, 8, 9, 15, 16, 17, 24, 31, 32]))
+    x_dtype = ("bf16", "f32", "i8")[i % 3]
+    base = {"bf16": "cfg2", "f32": "cfg1", "i8": "cfg5_d20"}[x_dtype]
+    density = float(g.choice([0.05, 0.28, 0.7]))
+    spec = gen.scaled(gen.CONFIGS[base], name=f"cluster{i}_{x_dtype}_{M}x{N}x{K}_B{B}", M=M, N=N, K=K, B=B,
+                      density=density, seed=9500 + i)
+    U, V, S = gen.make_weights(spec)
+    S = (S * g.choice([-1.0, 1.0], K)).astype(np.float32)
+    scale = {"bf16": 1.0, "f32": 1.0, "i8": 74.0}[x_dtype] * max(1.0, density * np.sqrt(float(K) * float(N)))
+    bias = (scale * g.standard_normal(M)).astype(np.float32) if i % 2 else None
+    flags = 0x40 | (0x200 if x_dtype == "bf16" and i % 4 == 0 else 0)
+    return spec, (U, V, S), bias, flags
+
+
+@pytest.mark.parametrize("i", range(30))
+def test_random_case_cluster_kernels(i):
+    spec, weights, bias, flags = _cluster_case(i)
+    _util.run_and_check(spec, weights=weights, bias=bias, flags=flags, expect_status=(0, 10))
