@@ -60,13 +60,19 @@ struct MidParams {
     PatchGather pg;       // V-stage: the tokens are patches of the image batch at `in` (C = 0: rows of a matrix)
 };
 
+#ifdef TSVD_PHASES   // development builds: finer time stamps from single threads of a middle CTA
+#define PH(k, thread) do { if (p.stamp && blockIdx.x == (gridDim.x / 2) && tid == (thread)) p.stamp[2 + (k)] = tsvd_globaltimer(); } while (0)
+#else
+#define PH(k, thread) do { } while (0)
+#endif
+
 __device__ __forceinline__ void st_cluster_b32(uint32_t cluster_addr, uint32_t bits)
 {
     asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(cluster_addr), "r"(bits) : "memory");
 }
 
 // grid: (R_pad / 128) * CL CTAs in clusters of CL; CTA c of a cluster takes blocks [c KB / CL, (c+1) KB / CL).
-// Dynamic shared memory (1024-aligned): digits [blocks][NT rows][128] | slots [CL][TOK][128 / CL] |
+// Dynamic shared memory (1024-aligned): digits [blocks][NT rows][128] | packed codes [blocks][4 KiB] | slots [CL][TOK][128 / CL] |
 // scale [TOK] | barriers
 template <typename IN_T, int ND, int TOK, int STAGE, int CL>
 __global__ void __launch_bounds__(MID_THREADS, 1)
@@ -89,12 +95,14 @@ ternary_cluster_mma_kernel(const MidParams p)
     const int n_blk = kb1 - kb0;                       // 0 .. MID_MAX_BLOCKS (the host checks the upper end)
     const int blk_cap = (p.KB + CL - 1) / CL;          // the most any CTA of the cluster has: same layout in all
     int8_t* digits = reinterpret_cast<int8_t*>(smem);
-    uint32_t* slots = reinterpret_cast<uint32_t*>(smem + (size_t)blk_cap * TILE_BYTES);   // [CL][TOK][ROWS_OWN]
+    uint4* codes = reinterpret_cast<uint4*>(smem + (size_t)blk_cap * TILE_BYTES);        // [blocks][2][128] packed units
+    uint32_t* slots = reinterpret_cast<uint32_t*>(codes + (size_t)blk_cap * 256);         // [CL][TOK][ROWS_OWN]
     float* scale = reinterpret_cast<float*>(slots + CL * TOK * ROWS_OWN);
     uint64_t* a_ready = reinterpret_cast<uint64_t*>(scale + TOK);   // [MID_MAX_BLOCKS] block j of A is in tensor memory
     uint64_t* d_ready = a_ready + MID_MAX_BLOCKS;                   // the slab's digits are in shared memory
     uint64_t* done = d_ready + 1;                                   // all MMAs have completed
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
+    uint64_t* c_ready = done + 1;                                   // the slab's packed codes are in shared memory
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(c_ready + 1);
     volatile int* ctl = reinterpret_cast<volatile int*>(tmem_slot + 1);   // [2]: abort flag, wait limit
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -102,17 +110,16 @@ ternary_cluster_mma_kernel(const MidParams p)
         for (int j = 0; j < MID_MAX_BLOCKS; ++j) mbar_init(&a_ready[j], 4);
         mbar_init(d_ready, MID_CONV_WARPS);
         mbar_init(done, 1);
+        mbar_init(c_ready, 1);
         ctl[0] = 0;
         ctl[1] = p.wait_limit > 0 ? p.wait_limit : kWaitLimitDefault;
         fence_mbar_init();
     }
-    // the first blocks of codes are requested before anything else (no kernel writes them), so that they
-    // travel while the kernel before this one still runs
-    const uint4* my_units = p.units + ((size_t)tile * (size_t)(p.C_pad >> 6) + (size_t)(2 * kb0)) * 128 + (tid & 127);
-    uint4 u_next[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-    if (warp < 4 && n_blk > 0) {
-        u_next[0] = __ldg(my_units);
-        u_next[1] = __ldg(my_units + 128);
+    // The slab's packed codes (contiguous: 4 KiB per block) are requested as one bulk copy before anything
+    // else -- no kernel writes them -- so that they travel while the kernel before this one still runs.
+    if (tid == 0 && n_blk > 0) {
+        mbar_arrive_expect_tx(c_ready, (uint32_t)n_blk * 4096u);
+        bulk_g2s(codes, p.units + ((size_t)tile * (size_t)(p.C_pad >> 6) + (size_t)(2 * kb0)) * 128, (uint32_t)n_blk * 4096u, c_ready);
     }
     if (warp == MID_MMA_WARP) {
         tmem_alloc(tmem_slot, MID_TMEM_COLS);
@@ -130,12 +137,9 @@ ternary_cluster_mma_kernel(const MidParams p)
     if (warp < 4) {
         // ---- expanders: thread = row of the tile = tensor-memory lane ----
         const uint32_t a_lane = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)MID_A_COL0;
-        for (int j = 0; j < n_blk; ++j) {
-            const uint4 u0 = u_next[0], u1 = u_next[1];
-            if (j + 1 < n_blk) {
-                u_next[0] = __ldg(my_units + (size_t)(2 * (j + 1)) * 128);
-                u_next[1] = __ldg(my_units + (size_t)(2 * (j + 1) + 1) * 128);
-            }
+        bool arrived = n_blk == 0 || mbar_wait(c_ready, 0, ctl);
+        for (int j = 0; j < n_blk && arrived; ++j) {
+            const uint4 u0 = codes[j * 256 + tid], u1 = codes[j * 256 + 128 + tid];
             uint32_t o[32];   // the row's 128 int8 values of this block, four per 32-bit column
             tsvd_expand16(u0.x, *reinterpret_cast<uint32_t(*)[4]>(&o[0]));
             tsvd_expand16(u0.y, *reinterpret_cast<uint32_t(*)[4]>(&o[4]));
@@ -156,6 +160,7 @@ ternary_cluster_mma_kernel(const MidParams p)
         //      between the maximum and the conversion ----
         pdl_wait();
         if (warp == MID_CONV_WARP0) tsvd_stamp_begin_any(p.stamp);
+        PH(0, MID_CONV_WARP0 * 32);
         const IN_T* in = reinterpret_cast<const IN_T*>(p.in);
         const int col0 = kb0 * 128;
         const int n_chunks = n_blk * 8;
@@ -189,6 +194,7 @@ ternary_cluster_mma_kernel(const MidParams p)
                 }
             }
             float qscale = 1.f;
+            PH(1, MID_CONV_WARP0 * 32);
             if constexpr (!kInt) {
                 for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
                 const int E = tsvd_quant_exponent(amax);
@@ -239,6 +245,7 @@ ternary_cluster_mma_kernel(const MidParams p)
         fence_proxy_async_smem();   // the MMAs read these through the async proxy
         __syncwarp();
         if (lane == 0 && !p.test_stall) mbar_arrive(d_ready);
+        PH(2, MID_CONV_WARP0 * 32);
     } else {
         // ---- MMA issue: the whole warp walks the blocks, one elected lane issues ----
         bool alive = n_blk == 0 || mbar_wait(d_ready, 0, ctl);
@@ -256,6 +263,7 @@ ternary_cluster_mma_kernel(const MidParams p)
         }
         if (alive && n_blk > 0 && elect_one()) umma_commit(done);
         __syncwarp();
+        PH(3, MID_MMA_WARP * 32);
     }
 
     if (warp < 4) {
@@ -269,6 +277,7 @@ ternary_cluster_mma_kernel(const MidParams p)
         if (have && n_blk > 0) have = mbar_wait(done, 0, ctl);
         else have = false;
         tc_fence_after_sync();
+        PH(4, 0);
         const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
 #pragma unroll 1
         for (int g = 0; g < TOK / 8; ++g) {
@@ -309,6 +318,7 @@ ternary_cluster_mma_kernel(const MidParams p)
     tc_fence_before_sync();
     cluster_sync_all();
     pdl_wait();
+    PH(5, 0);
 
     // ---- owner: rows c*ROWS_OWN .. of the tile, all tokens ----
     for (int item = tid; item < TOK * ROWS_OWN; item += MID_THREADS) {
@@ -361,7 +371,7 @@ inline int mid_cluster(int KB, int nt)
 inline size_t mid_smem_bytes(int KB, int nt, int tok, int cl)
 {
     const size_t cap = (KB + cl - 1) / cl;
-    return 1024 + cap * nt * 128 + (size_t)tok * 128 * 4 + (size_t)tok * 4 + (MID_MAX_BLOCKS + 2) * 8 + 16;
+    return 1024 + cap * nt * 128 + cap * 4096 + (size_t)tok * 128 * 4 + (size_t)tok * 4 + (MID_MAX_BLOCKS + 3) * 8 + 16;
 }
 
 template <typename IN_T, int ND, int TOK, int STAGE, int CL>
