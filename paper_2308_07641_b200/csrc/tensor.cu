@@ -1163,6 +1163,27 @@ int pick_ksplit(int out_tiles, int KB)
     return ks < 1 ? 1 : ks;
 }
 
+// Whether a batch of at most SMALL_MAX_B tokens runs the split-contraction form below rather than the tile
+// kernels (one tile of tokens per row tile).  Both are bound by the blocks of 128 columns a CTA walks through
+// (about 0.2 us each): per stage the tile kernels take rounds x KB of them, the split form rounds x KB / parts,
+// but its integer atomics, last-arriver tails and heavier launches cost about 8 us more per forward (40 blocks).
+// Measured (bf16, 20 to 48 tokens, us, split / tiles): 4096^3 38 / 29, 768^3 24 / 16, 2048 x 8192 x 2048 28 / 31,
+// 1024 x 16384 x 1024 28 / 43, 256 x 32768 x 256 27 / 70, 128 x 16384 x 16384 92 / 77: the rule reproduces each.
+bool prefer_split_form(const tsvd_handle_s* h, int B)
+{
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int j16 = (B + SMALL_TOK - 1) / SMALL_TOK;
+    long long tiles_cost = 0, split_cost = 40;
+    for (const PackedMat* m : {&h->V, &h->U}) {
+        const int rows = m->R_pad / BLOCK_R, KB = m->C_pad / BLOCK_C;
+        tiles_cost += (long long)((rows + sms - 1) / sms) * KB;
+        const int parts = pick_ksplit(rows * j16, KB);
+        split_cost += (long long)((rows * j16 * parts + sms - 1) / sms) * ((KB + parts - 1) / parts);
+    }
+    return split_cost < tiles_cost;
+}
+
 // Four launches: x -> digits (clears the V-stage sums) | V-stage parts, the last part of each tile
 // writes t = S*z and the per-token max |t| | t -> digits (clears the U-stage sums) | U-stage
 // parts, the last part of each tile writes y.
@@ -1226,7 +1247,7 @@ int tsvd_tensor_digits_t() { return ND_T; }
 
 size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x)
 {
-    if (B <= SMALL_MAX_B) return carve_small(h, B, dt, wide_x, nullptr).total;
+    if (B <= SMALL_MAX_B && prefer_split_form(h, B)) return carve_small(h, B, dt, wide_x, nullptr).total;
     return carve(h, B, dt, wide_x, nullptr).total;
 }
 
@@ -1234,8 +1255,8 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
 {
     tsvd_handle_s* h = a.h;
     if (tsvd_mid_fits(h, a.B, a.dtype, a.wide_x)) return tsvd_forward_mid(a, ws);   // (its scratch is the smaller)
-    if (a.B <= SMALL_MAX_B) {
-        // small batches: 16-token tiles, the contraction split across CTAs
+    if (a.B <= SMALL_MAX_B && prefer_split_form(h, a.B)) {
+        // few tokens on few row tiles with long contractions: 16-token tiles, the contraction split across CTAs
         const SmallWs sw = carve_small(h, a.B, a.dtype, a.wide_x, ws);
         switch (a.dtype) {
             case TSVD_F32: return forward_small<float, 4>(a, sw);

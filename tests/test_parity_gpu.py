@@ -414,15 +414,17 @@ def test_bounded_wait_gives_up_and_reports_timeout(B):
 
 @pytest.mark.parametrize("B", [63, 64, 65, 128])
 def test_batch_sizes_around_the_small_batch_switch(B):
-    """B <= 64 takes 16-token tiles with a split contraction, B > 64 the 192-column tiles."""
+    """Up to 64 tokens the tile kernels run one (padded) token tile per row tile unless the split form is
+    estimated faster (not here: short contractions); beyond 64 always the tile kernels."""
     spec = gen.scaled(C["cfg2"], name=f"switch_B{B}", M=300, N=520, K=390, B=B, seed=51)
     _util.run_and_check(spec)
 
 
-def test_small_batch_with_many_row_tiles_runs_unsplit():
-    """More output tiles than SMs: the contraction is not split (every part is the last one)."""
-    spec = gen.scaled(C["cfg5_d20"], name="unsplit", M=128 * 80, N=256, K=128 * 80, B=17, seed=52)
-    _util.run_and_check(spec, sample_tokens=[0, 8, 16])
+def test_split_form_with_one_stage_unsplit():
+    """Few row tiles on a long contraction: the split form (U-stage: 4 row tiles x 2 token tiles, 16 parts
+    each); its V-stage has 128 output tiles, about one per SM, and is not split (every part is the last one)."""
+    spec = gen.scaled(C["cfg5_d20"], name="unsplit", M=512, N=8192, K=8192, B=20, seed=52, density=0.05)
+    _util.run_and_check(spec, sample_tokens=[0, 8, 16, 19])
 
 
 @pytest.mark.parametrize("B", [385, 400, 448])
