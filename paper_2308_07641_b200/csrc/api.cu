@@ -320,6 +320,15 @@ static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, u
     // tokens 11.5 / 13.1, 12.9 / 13.1, 16.5 / 14.1 and 21.2 / 14.6; at four tokens and fewer the decode
     // kernels win everywhere (4096^3: 9.1 / 13.0).
     if (tsvd_mid_fits(h, B, dtype, wide_x) && (B >= 9 || !tsvd_decode_cluster_form(h, B))) return TSVD_FLAG_PATH_TENSOR;
+    // Nine to sixteen tokens on very tall matrices: the decode kernels' clusters (four CTAs per 128 rows) would
+    // run in more than two rounds, and one padded token tile on the tile kernels is faster (16384 x 4096 x 4096:
+    // 33-35 us against 30).
+    if (fits && B >= 9) {
+        int sms = 148, dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int rows = (h->V.R_pad > h->U.R_pad ? h->V.R_pad : h->U.R_pad) / 128;
+        if (4 * rows > 2 * sms) return TSVD_FLAG_PATH_TENSOR;
+    }
     return fits ? TSVD_FLAG_PATH_DECODE : TSVD_FLAG_PATH_TENSOR;
 }
 

@@ -423,6 +423,13 @@ inline int digits_for_x(tsvd_dtype_t dt, bool wide) { return dt == TSVD_I8 ? 1 :
 bool tsvd_mid_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x)
 {
     if (B < MID_MIN_B || B > MID_MAX_B) return false;
+    // one round of clusters: with more row tiles than a quarter of the SMs the launch runs in several rounds of
+    // about 6 us each, and one padded token tile on the tile kernels is faster (16384 x 4096 x 4096 at 17 and
+    // 32 tokens: 42 and 48 us against 30)
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int rows = (h->V.R_pad > h->U.R_pad ? h->V.R_pad : h->U.R_pad) / 128;
+    if (rows * MID_CL > sms) return false;
     const int tok = mid_tok(B);
     return mid_cluster(h->V.C_pad / 128, digits_for_x(dt, wide_x) * tok) != 0 && mid_cluster(h->U.C_pad / 128, ND_T * tok) != 0;
 }
