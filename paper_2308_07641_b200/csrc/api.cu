@@ -320,14 +320,15 @@ static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, u
     // tokens 11.5 / 13.1, 12.9 / 13.1, 16.5 / 14.1 and 21.2 / 14.6; at four tokens and fewer the decode
     // kernels win everywhere (4096^3: 9.1 / 13.0).
     if (tsvd_mid_fits(h, B, dtype, wide_x) && (B >= 9 || !tsvd_decode_cluster_form(h, B))) return TSVD_FLAG_PATH_TENSOR;
-    // Nine to sixteen tokens on very tall matrices: the decode kernels' clusters (four CTAs per 128 rows) would
-    // run in more than two rounds, and one padded token tile on the tile kernels is faster (16384 x 4096 x 4096:
-    // 33-35 us against 30).
+    // Nine to sixteen tokens on tall matrices: where the decode kernels' clusters (four CTAs per 128 rows) need
+    // four rounds or more over the two stages, one padded token tile on the tile kernels is as fast or faster
+    // (16384 x 4096 x 4096: 33-35 us against 30; 8192^3: 41-51 against 43; but 4096 x 4096 x 8192, three
+    // rounds: 23-29 against 36).
     if (fits && B >= 9) {
         int sms = 148, dev = 0;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        const int rows = (h->V.R_pad > h->U.R_pad ? h->V.R_pad : h->U.R_pad) / 128;
-        if (4 * rows > 2 * sms) return TSVD_FLAG_PATH_TENSOR;
+        const int rounds = (h->V.R_pad / 128 * 4 + sms - 1) / sms + (h->U.R_pad / 128 * 4 + sms - 1) / sms;
+        if (rounds >= 4) return TSVD_FLAG_PATH_TENSOR;
     }
     return fits ? TSVD_FLAG_PATH_DECODE : TSVD_FLAG_PATH_TENSOR;
 }
@@ -459,13 +460,13 @@ extern "C" tsvd_status_t tsvd_reserve(tsvd_handle_t h, int B_max, tsvd_dtype_t d
     TSVD_CUDA_OK(cudaGetDevice(&dev));
     if (dev != h->device) return TSVD_E_CUDA;
     size_t need = 0;
-    const int marks[] = {B_max, 64, TSVD_DECODE_MAX_B, TSVD_INDEX_MAX_B};
+    for (int wide = 0; wide < 2; ++wide) {
+        const size_t t = tsvd_tensor_ws_bytes_upto(h, B_max, dtype, wide != 0);
+        if (t > need) need = t;
+    }
+    const int marks[] = {B_max, TSVD_DECODE_MAX_B, TSVD_INDEX_MAX_B};
     for (int B : marks) {
         if (B > B_max) continue;
-        for (int wide = 0; wide < 2; ++wide) {
-            const size_t t = tsvd_tensor_ws_bytes(h, B, dtype, wide != 0);
-            if (t > need) need = t;
-        }
         const size_t d = tsvd_decode_ws_bytes(h, B), s = tsvd_simple_ws_bytes(h, B);
         if (d > need) need = d;
         if (s > need) need = s;

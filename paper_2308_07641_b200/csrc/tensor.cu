@@ -1113,7 +1113,7 @@ TensorWs carve(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide, void* 
 namespace {
 
 constexpr int SMALL_TOK = 16;        // tokens per tile on the small-batch path
-constexpr int SMALL_MAX_B = 64;
+constexpr int SMALL_MAX_B = 512;   // (the split form also has to be preferred: few row tiles, long contractions)
 
 struct SmallWs {
     int8_t* Dx; float* scale_x; int* zacc; float* t; int8_t* Dt; float* scale_t; int* yacc;
@@ -1179,7 +1179,10 @@ bool prefer_split_form(const tsvd_handle_s* h, int B)
         const int rows = m->R_pad / BLOCK_R, KB = m->C_pad / BLOCK_C;
         tiles_cost += (long long)((rows + sms - 1) / sms) * KB;
         const int parts = pick_ksplit(rows * j16, KB);
-        split_cost += (long long)((rows * j16 * parts + sms - 1) / sms) * ((KB + parts - 1) / parts);
+        // a split stage of more than one round is slow beyond this estimate (its many short tiles each end in
+        // atomics): 1024 x 1024 x 16384 at 17 to 64 tokens took 56 to 82 us in the split form, 55 on the tiles
+        if (rows * j16 * parts > sms) return false;
+        split_cost += (KB + parts - 1) / parts;
     }
     return split_cost < tiles_cost;
 }
@@ -1249,6 +1252,15 @@ size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool
 {
     if (B <= SMALL_MAX_B && prefer_split_form(h, B)) return carve_small(h, B, dt, wide_x, nullptr).total;
     return carve(h, B, dt, wide_x, nullptr).total;
+}
+
+// An upper bound of the scratch of any batch of up to B_max tokens (both forms grow with the batch; which of
+// them a batch takes depends on the batch).
+size_t tsvd_tensor_ws_bytes_upto(const tsvd_handle_s* h, int B_max, tsvd_dtype_t dt, bool wide_x)
+{
+    const size_t tiles = carve(h, B_max, dt, wide_x, nullptr).total;
+    const size_t split = carve_small(h, B_max < SMALL_MAX_B ? B_max : SMALL_MAX_B, dt, wide_x, nullptr).total;
+    return tiles > split ? tiles : split;
 }
 
 tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)

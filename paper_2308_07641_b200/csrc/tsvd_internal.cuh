@@ -231,6 +231,7 @@ size_t tsvd_simple_ws_bytes(const tsvd_handle_s* h, int B);
 // tensor.cu -- tcgen05 path
 tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws);
 size_t tsvd_tensor_ws_bytes(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_x);
+size_t tsvd_tensor_ws_bytes_upto(const tsvd_handle_s* h, int B_max, tsvd_dtype_t dt, bool wide_x);
 int tsvd_tensor_digits_x(tsvd_dtype_t dt, bool wide_x);
 int tsvd_tensor_digits_t();
 

@@ -261,3 +261,30 @@ def test_reserve_sizes_the_scratch_once():
         assert free1 == free0
     finally:
         layer.close()
+
+
+def test_reserve_covers_both_forms_of_the_tensor_core_path():
+    """Two row tiles per stage and a contraction of 20000 columns: batches of up to 512 tokens take the
+    split-contraction form, whose scratch per token is the larger one; after tsvd_reserve(300) no batch up
+    to 300 tokens allocates on either form."""
+    import torch
+    from paper_2308_07641_b200 import TSVDLinear
+    spec = gen.scaled(C["cfg2"], name="reserve_split", M=200, N=20000, K=250, B=300, seed=314, density=0.05)
+    U, V, S = gen.make_weights(spec)
+    x = _util.torch_x(gen.make_x(spec), "bf16")
+    layer = TSVDLinear(U, S, V)
+    try:
+        layer.reserve(300, "bf16")
+        y = torch.empty((300, spec.M), dtype=torch.bfloat16, device="cuda")
+        for B, flags in ((300, 0), (2, 0), (6, 0), (40, 0), (5, SIMPLE)):     # (lazy module loading, as above)
+            layer.forward(x[:B], out=y[:B], flags=flags)
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        for B in (300, 192, 100, 65, 64, 20, 5, 1):
+            for flags in (0, WIDE, TENSOR):
+                layer.forward(x[:B], out=y[:B], flags=flags)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0
+    finally:
+        layer.close()

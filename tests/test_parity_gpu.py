@@ -441,3 +441,12 @@ def test_int8_v_stage_in_tiles_of_128_tokens(B):
     """int8 activations: 128-token tiles where they leave fewer padded tokens than 192-token ones (z bit-exact)."""
     spec = gen.scaled(C["cfg5_d20"], name=f"narrow_i8_B{B}", M=200, N=1500, K=700, B=B, seed=54)
     _util.run_and_check(spec)
+
+
+@pytest.mark.parametrize("B", [65, 100, 192, 300, 512])
+@pytest.mark.parametrize("x_dtype,base", [("bf16", "cfg2"), ("f32", "cfg1"), ("i8", "cfg5_d20")])
+def test_split_form_beyond_64_tokens(B, x_dtype, base):
+    """Two row tiles in each stage and a contraction of 20000 columns: the split form is preferred up to 512
+    tokens (16-token tiles, up to sixteen parts per tile, integer atomics, last-arriver tail)."""
+    spec = gen.scaled(C[base], name=f"split_{x_dtype}_B{B}", M=200, N=20000, K=250, B=B, seed=55, density=0.05)
+    _util.run_and_check(spec, sample_tokens=[0, 15, 16, B // 2, B - 1])
