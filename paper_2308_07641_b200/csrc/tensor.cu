@@ -1053,7 +1053,7 @@ constexpr int TOK_I8_NARROW = 128;
 // would overlap with a second buffer anyway (4096 rows x 256 tokens: 32 x 6 = 192 tiles in two rounds
 // against 32 x 4 = 128 in one).
 constexpr int TOK_T_WIDE = 64;
-inline int tokens_of_t_tile(const tsvd_handle_s* h, int B)
+inline int tokens_of_four_digit_tile(int row_tiles, int B)
 {
     static int sms = 0;
     if (sms == 0) {
@@ -1061,14 +1061,16 @@ inline int tokens_of_t_tile(const tsvd_handle_s* h, int B)
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
         sms = n;
     }
-    const int rows = h->U.R_pad / BLOCK_R;
     const int regular = tokens_per_tile(ND_T);
-    const long long tiles_regular = (long long)rows * ((B + regular - 1) / regular);
-    const long long tiles_wide = (long long)rows * ((B + TOK_T_WIDE - 1) / TOK_T_WIDE);
+    const long long tiles_regular = (long long)row_tiles * ((B + regular - 1) / regular);
+    const long long tiles_wide = (long long)row_tiles * ((B + TOK_T_WIDE - 1) / TOK_T_WIDE);
     return tiles_regular > sms && tiles_wide <= sms ? TOK_T_WIDE : regular;
 }
-inline int tokens_of_x_tile(int ndx, int B)
+inline int tokens_of_t_tile(const tsvd_handle_s* h, int B) { return tokens_of_four_digit_tile(h->U.R_pad / BLOCK_R, B); }
+// (the V-stage of four-digit activations -- fp32, or bf16 on request -- follows the same rule)
+inline int tokens_of_x_tile(const tsvd_handle_s* h, int ndx, int B)
 {
+    if (ndx == 4) return tokens_of_four_digit_tile(h->V.R_pad / BLOCK_R, B);
     const int wide_tile = tokens_per_tile(ndx);
     if (ndx != 1) return wide_tile;
     const long long padded_wide = (B + wide_tile - 1LL) / wide_tile * wide_tile;
@@ -1084,7 +1086,7 @@ struct TensorWs {
 TensorWs carve(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide, void* base)
 {
     const int ndx = digits_for_x(dt, wide);
-    const int tokx = tokens_of_x_tile(ndx, B), tokt = tokens_of_t_tile(h, B);
+    const int tokx = tokens_of_x_tile(h, ndx, B), tokt = tokens_of_t_tile(h, B);
     const size_t Bx = align_up(B, tokx), Bt = align_up(B, tokt);
     const size_t Bmax = Bx > Bt ? Bx : Bt;
     const size_t KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
@@ -1279,7 +1281,8 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     }
     const TensorWs w = carve(h, a.B, a.dtype, a.wide_x, ws);
     const bool wide_bf16 = a.dtype == TSVD_BF16 && a.wide_x;
-    const bool narrow_i8 = a.dtype == TSVD_I8 && tokens_of_x_tile(1, a.B) == TOK_I8_NARROW;
+    const bool narrow_i8 = a.dtype == TSVD_I8 && tokens_of_x_tile(h, 1, a.B) == TOK_I8_NARROW;
+    const bool wide_x4 = (a.dtype == TSVD_F32 || wide_bf16) && tokens_of_x_tile(h, 4, a.B) == TOK_T_WIDE;
     const int KBv = h->V.C_pad / BLOCK_C, KBu = h->U.C_pad / BLOCK_C;
     cudaStream_t st = a.stream;
     cudaError_t e;
@@ -1289,11 +1292,19 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     h->prof.begin(0, st);
     switch (a.dtype) {
         case TSVD_F32:
-            e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, nullptr, 0,
-                                          h->dev_status, stamp0, st, a.gather);
+            if (wide_x4)
+                e = launch_digitise<float, 4, TOK_T_WIDE>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x,
+                                                          nullptr, 0, h->dev_status, stamp0, st, a.gather);
+            else
+                e = launch_digitise<float, 4>((const float*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx, w.scale_x, nullptr, 0,
+                                              h->dev_status, stamp0, st, a.gather);
             break;
         case TSVD_BF16:
-            if (wide_bf16)
+            if (wide_bf16 && wide_x4)
+                e = launch_digitise<__nv_bfloat16, 4, TOK_T_WIDE>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr,
+                                                                  w.Dx, w.scale_x, nullptr, 0, h->dev_status, stamp0, st,
+                                                                  a.gather);
+            else if (wide_bf16)
                 e = launch_digitise<__nv_bfloat16, 4>((const __nv_bfloat16*)a.x, a.ldx, a.B, h->N, KBv, nullptr, w.Dx,
                                                       w.scale_x, nullptr, 0, h->dev_status, stamp0, st, a.gather);
             else
@@ -1322,7 +1333,8 @@ tsvd_status_t tsvd_forward_tensor(const ForwardArgs& a, void* ws)
     if (a.test_stall) { p.test_stall = 1; p.wait_limit = 16; }   // ~8 ms instead of ~2 s
     const int v_tiles = h->V.R_pad / BLOCK_R;
     h->prof.begin(1, st);
-    if (a.dtype == TSVD_F32 || wide_bf16) e = launch_gemm<4, EPI_V>(p, v_tiles, st);
+    if (wide_x4) e = launch_gemm<4, EPI_V, TOK_T_WIDE>(p, v_tiles, st);
+    else if (a.dtype == TSVD_F32 || wide_bf16) e = launch_gemm<4, EPI_V>(p, v_tiles, st);
     else if (a.dtype == TSVD_BF16) e = launch_gemm<3, EPI_V>(p, v_tiles, st);
     else if (narrow_i8) e = launch_gemm<1, EPI_V, TOK_I8_NARROW>(p, v_tiles, st);
     else e = launch_gemm<1, EPI_V>(p, v_tiles, st);

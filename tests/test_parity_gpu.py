@@ -450,3 +450,12 @@ def test_split_form_beyond_64_tokens(B, x_dtype, base):
     tokens (16-token tiles, up to sixteen parts per tile, integer atomics, last-arriver tail)."""
     spec = gen.scaled(C[base], name=f"split_{x_dtype}_B{B}", M=200, N=20000, K=250, B=B, seed=55, density=0.05)
     _util.run_and_check(spec, sample_tokens=[0, 15, 16, B // 2, B - 1])
+
+
+@pytest.mark.parametrize("B", [385, 448])
+@pytest.mark.parametrize("x_dtype,base,flags", [("f32", "cfg1", 0), ("bf16", "cfg2", 0x200)])
+def test_four_digit_v_stage_in_one_round_of_256_column_tiles(B, x_dtype, base, flags):
+    """fp32 activations (or bf16 with four digits): 20 row tiles of V x 9 or 10 token tiles of 48 are more
+    tiles than SMs, 20 x 7 of 64 tokens are not: the V-stage, too, then runs tiles of 256 columns."""
+    spec = gen.scaled(C[base], name=f"wide_v_{x_dtype}_B{B}", M=300, N=1300, K=2560 - 9, B=B, seed=56)
+    _util.run_and_check(spec, flags=flags, sample_tokens=[0, 47, 48, 63, 64, 191, 192, B - 1])
