@@ -694,6 +694,14 @@ size_t gemv_smem_bytes(int nd, int ntok, int C_pad)
            (size_t)ntok * sizeof(float) + (size_t)GEMV_WARPS * ntok * sizeof(float);
 }
 
+// One and two tokens take the cluster form only where the digits of a whole row do not fit one CTA's shared
+// memory (contractions of tens of thousands of columns) while a quarter of them does.
+inline bool stage_in_cluster_form(int nd, int C_pad, int B)
+{
+    if (use_cluster_form(C_pad, B)) return true;
+    return B <= 2 && (C_pad >> 6) >= CLUSTER_MIN_GROUPS && gemv_smem_bytes(nd, B, C_pad) > (size_t)GEMV_MAX_SMEM;
+}
+
 template <typename IN_T, int ND, int NTOK, int STAGE>
 cudaError_t launch_gemv(const GemvParams& p, int R_pad, cudaStream_t stream)
 {
@@ -750,7 +758,7 @@ cudaError_t launch_gemv_cluster(const GemvParams& p, int R_pad, cudaStream_t str
 template <typename IN_T, int ND, int STAGE>
 cudaError_t launch_gemv_tokens(const GemvParams& p, int R_pad, cudaStream_t stream)
 {
-    if (use_cluster_form(p.C_pad, p.B)) {
+    if (stage_in_cluster_form(ND, p.C_pad, p.B)) {
         if (p.B == 1) return launch_gemv_cluster<IN_T, ND, 1, STAGE>(p, R_pad, stream);
         if (p.B == 2) return launch_gemv_cluster<IN_T, ND, 2, STAGE>(p, R_pad, stream);
         if (p.B <= 4) return launch_gemv_cluster<IN_T, ND, 4, STAGE>(p, R_pad, stream);
@@ -778,7 +786,7 @@ bool tsvd_decode_fits(const tsvd_handle_s* h, int B, tsvd_dtype_t dt, bool wide_
     // nine to sixteen tokens: the cluster form only
     if (B > 8 && !(use_cluster_form(h->V.C_pad, B) && use_cluster_form(h->U.C_pad, B))) return false;
     auto need = [&](int nd, int C_pad) {
-        if (!use_cluster_form(C_pad, B)) return gemv_smem_bytes(nd, ntok, C_pad);
+        if (!stage_in_cluster_form(nd, C_pad, B)) return gemv_smem_bytes(nd, ntok, C_pad);
         return gemv_cluster_smem_bytes(nd, (B == 5 || B == 6) ? 6 : ntok, C_pad);   // (the cluster form also has six)
     };
     return need(digits_for_x(dt, wide_x), h->V.C_pad) <= (size_t)GEMV_MAX_SMEM && need(ND_T, h->U.C_pad) <= (size_t)GEMV_MAX_SMEM;

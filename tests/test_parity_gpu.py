@@ -263,12 +263,12 @@ def test_decode_falls_back_when_the_digits_do_not_fit_shared_memory():
             assert binding.tsvd_plan(h, B, binding.TSVD_F32)["path"] == "decode"
     finally:
         binding.tsvd_destroy(h)
-    N = 40000                       # 40064 padded columns x 4 digits: one token fits, two do not; a quarter at four tokens fits, at eight not
+    N = 40000                       # 40064 padded columns x 4 digits: one token fits; two and four on a quarter each (cluster form); eight do not
     V = np.zeros((8, N), np.int8)
     h = binding.tsvd_pack(U, S, V)
     try:
         assert binding.tsvd_plan(h, 1, binding.TSVD_F32)["path"] == "decode"
-        assert binding.tsvd_plan(h, 2, binding.TSVD_F32)["path"] == "tensor"
+        assert binding.tsvd_plan(h, 2, binding.TSVD_F32)["path"] == "decode"
         assert binding.tsvd_plan(h, 4, binding.TSVD_F32)["path"] == "decode"
         assert binding.tsvd_plan(h, 8, binding.TSVD_F32)["path"] == "tensor"
         with pytest.raises(binding.TSVDError) as ei:
@@ -459,3 +459,13 @@ def test_four_digit_v_stage_in_one_round_of_256_column_tiles(B, x_dtype, base, f
     tiles than SMs, 20 x 7 of 64 tokens are not: the V-stage, too, then runs tiles of 256 columns."""
     spec = gen.scaled(C[base], name=f"wide_v_{x_dtype}_B{B}", M=300, N=1300, K=2560 - 9, B=B, seed=56)
     _util.run_and_check(spec, flags=flags, sample_tokens=[0, 47, 48, 63, 64, 191, 192, B - 1])
+
+
+@pytest.mark.parametrize("B,N", [(1, 60000), (2, 40000), (2, 65280)])
+def test_decode_one_and_two_tokens_on_rows_too_long_for_one_cta(B, N):
+    """fp32 activations, four digits: the digits of a whole row exceed a CTA's shared memory, a quarter fits:
+    the cluster form serves one and two tokens as well."""
+    from paper_2308_07641_b200 import binding
+    spec = gen.scaled(C["cfg1"], name=f"long_row_B{B}_{N}", M=200, N=N, K=300, B=B, seed=57, density=0.02)
+    res = _util.run_and_check(spec, flags=0x20)
+    assert res["status"] in (0, 10)
