@@ -89,9 +89,9 @@ typedef enum {
  * pair of cluster kernels of the tensor-core path (TSVD_FLAG_PATH_TENSOR; one launch per stage,
  * contractions of up to 4096 columns), and the tile kernels of that path otherwise.
  * Forcing the decode kernels for a larger batch, or for a contraction too long for the digits to fit in
- * shared memory (the whole range of contractions at one and two tokens, about 40,000 columns at four,
- * 12,000 at sixteen; nine to
- * sixteen tokens also need 1024 columns or more in both stages), returns TSVD_E_TOOBIG. */
+ * shared memory, returns TSVD_E_TOOBIG (one and two tokens fit at any supported length, four up to about
+ * 40,000 columns, sixteen up to about 12,000; nine to sixteen tokens also need 1024 columns or more in
+ * both stages). */
 #define TSVD_DECODE_MAX_B 16
 /* the index-list kernels serve at most this many tokens */
 #define TSVD_INDEX_MAX_B 4
