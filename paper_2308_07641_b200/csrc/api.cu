@@ -320,15 +320,21 @@ static unsigned choose_path(const tsvd_handle_s* h, int B, tsvd_dtype_t dtype, u
     // tokens 11.5 / 13.1, 12.9 / 13.1, 16.5 / 14.1 and 21.2 / 14.6; at four tokens and fewer the decode
     // kernels win everywhere (4096^3: 9.1 / 13.0).
     if (tsvd_mid_fits(h, B, dtype, wide_x) && (B >= 9 || !tsvd_decode_cluster_form(h, B))) return TSVD_FLAG_PATH_TENSOR;
-    // Nine to sixteen tokens on tall matrices: where the decode kernels' clusters (four CTAs per 128 rows) need
-    // four rounds or more over the two stages, one padded token tile on the tile kernels is as fast or faster
-    // (16384 x 4096 x 4096: 33-35 us against 30; 8192^3: 41-51 against 43; but 4096 x 4096 x 8192, three
-    // rounds: 23-29 against 36).
-    if (fits && B >= 9) {
+    // Three tokens and more on tall matrices: the decode kernels run one CTA per 32 rows and SM, so a stage of
+    // R rows takes ceil(R / 32 / SMs) rounds of about 3.8 us (three and four tokens), 5 us (up to eight) or 7 us
+    // (up to sixteen), while one padded token tile on the tile kernels costs about 16 us plus 0.2 us per block of
+    // 128 columns a CTA walks through.  Measured, decode / tiles: 32768 x 1024 x 1024 at 3 and 8 tokens 29 / 17
+    // and 38 / 17 us; 16384 x 4096 x 4096 at 4, 8 and 9-16 tokens 23 / 30, 33 / 30 and 33-35 / 30; 8192^3 at
+    // 4 and 9-16 tokens 29 / 43 and 41-51 / 43; 4096 x 4096 x 8192 at 9-16 tokens 23-29 / 36.
+    if (fits && B >= 3) {
         int sms = 148, dev = 0;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        const int rounds = (h->V.R_pad / 128 * 4 + sms - 1) / sms + (h->U.R_pad / 128 * 4 + sms - 1) / sms;
-        if (rounds >= 4) return TSVD_FLAG_PATH_TENSOR;
+        const int rv = h->V.R_pad / 128, ru = h->U.R_pad / 128;
+        const int rounds = (4 * rv + sms - 1) / sms + (4 * ru + sms - 1) / sms;
+        const double decode_us = rounds * (B <= 4 ? 3.8 : B <= 8 ? 5.0 : 7.0);
+        const double tiles_us = 16.0 + 0.195 * ((double)((rv + sms - 1) / sms) * (h->V.C_pad / 128) +
+                                                (double)((ru + sms - 1) / sms) * (h->U.C_pad / 128));
+        if (decode_us > tiles_us || (B >= 9 && rounds >= 4)) return TSVD_FLAG_PATH_TENSOR;
     }
     return fits ? TSVD_FLAG_PATH_DECODE : TSVD_FLAG_PATH_TENSOR;
 }
